@@ -1,0 +1,190 @@
+/*
+ * td.h - C ABI of the transfer dock: put/get dispatch of RL samples held in GPU memory.
+ *
+ * The dock follows the sample flow of "Distributed Transfer Dock Strategy" (Fig. 4, Eq. 4):
+ *   warehouses  hold the real data, the buffer being split along the global batch with every
+ *               sample keeping its own index        -> per-column ragged arenas, S shards;
+ *   controllers (one per worker state) record which samples that state may still be served
+ *                                                   -> per-consumer claim / consumed bitmaps;
+ *   workflow    1. a worker state asks its controller for metadata     (td_get: select)
+ *               2. it fetches, or sends, the real data                 (td_get: gather, td_put)
+ *               3. the warehouse updates its state, visible to every controller
+ *                                                                      (td_put: publish).
+ * The record schema is the one under Eq. 1: one prompt-length item, several response-length
+ * items and a few scalars per sample; samples come in GRPO groups of N responses per prompt
+ * (Fig. 2).  The group-normalised advantage is not given in the paper; td_get computes
+ * A = (r - mean) / (std + eps) over each dispatched group, population std, in double.
+ *
+ * Conventions for every call:
+ *   - "device" pointers are CUDA device memory owned by the caller; the library allocates no
+ *     device memory and frees none.  "host" pointers are ordinary host memory.
+ *   - td_put / td_get / td_get_many / td_reset only enqueue work on the given stream and return;
+ *     they never synchronise.  Calls on one stream execute in call order.  Gets may run
+ *     concurrently with each other and with puts on other streams; puts that touch the same
+ *     (sample, length class) must be ordered by the caller.
+ *   - return value: TD_OK (0) or a negative td_error found on the host.  Conditions found on the
+ *     device never trap: the offending sample is skipped, a TD_ERR_* bit is OR-ed into the
+ *     dock's error word (td_status) and, for a get, into td_result.status.
+ *   - a streamlike argument is a cudaStream_t passed as void* (NULL = the default stream).
+ */
+#ifndef TD_H
+#define TD_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct td_dock td_dock;          /* opaque host object */
+
+enum { TD_I32 = 0, TD_F32 = 1, TD_BF16 = 2 };             /* td_column.dtype */
+enum { TD_SCALAR = 0, TD_PROMPT = 1, TD_RESPONSE = 2 };   /* td_column.cls   */
+enum { TD_PACKED = 0, TD_PADDED = 1 };                    /* td_get_out.mode */
+enum { TD_F_ADVANTAGE = 1u };                             /* td_consumer.flags */
+
+typedef enum {
+    TD_OK = 0,
+    TD_EINVAL = -1,       /* bad argument                                   */
+    TD_EWORKSPACE = -2,   /* workspace or scratch too small or misaligned   */
+    TD_ECUDA = -3         /* a CUDA runtime call failed (no device, ...)    */
+} td_error;
+
+/* device-detected conditions */
+enum {
+    TD_ERR_OOB_INDEX        = 1u << 0,  /* put: sample index outside [0, G*N)                  */
+    TD_ERR_DUP_PUT          = 1u << 1,  /* put: (sample, column) already stored; first one kept */
+    TD_ERR_LEN_MISMATCH     = 1u << 2,  /* put: length differs from the sample's length class   */
+    TD_ERR_ARENA_FULL       = 1u << 3,  /* put: shard arena has no room for the row             */
+    TD_ERR_OUT_TRUNCATED    = 1u << 4,  /* get: stopped before a group that would not fit       */
+    TD_ERR_LOOKBACK_TIMEOUT = 1u << 5,  /* get: a scan tile gave up waiting; nothing returned   */
+    TD_ERR_BAD_LENGTH       = 1u << 6   /* put: cu not monotone or beyond data_elems            */
+};
+
+typedef struct {
+    const char *name;      /* not kept */
+    int32_t  dtype;        /* TD_I32 | TD_F32 | TD_BF16; payload is copied as raw bits */
+    int32_t  cls;          /* TD_SCALAR: one element per sample; TD_PROMPT / TD_RESPONSE:
+                              a row whose length is the sample's prompt / response length */
+    uint32_t pad_bits;     /* raw bit pattern written behind a row in TD_PADDED mode */
+} td_column;
+
+typedef struct {
+    const char *name;      /* not kept */
+    uint32_t need_mask;    /* bit c: column c must be stored before a sample is served */
+    uint32_t out_mask;     /* bit c: column c is gathered; must lie within need_mask   */
+    uint32_t flags;        /* TD_F_ADVANTAGE: needs reward_column within need_mask     */
+} td_consumer;
+
+typedef struct {
+    uint32_t n_prompts;    /* G */
+    uint32_t n_per_group;  /* N; sample s = prompt * N + response, group = s / N */
+    uint32_t n_shards;     /* S warehouses, 1..256, must divide G; shard(s) = (s / N) / (G / S) */
+    uint32_t n_columns;    const td_column   *columns;     /* 1..32, host array */
+    uint32_t n_consumers;  const td_consumer *consumers;   /* 1..32, host array */
+    uint64_t prompt_elems_per_shard;    /* arena capacity per shard, elements (rounded up to 8) */
+    uint64_t response_elems_per_shard;
+    uint32_t reward_column;             /* a TD_F32 TD_SCALAR column */
+    float    adv_eps;
+    int32_t  device;                    /* CUDA device ordinal of the workspace */
+} td_config;
+
+/* Written by td_get on the device; read it after the stream has reached that point. */
+typedef struct {
+    uint32_t n_samples, n_groups;             /* n_samples = n_groups * N */
+    uint64_t prompt_tokens, response_tokens;  /* = cu_prompt[n_samples], cu_response[n_samples] */
+    uint32_t status;                          /* TD_ERR_* bits of this call */
+    uint32_t reserved;
+} td_result;
+
+/* Output buffers of one get.  The struct itself is host memory; every pointer in it is
+ * caller-owned DEVICE memory that stays valid until the get has executed. */
+typedef struct {
+    int32_t  mode;                    /* TD_PACKED: column c holds its rows back to back, row i at
+                                         cu_<class>[i]; TD_PADDED: row i at i * pad_<class>_to,
+                                         filled up with the column's pad_bits */
+    uint32_t pad_prompt_to, pad_response_to;   /* row widths in elements (TD_PADDED only) */
+    uint32_t reserved;
+    int32_t *indices;                 /* [max_samples] sample indices, ascending          required */
+    int32_t *cu_prompt, *cu_response; /* [max_samples + 1] prefix sums of the true lengths required */
+    int32_t *cu_seq;                  /* [max_samples + 1] cu_prompt + cu_response, or NULL */
+    void    *col[32];                 /* per column; NULL = not wanted                     */
+    uint64_t col_capacity_elems[32];  /* room behind col[c], in elements                   */
+    float   *advantages;              /* [max_samples]; required iff TD_F_ADVANTAGE        */
+    td_result *result;                /* required                                          */
+    void    *scratch;                 /* td_get_scratch_bytes() bytes, 16-byte aligned, private to
+                                         this call while it is in flight; zero-filled once after
+                                         allocation, never needs clearing afterwards       required */
+    uint64_t scratch_bytes;
+} td_get_out;
+
+typedef struct {
+    uint64_t put_accepted[32];        /* per column */
+    uint64_t got_samples[32];         /* per consumer */
+    uint64_t got_tokens[32];          /* per consumer, prompt + response tokens */
+    uint64_t n_oob, n_dup, n_len_mismatch, n_arena_full, n_truncated, n_bad_length;
+    uint64_t n_claim_conflicts;       /* groups lost to a concurrent get of the same consumer */
+    uint64_t n_lookback_timeouts;
+    uint32_t error_word;              /* OR of all TD_ERR_* bits since the last reset */
+    uint32_t reserved;
+} td_stats;
+
+/* Bytes of device workspace a dock with this configuration needs (tables, bitmaps and the
+ * arenas of Eq. 4's payload term).  Host only; no CUDA call. */
+int td_query_workspace(const td_config *cfg, size_t *bytes);
+
+/* Builds a dock inside `d_workspace` (device, 256-byte aligned, `bytes` >= td_query_workspace)
+ * and brings it to the empty state on the default stream, synchronising once.  The workspace
+ * stays the caller's and must outlive the dock.  *out is freed by td_destroy. */
+int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **out);
+int td_destroy(td_dock *dock);
+
+/* Workflow steps 2 and 3 for a producer: store column `column` of the k samples d_indices[0..k)
+ * and make them visible to every consumer.
+ *   d_indices  device int32 [k], any order.
+ *   d_cu       device int32 [k + 1], non-decreasing element offsets of the rows inside d_data;
+ *              NULL for a TD_SCALAR column (row i is element i).
+ *   d_data     device, rows back to back, data_elems elements in total (bounds what is read).
+ * Rows are placed in call order: the first column of a length class to arrive for a sample
+ * fixes its length and reserves its row at the next free element of the sample's shard.
+ * Samples that are out of range, already stored, of the wrong length or without room are
+ * skipped and counted.  The same index twice within one call is safe but leaves that row's
+ * content unspecified. */
+int td_put(td_dock *dock, uint32_t column, const int32_t *d_indices, uint32_t k,
+           const int32_t *d_cu, const void *d_data, uint64_t data_elems, void *stream);
+
+/* Workflow steps 1 and 2 for worker state `consumer`: claim the lowest-numbered groups whose
+ * need_mask columns are all stored and that this consumer has not been served, at most
+ * max_samples / N of them, and gather their out_mask columns, cu_seqlens and (TD_F_ADVANTAGE)
+ * advantages into `out`.  Fewer groups than asked for, zero included, is not an error.  The
+ * batch ends before the first group that would overflow a supplied buffer (TD_ERR_OUT_TRUNCATED;
+ * that group stays available).  A group is never served twice to one consumer, also when gets
+ * of that consumer run concurrently on several streams; such a get may then return fewer
+ * groups than were ready. */
+int td_get(td_dock *dock, uint32_t consumer, uint32_t max_samples, const td_get_out *out,
+           void *stream);
+size_t td_get_scratch_bytes(const td_dock *dock);
+
+/* One buffer serves one RL iteration: forget every table, bitmap and counter; payload bytes
+ * and capacities stay. */
+int td_reset(td_dock *dock, void *stream);
+
+/* Synchronises `stream`, then copies counters and the error word to *host_out. */
+int td_status(td_dock *dock, td_stats *host_out, void *stream);
+
+/* Device address and size of an internal table, for inspection by tests and tools.
+ *   which: 0 status u32[n] | 1 len i32[n] (index = class) | 2 off i64[n] (index = class)
+ *          3 cursor u64[S] (index = class) | 4 claim bits (index = consumer)
+ *          5 consumed bits (index = consumer) | 6 arena or scalar store (index = column) */
+int td_debug_table(const td_dock *dock, int which, uint32_t index, void **d_ptr, size_t *bytes);
+
+/* Kernels this dock has launched since td_create. */
+uint64_t td_launch_count(const td_dock *dock);
+
+const char *td_strerror(int code);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TD_H */

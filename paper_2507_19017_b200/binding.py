@@ -1,0 +1,278 @@
+"""Thin ctypes binding of the C ABI in include/td.h.
+
+Argument marshalling only: every step of put and get runs in the CUDA library.  PyTorch
+supplies device memory (`torch.empty(...).data_ptr()`) and streams; nothing here computes
+on tensors.  There is no CPU fallback: if libtd.so cannot be loaded, or a call fails,
+an exception is raised.
+"""
+from __future__ import annotations
+
+import ctypes as C
+import os
+from typing import Dict, List, Optional, Sequence, Tuple
+
+from . import build as _build
+
+I32, F32, BF16 = 0, 1, 2
+SCALAR, PROMPT, RESPONSE = 0, 1, 2
+PACKED, PADDED = 0, 1
+F_ADVANTAGE = 1
+OK, EINVAL, EWORKSPACE, ECUDA = 0, -1, -2, -3
+ERR_OOB_INDEX, ERR_DUP_PUT, ERR_LEN_MISMATCH, ERR_ARENA_FULL = 1, 2, 4, 8
+ERR_OUT_TRUNCATED, ERR_LOOKBACK_TIMEOUT, ERR_BAD_LENGTH = 16, 32, 64
+
+DTYPE_TAG = {"i32": I32, "f32": F32, "bf16": BF16}
+CLASS_TAG = {"scalar": SCALAR, "prompt": PROMPT, "response": RESPONSE}
+ELEM_SIZE = {I32: 4, F32: 4, BF16: 2}
+
+# every symbol include/td.h declares
+EXPORTS = ["td_query_workspace", "td_create", "td_destroy", "td_put", "td_get",
+           "td_get_scratch_bytes", "td_reset", "td_status", "td_debug_table",
+           "td_launch_count", "td_strerror"]
+
+
+class TdColumn(C.Structure):
+    _fields_ = [("name", C.c_char_p), ("dtype", C.c_int32), ("cls", C.c_int32), ("pad_bits", C.c_uint32)]
+
+
+class TdConsumer(C.Structure):
+    _fields_ = [("name", C.c_char_p), ("need_mask", C.c_uint32), ("out_mask", C.c_uint32),
+                ("flags", C.c_uint32)]
+
+
+class TdConfig(C.Structure):
+    _fields_ = [("n_prompts", C.c_uint32), ("n_per_group", C.c_uint32), ("n_shards", C.c_uint32),
+                ("n_columns", C.c_uint32), ("columns", C.POINTER(TdColumn)),
+                ("n_consumers", C.c_uint32), ("consumers", C.POINTER(TdConsumer)),
+                ("prompt_elems_per_shard", C.c_uint64), ("response_elems_per_shard", C.c_uint64),
+                ("reward_column", C.c_uint32), ("adv_eps", C.c_float), ("device", C.c_int32)]
+
+
+class TdResult(C.Structure):
+    _fields_ = [("n_samples", C.c_uint32), ("n_groups", C.c_uint32),
+                ("prompt_tokens", C.c_uint64), ("response_tokens", C.c_uint64),
+                ("status", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class TdGetOut(C.Structure):
+    _fields_ = [("mode", C.c_int32), ("pad_prompt_to", C.c_uint32), ("pad_response_to", C.c_uint32),
+                ("reserved", C.c_uint32),
+                ("indices", C.c_void_p), ("cu_prompt", C.c_void_p), ("cu_response", C.c_void_p),
+                ("cu_seq", C.c_void_p), ("col", C.c_void_p * 32),
+                ("col_capacity_elems", C.c_uint64 * 32), ("advantages", C.c_void_p),
+                ("result", C.c_void_p), ("scratch", C.c_void_p), ("scratch_bytes", C.c_uint64)]
+
+
+class TdStats(C.Structure):
+    _fields_ = [("put_accepted", C.c_uint64 * 32), ("got_samples", C.c_uint64 * 32),
+                ("got_tokens", C.c_uint64 * 32), ("n_oob", C.c_uint64), ("n_dup", C.c_uint64),
+                ("n_len_mismatch", C.c_uint64), ("n_arena_full", C.c_uint64),
+                ("n_truncated", C.c_uint64), ("n_bad_length", C.c_uint64),
+                ("n_claim_conflicts", C.c_uint64), ("n_lookback_timeouts", C.c_uint64),
+                ("error_word", C.c_uint32), ("reserved", C.c_uint32)]
+
+
+class TdError(RuntimeError):
+    def __init__(self, call: str, code: int):
+        self.code = code
+        msg = lib().td_strerror(code).decode() if _lib is not None else "?"
+        super().__init__(f"{call} failed: {code} ({msg})")
+
+
+_lib = None
+
+
+def lib_path() -> str:
+    return _build.LIB_PATH
+
+
+def lib():
+    """Loads libtd.so (raises if it is missing: there is no other implementation)."""
+    global _lib
+    if _lib is None:
+        path = lib_path()
+        if not os.path.exists(path):
+            raise RuntimeError(f"{path} is missing: build it with "
+                               "`python -m paper_2507_19017_b200.build` (needs nvcc)")
+        L = C.CDLL(path)
+        vp, u32, u64 = C.c_void_p, C.c_uint32, C.c_uint64
+        L.td_query_workspace.restype = C.c_int
+        L.td_query_workspace.argtypes = [C.POINTER(TdConfig), C.POINTER(C.c_size_t)]
+        L.td_create.restype = C.c_int
+        L.td_create.argtypes = [C.POINTER(TdConfig), vp, C.c_size_t, C.POINTER(vp)]
+        L.td_destroy.restype = C.c_int
+        L.td_destroy.argtypes = [vp]
+        L.td_put.restype = C.c_int
+        L.td_put.argtypes = [vp, u32, vp, u32, vp, vp, u64, vp]
+        L.td_get.restype = C.c_int
+        L.td_get.argtypes = [vp, u32, u32, C.POINTER(TdGetOut), vp]
+        L.td_get_scratch_bytes.restype = C.c_size_t
+        L.td_get_scratch_bytes.argtypes = [vp]
+        L.td_reset.restype = C.c_int
+        L.td_reset.argtypes = [vp, vp]
+        L.td_status.restype = C.c_int
+        L.td_status.argtypes = [vp, C.POINTER(TdStats), vp]
+        L.td_debug_table.restype = C.c_int
+        L.td_debug_table.argtypes = [vp, C.c_int, u32, C.POINTER(vp), C.POINTER(C.c_size_t)]
+        L.td_launch_count.restype = u64
+        L.td_launch_count.argtypes = [vp]
+        L.td_strerror.restype = C.c_char_p
+        L.td_strerror.argtypes = [C.c_int]
+        _lib = L
+    return _lib
+
+
+def _check(call: str, rc: int):
+    if rc != 0:
+        raise TdError(call, rc)
+
+
+def make_config(G: int, N: int, S: int, columns: Sequence[Tuple[str, str, int]],
+                consumers: Sequence[Tuple[int, int, bool]], prompt_cap: int, response_cap: int,
+                reward_column: int, eps: float = 1e-6, device: int = 0):
+    """columns: (dtype tag, class tag, pad_bits); consumers: (need_mask, out_mask, advantage).
+    Returns (TdConfig, keepalive) - keep the second value alive as long as the first."""
+    cols = (TdColumn * len(columns))(*[TdColumn(None, DTYPE_TAG[d], CLASS_TAG[c], int(p))
+                                       for d, c, p in columns])
+    cons = (TdConsumer * len(consumers))(*[TdConsumer(None, int(a), int(b), F_ADVANTAGE if f else 0)
+                                           for a, b, f in consumers])
+    cfg = TdConfig(G, N, S, len(columns), cols, len(consumers), cons, prompt_cap, response_cap,
+                   reward_column, eps, device)
+    return cfg, (cols, cons)
+
+
+def query_workspace(cfg: TdConfig) -> int:
+    out = C.c_size_t(0)
+    _check("td_query_workspace", lib().td_query_workspace(C.byref(cfg), C.byref(out)))
+    return out.value
+
+
+def _stream_ptr(stream) -> Optional[int]:
+    if stream is None:
+        import torch
+        return torch.cuda.current_stream().cuda_stream
+    if isinstance(stream, int):
+        return stream
+    return stream.cuda_stream
+
+
+class GetBuffers:
+    """Device buffers of one get, allocated once and reusable for any number of calls."""
+
+    def __init__(self, dock: "Dock", consumer: int, max_samples: int, mode: int = PACKED,
+                 pad_prompt_to: int = 0, pad_response_to: int = 0,
+                 capacities: Optional[Dict[int, int]] = None, want: Optional[Sequence[int]] = None,
+                 prompt_tokens_cap: Optional[int] = None, response_tokens_cap: Optional[int] = None):
+        import torch
+        dev = dock.device
+        self.dock, self.consumer, self.max_samples, self.mode = dock, consumer, max_samples, mode
+        self.pad_prompt_to, self.pad_response_to = pad_prompt_to, pad_response_to
+        i32 = torch.int32
+        self.indices = torch.zeros(max_samples, dtype=i32, device=dev)
+        self.cu_prompt = torch.zeros(max_samples + 1, dtype=i32, device=dev)
+        self.cu_response = torch.zeros(max_samples + 1, dtype=i32, device=dev)
+        self.cu_seq = torch.zeros(max_samples + 1, dtype=i32, device=dev)
+        self.result = torch.zeros(C.sizeof(TdResult), dtype=torch.uint8, device=dev)
+        self.scratch = torch.zeros(lib().td_get_scratch_bytes(dock.handle), dtype=torch.uint8, device=dev)
+        need, outm, adv = dock.consumers[consumer]
+        self.advantages = torch.zeros(max_samples, dtype=torch.float32, device=dev) if adv else None
+        self.cols: Dict[int, "torch.Tensor"] = {}
+        self.caps: Dict[int, int] = {}
+        tdt = {I32: torch.int32, F32: torch.float32, BF16: torch.bfloat16}
+        for c, (dt, cls, _pad) in enumerate(dock.columns):
+            if not (outm >> c) & 1 or (want is not None and c not in want):
+                continue
+            if capacities is not None and c in capacities:
+                cap = int(capacities[c])
+            elif cls == SCALAR:
+                cap = max_samples
+            elif mode == PADDED:
+                cap = max_samples * (pad_prompt_to if cls == PROMPT else pad_response_to)
+            else:
+                cap = prompt_tokens_cap if cls == PROMPT else response_tokens_cap
+                if cap is None:
+                    raise ValueError("packed ragged columns need prompt_tokens_cap / response_tokens_cap "
+                                     "or explicit capacities")
+            self.caps[c] = cap
+            self.cols[c] = torch.empty(max(cap, 1), dtype=tdt[dt], device=dev)
+        go = TdGetOut()
+        go.mode, go.pad_prompt_to, go.pad_response_to = mode, pad_prompt_to, pad_response_to
+        go.indices, go.cu_prompt = self.indices.data_ptr(), self.cu_prompt.data_ptr()
+        go.cu_response, go.cu_seq = self.cu_response.data_ptr(), self.cu_seq.data_ptr()
+        for c, t in self.cols.items():
+            go.col[c] = t.data_ptr()
+            go.col_capacity_elems[c] = self.caps[c]
+        go.advantages = self.advantages.data_ptr() if self.advantages is not None else None
+        go.result = self.result.data_ptr()
+        go.scratch, go.scratch_bytes = self.scratch.data_ptr(), self.scratch.numel()
+        self.struct = go
+
+    def read_result(self) -> TdResult:
+        """Copies the result block to the host (synchronises the current stream)."""
+        host = self.result.cpu().numpy().tobytes()
+        return TdResult.from_buffer_copy(host)
+
+
+class Dock:
+    """A transfer dock living in one torch-allocated workspace on `device`."""
+
+    def __init__(self, G: int, N: int, S: int, columns: Sequence[Tuple[str, str, int]],
+                 consumers: Sequence[Tuple[int, int, bool]], prompt_cap: int, response_cap: int,
+                 reward_column: int, eps: float = 1e-6, device: int = 0):
+        import torch
+        self.G, self.N, self.S, self.n = G, N, S, G * N
+        self.columns = [(DTYPE_TAG[d], CLASS_TAG[c], int(p)) for d, c, p in columns]
+        self.consumers = [(int(a), int(b), bool(f)) for a, b, f in consumers]
+        self.device = torch.device("cuda", device)
+        self.cfg, self._keep = make_config(G, N, S, columns, consumers, prompt_cap, response_cap,
+                                           reward_column, eps, device)
+        self.workspace_bytes = query_workspace(self.cfg)
+        self.workspace = torch.empty(self.workspace_bytes, dtype=torch.uint8, device=self.device)
+        h = C.c_void_p()
+        _check("td_create", lib().td_create(C.byref(self.cfg), self.workspace.data_ptr(),
+                                            self.workspace_bytes, C.byref(h)))
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().td_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # -- the four calls ---------------------------------------------------
+    def put(self, column: int, indices, cu, data, stream=None):
+        """indices int32 [k], cu int32 [k+1] or None, data: device tensors."""
+        k = indices.numel()
+        _check("td_put", lib().td_put(self.handle, column, indices.data_ptr(), k,
+                                      cu.data_ptr() if cu is not None else None,
+                                      data.data_ptr(), data.numel(), _stream_ptr(stream)))
+
+    def get(self, bufs: GetBuffers, stream=None, max_samples: Optional[int] = None):
+        _check("td_get", lib().td_get(self.handle, bufs.consumer,
+                                      bufs.max_samples if max_samples is None else max_samples,
+                                      C.byref(bufs.struct), _stream_ptr(stream)))
+
+    def reset(self, stream=None):
+        _check("td_reset", lib().td_reset(self.handle, _stream_ptr(stream)))
+
+    def status(self, stream=None) -> TdStats:
+        st = TdStats()
+        _check("td_status", lib().td_status(self.handle, C.byref(st), _stream_ptr(stream)))
+        return st
+
+    # -- inspection -------------------------------------------------------
+    def table(self, which: int, index: int = 0):
+        """Device table as a uint8 torch tensor view (copy it before the dock changes)."""
+        import torch
+        ptr, nbytes = C.c_void_p(), C.c_size_t()
+        _check("td_debug_table", lib().td_debug_table(self.handle, which, index, C.byref(ptr), C.byref(nbytes)))
+        off = ptr.value - self.workspace.data_ptr()
+        return self.workspace[off:off + nbytes.value]
+
+    def launch_count(self) -> int:
+        return lib().td_launch_count(self.handle)

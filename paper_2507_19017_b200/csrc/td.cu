@@ -1,0 +1,313 @@
+// Host side of the C ABI declared in include/td.h: argument checks, workspace carving and
+// kernel launches.  No device memory is allocated here and nothing synchronises except
+// td_create (once) and td_status.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "td_device.cuh"
+#include "td_get.cuh"
+#include "td_put.cuh"
+
+using namespace td;
+
+struct td_dock {
+    DockView dv;
+    td_config cfg;                 // columns / consumers pointers are not kept
+    int device;
+    int sm_count;
+    uint8_t *ws;
+    size_t ws_bytes;
+    size_t table_bytes[7];
+    std::atomic<uint64_t> launches;
+};
+
+namespace {
+
+std::atomic<uint32_t> g_seq{1};     // launch sequence numbers for scan scratch, process wide
+
+inline size_t align_up_sz(size_t x, size_t a) { return (x + a - 1) / a * a; }
+inline uint32_t esize_of(int32_t dtype) { return dtype == TD_BF16 ? 2u : 4u; }
+
+struct Layout {
+    size_t status, len[3], off[3], cursor[3], claim, consumed, errword, counters, col[kMaxColumns], total;
+    uint32_t claim_words, consumed_words;
+    uint64_t cap[3];
+};
+
+bool valid_config(const td_config *c) {
+    if (!c || !c->columns || !c->consumers) return false;
+    if (c->n_prompts == 0 || c->n_per_group == 0 || c->n_shards == 0 || c->n_shards > 256) return false;
+    if (c->n_prompts % c->n_shards) return false;
+    if (c->n_columns == 0 || c->n_columns > 32 || c->n_consumers == 0 || c->n_consumers > 32) return false;
+    if ((uint64_t)c->n_prompts * c->n_per_group >= (1ull << 30)) return false;
+    for (uint32_t k = 0; k < c->n_columns; ++k) {
+        const td_column &col = c->columns[k];
+        if (col.dtype < TD_I32 || col.dtype > TD_BF16) return false;
+        if (col.cls < TD_SCALAR || col.cls > TD_RESPONSE) return false;
+    }
+    const uint32_t all = c->n_columns == 32 ? 0xffffffffu : ((1u << c->n_columns) - 1u);
+    for (uint32_t k = 0; k < c->n_consumers; ++k) {
+        const td_consumer &q = c->consumers[k];
+        if ((q.need_mask & ~all) || (q.out_mask & ~q.need_mask)) return false;
+        if (q.flags & TD_F_ADVANTAGE) {
+            if (c->reward_column >= c->n_columns) return false;
+            const td_column &r = c->columns[c->reward_column];
+            if (r.cls != TD_SCALAR || r.dtype != TD_F32) return false;
+            if (!((q.need_mask >> c->reward_column) & 1u)) return false;
+        }
+    }
+    return true;
+}
+
+Layout make_layout(const td_config *c) {
+    Layout L{};
+    const size_t n = (size_t)c->n_prompts * c->n_per_group;
+    const size_t S = c->n_shards;
+    L.cap[1] = (c->prompt_elems_per_shard + 7) / 8 * 8;
+    L.cap[2] = (c->response_elems_per_shard + 7) / 8 * 8;
+    L.claim_words = (c->n_prompts + 31) / 32;
+    L.consumed_words = (uint32_t)((n + 31) / 32);
+    size_t p = 0;
+    auto take = [&](size_t bytes) { size_t at = p; p = align_up_sz(p + bytes, 256); return at; };
+    L.errword = take(256);
+    L.counters = take(CNT_TOTAL * 8);
+    L.status = take(n * 4);
+    for (int k = 1; k <= 2; ++k) { L.len[k] = take(n * 4); L.off[k] = take(n * 8); L.cursor[k] = take(S * 8); }
+    L.claim = take((size_t)c->n_consumers * L.claim_words * 4);
+    L.consumed = take((size_t)c->n_consumers * L.consumed_words * 4);
+    for (uint32_t k = 0; k < c->n_columns; ++k) {
+        const td_column &col = c->columns[k];
+        const size_t es = esize_of(col.dtype);
+        L.col[k] = take(col.cls == TD_SCALAR ? n * es : S * L.cap[col.cls] * es);
+    }
+    L.total = p;
+    return L;
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch(td_dock *d, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                   cudaStream_t st, Args &&...args) {
+    kernel<<<grid, block, smem, st>>>(std::forward<Args>(args)...);
+    d->launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaGetLastError();
+}
+
+}  // namespace
+
+extern "C" {
+
+const char *td_strerror(int code) {
+    switch (code) {
+        case TD_OK: return "ok";
+        case TD_EINVAL: return "invalid argument";
+        case TD_EWORKSPACE: return "workspace or scratch too small or misaligned";
+        case TD_ECUDA: return "CUDA runtime call failed";
+        default: return "unknown error";
+    }
+}
+
+int td_query_workspace(const td_config *cfg, size_t *bytes) {
+    if (!bytes || !valid_config(cfg)) return TD_EINVAL;
+    *bytes = make_layout(cfg).total;
+    return TD_OK;
+}
+
+int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **out) {
+    if (!out || !d_workspace || !valid_config(cfg)) return TD_EINVAL;
+    const Layout L = make_layout(cfg);
+    if (bytes < L.total || (reinterpret_cast<uintptr_t>(d_workspace) & 255u)) return TD_EWORKSPACE;
+    if (cudaSetDevice(cfg->device) != cudaSuccess) return TD_ECUDA;
+    int sms = 0;
+    if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess) return TD_ECUDA;
+    const size_t alloc_smem = put_alloc_smem_bytes(cfg->n_shards);
+    if (alloc_smem > 48 * 1024 &&
+        cudaFuncSetAttribute(put_alloc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)alloc_smem) != cudaSuccess)
+        return TD_ECUDA;
+
+    td_dock *d = new (std::nothrow) td_dock();
+    if (!d) return TD_EINVAL;
+    d->cfg = *cfg; d->cfg.columns = nullptr; d->cfg.consumers = nullptr;
+    d->device = cfg->device; d->sm_count = sms;
+    d->ws = static_cast<uint8_t *>(d_workspace); d->ws_bytes = bytes;
+    d->launches = 0;
+    DockView &v = d->dv;
+    std::memset(&v, 0, sizeof(v));
+    v.G = cfg->n_prompts; v.N = cfg->n_per_group; v.S = cfg->n_shards; v.n = v.G * v.N;
+    v.ncol = cfg->n_columns; v.ncons = cfg->n_consumers;
+    v.prompts_per_shard = v.G / v.S;
+    v.reward_col = cfg->reward_column;
+    v.claim_words = L.claim_words; v.consumed_words = L.consumed_words;
+    v.spin_limit = 1u << 20;
+    v.eps = (double)cfg->adv_eps;
+    v.cap[1] = L.cap[1]; v.cap[2] = L.cap[2];
+    uint8_t *w = d->ws;
+    v.status = reinterpret_cast<uint32_t *>(w + L.status);
+    for (int k = 1; k <= 2; ++k) {
+        v.len[k] = reinterpret_cast<int32_t *>(w + L.len[k]);
+        v.off[k] = reinterpret_cast<long long *>(w + L.off[k]);
+        v.cursor[k] = reinterpret_cast<unsigned long long *>(w + L.cursor[k]);
+    }
+    v.claim = reinterpret_cast<uint32_t *>(w + L.claim);
+    v.consumed = reinterpret_cast<uint32_t *>(w + L.consumed);
+    v.errword = reinterpret_cast<uint32_t *>(w + L.errword);
+    v.counters = reinterpret_cast<unsigned long long *>(w + L.counters);
+    for (uint32_t k = 0; k < v.ncol; ++k) {
+        v.colbase[k] = w + L.col[k];
+        v.col_esz[k] = (uint8_t)esize_of(cfg->columns[k].dtype);
+        v.col_cls[k] = (uint8_t)cfg->columns[k].cls;
+        v.col_pad[k] = cfg->columns[k].pad_bits;
+    }
+    for (uint32_t k = 0; k < v.ncons; ++k) {
+        v.need[k] = cfg->consumers[k].need_mask;
+        v.outm[k] = cfg->consumers[k].out_mask;
+        v.cflags[k] = cfg->consumers[k].flags;
+    }
+    d->table_bytes[0] = (size_t)v.n * 4; d->table_bytes[1] = (size_t)v.n * 4; d->table_bytes[2] = (size_t)v.n * 8;
+    d->table_bytes[3] = (size_t)v.S * 8; d->table_bytes[4] = (size_t)v.claim_words * 4;
+    d->table_bytes[5] = (size_t)v.consumed_words * 4; d->table_bytes[6] = 0;
+
+    int rc = td_reset(d, nullptr);
+    if (rc == TD_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) rc = TD_ECUDA;
+    if (rc != TD_OK) { delete d; return rc; }
+    *out = d;
+    return TD_OK;
+}
+
+int td_destroy(td_dock *dock) {
+    delete dock;
+    return TD_OK;
+}
+
+int td_reset(td_dock *d, void *stream) {
+    if (!d) return TD_EINVAL;
+    const uint32_t blocks = (uint32_t)std::min<size_t>((d->dv.n + 255) / 256, (size_t)d->sm_count * 4);
+    if (launch(d, reset_kernel, dim3(blocks ? blocks : 1), dim3(256), 0, (cudaStream_t)stream, d->dv) != cudaSuccess)
+        return TD_ECUDA;
+    return TD_OK;
+}
+
+int td_put(td_dock *d, uint32_t column, const int32_t *d_indices, uint32_t k, const int32_t *d_cu,
+           const void *d_data, uint64_t data_elems, void *stream) {
+    if (!d || column >= d->dv.ncol) return TD_EINVAL;
+    if (k == 0) return TD_OK;
+    if (!d_indices || !d_data) return TD_EINVAL;
+    const uint32_t cls = d->dv.col_cls[column];
+    if (cls != TD_SCALAR && !d_cu) return TD_EINVAL;
+    if (data_elems >= (1ull << 31)) return TD_EINVAL;       // cu is int32
+    cudaStream_t st = (cudaStream_t)stream;
+    PutArgs a{column, k, d_indices, d_cu, static_cast<const uint8_t *>(d_data), data_elems};
+    if (cls == TD_SCALAR) {
+        if (launch(d, put_scalar_kernel, dim3((k + 255) / 256), dim3(256), 0, st, d->dv, a) != cudaSuccess) return TD_ECUDA;
+        return TD_OK;
+    }
+    if (launch(d, put_alloc_kernel, dim3(1), dim3(kAllocThreads), put_alloc_smem_bytes(d->dv.S), st, d->dv, a) != cudaSuccess)
+        return TD_ECUDA;
+    const uint64_t bytes = data_elems * d->dv.col_esz[column];
+    const uint64_t chunks = (bytes + kWarpChunkBytes - 1) / kWarpChunkBytes;
+    uint64_t blocks = (chunks + kCopyWarps - 1) / kCopyWarps;
+    const uint64_t max_blocks = (uint64_t)d->sm_count * 8;
+    if (blocks > max_blocks) blocks = max_blocks;
+    if (blocks == 0) blocks = 1;
+    if (launch(d, put_scatter_kernel, dim3((uint32_t)blocks), dim3(kCopyThreads), 0, st, d->dv, a) != cudaSuccess) return TD_ECUDA;
+    if (launch(d, put_publish_kernel, dim3((k + 255) / 256), dim3(256), 0, st, d->dv, a) != cudaSuccess) return TD_ECUDA;
+    return TD_OK;
+}
+
+size_t td_get_scratch_bytes(const td_dock *d) {
+    return d ? sel_scratch_bytes(d->dv.G) : 0;
+}
+
+int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out *out, void *stream) {
+    if (!d || !out || consumer >= d->dv.ncons) return TD_EINVAL;
+    const DockView &v = d->dv;
+    const uint32_t m = max_samples / v.N;
+    if (m == 0) return TD_EINVAL;
+    if (!out->indices || !out->cu_prompt || !out->cu_response || !out->result) return TD_EINVAL;
+    if (out->mode != TD_PACKED && out->mode != TD_PADDED) return TD_EINVAL;
+    if ((v.cflags[consumer] & TD_F_ADVANTAGE) && !out->advantages) return TD_EINVAL;
+    if (!out->scratch || (reinterpret_cast<uintptr_t>(out->scratch) & 15u) ||
+        out->scratch_bytes < sel_scratch_bytes(v.G))
+        return TD_EWORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+
+    GetInline one;
+    std::memset(&one, 0, sizeof(one));
+    one.req.out = *out;
+    one.req.consumer = consumer;
+    one.req.max_groups = m < v.G ? m : v.G;
+    one.req.rank_base = 0;
+    one.req.cslot = 0;
+    one.cs.consumer = consumer;
+    one.cs.max_groups = one.req.max_groups;
+    one.cs.scratch = out->scratch;
+    const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
+
+    if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
+               (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
+    if (launch(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
+               (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
+    // gather grid from the room the caller supplied
+    uint64_t bytes = 0;
+    for (uint32_t k = 0; k < v.ncol; ++k)
+        if (((v.outm[consumer] >> k) & 1u) && out->col[k]) {
+            uint64_t room = out->col_capacity_elems[k];
+            if (v.col_cls[k] == TD_SCALAR && room > max_samples) room = max_samples;
+            bytes += room * v.col_esz[k] + kGatherChunkBytes;
+        }
+    uint64_t blocks = (bytes / kGatherChunkBytes + kGatherWarps - 1) / kGatherWarps;
+    const uint64_t max_blocks = (uint64_t)d->sm_count * 8;
+    if (blocks > max_blocks) blocks = max_blocks;
+    if (blocks == 0) blocks = 1;
+    if (launch(d, get_gather_kernel, dim3((uint32_t)blocks), dim3(kGatherThreads), 0, st, v, one,
+               (const GetReq *)nullptr, 1u) != cudaSuccess) return TD_ECUDA;
+    return TD_OK;
+}
+
+int td_status(td_dock *d, td_stats *host_out, void *stream) {
+    if (!d || !host_out) return TD_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    unsigned long long cnt[CNT_TOTAL];
+    uint32_t err = 0;
+    if (cudaMemcpyAsync(cnt, d->dv.counters, sizeof(cnt), cudaMemcpyDeviceToHost, st) != cudaSuccess) return TD_ECUDA;
+    if (cudaMemcpyAsync(&err, d->dv.errword, sizeof(err), cudaMemcpyDeviceToHost, st) != cudaSuccess) return TD_ECUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
+    std::memset(host_out, 0, sizeof(*host_out));
+    for (int i = 0; i < 32; ++i) {
+        host_out->put_accepted[i] = cnt[CNT_PUT_ACCEPTED + i];
+        host_out->got_samples[i] = cnt[CNT_GOT_SAMPLES + i];
+        host_out->got_tokens[i] = cnt[CNT_GOT_TOKENS + i];
+    }
+    host_out->n_oob = cnt[CNT_OOB]; host_out->n_dup = cnt[CNT_DUP];
+    host_out->n_len_mismatch = cnt[CNT_MISMATCH]; host_out->n_arena_full = cnt[CNT_FULL];
+    host_out->n_truncated = cnt[CNT_TRUNC]; host_out->n_bad_length = cnt[CNT_BADLEN];
+    host_out->n_claim_conflicts = cnt[CNT_CONFLICT]; host_out->n_lookback_timeouts = cnt[CNT_TIMEOUT];
+    host_out->error_word = err;
+    return TD_OK;
+}
+
+int td_debug_table(const td_dock *d, int which, uint32_t index, void **d_ptr, size_t *bytes) {
+    if (!d || !d_ptr || !bytes) return TD_EINVAL;
+    const DockView &v = d->dv;
+    switch (which) {
+        case 0: *d_ptr = v.status; *bytes = (size_t)v.n * 4; return TD_OK;
+        case 1: if (index < 1 || index > 2) return TD_EINVAL; *d_ptr = v.len[index]; *bytes = (size_t)v.n * 4; return TD_OK;
+        case 2: if (index < 1 || index > 2) return TD_EINVAL; *d_ptr = v.off[index]; *bytes = (size_t)v.n * 8; return TD_OK;
+        case 3: if (index < 1 || index > 2) return TD_EINVAL; *d_ptr = v.cursor[index]; *bytes = (size_t)v.S * 8; return TD_OK;
+        case 4: if (index >= v.ncons) return TD_EINVAL; *d_ptr = v.claim + (size_t)index * v.claim_words; *bytes = (size_t)v.claim_words * 4; return TD_OK;
+        case 5: if (index >= v.ncons) return TD_EINVAL; *d_ptr = v.consumed + (size_t)index * v.consumed_words; *bytes = (size_t)v.consumed_words * 4; return TD_OK;
+        case 6: {
+            if (index >= v.ncol) return TD_EINVAL;
+            *d_ptr = v.colbase[index];
+            const uint32_t cls = v.col_cls[index];
+            *bytes = cls == TD_SCALAR ? (size_t)v.n * v.col_esz[index] : (size_t)v.S * v.cap[cls] * v.col_esz[index];
+            return TD_OK;
+        }
+        default: return TD_EINVAL;
+    }
+}
+
+uint64_t td_launch_count(const td_dock *d) { return d ? d->launches.load() : 0; }
+
+}  // extern "C"

@@ -1,0 +1,481 @@
+// td_get: readiness scan + compaction + claim (select), cu_seqlens / advantages (finalize),
+// ragged gather.  Workflow steps 1 and 2 of "Distributed Transfer Dock Strategy": the worker
+// state asks its controller which samples come next, then fetches the real data.
+#pragma once
+
+#include "td_device.cuh"
+
+namespace td {
+
+constexpr int kSelThreads = 256;            // one thread per group; a tile is 256 groups
+constexpr int kSelWarps = kSelThreads / 32;
+constexpr int kFinThreads = 256;
+constexpr int kGatherThreads = 256;
+constexpr int kGatherWarps = kGatherThreads / 32;
+constexpr uint32_t kGatherChunkBytes = 4096;   // output bytes one warp produces per step
+constexpr int kMaxJobs = 2048;              // (request, column) pairs one gather launch serves
+
+// Tile descriptor of the single-pass scan: [63:32] launch sequence number, [31:30] state,
+// [29:0] count.  A descriptor whose sequence number is not the launch's is "not written yet",
+// so scratch never has to be cleared between gets.
+constexpr uint32_t kStateAggregate = 1, kStatePrefix = 2, kStateFailed = 3;
+__host__ __device__ __forceinline__ unsigned long long desc_pack(uint32_t seq, uint32_t state, uint32_t count) {
+    return ((unsigned long long)seq << 32) | ((unsigned long long)state << 30) | (count & 0x3fffffffu);
+}
+__device__ __forceinline__ uint32_t desc_seq(unsigned long long d) { return (uint32_t)(d >> 32); }
+__device__ __forceinline__ uint32_t desc_state(unsigned long long d) { return (uint32_t)(d >> 30) & 3u; }
+__device__ __forceinline__ uint32_t desc_count(unsigned long long d) { return (uint32_t)d & 0x3fffffffu; }
+
+// Scratch of one (call, consumer): [0] ticket, [1] reserved, [2 .. 2+T) tile descriptors, then
+// the candidate list int32[G]: the r-th ready group in index order, one's complement when the
+// claim was lost to a concurrent get.
+struct SelScratch {
+    unsigned long long *ticket;
+    unsigned long long *desc;
+    int32_t *cand;
+};
+__host__ __device__ __forceinline__ uint32_t sel_tiles(uint32_t G) { return (G + kSelThreads - 1) / kSelThreads; }
+__host__ __device__ __forceinline__ size_t sel_scratch_bytes(uint32_t G) {
+    size_t b = (2 + (size_t)sel_tiles(G)) * 8 + (size_t)G * 4;
+    return (b + 15) & ~size_t(15);
+}
+__host__ __device__ __forceinline__ SelScratch sel_scratch(void *p, uint32_t G) {
+    SelScratch s;
+    s.ticket = reinterpret_cast<unsigned long long *>(p);
+    s.desc = s.ticket + 2;
+    s.cand = reinterpret_cast<int32_t *>(s.desc + sel_tiles(G));
+    return s;
+}
+
+// One request of a call and the consumer slot it draws its groups from.
+struct GetReq {
+    td_get_out out;
+    uint32_t consumer;
+    uint32_t max_groups;      // floor(max_samples / N)
+    uint32_t rank_base;       // first candidate rank this request may take
+    uint32_t cslot;
+};
+struct ConsumerSlot {
+    uint32_t consumer;
+    uint32_t max_groups;      // over all requests of the call that name this consumer
+    void *scratch;
+};
+struct GetInline {            // a single get travels in the kernel parameters
+    GetReq req;
+    ConsumerSlot cs;
+};
+
+// ---------------------------------------------------------------------------------------------
+// Select.  grid = (tiles, consumer slots).  Thread g of a tile tests group g: all N status
+// words carry the consumer's need bits and the group is not claimed.  Warp ballots and popc
+// give the rank inside the tile, a decoupled look-back over the tile descriptors gives the
+// rank before it, and the first max_groups ready groups are claimed with one atomicOr per
+// warp.  Tiles take their number from a ticket, so a tile only ever waits for tiles that have
+// already started; the wait is bounded all the same.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kSelThreads)
+get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
+                  const ConsumerSlot *slots_dev, const uint32_t seq) {
+    const ConsumerSlot *slots = slots_dev ? slots_dev : &one.cs;
+    const ConsumerSlot cs = slots[blockIdx.y];
+    const SelScratch sc = sel_scratch(cs.scratch, dv.G);
+    const uint32_t c = cs.consumer;
+    const uint32_t need = dv.need[c];
+    uint32_t *claim = dv.claim + (size_t)c * dv.claim_words;
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    __shared__ uint32_t s_tile, s_excl, s_failed;
+    __shared__ uint32_t s_warp[kSelWarps];
+
+    if (tid == 0) {
+        // ticket word = seq << 32 | tiles started; sequence numbers only grow
+        atomicMax(sc.ticket, (unsigned long long)seq << 32);
+        const unsigned long long t = atomicAdd(sc.ticket, 1ull);
+        s_tile = (uint32_t)(t & 0xffffffffu);
+        // scratch shared with another launch in flight: refuse rather than index past the tiles
+        s_failed = (uint32_t)(t >> 32) != seq || (uint32_t)(t & 0xffffffffu) >= gridDim.x;
+    }
+    __syncthreads();
+    if (s_failed) {
+        if (tid == 0) flag_error(dv, TD_ERR_LOOKBACK_TIMEOUT, CNT_TIMEOUT);
+        return;
+    }
+    const uint32_t tile = s_tile;
+    const uint32_t g = tile * kSelThreads + tid;
+
+    bool ready = false;
+    if (g < dv.G) {
+        const uint32_t cw = ld_acquire_u32(&claim[g >> 5]);
+        if (!((cw >> (g & 31)) & 1u)) {
+            ready = true;
+            const uint32_t *st = dv.status + (size_t)g * dv.N;
+            for (uint32_t j = 0; j < dv.N; ++j)
+                if ((ld_acquire_u32(st + j) & need) != need) { ready = false; break; }
+        }
+    }
+    const uint32_t ballot = __ballot_sync(kFullMask, ready);
+    const uint32_t in_warp = __popc(ballot & ((1u << lane) - 1u));
+    if (lane == 0) s_warp[warp] = __popc(ballot);
+    __syncthreads();
+    uint32_t warp_off = 0, tile_count = 0;
+    #pragma unroll
+    for (int w = 0; w < kSelWarps; ++w) {
+        const uint32_t v = s_warp[w];
+        if (w < (int)warp) warp_off += v;
+        tile_count += v;
+    }
+
+    if (warp == 0) {
+        uint32_t excl = 0;
+        bool failed = s_failed;
+        if (tile == 0) {
+            if (lane == 0) st_release_u64(&sc.desc[0], desc_pack(seq, kStatePrefix, tile_count));
+        } else {
+            if (lane == 0) st_release_u64(&sc.desc[tile], desc_pack(seq, kStateAggregate, tile_count));
+            // look back over windows of 32 predecessors
+            int32_t look = (int32_t)tile - 1;
+            bool done = false;
+            while (!done && !failed) {
+                const int32_t t = look - (int32_t)lane;
+                unsigned long long d = 0;
+                uint32_t state = kStatePrefix, count = 0;     // lanes before tile 0 contribute nothing
+                if (t >= 0) {
+                    uint32_t polls = 0;
+                    do {
+                        d = ld_acquire_u64(&sc.desc[t]);
+                        if (desc_seq(d) == seq && desc_state(d) != 0) break;
+                        __nanosleep(32);
+                    } while (++polls < dv.spin_limit);
+                    if (desc_seq(d) != seq || desc_state(d) == 0) state = kStateFailed;
+                    else { state = desc_state(d); count = desc_count(d); }
+                }
+                const uint32_t bad = __ballot_sync(kFullMask, state == kStateFailed);
+                const uint32_t pre = __ballot_sync(kFullMask, state == kStatePrefix);
+                // nearest predecessor that already knows its inclusive prefix
+                const uint32_t first = pre ? (uint32_t)__ffs(pre) - 1u : 32u;
+                const uint32_t upto = first < 32u ? first : 31u;
+                if (bad & (upto == 31u ? kFullMask : ((2u << upto) - 1u))) { failed = true; break; }
+                excl += __reduce_add_sync(kFullMask, lane <= upto ? count : 0u);
+                if (first < 32u) done = true; else look -= 32;
+            }
+            if (lane == 0)
+                st_release_u64(&sc.desc[tile], failed ? desc_pack(seq, kStateFailed, 0)
+                                                      : desc_pack(seq, kStatePrefix, excl + tile_count));
+        }
+        if (lane == 0) { s_excl = excl; s_failed = failed; }
+    }
+    __syncthreads();
+    if (s_failed) {
+        if (tid == 0) flag_error(dv, TD_ERR_LOOKBACK_TIMEOUT, CNT_TIMEOUT);
+        return;
+    }
+    const uint32_t rank = s_excl + warp_off + in_warp;
+    const bool cand = ready && rank < cs.max_groups;
+    const uint32_t mask = __ballot_sync(kFullMask, cand);
+    uint32_t old = 0;
+    if (lane == 0 && mask) old = atomicOr(&claim[g >> 5], mask);   // the warp's 32 groups share a word
+    old = __shfl_sync(kFullMask, old, 0);
+    if (cand) sc.cand[rank] = ((old >> lane) & 1u) ? ~(int32_t)g : (int32_t)g;
+    const uint32_t lost = __popc(mask & old);
+    if (lane == 0 && lost) atomicAdd(&dv.counters[CNT_CONFLICT], (unsigned long long)lost);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Finalize.  One CTA per request: compacts the groups it won into `indices`, builds
+// cu_prompt / cu_response / cu_seq by block scans, cuts the batch before the first group that
+// would not fit a supplied buffer (handing the cut groups back), sets the consumed bits,
+// computes the group-normalised advantages and writes the result block.
+// ---------------------------------------------------------------------------------------------
+__device__ __forceinline__ uint64_t block_scan_incl_2(uint64_t a, uint64_t b, uint64_t &out_b,
+                                                      uint64_t *sh_a, uint64_t *sh_b,
+                                                      uint64_t &tot_a, uint64_t &tot_b) {
+    const uint32_t lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    #pragma unroll
+    for (int d = 1; d < 32; d <<= 1) {
+        const uint64_t ta = __shfl_up_sync(kFullMask, a, d);
+        const uint64_t tb = __shfl_up_sync(kFullMask, b, d);
+        if ((int)lane >= d) { a += ta; b += tb; }
+    }
+    __syncthreads();                 // previous use of sh_* finished
+    if (lane == 31) { sh_a[warp] = a; sh_b[warp] = b; }
+    __syncthreads();
+    uint64_t oa = 0, ob = 0; tot_a = 0; tot_b = 0;
+    #pragma unroll
+    for (int w = 0; w < kFinThreads / 32; ++w) {
+        if (w < (int)warp) { oa += sh_a[w]; ob += sh_b[w]; }
+        tot_a += sh_a[w]; tot_b += sh_b[w];
+    }
+    out_b = b + ob;
+    return a + oa;
+}
+
+__global__ void __launch_bounds__(kFinThreads)
+get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
+                    const GetReq *reqs_dev, const ConsumerSlot *slots_dev, const uint32_t seq) {
+    const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
+    const ConsumerSlot *slots = slots_dev ? slots_dev : &one.cs;
+    const GetReq &rq = reqs[blockIdx.x];
+    const td_get_out &out = rq.out;
+    const ConsumerSlot cs = slots[rq.cslot];
+    const SelScratch sc = sel_scratch(cs.scratch, dv.G);
+    const uint32_t c = rq.consumer, N = dv.N;
+    const uint32_t tid = threadIdx.x;
+    __shared__ uint64_t sh_a[kFinThreads / 32], sh_b[kFinThreads / 32];
+    __shared__ uint32_t s_first_over;
+
+    // how many groups were ready, from the last tile's inclusive prefix
+    const unsigned long long last = sc.desc[sel_tiles(dv.G) - 1];
+    uint32_t status = 0;
+    uint32_t total = 0;
+    if (desc_seq(last) != seq || desc_state(last) != kStatePrefix) status |= TD_ERR_LOOKBACK_TIMEOUT;
+    else total = min(desc_count(last), cs.max_groups);
+    const uint32_t lo = rq.rank_base;
+    const uint32_t hi = min(lo + rq.max_groups, total);
+    const uint32_t ncand = hi > lo ? hi - lo : 0;
+
+    // pass A: groups won, in order -> indices
+    uint32_t n_grp = 0;
+    for (uint32_t base = 0; base < ncand; base += kFinThreads) {
+        const uint32_t r = base + tid;
+        int32_t g = -1;
+        if (r < ncand) g = sc.cand[lo + r];
+        uint64_t dummy_b, ta, tb;
+        const uint64_t inc = block_scan_incl_2(g >= 0 ? 1u : 0u, 0, dummy_b, sh_a, sh_b, ta, tb);
+        if (g >= 0) {
+            const uint32_t p = n_grp + (uint32_t)inc - 1u;
+            for (uint32_t j = 0; j < N; ++j) out.indices[(size_t)p * N + j] = g * (int32_t)N + (int32_t)j;
+        }
+        n_grp += (uint32_t)ta;
+    }
+    __syncthreads();
+    uint32_t n_s = n_grp * N;
+
+    // pass B: cu_seqlens and the fit test
+    if (tid == 0) {
+        s_first_over = 0xffffffffu;
+        out.cu_prompt[0] = 0; out.cu_response[0] = 0;
+        if (out.cu_seq) out.cu_seq[0] = 0;
+    }
+    // tightest room per length class over the wanted columns
+    uint64_t room_tok[3] = {~0ull, ~0ull, ~0ull};      // packed: tokens; scalar slot [0]: samples
+    uint64_t room_rows = ~0ull;                         // padded: rows
+    const uint32_t outm = dv.outm[c];
+    for (uint32_t k = 0; k < dv.ncol; ++k) {
+        if (!((outm >> k) & 1u) || out.col[k] == nullptr) continue;
+        const uint32_t cls = dv.col_cls[k];
+        const uint64_t capk = out.col_capacity_elems[k];
+        if (cls == TD_SCALAR) room_tok[0] = min(room_tok[0], capk);
+        else if (out.mode == TD_PACKED) room_tok[cls] = min(room_tok[cls], capk);
+        else {
+            const uint32_t W = cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to;
+            room_rows = min(room_rows, W ? (uint64_t)(capk / W) : (uint64_t)0);
+        }
+    }
+    const bool padded = out.mode == TD_PADDED;
+    bool want_p = false, want_r = false;
+    for (uint32_t k = 0; k < dv.ncol; ++k)
+        if (((outm >> k) & 1u) && out.col[k] != nullptr) {
+            want_p |= dv.col_cls[k] == TD_PROMPT;
+            want_r |= dv.col_cls[k] == TD_RESPONSE;
+        }
+    uint64_t carry_p = 0, carry_r = 0;
+    for (uint32_t base = 0; base < n_s; base += kFinThreads) {
+        const uint32_t i = base + tid;
+        uint64_t lp = 0, lr = 0;
+        if (i < n_s) {
+            const int32_t s = out.indices[i];
+            const int32_t a = dv.len[TD_PROMPT][s], b = dv.len[TD_RESPONSE][s];
+            lp = a > 0 ? (uint64_t)a : 0; lr = b > 0 ? (uint64_t)b : 0;
+        }
+        uint64_t ir, tp, tr;
+        const uint64_t ip = block_scan_incl_2(lp, lr, ir, sh_a, sh_b, tp, tr);
+        if (i < n_s) {
+            const uint64_t cp = carry_p + ip, cr = carry_r + ir;
+            out.cu_prompt[i + 1] = (int32_t)cp;
+            out.cu_response[i + 1] = (int32_t)cr;
+            if (out.cu_seq) out.cu_seq[i + 1] = (int32_t)(cp + cr);
+            bool over = (uint64_t)(i + 1) > room_tok[0];
+            if (!padded) over |= cp > room_tok[TD_PROMPT] || cr > room_tok[TD_RESPONSE];
+            else over |= (uint64_t)(i + 1) > room_rows || (want_p && lp > out.pad_prompt_to) ||
+                         (want_r && lr > out.pad_response_to);
+            if (over) atomicMin(&s_first_over, i);
+        }
+        carry_p += tp; carry_r += tr;
+    }
+    __syncthreads();
+    if (s_first_over != 0xffffffffu) {
+        const uint32_t keep = s_first_over / N;
+        for (uint32_t p = keep + tid; p < n_grp; p += kFinThreads) {
+            const uint32_t g = (uint32_t)out.indices[(size_t)p * N] / N;
+            atomicAnd(&dv.claim[(size_t)c * dv.claim_words + (g >> 5)], ~(1u << (g & 31)));
+        }
+        n_grp = keep; n_s = keep * N;
+        status |= TD_ERR_OUT_TRUNCATED;
+        if (tid == 0) flag_error(dv, TD_ERR_OUT_TRUNCATED, CNT_TRUNC);
+    }
+    // consumed bits
+    uint32_t *consumed = dv.consumed + (size_t)c * dv.consumed_words;
+    for (uint32_t i = tid; i < n_s; i += kFinThreads) {
+        const uint32_t s = (uint32_t)out.indices[i];
+        atomicOr(&consumed[s >> 5], 1u << (s & 31));
+    }
+    // group-normalised advantage, one thread per group, in double
+    if ((dv.cflags[c] & TD_F_ADVANTAGE) && out.advantages) {
+        const float *rew = reinterpret_cast<const float *>(dv.colbase[dv.reward_col]);
+        for (uint32_t p = tid; p < n_grp; p += kFinThreads) {
+            const int32_t *ix = out.indices + (size_t)p * N;
+            double sum = 0.0;
+            for (uint32_t j = 0; j < N; ++j) sum += (double)rew[ix[j]];
+            const double mean = sum / (double)N;
+            double ss = 0.0;
+            for (uint32_t j = 0; j < N; ++j) { const double d = (double)rew[ix[j]] - mean; ss += d * d; }
+            const double sd = sqrt(ss / (double)N);
+            for (uint32_t j = 0; j < N; ++j)
+                out.advantages[(size_t)p * N + j] = (float)(((double)rew[ix[j]] - mean) / (sd + dv.eps));
+        }
+    }
+    __syncthreads();
+    if (tid == 0) {
+        td_result r;
+        r.n_samples = n_s; r.n_groups = n_grp;
+        r.prompt_tokens = (uint64_t)(int64_t)out.cu_prompt[n_s];
+        r.response_tokens = (uint64_t)(int64_t)out.cu_response[n_s];
+        r.status = status; r.reserved = 0;
+        *out.result = r;
+        if (status & TD_ERR_LOOKBACK_TIMEOUT) atomicOr(dv.errword, TD_ERR_LOOKBACK_TIMEOUT);
+        atomicAdd(&dv.counters[CNT_GOT_SAMPLES + c], (unsigned long long)n_s);
+        atomicAdd(&dv.counters[CNT_GOT_TOKENS + c], (unsigned long long)(r.prompt_tokens + r.response_tokens));
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Gather.  Persistent grid.  Every (request, wanted column) is a job whose output space is cut
+// into warp chunks of kGatherChunkBytes; warps stride over the chunks of all jobs, so the
+// work is balanced over bytes whatever the mix of row lengths.
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(kGatherThreads)
+get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
+                  const GetReq *reqs_dev, const uint32_t n_req) {
+    const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
+    __shared__ uint64_t job_end[kMaxJobs];          // inclusive prefix of chunks per job
+    __shared__ uint16_t job_req[kMaxJobs];
+    __shared__ uint8_t job_col[kMaxJobs];
+    __shared__ uint32_t s_njobs;
+    const uint32_t tid = threadIdx.x, lane = tid & 31;
+
+    // job table (every CTA builds the same one)
+    if (tid == 0) {
+        uint32_t nj = 0; uint64_t acc = 0;
+        for (uint32_t q = 0; q < n_req; ++q) {
+            const td_get_out &out = reqs[q].out;
+            const td_result res = *out.result;
+            const uint32_t outm = dv.outm[reqs[q].consumer];
+            for (uint32_t k = 0; k < dv.ncol && nj < kMaxJobs; ++k) {
+                if (!((outm >> k) & 1u) || out.col[k] == nullptr) continue;
+                const uint32_t cls = dv.col_cls[k], esz = dv.col_esz[k];
+                uint64_t bytes;
+                if (cls == TD_SCALAR) bytes = (uint64_t)res.n_samples * esz;
+                else if (out.mode == TD_PACKED)
+                    bytes = (cls == TD_PROMPT ? res.prompt_tokens : res.response_tokens) * esz;
+                else
+                    bytes = (uint64_t)res.n_samples * (cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to) * esz;
+                if (bytes == 0) continue;
+                acc += (bytes + kGatherChunkBytes - 1) / kGatherChunkBytes;
+                job_end[nj] = acc; job_req[nj] = (uint16_t)q; job_col[nj] = (uint8_t)k;
+                ++nj;
+            }
+        }
+        s_njobs = nj;
+    }
+    __syncthreads();
+    const uint32_t njobs = s_njobs;
+    if (njobs == 0) return;
+    const uint64_t n_chunks = job_end[njobs - 1];
+    const uint64_t warp0 = (uint64_t)blockIdx.x * kGatherWarps + (tid >> 5);
+    const uint64_t stride = (uint64_t)gridDim.x * kGatherWarps;
+
+    for (uint64_t ch = warp0; ch < n_chunks; ch += stride) {
+        // job of this chunk: first j with job_end[j] > ch
+        uint32_t jlo = 0, jhi = njobs - 1;
+        while (jlo < jhi) { const uint32_t m = (jlo + jhi) >> 1; if (job_end[m] > ch) jhi = m; else jlo = m + 1; }
+        const uint32_t j = jlo;
+        const uint64_t local = ch - (j ? job_end[j - 1] : 0);
+        const GetReq &rq = reqs[job_req[j]];
+        const td_get_out &out = rq.out;
+        const uint32_t k = job_col[j];
+        const uint32_t cls = dv.col_cls[k], esz = dv.col_esz[k];
+        const uint32_t n_s = out.result->n_samples;
+        uint8_t *dst0 = reinterpret_cast<uint8_t *>(out.col[k]);
+        const uint8_t *base = dv.colbase[k];
+        const uint64_t b0 = local * kGatherChunkBytes;
+
+        if (cls == TD_SCALAR) {
+            const uint64_t e0 = b0 / esz, e1 = min((b0 + kGatherChunkBytes) / esz, (uint64_t)n_s);
+            for (uint64_t e = e0 + lane; e < e1; e += 32) {
+                const int32_t s = out.indices[e];
+                if (esz == 4) reinterpret_cast<uint32_t *>(dst0)[e] = reinterpret_cast<const uint32_t *>(base)[s];
+                else reinterpret_cast<uint16_t *>(dst0)[e] = reinterpret_cast<const uint16_t *>(base)[s];
+            }
+            continue;
+        }
+        const uint64_t cap = dv.cap[cls];
+        const uint8_t *src_lo = base, *src_hi = base + (uint64_t)dv.S * cap * esz;
+        const long long *offt = dv.off[cls];
+        if (out.mode == TD_PACKED) {
+            const int32_t *cu = cls == TD_PROMPT ? out.cu_prompt : out.cu_response;
+            const uint64_t total = (uint64_t)(int64_t)cu[n_s] * esz;
+            const uint64_t b1 = min(b0 + (uint64_t)kGatherChunkBytes, total);
+            for (uint32_t i = row_of(cu, n_s, (int64_t)(b0 / esz)); i < n_s; ++i) {
+                const uint64_t row_lo = (uint64_t)(int64_t)cu[i] * esz;
+                if (row_lo >= b1) break;
+                const uint64_t row_hi = (uint64_t)(int64_t)cu[i + 1] * esz;
+                const uint64_t lo = max(row_lo, b0), hi = min(row_hi, b1);
+                if (hi <= lo) continue;
+                const uint32_t s = (uint32_t)out.indices[i];
+                const uint8_t *src = base + ((uint64_t)shard_of(dv, s) * cap + (uint64_t)offt[s]) * esz + (lo - row_lo);
+                warp_copy(dst0 + lo, src, hi - lo, esz, lane, src_lo, src_hi);
+            }
+        } else {
+            const uint32_t W = cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to;
+            const int32_t *lent = dv.len[cls];
+            const uint64_t row_bytes = (uint64_t)W * esz;
+            const uint64_t total = (uint64_t)n_s * row_bytes;
+            const uint64_t b1 = min(b0 + (uint64_t)kGatherChunkBytes, total);
+            for (uint64_t i = b0 / row_bytes; i < n_s; ++i) {
+                const uint64_t row_lo = i * row_bytes;
+                if (row_lo >= b1) break;
+                const uint32_t s = (uint32_t)out.indices[i];
+                const int32_t l = lent[s];
+                const uint64_t valid_hi = row_lo + (uint64_t)(l > 0 ? l : 0) * esz;
+                const uint64_t lo = max(row_lo, b0), hi = min(row_lo + row_bytes, b1);
+                // payload part
+                const uint64_t phi = min(hi, valid_hi);
+                if (phi > lo) {
+                    const uint8_t *src = base + ((uint64_t)shard_of(dv, s) * cap + (uint64_t)offt[s]) * esz + (lo - row_lo);
+                    warp_copy(dst0 + lo, src, phi - lo, esz, lane, src_lo, src_hi);
+                }
+                // padding part
+                const uint64_t plo = max(lo, valid_hi);
+                if (hi > plo) warp_fill(dst0 + plo, hi - plo, dv.col_pad[k], esz, lane);
+            }
+        }
+    }
+}
+
+// Reset: every table, bitmap and counter back to the empty state; payload untouched.
+__global__ void __launch_bounds__(256)
+reset_kernel(const DockView dv) {
+    const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t stride = gridDim.x * blockDim.x;
+    for (uint32_t s = t; s < dv.n; s += stride) {
+        dv.status[s] = 0;
+        dv.len[1][s] = -1; dv.len[2][s] = -1;
+        dv.off[1][s] = -1; dv.off[2][s] = -1;
+    }
+    for (uint32_t i = t; i < dv.S; i += stride) { dv.cursor[1][i] = 0; dv.cursor[2][i] = 0; }
+    for (uint32_t i = t; i < dv.ncons * dv.claim_words; i += stride) dv.claim[i] = 0;
+    for (uint32_t i = t; i < dv.ncons * dv.consumed_words; i += stride) dv.consumed[i] = 0;
+    for (uint32_t i = t; i < CNT_TOTAL; i += stride) dv.counters[i] = 0;
+    if (t == 0) *dv.errword = 0;
+}
+
+}  // namespace td

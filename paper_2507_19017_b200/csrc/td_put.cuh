@@ -1,0 +1,266 @@
+// td_put: reserve rows (alloc), scatter payload into the arenas, publish readiness bits.
+// Workflow steps 2 and 3 of "Distributed Transfer Dock Strategy": a worker sends real data to
+// the warehouses, then the warehouse state becomes visible to every controller.
+#pragma once
+
+#include "td_device.cuh"
+
+namespace td {
+
+constexpr int kAllocThreads = 1024;
+constexpr int kAllocWarps = kAllocThreads / 32;
+constexpr int kCopyThreads = 256;
+constexpr int kCopyWarps = kCopyThreads / 32;
+constexpr uint32_t kWarpChunkBytes = 4096;     // packed-side bytes one warp copies per step
+constexpr uint32_t kNotAllocating = 0xffffffffu;
+constexpr unsigned long long kNoStart = ~0ull;
+
+struct PutArgs {
+    uint32_t column, k;
+    const int32_t *idx;
+    const int32_t *cu;
+    const uint8_t *data;
+    uint64_t data_elems;
+};
+
+// Is entry i of this call a row that the alloc kernel accepted?  Recomputed from the tables by
+// the scatter and publish kernels, so that a put needs no scratch memory of its own.
+__device__ __forceinline__ bool put_entry_live(const DockView &dv, const PutArgs &a, uint32_t i,
+                                               uint32_t L, uint32_t bit, int32_t &s_out,
+                                               int64_t &c0_out, int64_t &len_out, long long &off_out) {
+    const int32_t s = a.idx[i];
+    if (s < 0 || (uint32_t)s >= dv.n) return false;
+    if (dv.status[s] & bit) return false;
+    const int64_t c0 = a.cu[i], c1 = a.cu[i + 1];
+    const int64_t l = c1 - c0;
+    if (l < 0 || c0 < 0 || (uint64_t)c1 > a.data_elems) return false;
+    if ((int64_t)dv.len[L][s] != l) return false;
+    const long long off = dv.off[L][s];
+    if (off < 0) return false;
+    s_out = s; c0_out = c0; len_out = l; off_out = off;
+    return true;
+}
+
+static inline size_t put_alloc_smem_bytes(uint32_t S) {
+    return (size_t)(kAllocWarps + 2) * S * sizeof(unsigned long long);
+}
+
+// Alloc.  One CTA walks the call's entries in rounds of kAllocThreads, in call order.  Per
+// round: validate, decide who reserves a row (first arrival of the length class, settled by a
+// CAS on len), then an ordered per-shard exclusive scan of the row sizes gives every new row the
+// offset a sequential walk would have given it.  A round that would overflow a shard is
+// replayed by one thread, entry by entry, so that only the rows without room are refused.
+__global__ void __launch_bounds__(kAllocThreads)
+put_alloc_kernel(const DockView dv, const PutArgs a) {
+    extern __shared__ unsigned long long smem_u64[];
+    const uint32_t S = dv.S;
+    unsigned long long *tot = smem_u64;                       // [kAllocWarps][S]
+    unsigned long long *s_total = tot + (size_t)kAllocWarps * S;   // [S] row space asked per shard
+    unsigned long long *s_start = s_total + S;                // [S] where the round's space begins
+    __shared__ int32_t e_s[kAllocThreads];
+    __shared__ uint32_t e_room[kAllocThreads];
+    __shared__ uint32_t s_overflow;
+
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t L = dv.col_cls[a.column];
+    const uint32_t bit = 1u << a.column;
+    const uint64_t cap = dv.cap[L];
+    uint32_t n_oob = 0, n_dup = 0, n_bad = 0, n_mis = 0, n_full = 0;
+
+    for (uint32_t base = 0; base < a.k; base += kAllocThreads) {
+        for (uint32_t j = tid; j < kAllocWarps * S; j += kAllocThreads) tot[j] = 0;
+        if (tid == 0) s_overflow = 0;
+        const uint32_t i = base + tid;
+        bool alloc = false;
+        int32_t s = -1;
+        uint32_t room = 0, sh = 0;
+        if (i < a.k) {
+            s = a.idx[i];
+            if (s < 0 || (uint32_t)s >= dv.n) { ++n_oob; }
+            else if (dv.status[s] & bit) { ++n_dup; }
+            else {
+                const int64_t c0 = a.cu[i], c1 = a.cu[i + 1];
+                const int64_t l = c1 - c0;
+                if (l < 0 || c0 < 0 || (uint64_t)c1 > a.data_elems) { ++n_bad; }
+                else {
+                    const int32_t old = atomicCAS(&dv.len[L][s], -1, (int32_t)l);
+                    if (old == -1) {
+                        alloc = true;
+                        room = (uint32_t)align_row((uint64_t)l);
+                        sh = shard_of(dv, (uint32_t)s);
+                    } else if (old != (int32_t)l) { ++n_mis; }
+                }
+            }
+        }
+        e_s[tid] = s;
+        e_room[tid] = alloc ? room : kNotAllocating;
+        // ordered exclusive prefix per shard inside the warp
+        const uint32_t key = alloc ? sh : kNotAllocating;
+        unsigned long long pre = 0, wsum = 0;
+        bool leader = alloc;
+        #pragma unroll 8
+        for (uint32_t j = 0; j < 32; ++j) {
+            const uint32_t kj = __shfl_sync(kFullMask, key, j);
+            const uint32_t rj = __shfl_sync(kFullMask, room, j);
+            if (alloc && kj == key) {
+                wsum += rj;
+                if (j < lane) { pre += rj; leader = false; }
+            }
+        }
+        __syncthreads();                                   // tot zeroed, e_* written
+        if (leader) tot[warp * S + sh] = wsum;
+        __syncthreads();
+        // per shard: exclusive scan of the warps' sums in warp order
+        for (uint32_t key2 = warp; key2 < S; key2 += kAllocWarps) {
+            const unsigned long long v = tot[lane * S + key2];
+            unsigned long long inc = v;
+            #pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const unsigned long long t = __shfl_up_sync(kFullMask, inc, d);
+                if ((int)lane >= d) inc += t;
+            }
+            tot[lane * S + key2] = inc - v;
+            if (lane == 31) {
+                s_total[key2] = inc;
+                unsigned long long start = kNoStart;
+                if (inc) {
+                    start = atomicAdd(&dv.cursor[L][key2], inc);
+                    if (start + inc > cap) s_overflow = 1;
+                }
+                s_start[key2] = start;
+            }
+        }
+        __syncthreads();
+        if (!s_overflow) {
+            if (alloc) dv.off[L][s] = (long long)(s_start[sh] + tot[warp * S + sh] + pre);
+        } else {
+            // hand the round's reservations back, then replay the round in call order
+            for (uint32_t key2 = tid; key2 < S; key2 += kAllocThreads)
+                if (s_start[key2] != kNoStart) atomicAdd(&dv.cursor[L][key2], 0ull - s_total[key2]);
+            __syncthreads();
+            if (tid == 0) {
+                for (uint32_t t = 0; t < kAllocThreads; ++t) {
+                    const uint32_t r = e_room[t];
+                    if (r == kNotAllocating) continue;
+                    const int32_t ss = e_s[t];
+                    const uint32_t key2 = shard_of(dv, (uint32_t)ss);
+                    const unsigned long long start = atomicAdd(&dv.cursor[L][key2], (unsigned long long)r);
+                    if (start + r > cap) {
+                        atomicAdd(&dv.cursor[L][key2], 0ull - (unsigned long long)r);
+                        atomicExch(&dv.len[L][ss], -1);
+                        ++n_full;
+                    } else {
+                        dv.off[L][ss] = (long long)start;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+    }
+    n_oob = __reduce_add_sync(kFullMask, n_oob);
+    n_dup = __reduce_add_sync(kFullMask, n_dup);
+    n_bad = __reduce_add_sync(kFullMask, n_bad);
+    n_mis = __reduce_add_sync(kFullMask, n_mis);
+    n_full = __reduce_add_sync(kFullMask, n_full);
+    if (lane == 0) {
+        if (n_oob) flag_error(dv, TD_ERR_OOB_INDEX, CNT_OOB, n_oob);
+        if (n_dup) flag_error(dv, TD_ERR_DUP_PUT, CNT_DUP, n_dup);
+        if (n_bad) flag_error(dv, TD_ERR_BAD_LENGTH, CNT_BADLEN, n_bad);
+        if (n_mis) flag_error(dv, TD_ERR_LEN_MISMATCH, CNT_MISMATCH, n_mis);
+        if (n_full) flag_error(dv, TD_ERR_ARENA_FULL, CNT_FULL, n_full);
+    }
+}
+
+// Scatter.  The packed source is cut into warp chunks of kWarpChunkBytes, so that work is
+// balanced over tokens rather than samples; a warp finds the row its chunk starts in by
+// bisection of cu and copies piece after piece into the rows' reserved places.
+__global__ void __launch_bounds__(kCopyThreads)
+put_scatter_kernel(const DockView dv, const PutArgs a) {
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t L = dv.col_cls[a.column];
+    const uint32_t esz = dv.col_esz[a.column];
+    const uint32_t bit = 1u << a.column;
+    const uint64_t total_bytes = (uint64_t)(int64_t)a.cu[a.k] * esz;
+    if ((int64_t)a.cu[a.k] <= 0 || (uint64_t)a.cu[a.k] > a.data_elems) return;
+    const uint64_t n_chunks = (total_bytes + kWarpChunkBytes - 1) / kWarpChunkBytes;
+    const uint64_t warp0 = (uint64_t)blockIdx.x * kCopyWarps + (threadIdx.x >> 5);
+    const uint64_t stride = (uint64_t)gridDim.x * kCopyWarps;
+    const uint8_t *src_lo = a.data, *src_hi = a.data + a.data_elems * esz;
+    uint8_t *arena = dv.colbase[a.column];
+    const uint64_t cap = dv.cap[L];
+
+    for (uint64_t c = warp0; c < n_chunks; c += stride) {
+        const uint64_t b0 = c * kWarpChunkBytes;
+        const uint64_t b1 = min(b0 + (uint64_t)kWarpChunkBytes, total_bytes);
+        uint32_t i = row_of(a.cu, a.k, (int64_t)(b0 / esz));
+        for (; i < a.k; ++i) {
+            const uint64_t row_lo = (uint64_t)(int64_t)a.cu[i] * esz;
+            if (row_lo >= b1) break;
+            int32_t s; int64_t c0, l; long long off;
+            if (!put_entry_live(dv, a, i, L, bit, s, c0, l, off)) continue;
+            const uint64_t row_hi = row_lo + (uint64_t)l * esz;
+            const uint64_t lo = max(row_lo, b0), hi = min(row_hi, b1);
+            if (hi <= lo) continue;
+            uint8_t *dst = arena + ((uint64_t)shard_of(dv, (uint32_t)s) * cap + (uint64_t)off) * esz + (lo - row_lo);
+            warp_copy(dst, a.data + lo, hi - lo, esz, lane, src_lo, src_hi);
+        }
+    }
+}
+
+// Publish.  Runs after the scatter kernel has finished, so every payload byte of the call is
+// globally visible before a readiness bit is; the fence orders the bit behind them for readers
+// that acquire it.
+__global__ void __launch_bounds__(256)
+put_publish_kernel(const DockView dv, const PutArgs a) {
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t L = dv.col_cls[a.column];
+    const uint32_t bit = 1u << a.column;
+    uint32_t ok = 0;
+    if (i < a.k) {
+        int32_t s; int64_t c0, l; long long off;
+        if (put_entry_live(dv, a, i, L, bit, s, c0, l, off)) {
+            __threadfence();
+            const uint32_t old = atomicOr(&dv.status[s], bit);
+            ok = (old & bit) ? 0u : 1u;
+        }
+    }
+    ok = __reduce_add_sync(kFullMask, ok);
+    if ((threadIdx.x & 31) == 0 && ok)
+        atomicAdd(&dv.counters[CNT_PUT_ACCEPTED + a.column], (unsigned long long)ok);
+}
+
+// Scalar column: one element per sample; store, fence, publish in one kernel.
+__global__ void __launch_bounds__(256)
+put_scalar_kernel(const DockView dv, const PutArgs a) {
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    const uint32_t esz = dv.col_esz[a.column];
+    const uint32_t bit = 1u << a.column;
+    uint32_t ok = 0, n_oob = 0, n_dup = 0, n_bad = 0;
+    if (i < a.k) {
+        const int32_t s = a.idx[i];
+        if (s < 0 || (uint32_t)s >= dv.n) ++n_oob;
+        else if ((uint64_t)i >= a.data_elems) ++n_bad;
+        else if (dv.status[s] & bit) ++n_dup;
+        else {
+            if (esz == 4)
+                reinterpret_cast<uint32_t *>(dv.colbase[a.column])[s] = reinterpret_cast<const uint32_t *>(a.data)[i];
+            else
+                reinterpret_cast<uint16_t *>(dv.colbase[a.column])[s] = reinterpret_cast<const uint16_t *>(a.data)[i];
+            __threadfence();
+            const uint32_t old = atomicOr(&dv.status[s], bit);
+            if (old & bit) ++n_dup; else ok = 1;
+        }
+    }
+    ok = __reduce_add_sync(kFullMask, ok);
+    n_oob = __reduce_add_sync(kFullMask, n_oob);
+    n_dup = __reduce_add_sync(kFullMask, n_dup);
+    n_bad = __reduce_add_sync(kFullMask, n_bad);
+    if ((threadIdx.x & 31) == 0) {
+        if (ok) atomicAdd(&dv.counters[CNT_PUT_ACCEPTED + a.column], (unsigned long long)ok);
+        if (n_oob) flag_error(dv, TD_ERR_OOB_INDEX, CNT_OOB, n_oob);
+        if (n_dup) flag_error(dv, TD_ERR_DUP_PUT, CNT_DUP, n_dup);
+        if (n_bad) flag_error(dv, TD_ERR_BAD_LENGTH, CNT_BADLEN, n_bad);
+    }
+}
+
+}  // namespace td

@@ -1,0 +1,263 @@
+"""Parity of the CUDA library with the CPU oracle on the same seeded inputs, through the C ABI.
+Indices, offsets, bitmaps, cu_seqlens and payload are compared bit for bit; the fp32 advantages
+within 1e-6 relative / 1e-7 absolute (both sides accumulate in double)."""
+import numpy as np
+import pytest
+
+torch = pytest.importorskip("torch")
+
+from oracle import td_oracle as ora
+from paper_2507_19017_b200 import binding as td
+from paper_2507_19017_b200 import workloads as wl
+from tests import helpers as H
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def G():
+    if not torch.cuda.is_available():
+        pytest.skip("no CUDA device")
+    from paper_2507_19017_b200 import build
+    build.build()
+    from tests import gpu_helpers
+    return gpu_helpers
+
+
+# ------------------------------------------------------------------ the five shapes
+def test_config1_tiny_random_order(G):
+    w = wl.make_config(1)
+    g, o, batches = G.replay_both(w, check_state_every=5)
+    assert sum(b.n_samples for _, b in batches) == w.n * len(w.consumers)
+
+
+def test_config1_padded(G):
+    w = wl.make_config(1)
+    G.replay_both(w, mode=td.PADDED)
+
+
+@pytest.mark.parametrize("cid", [2, 3])
+def test_bulk_configs_full_size(G, cid):
+    w = wl.make_config(cid)
+    g, o, batches = G.replay_both(w)
+    assert sum(b.n_samples for _, b in batches) == w.n * len(w.consumers)
+
+
+def test_config5_full_size_packed_and_padded(G):
+    w = wl.make_config(5)
+    g, o, batches = G.replay_both(w)
+    assert sum(b.n_samples for _, b in batches) == w.n * len(w.consumers)
+    # right-padded gets of the same dock: reset the claims by re-running puts on fresh docks is
+    # costly at this size, so gather parity is checked on sampled micro-batches instead
+    rng = np.random.default_rng(5)
+    g.dock.reset(); o.reset()
+    for c in range(len(w.columns)):
+        cu, data = w.pack(c, np.arange(w.n, dtype=np.int32))
+        o.put(c, np.arange(w.n), cu, data); g.put(c, np.arange(w.n), cu, data)
+    for _ in range(3):
+        for cons in (0, 3):
+            want = o.get(cons, w.micro_batch, ora.PADDED, w.pad_prompt_to, w.pad_response_to)
+            got = g.get(cons, w.micro_batch, td.PADDED, w.pad_prompt_to, w.pad_response_to)
+            G.assert_batch_equal(got, want, f"padded consumer {cons}")
+    del rng
+
+
+def test_config4_interleaved_serialized(G):
+    """The out-of-order schedule executed in order on one stream is deterministic: bit-exact."""
+    w = wl.make_config(4)
+    g, o, batches = G.replay_both(w, check_state_every=400, arenas=False)
+    per = {c: 0 for c in range(len(w.consumers))}
+    partial = 0
+    for c, b in batches:
+        per[c] += b.n_samples
+        partial += b.n_samples < w.micro_batch
+    assert all(v == w.n for v in per.values())
+    assert partial > 100          # the schedule really met partially ready docks
+
+
+# --------------------------------------------------------------- shapes that stress the kernels
+@pytest.mark.parametrize("N,Gp,S", [(1, 12, 3), (3, 10, 5), (5, 8, 2), (7, 6, 1), (32, 4, 4), (33, 3, 3)])
+def test_group_sizes_that_do_not_divide_a_warp(G, N, Gp, S):
+    w = wl.make_custom("odd", Gp, N, S, prompt_len=(1, 70), response=("uniform", 0, 200), vocab=50000,
+                       micro_batch=2 * N, seed=100 + N, with_entropy=True, schedule="random_order", chunk=(1, 9))
+    G.replay_both(w, check_state_every=7)
+    G.replay_both(w, mode=td.PADDED)
+
+
+def test_all_row_alignments_and_lengths(G):
+    """Row lengths 0..70 in every order: every source/destination misalignment of the 16-byte
+    copy path, for 4-byte and 2-byte elements, heads and tails included."""
+    w = wl.make_custom("align", 64, 2, 4, prompt_len=(0, 37), response=("uniform", 0, 70), vocab=1 << 20,
+                       micro_batch=6, seed=11, with_entropy=True, schedule="random_order", chunk=(1, 7))
+    G.replay_both(w)
+    w2 = wl.make_custom("align2", 64, 2, 4, prompt_len=(0, 37), response=("uniform", 0, 70), vocab=1 << 20,
+                        micro_batch=128, seed=12, with_entropy=True, schedule="bulk")
+    G.replay_both(w2)
+
+
+def test_source_buffer_edges_are_not_overread(G):
+    """Put from, and get into, tensors that sit at odd element offsets inside guard regions:
+    the guards must stay untouched and the payload exact."""
+    w = wl.make_custom("edge", 8, 2, 2, prompt_len=(1, 50), response=("uniform", 1, 300), vocab=1000,
+                       micro_batch=16, seed=5, with_entropy=True, schedule="none")
+    o = H.make_oracle(w)
+    g = G.GpuDock(w)
+    idx = np.arange(w.n, dtype=np.int32)
+    for c, spec in enumerate(w.columns):
+        cu, data = w.pack(c, idx)
+        o.put(c, idx, cu, data)
+        dev = G.to_device(data, g.device)
+        guard = torch.full((dev.numel() + 64,), -1 if dev.dtype != torch.bfloat16 else 1.0, dtype=dev.dtype, device=g.device)
+        shift = 3 if spec.cls != wl.SCALAR else 1
+        guard[shift:shift + dev.numel()] = dev
+        view = guard[shift:shift + dev.numel()]
+        g.dock.put(c, G.to_device(idx, g.device), G.to_device(cu, g.device) if cu is not None else None, view)
+    torch.cuda.synchronize()
+    want = o.get(3, w.n)
+    bufs = g.buffers(3, w.n)
+    # exact-size outputs embedded in guard buffers
+    embedded = {}
+    for c, t in list(bufs.cols.items()):
+        need = want.columns[c].size
+        big = torch.zeros(need + 48, dtype=t.dtype, device=g.device)
+        fill = torch.full_like(big, 7)
+        big.copy_(fill)
+        shift = 5
+        bufs.cols[c] = big[shift:shift + need]
+        bufs.caps[c] = need
+        bufs.struct.col[c] = bufs.cols[c].data_ptr()
+        bufs.struct.col_capacity_elems[c] = need
+        embedded[c] = (big, shift, need)
+    g.dock.get(bufs)
+    got = g.read(bufs)
+    G.assert_batch_equal(got, want, "edge")
+    for c, (big, shift, need) in embedded.items():
+        host = G.to_host(big)
+        ref = G.to_host(torch.full((1,), 7, dtype=big.dtype))[0]
+        assert np.all(host[:shift] == ref) and np.all(host[shift + need:] == ref), f"guard of column {c}"
+
+
+def test_many_tiles_look_back(G):
+    """More groups than one scan tile holds (256), random readiness, several consumers and
+    batch sizes: ranks must come from the look-back chain across tiles."""
+    w = wl.make_custom("tiles", 3000, 1, 8, prompt_len=(0, 4), response=("uniform", 0, 6), vocab=100,
+                       micro_batch=700, seed=21, schedule="interleaved", chunk=(1, 900), poll_every=3)
+    g, o, batches = G.replay_both(w, arenas=False)
+    assert max(b.n_groups for _, b in batches) > 256
+    w2 = wl.make_custom("tiles2", 1100, 2, 4, prompt_len=(0, 4), response=("uniform", 0, 6), vocab=100,
+                        micro_batch=2200, seed=22, schedule="bulk")
+    g, o, batches = G.replay_both(w2)
+    assert batches[0][1].n_samples == 2200
+
+
+# ----------------------------------------------------------------------------- error paths
+def test_put_errors_are_counted_and_skipped(G):
+    w = wl.make_custom("err", 8, 4, 2, prompt_len=(3, 40), response=("uniform", 1, 90), vocab=1000,
+                       micro_batch=8, seed=7, schedule="none")
+    o = H.make_oracle(w)
+    g = G.GpuDock(w)
+    rid, old, rew = w.column_index("response_ids"), w.column_index("old_logprob"), w.column_index("reward")
+
+    def both(col, idx, cu, data):
+        idx = np.asarray(idx, np.int32)
+        o.put(col, idx, cu, data)
+        g.put(col, idx, cu, data)
+
+    both(rid, [0, 1, 2], *w.pack(rid, np.array([0, 1, 2], np.int32)))
+    both(rid, [1, -1, w.n, 3], *w.pack(rid, np.array([1, 0, 0, 3], np.int32)))       # dup, 2 x oob, ok
+    bad_cu = np.array([0, int(w.len_response[0]) + 1], np.int32)
+    both(old, [0], bad_cu, np.zeros(bad_cu[1], np.float32))                           # length mismatch
+    both(rid, [5], np.array([4, 2], np.int32), np.zeros(8, np.int32))                 # decreasing cu
+    both(rew, [0, 0 + w.n, 1], None, np.array([1.0, 2.0, 3.0], np.float32))           # scalar oob
+    both(rew, [1, 2], None, np.array([9.0, 4.0], np.float32))                         # scalar dup
+    G.assert_state_equal(g, o, ctx="errors")
+    G.assert_stats_equal(g, o, "errors")
+    st = g.dock.status()
+    assert st.error_word == td.ERR_OOB_INDEX | td.ERR_DUP_PUT | td.ERR_LEN_MISMATCH | td.ERR_BAD_LENGTH
+
+
+def test_arena_full_refuses_only_rows_without_room(G):
+    w = wl.make_custom("full", 4, 4, 2, prompt_len=(10, 10), response=("uniform", 5, 60), vocab=1000,
+                       micro_batch=16, seed=9, schedule="none")
+    room =(w.len_response.reshape(2, -1).astype(np.int64) + 7) // 8 * 8
+    cap = int(room.sum(axis=1).min() // 2 // 8 * 8)            # about half of what a shard needs
+    o = H.make_oracle(w, response_cap=cap)
+    g = G.GpuDock(w, response_cap=cap)
+    rid = w.column_index("response_ids")
+    order = np.random.default_rng(1).permutation(w.n).astype(np.int32)
+    cu, data = w.pack(rid, order)
+    accepted = o.put(rid, order, cu, data)
+    g.put(rid, order, cu, data)
+    assert 0 < accepted < w.n
+    G.assert_state_equal(g, o, ctx="arena full")
+    G.assert_stats_equal(g, o, "arena full")
+    assert g.dock.status().error_word == td.ERR_ARENA_FULL
+
+
+def test_output_capacity_truncation_matches(G):
+    w = wl.make_custom("trunc", 8, 2, 2, prompt_len=(3, 40), response=("uniform", 1, 90), vocab=1000,
+                       micro_batch=16, seed=7, schedule="none")
+    o = H.make_oracle(w)
+    g = G.GpuDock(w)
+    idx = np.arange(w.n, dtype=np.int32)
+    for c in range(len(w.columns)):
+        cu, data = w.pack(c, idx)
+        o.put(c, idx, cu, data); g.put(c, idx, cu, data)
+    rid = w.column_index("response_ids")
+    room = int(w.len_response[:6].sum()) + 1
+    caps = {rid: room, w.column_index("prompt_ids"): int(w.len_prompt.sum())}
+    want = o.get(0, w.n, capacities=caps)
+    got = g.get(0, w.n, capacities=caps)
+    assert want.status == ora.ERR_OUT_TRUNC and want.n_samples == 6
+    G.assert_batch_equal(got, want, "truncated")
+    G.assert_state_equal(g, o, ctx="after truncation")
+    G.assert_batch_equal(g.get(0, w.n), o.get(0, w.n), "rest")
+    # padded: a row longer than the width ends the batch before its group
+    wide = int(w.len_response.max())
+    want = o.get(1, w.n, ora.PADDED, 40, wide - 1)
+    got = g.get(1, w.n, td.PADDED, 40, wide - 1)
+    G.assert_batch_equal(got, want, "padded truncation")
+    G.assert_stats_equal(g, o, "truncation")
+
+
+def test_host_argument_checks(G):
+    w = wl.make_config(1)
+    g = G.GpuDock(w)
+    bufs = g.buffers(0, 8)
+    with pytest.raises(td.TdError):
+        g.dock.get(bufs, max_samples=3)             # fewer than one group
+    idx = torch.zeros(4, dtype=torch.int32, device=g.device)
+    with pytest.raises(td.TdError):
+        g.dock.put(1, idx, None, idx)               # ragged column without cu
+    with pytest.raises(td.TdError):
+        g.dock.put(99, idx, idx, idx)
+    small = td.GetBuffers(g.dock, 0, 8, prompt_tokens_cap=8, response_tokens_cap=8)
+    small.struct.scratch_bytes = 8
+    with pytest.raises(td.TdError) as e:
+        g.dock.get(small)
+    assert e.value.code == td.EWORKSPACE
+
+
+def test_reset_and_reuse(G):
+    w = wl.make_config(1)
+    g, o, _ = G.replay_both(w)
+    g.dock.reset(); o.reset()
+    G.assert_state_equal(g, o, arenas=False, ctx="after reset")
+    assert g.get(0, 8).n_samples == 0
+    for op in w.ops:
+        if op.kind == "put":
+            cu, data = w.pack(op.column, op.indices)
+            o.put(op.column, op.indices, cu, data); g.put(op.column, op.indices, cu, data)
+    G.assert_batch_equal(g.get(3, w.n), o.get(3, w.n), "after reuse")
+
+
+def test_zero_variance_groups_give_exact_zero(G):
+    w = wl.make_custom("zv", 6, 5, 1, prompt_len=(1, 4), response=("uniform", 1, 4), vocab=10,
+                       micro_batch=30, seed=2, schedule="none")
+    w.data["reward"][:5] = np.float32(0.3)
+    w.data["reward"][5:10] = np.array([0, 1, 1, 0, 1], np.float32)
+    w.data["reward"][10:15] = np.float32(1e4) + np.float32(1e-3) * np.arange(5, dtype=np.float32)
+    w.ops = wl._bulk_ops(w)
+    g, o, batches = G.replay_both(w)
+    adv = [b for c, b in batches if c == 3][0].advantages
+    assert np.all(adv[:5] == 0.0)
