@@ -192,7 +192,7 @@ int td_put(td_dock *d, uint32_t column, const int32_t *d_indices, uint32_t k, co
            const void *d_data, uint64_t data_elems, void *stream) {
     if (!d || column >= d->dv.ncol) return TD_EINVAL;
     if (k == 0) return TD_OK;
-    if (!d_indices || !d_data) return TD_EINVAL;
+    if (!d_indices || (!d_data && data_elems)) return TD_EINVAL;
     const uint32_t cls = d->dv.col_cls[column];
     if (cls != TD_SCALAR && !d_cu) return TD_EINVAL;
     if (data_elems >= (1ull << 31)) return TD_EINVAL;       // cu is int32

@@ -122,11 +122,9 @@ put_alloc_kernel(const DockView dv, const PutArgs a) {
             tot[lane * S + key2] = inc - v;
             if (lane == 31) {
                 s_total[key2] = inc;
-                unsigned long long start = kNoStart;
-                if (inc) {
-                    start = atomicAdd(&dv.cursor[L][key2], inc);
-                    if (start + inc > cap) s_overflow = 1;
-                }
+                // rows of length zero still get a place: the cursor as it stands
+                const unsigned long long start = atomicAdd(&dv.cursor[L][key2], inc);
+                if (start + inc > cap) s_overflow = 1;
                 s_start[key2] = start;
             }
         }

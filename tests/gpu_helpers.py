@@ -131,16 +131,22 @@ def assert_batch_equal(got: ora.Batch, want: ora.Batch, ctx=""):
         assert np.array_equal(got.advantages == 0.0, want.advantages == 0.0), ctx
 
 
+def _same(got: np.ndarray, want: np.ndarray, what: str):
+    if not np.array_equal(got, want):
+        bad = np.where(got != want)[0][:8]
+        raise AssertionError(f"{what}: differs at {bad.tolist()}: got {got[bad].tolist()} want {want[bad].tolist()}")
+
+
 def assert_state_equal(g: GpuDock, o: ora.OracleDock, arenas: bool = True, ctx=""):
     w = g.w
-    assert np.array_equal(g.table(0, 0, np.uint32), o.status()), ctx + " status"
+    _same(g.table(0, 0, np.uint32), o.status(), ctx + " status")
     for cls in (1, 2):
-        assert np.array_equal(g.table(1, cls, np.int32), o.lengths(cls)), ctx + f" len[{cls}]"
-        assert np.array_equal(g.table(2, cls, np.int64), o.offsets(cls)), ctx + f" off[{cls}]"
-        assert np.array_equal(g.table(3, cls, np.uint64), o.cursors(cls)), ctx + f" cursor[{cls}]"
+        _same(g.table(1, cls, np.int32), o.lengths(cls), ctx + f" len[{cls}]")
+        _same(g.table(2, cls, np.int64), o.offsets(cls), ctx + f" off[{cls}]")
+        _same(g.table(3, cls, np.uint64), o.cursors(cls), ctx + f" cursor[{cls}]")
     for c in range(len(w.consumers)):
-        assert np.array_equal(g.table(4, c, np.uint32), o.claim_words(c)), ctx + f" claim[{c}]"
-        assert np.array_equal(g.table(5, c, np.uint32), o.consumed_words(c)), ctx + f" consumed[{c}]"
+        _same(g.table(4, c, np.uint32), o.claim_words(c), ctx + f" claim[{c}]")
+        _same(g.table(5, c, np.uint32), o.consumed_words(c), ctx + f" consumed[{c}]")
     if arenas:
         for c, spec in enumerate(w.columns):
             dt = wl.DTYPE_NUMPY[spec.dtype]
