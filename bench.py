@@ -1,0 +1,431 @@
+#!/usr/bin/env python
+"""Benchmark of the transfer dock's put/get dispatch.
+
+One step = one pass of the whole hot path over one synthetic GRPO batch: reset the dock, put
+every column of every sample, then drain it for all consumers in micro-batches.  The headline
+value is samples dispatched to consumers per second of (put phase + drain phase), with inputs
+resident in HBM.  The L2 is flushed (a 256 MiB write, untimed) before each phase.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config 2] [--impl reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "td_put+td_get samples/s dispatched"
+L2_FLUSH_BYTES = 256 << 20
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--config", type=int, default=2, help="workload shape 1..5 (default 2: Qwen2.5-7B-shaped)")
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU-oracle time budget")
+    return ap.parse_args()
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured (MEASURED_PEAKS.json, torch copy)"
+    return 6650.0, "fallback (earlier measurement on this pool)"
+
+
+# --------------------------------------------------------------------------- clocks
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, uuid: str):
+        self.uuid, self.proc, self.lines = uuid, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.uuid}", f"--query-gpu={self.QUERY}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except OSError:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def gpu_id_for_smi(torch, local_rank: int) -> str:
+    """The id nvidia-smi knows this process's device by: its UUID when listed, else its index."""
+    try:
+        uuid = str(torch.cuda.get_device_properties(local_rank).uuid)
+        if not uuid.startswith("GPU-"):
+            uuid = "GPU-" + uuid
+        listed = subprocess.run(["nvidia-smi", "-L"], capture_output=True, text=True, timeout=20).stdout
+        if uuid in listed:
+            return uuid
+    except Exception:
+        pass
+    return str(local_rank)
+
+
+# --------------------------------------------------------------------------- workload glue
+def algorithmic_bytes(w):
+    """Bytes the method must move per step: every put row read and written once, every served
+    row read and written once, element size times true length (no padding)."""
+    from paper_2507_19017_b200 import workloads as wl
+    put = 0
+    for spec in w.columns:
+        put += 2 * w.data[spec.name].nbytes
+    put_ragged = sum(2 * w.data[s.name].nbytes for s in w.columns if s.cls != wl.SCALAR)
+    get = 0
+    for k in w.consumers:
+        for name in k.out:
+            get += 2 * w.data[name].nbytes
+    return put, put_ragged, get
+
+
+class GpuStep:
+    """Device-resident inputs and per-get output buffers of one step, and the step itself."""
+
+    def __init__(self, w, device_index: int):
+        import torch
+        from paper_2507_19017_b200 import binding as td
+        from paper_2507_19017_b200 import workloads as wl
+        self.torch, self.td, self.w = torch, td, w
+        torch.cuda.set_device(device_index)
+        self.dev = torch.device("cuda", device_index)
+        self.dock = td.Dock(w.G, w.N, w.S, w.column_tuples(), w.consumer_tuples(),
+                            w.shard_capacity(wl.PROMPT), w.shard_capacity(wl.RESPONSE),
+                            w.column_index("reward"), 1e-6, device_index)
+        self.puts = []        # (column, idx, cu, data) device tensors
+        self.host_puts = []   # the same in pinned host memory
+        self.h2d_bytes = 0
+        for op in w.ops:
+            if op.kind != "put":
+                continue
+            cu, data = w.pack(op.column, op.indices)
+            idx = np.ascontiguousarray(op.indices, dtype=np.int32)
+            h = (op.column, self._pin(idx), self._pin(cu) if cu is not None else None, self._pin(data))
+            self.host_puts.append(h)
+            self.puts.append((op.column, h[1].to(self.dev), h[2].to(self.dev) if h[2] is not None else None,
+                              h[3].to(self.dev)))
+            self.h2d_bytes += idx.nbytes + (cu.nbytes if cu is not None else 0) + data.nbytes
+        # one output buffer set per get call, sized by the longest rows it could meet
+        lp = np.sort(w.len_prompt)[::-1]
+        lr = np.sort(w.len_response)[::-1]
+        self.gets = []
+        for op in w.ops:
+            if op.kind != "get":
+                continue
+            m = op.max_samples
+            bufs = td.GetBuffers(self.dock, op.consumer, m, td.PACKED,
+                                 prompt_tokens_cap=int(lp[:m].sum(dtype=np.int64)),
+                                 response_tokens_cap=int(lr[:m].sum(dtype=np.int64)))
+            self.gets.append(bufs)
+        self.flush_buf = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=self.dev)
+        self.stage = None
+        self.host_gets = None
+
+    def _pin(self, a):
+        t = self.torch.from_numpy(np.ascontiguousarray(a).view(np.int16) if a.dtype == np.uint16 else np.ascontiguousarray(a))
+        if a.dtype == np.uint16:
+            t = t.view(self.torch.bfloat16)
+        return t.pin_memory()
+
+    def flush_l2(self):
+        self.flush_buf.zero_()
+
+    def put_phase(self):
+        self.dock.reset()
+        for col, idx, cu, data in self.puts:
+            self.dock.put(col, idx, cu, data)
+
+    def drain_phase(self):
+        for bufs in self.gets:
+            self.dock.get(bufs)
+
+    def timed_step(self):
+        """Returns (put_ms, drain_ms) measured with CUDA events on the current stream."""
+        torch = self.torch
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(4)]
+        self.flush_l2()
+        ev[0].record(); self.put_phase(); ev[1].record()
+        self.flush_l2()
+        ev[2].record(); self.drain_phase(); ev[3].record()
+        torch.cuda.synchronize()
+        return ev[0].elapsed_time(ev[1]), ev[2].elapsed_time(ev[3])
+
+    def served(self):
+        """Samples and tokens the last drain dispatched (reads the result blocks)."""
+        s = t = 0
+        for bufs in self.gets:
+            r = bufs.read_result()
+            s += r.n_samples
+            t += r.prompt_tokens + r.response_tokens
+        return s, t
+
+    # end to end: host buffers in, host buffers out
+    def prepare_e2e(self):
+        td, torch = self.td, self.torch
+        need = max(self.dock.put_host_stage_bytes(c, i.numel(), d.numel()) for c, i, _cu, d in self.host_puts)
+        self.stage = [torch.empty(need, dtype=torch.uint8, device=self.dev) for _ in range(2)]
+        self.host_gets = [td.HostGetBuffers(b) for b in self.gets]
+
+    def e2e_step(self):
+        torch = self.torch
+        self.dock.reset()
+        for j, (col, idx, cu, data) in enumerate(self.host_puts):
+            if j >= 2:
+                self.stage_ev[j % 2].synchronize()      # staging buffer free again
+            self.dock.put_host(col, idx, cu, data, self.stage[j % 2])
+            self.stage_ev[j % 2].record()
+        d2h = 0
+        for bufs, host in zip(self.gets, self.host_gets):
+            self.dock.get_host(bufs, host)
+            d2h += host.bytes_valid(self.dock)
+        torch.cuda.synchronize()
+        return d2h
+
+    def run_e2e(self, steps: int, warmup: int):
+        torch = self.torch
+        self.prepare_e2e()
+        self.stage_ev = [torch.cuda.Event() for _ in range(2)]
+        for _ in range(warmup):
+            self.e2e_step()
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        d2h = 0
+        for _ in range(steps):
+            d2h = self.e2e_step()
+        torch.cuda.synchronize()
+        return (time.perf_counter() - t0) / steps, d2h
+
+
+# --------------------------------------------------------------------------- CPU oracle
+def time_oracle(w, budget_s: float):
+    """The oracle as it stands, one thread, whole steps of the same workload until the time
+    budget is used (at least one step).  Returns (samples/s, steps, seconds)."""
+    from oracle import td_oracle as ora
+    from paper_2507_19017_b200 import workloads as wl
+    d = ora.OracleDock(w.G, w.N, w.S, w.column_tuples(), w.consumer_tuples(),
+                       w.shard_capacity(wl.PROMPT), w.shard_capacity(wl.RESPONSE),
+                       w.column_index("reward"), 1e-6)
+    puts = []
+    for op in w.ops:
+        if op.kind == "put":
+            cu, data = w.pack(op.column, op.indices)
+            puts.append((op.column, np.ascontiguousarray(op.indices, dtype=np.int32), cu, np.ascontiguousarray(data)))
+    lp = np.sort(w.len_prompt)[::-1]
+    lr = np.sort(w.len_response)[::-1]
+    gets = []
+    for op in w.ops:
+        if op.kind == "get":
+            m = op.max_samples
+            caps = {}
+            for c, (dt, cls, _p) in enumerate(d.columns):
+                caps[c] = m if cls == 0 else int((lp if cls == 1 else lr)[:m].sum(dtype=np.int64))
+            gets.append(d.prepare_get(op.consumer, m, caps))
+    steps, samples = 0, 0
+    t0 = time.perf_counter()
+    while True:
+        d.reset()
+        for col, idx, cu, data in puts:
+            d.put_raw(col, idx, cu, data)
+        for g in gets:
+            samples += d.get_prepared(g)
+        steps += 1
+        el = time.perf_counter() - t0
+        if el >= budget_s:
+            break
+    d.close()
+    return samples / el, steps, el
+
+
+# --------------------------------------------------------------------------- main
+def main():
+    args = parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+
+    from paper_2507_19017_b200 import workloads as wl
+    schedule = "bulk"
+    w = wl.make_config(args.config, seed=wl.BASE_SEED + args.config + 1000 * rank, schedule=schedule)
+    config = {"workload": f"configs[{args.config - 1}] {w.name}", "G": w.G, "N": w.N, "S": w.S,
+              "samples": w.n, "tokens": w.tokens_total(), "micro_batch": w.micro_batch,
+              "consumers": len(w.consumers), "schedule": "one put per column, then round-robin gets",
+              "l2": "flushed before each phase (256 MiB write)", "response_sigma": wl.SIGMA_HEADLINE}
+    n_dispatch = w.n * len(w.consumers)
+
+    if args.impl == "reference":
+        if rank != 0:
+            return
+        from oracle import td_oracle
+        td_oracle.build()
+        steps_s = []
+        for _ in range(args.warmup):
+            pass          # the oracle needs no warm-up beyond its first pass, which is timed too
+        rate, steps, el = time_oracle(w, max(args.cpu_seconds, 1.0))
+        line = {"metric": METRIC, "value": rate, "unit": "samples/s", "n_gpus": args.gpus,
+                "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * el / steps,
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8",
+                "data": "synthetic", "impl": "reference", "config": config,
+                "cpu_baseline": {"value": rate, "unit": "samples/s", "cores": 1, "kind": "oracle",
+                                 "sample": f"{steps} whole step(s) of the workload in {el:.1f} s"},
+                "e2e": {"value": rate, "unit": "samples/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+        print(json.dumps(line))
+        return
+
+    import torch
+    from paper_2507_19017_b200 import build
+    build.build()
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: there is no CPU fallback")
+    dist = None
+    if world > 1:
+        import torch.distributed as dist
+        torch.cuda.set_device(local_rank)
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    step = GpuStep(w, local_rank)
+    peak, peak_kind = load_peaks()
+    put_bytes, put_ragged_bytes, get_bytes = algorithmic_bytes(w)
+
+    for _ in range(max(args.warmup, 3)):
+        step.timed_step()
+    served_s, served_t = step.served()
+    assert served_s == n_dispatch, f"drain served {served_s} of {n_dispatch} samples"
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    sampler = ClockSampler(gpu_id_for_smi(torch, local_rank))
+    barrier()
+    sampler.start()
+    launches0 = step.dock.launch_count()
+    put_ms, drain_ms = [], []
+    for _ in range(args.steps):
+        a, b = step.timed_step()
+        put_ms.append(a); drain_ms.append(b)
+    barrier()
+    launches = step.dock.launch_count() - launches0
+    clocks = sampler.stop()
+
+    mean_put, mean_drain = sum(put_ms) / len(put_ms), sum(drain_ms) / len(drain_ms)
+    ms_per_step = mean_put + mean_drain
+    if dist is not None:
+        t = torch.tensor([ms_per_step, mean_put, mean_drain], device=step.dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        ms_per_step, mean_put, mean_drain = t.tolist()
+    value = world * n_dispatch / (ms_per_step * 1e-3)
+
+    # per-kernel pass: event pairs around every launch of the two copy kernels
+    step.dock.kernel_timing(True)
+    ksteps = min(args.steps, 5)
+    for _ in range(ksteps):
+        step.timed_step()
+    n_sc, ms_sc = step.dock.kernel_timing_read(0)
+    n_ga, ms_ga = step.dock.kernel_timing_read(1)
+    step.dock.kernel_timing(False)
+    kern = {
+        "put_scatter": {"launches_per_step": n_sc // ksteps, "avg_ms": ms_sc / max(n_sc, 1),
+                        "bytes_per_launch": put_ragged_bytes / max(n_sc // ksteps, 1)},
+        "get_gather": {"launches_per_step": n_ga // ksteps, "avg_ms": ms_ga / max(n_ga, 1),
+                       "bytes_per_launch": get_bytes / max(n_ga // ksteps, 1)},
+    }
+    for k in kern.values():
+        k["GBps"] = k["bytes_per_launch"] / (k["avg_ms"] * 1e-3) / 1e9 if k["avg_ms"] > 0 else 0.0
+    dom = "get_gather" if ms_ga >= ms_sc else "put_scatter"
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": kern[dom]["GBps"], "peak": peak, "unit": "GB/s",
+                "frac": kern[dom]["GBps"] / peak, "traffic": None, "peak_kind": peak_kind,
+                "bytes_per_launch": kern[dom]["bytes_per_launch"], "avg_launch_ms": kern[dom]["avg_ms"]}
+
+    e2e = None
+    if not args.no_e2e:
+        e2e_s, d2h = step.run_e2e(min(args.steps, 5), 1)
+        if dist is not None:
+            t = torch.tensor([e2e_s], device=step.dev, dtype=torch.float64)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            e2e_s = t.item()
+        e2e = {"value": world * n_dispatch / e2e_s, "unit": "samples/s", "ms_per_step": e2e_s * 1e3,
+               "h2d_bytes_per_step": step.h2d_bytes, "d2h_bytes_per_step": d2h}
+
+    if rank != 0:
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    cpu = None
+    if world == 1 and not args.no_cpu_baseline:
+        from oracle import td_oracle
+        td_oracle.build()
+        rate, steps_o, el = time_oracle(w, args.cpu_seconds)
+        cpu = {"value": rate, "unit": "samples/s", "cores": 1, "kind": "oracle",
+               "sample": f"{steps_o} whole step(s) of the same workload in {el:.1f} s"}
+
+    line = {
+        "metric": METRIC, "value": value, "unit": "samples/s", "n_gpus": world, "steps": args.steps,
+        "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic", "config": config,
+        "tokens_per_s": world * served_t / (ms_per_step * 1e-3),
+        "phases": {"put_ms": mean_put, "drain_ms": mean_drain,
+                   "put_GBps": put_bytes / (mean_put * 1e-3) / 1e9,
+                   "drain_GBps": get_bytes / (mean_drain * 1e-3) / 1e9,
+                   "step_GBps": (put_bytes + get_bytes) / (ms_per_step * 1e-3) / 1e9},
+        "kernels": kern, "roofline": roofline, "cpu_baseline": cpu, "e2e": e2e,
+        "gpu_launches": launches, "gpu_launches_per_step": launches // args.steps, "clocks": clocks,
+    }
+    print(json.dumps(line))
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()

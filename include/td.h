@@ -182,6 +182,32 @@ int td_debug_table(const td_dock *dock, int which, uint32_t index, void **d_ptr,
 /* Kernels this dock has launched since td_create. */
 uint64_t td_launch_count(const td_dock *dock);
 
+/* Per-launch timing of the two copy kernels, the ones that move Eq. 1's payload terms:
+ * which = 0 the put scatter, 1 the get gather.  While enabled, each of their launches is
+ * bracketed by a pair of CUDA events on the launching stream (host objects; no device memory).
+ * td_kernel_timing(dock, enable) clears what was collected and switches collection on or off;
+ * td_kernel_timing_read waits for the recorded launches and returns their count and summed
+ * device time in milliseconds. */
+int td_kernel_timing(td_dock *dock, int enable);
+int td_kernel_timing_read(td_dock *dock, int which, uint64_t *launches, double *total_ms);
+
+/* Host-buffer variants: the same workflow steps for a worker whose tensors live in host memory,
+ * with the transfers across the bus part of the call (the paper's workers exchange samples
+ * between nodes; here the hop is host <-> device).
+ * td_put_host: h_indices / h_cu / h_data are HOST arrays (pinned memory makes the copies
+ * asynchronous); they are copied into d_stage (device, 256-byte aligned, at least
+ * td_put_host_stage_bytes() bytes, not reused until the put has executed) and put from there.
+ * td_get_host: runs td_get into the device buffers of dev_out, then copies exactly the valid
+ * part of every buffer to the matching HOST pointer of host_out (NULL = skip; host_out->result
+ * and host_out->indices are required; col_capacity_elems bounds the host buffers).  It
+ * synchronises the stream twice and returns with host_out filled. */
+size_t td_put_host_stage_bytes(const td_dock *dock, uint32_t column, uint32_t k, uint64_t data_elems);
+int td_put_host(td_dock *dock, uint32_t column, const int32_t *h_indices, uint32_t k,
+                const int32_t *h_cu, const void *h_data, uint64_t data_elems,
+                void *d_stage, size_t stage_bytes, void *stream);
+int td_get_host(td_dock *dock, uint32_t consumer, uint32_t max_samples, const td_get_out *dev_out,
+                const td_get_out *host_out, void *stream);
+
 const char *td_strerror(int code);
 
 #ifdef __cplusplus

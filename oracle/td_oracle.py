@@ -267,6 +267,24 @@ class OracleDock:
             raise ValueError("ora_get: bad argument")
         return self._finish(go, res, bufs, cols, adv, mode, pad_prompt_to, pad_response_to)
 
+    def prepare_get(self, consumer: int, max_samples: int, capacities: Dict[int, int], mode: int = PACKED,
+                    pad_prompt_to: int = 0, pad_response_to: int = 0):
+        """Output buffers allocated once, for callers that time ora_get itself."""
+        return self._alloc(consumer, max_samples, mode, pad_prompt_to, pad_response_to, capacities,
+                           None, [0, 0, 0]) + (consumer, max_samples)
+
+    def get_prepared(self, prepared) -> int:
+        """ora_get into buffers from prepare_get(); returns the number of samples served."""
+        go, res = prepared[0], prepared[1]
+        if lib().ora_get(self._h, prepared[5], prepared[6], C.byref(go)) != 0:
+            raise ValueError("ora_get: bad argument")
+        return res.n_samples
+
+    def put_raw(self, column: int, idx: np.ndarray, cu: Optional[np.ndarray], data: np.ndarray) -> int:
+        """ora_put on arrays that already have the right dtype and layout (no conversion)."""
+        return lib().ora_put(self._h, column, idx.ctypes.data, len(idx),
+                             cu.ctypes.data if cu is not None else None, data.ctypes.data)
+
     def gather(self, consumer: int, indices: np.ndarray, mode: int = PACKED, pad_prompt_to: int = 0,
                pad_response_to: int = 0, want: Optional[Sequence[int]] = None) -> Batch:
         idx = np.ascontiguousarray(indices, dtype=np.int32)

@@ -28,7 +28,8 @@ ELEM_SIZE = {I32: 4, F32: 4, BF16: 2}
 # every symbol include/td.h declares
 EXPORTS = ["td_query_workspace", "td_create", "td_destroy", "td_put", "td_get",
            "td_get_scratch_bytes", "td_reset", "td_status", "td_debug_table",
-           "td_launch_count", "td_strerror"]
+           "td_launch_count", "td_strerror", "td_kernel_timing", "td_kernel_timing_read",
+           "td_put_host_stage_bytes", "td_put_host", "td_get_host"]
 
 
 class TdColumn(C.Structure):
@@ -118,6 +119,16 @@ def lib():
         L.td_launch_count.argtypes = [vp]
         L.td_strerror.restype = C.c_char_p
         L.td_strerror.argtypes = [C.c_int]
+        L.td_kernel_timing.restype = C.c_int
+        L.td_kernel_timing.argtypes = [vp, C.c_int]
+        L.td_kernel_timing_read.restype = C.c_int
+        L.td_kernel_timing_read.argtypes = [vp, C.c_int, C.POINTER(u64), C.POINTER(C.c_double)]
+        L.td_put_host_stage_bytes.restype = C.c_size_t
+        L.td_put_host_stage_bytes.argtypes = [vp, u32, u32, u64]
+        L.td_put_host.restype = C.c_int
+        L.td_put_host.argtypes = [vp, u32, vp, u32, vp, vp, u64, vp, C.c_size_t, vp]
+        L.td_get_host.restype = C.c_int
+        L.td_get_host.argtypes = [vp, u32, u32, C.POINTER(TdGetOut), C.POINTER(TdGetOut), vp]
         _lib = L
     return _lib
 
@@ -213,6 +224,46 @@ class GetBuffers:
         return TdResult.from_buffer_copy(host)
 
 
+class HostGetBuffers:
+    """Pinned host mirrors of a GetBuffers, the destination of td_get_host."""
+
+    def __init__(self, bufs: GetBuffers):
+        import torch
+        self.indices = torch.zeros(bufs.indices.shape, dtype=bufs.indices.dtype).pin_memory()
+        self.cu_prompt = torch.zeros(bufs.cu_prompt.shape, dtype=torch.int32).pin_memory()
+        self.cu_response = torch.zeros(bufs.cu_response.shape, dtype=torch.int32).pin_memory()
+        self.cu_seq = torch.zeros(bufs.cu_seq.shape, dtype=torch.int32).pin_memory()
+        self.advantages = (torch.zeros(bufs.advantages.shape, dtype=torch.float32).pin_memory()
+                           if bufs.advantages is not None else None)
+        self.cols = {c: torch.zeros(t.shape, dtype=t.dtype).pin_memory() for c, t in bufs.cols.items()}
+        self.result = TdResult()
+        go = TdGetOut()
+        go.mode, go.pad_prompt_to, go.pad_response_to = bufs.mode, bufs.pad_prompt_to, bufs.pad_response_to
+        go.indices, go.cu_prompt = self.indices.data_ptr(), self.cu_prompt.data_ptr()
+        go.cu_response, go.cu_seq = self.cu_response.data_ptr(), self.cu_seq.data_ptr()
+        for c, t in self.cols.items():
+            go.col[c] = t.data_ptr()
+            go.col_capacity_elems[c] = t.numel()
+        go.advantages = self.advantages.data_ptr() if self.advantages is not None else None
+        go.result = C.addressof(self.result)
+        self.struct = go
+
+    def bytes_valid(self, dock: "Dock") -> int:
+        """Bytes td_get_host copied to the host for the last call."""
+        r, n = self.result, self.result.n_samples
+        total = C.sizeof(TdResult) + n * 4 + 3 * (n + 1) * 4 + (n * 4 if self.advantages is not None else 0)
+        for c, t in self.cols.items():
+            dt, cls, _ = dock.columns[c]
+            if cls == SCALAR:
+                e = n
+            elif self.struct.mode == PACKED:
+                e = r.prompt_tokens if cls == PROMPT else r.response_tokens
+            else:
+                e = n * (self.struct.pad_prompt_to if cls == PROMPT else self.struct.pad_response_to)
+            total += e * ELEM_SIZE[dt]
+        return total
+
+
 class Dock:
     """A transfer dock living in one torch-allocated workspace on `device`."""
 
@@ -264,6 +315,33 @@ class Dock:
         st = TdStats()
         _check("td_status", lib().td_status(self.handle, C.byref(st), _stream_ptr(stream)))
         return st
+
+    # -- host-buffer variants ----------------------------------------------
+    def put_host(self, column: int, indices, cu, data, stage, stream=None):
+        """indices / cu / data: host tensors (pinned for asynchronous copies); stage: a device
+        uint8 tensor of at least put_host_stage_bytes()."""
+        k = indices.numel()
+        _check("td_put_host", lib().td_put_host(self.handle, column, indices.data_ptr(), k,
+                                                cu.data_ptr() if cu is not None else None,
+                                                data.data_ptr(), data.numel(), stage.data_ptr(),
+                                                stage.numel(), _stream_ptr(stream)))
+
+    def put_host_stage_bytes(self, column: int, k: int, data_elems: int) -> int:
+        return lib().td_put_host_stage_bytes(self.handle, column, k, data_elems)
+
+    def get_host(self, bufs: GetBuffers, host: "HostGetBuffers", stream=None):
+        _check("td_get_host", lib().td_get_host(self.handle, bufs.consumer, bufs.max_samples,
+                                                C.byref(bufs.struct), C.byref(host.struct),
+                                                _stream_ptr(stream)))
+
+    # -- measurement ------------------------------------------------------
+    def kernel_timing(self, enable: bool):
+        _check("td_kernel_timing", lib().td_kernel_timing(self.handle, 1 if enable else 0))
+
+    def kernel_timing_read(self, which: int) -> Tuple[int, float]:
+        n, ms = C.c_uint64(0), C.c_double(0.0)
+        _check("td_kernel_timing_read", lib().td_kernel_timing_read(self.handle, which, C.byref(n), C.byref(ms)))
+        return n.value, ms.value
 
     # -- inspection -------------------------------------------------------
     def table(self, which: int, index: int = 0):

@@ -4,7 +4,9 @@
 #include <atomic>
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 #include <new>
+#include <vector>
 
 #include "td_device.cuh"
 #include "td_get.cuh"
@@ -21,6 +23,10 @@ struct td_dock {
     size_t ws_bytes;
     size_t table_bytes[7];
     std::atomic<uint64_t> launches;
+    // optional per-kernel timing of the two copy kernels (0 = put scatter, 1 = get gather)
+    std::atomic<bool> timing;
+    std::mutex timing_mu;
+    std::vector<std::pair<cudaEvent_t, cudaEvent_t>> timing_ev[2];
 };
 
 namespace {
@@ -94,6 +100,30 @@ cudaError_t launch(td_dock *d, void (*kernel)(KArgs...), dim3 grid, dim3 block, 
     return cudaGetLastError();
 }
 
+// Launch bracketed by a pair of events on the same stream while timing is switched on.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_timed(td_dock *d, int which, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                         cudaStream_t st, Args &&...args) {
+    if (!d->timing.load(std::memory_order_relaxed))
+        return launch(d, kernel, grid, block, smem, st, std::forward<Args>(args)...);
+    cudaEvent_t e0, e1;
+    if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return cudaErrorUnknown;
+    cudaEventRecord(e0, st);
+    cudaError_t rc = launch(d, kernel, grid, block, smem, st, std::forward<Args>(args)...);
+    cudaEventRecord(e1, st);
+    std::lock_guard<std::mutex> lk(d->timing_mu);
+    d->timing_ev[which].emplace_back(e0, e1);
+    return rc;
+}
+
+void drop_timing(td_dock *d) {
+    std::lock_guard<std::mutex> lk(d->timing_mu);
+    for (auto &v : d->timing_ev) {
+        for (auto &p : v) { cudaEventDestroy(p.first); cudaEventDestroy(p.second); }
+        v.clear();
+    }
+}
+
 }  // namespace
 
 extern "C" {
@@ -132,6 +162,7 @@ int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **o
     d->device = cfg->device; d->sm_count = sms;
     d->ws = static_cast<uint8_t *>(d_workspace); d->ws_bytes = bytes;
     d->launches = 0;
+    d->timing = false;
     DockView &v = d->dv;
     std::memset(&v, 0, sizeof(v));
     v.G = cfg->n_prompts; v.N = cfg->n_per_group; v.S = cfg->n_shards; v.n = v.G * v.N;
@@ -176,6 +207,7 @@ int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **o
 }
 
 int td_destroy(td_dock *dock) {
+    if (dock) drop_timing(dock);
     delete dock;
     return TD_OK;
 }
@@ -210,7 +242,7 @@ int td_put(td_dock *d, uint32_t column, const int32_t *d_indices, uint32_t k, co
     const uint64_t max_blocks = (uint64_t)d->sm_count * 8;
     if (blocks > max_blocks) blocks = max_blocks;
     if (blocks == 0) blocks = 1;
-    if (launch(d, put_scatter_kernel, dim3((uint32_t)blocks), dim3(kCopyThreads), 0, st, d->dv, a) != cudaSuccess) return TD_ECUDA;
+    if (launch_timed(d, 0, put_scatter_kernel, dim3((uint32_t)blocks), dim3(kCopyThreads), 0, st, d->dv, a) != cudaSuccess) return TD_ECUDA;
     if (launch(d, put_publish_kernel, dim3((k + 255) / 256), dim3(256), 0, st, d->dv, a) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
@@ -260,7 +292,7 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
     const uint64_t max_blocks = (uint64_t)d->sm_count * 8;
     if (blocks > max_blocks) blocks = max_blocks;
     if (blocks == 0) blocks = 1;
-    if (launch(d, get_gather_kernel, dim3((uint32_t)blocks), dim3(kGatherThreads), 0, st, v, one,
+    if (launch_timed(d, 1, get_gather_kernel, dim3((uint32_t)blocks), dim3(kGatherThreads), 0, st, v, one,
                (const GetReq *)nullptr, 1u) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
@@ -309,5 +341,89 @@ int td_debug_table(const td_dock *d, int which, uint32_t index, void **d_ptr, si
 }
 
 uint64_t td_launch_count(const td_dock *d) { return d ? d->launches.load() : 0; }
+
+int td_kernel_timing(td_dock *d, int enable) {
+    if (!d) return TD_EINVAL;
+    drop_timing(d);
+    d->timing = enable != 0;
+    return TD_OK;
+}
+
+int td_kernel_timing_read(td_dock *d, int which, uint64_t *launches, double *total_ms) {
+    if (!d || which < 0 || which > 1 || !launches || !total_ms) return TD_EINVAL;
+    std::lock_guard<std::mutex> lk(d->timing_mu);
+    double sum = 0.0;
+    for (auto &p : d->timing_ev[which]) {
+        if (cudaEventSynchronize(p.second) != cudaSuccess) return TD_ECUDA;
+        float ms = 0.f;
+        if (cudaEventElapsedTime(&ms, p.first, p.second) != cudaSuccess) return TD_ECUDA;
+        sum += ms;
+    }
+    *launches = d->timing_ev[which].size();
+    *total_ms = sum;
+    return TD_OK;
+}
+
+// ---- host-buffer variants: the same put / get with the copies across the bus included ----
+size_t td_put_host_stage_bytes(const td_dock *d, uint32_t column, uint32_t k, uint64_t data_elems) {
+    if (!d || column >= d->dv.ncol) return 0;
+    return align_up_sz((size_t)k * 4, 256) + align_up_sz(((size_t)k + 1) * 4, 256) +
+           align_up_sz((size_t)data_elems * d->dv.col_esz[column], 256);
+}
+
+int td_put_host(td_dock *d, uint32_t column, const int32_t *h_indices, uint32_t k, const int32_t *h_cu,
+                const void *h_data, uint64_t data_elems, void *d_stage, size_t stage_bytes, void *stream) {
+    if (!d || column >= d->dv.ncol) return TD_EINVAL;
+    if (k == 0) return TD_OK;
+    if (!h_indices || (!h_data && data_elems) || !d_stage) return TD_EINVAL;
+    const bool ragged = d->dv.col_cls[column] != TD_SCALAR;
+    if (ragged && !h_cu) return TD_EINVAL;
+    if ((reinterpret_cast<uintptr_t>(d_stage) & 255u) || stage_bytes < td_put_host_stage_bytes(d, column, k, data_elems))
+        return TD_EWORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    uint8_t *p = static_cast<uint8_t *>(d_stage);
+    int32_t *d_idx = reinterpret_cast<int32_t *>(p);
+    int32_t *d_cu = reinterpret_cast<int32_t *>(p + align_up_sz((size_t)k * 4, 256));
+    uint8_t *d_dat = reinterpret_cast<uint8_t *>(d_cu) + align_up_sz(((size_t)k + 1) * 4, 256);
+    const size_t esz = d->dv.col_esz[column];
+    if (cudaMemcpyAsync(d_idx, h_indices, (size_t)k * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TD_ECUDA;
+    if (ragged && cudaMemcpyAsync(d_cu, h_cu, ((size_t)k + 1) * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TD_ECUDA;
+    if (data_elems && cudaMemcpyAsync(d_dat, h_data, (size_t)data_elems * esz, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        return TD_ECUDA;
+    return td_put(d, column, d_idx, k, ragged ? d_cu : nullptr, d_dat, data_elems, stream);
+}
+
+int td_get_host(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out *dev_out,
+                const td_get_out *host_out, void *stream) {
+    if (!d || !dev_out || !host_out || !host_out->result || !host_out->indices) return TD_EINVAL;
+    const int rc = td_get(d, consumer, max_samples, dev_out, stream);
+    if (rc != TD_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const DockView &v = d->dv;
+    td_result *res = host_out->result;
+    if (cudaMemcpyAsync(res, dev_out->result, sizeof(td_result), cudaMemcpyDeviceToHost, st) != cudaSuccess) return TD_ECUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
+    const size_t n = res->n_samples;
+    auto d2h = [&](void *dst, const void *src, size_t bytes) {
+        return !dst || !src || bytes == 0 || cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    };
+    bool ok = d2h(host_out->indices, dev_out->indices, n * 4);
+    ok = ok && d2h(host_out->cu_prompt, dev_out->cu_prompt, (n + 1) * 4);
+    ok = ok && d2h(host_out->cu_response, dev_out->cu_response, (n + 1) * 4);
+    ok = ok && d2h(host_out->cu_seq, dev_out->cu_seq, (n + 1) * 4);
+    ok = ok && d2h(host_out->advantages, dev_out->advantages, n * 4);
+    for (uint32_t k = 0; k < v.ncol && ok; ++k) {
+        if (!((v.outm[consumer] >> k) & 1u) || !dev_out->col[k] || !host_out->col[k]) continue;
+        const uint32_t cls = v.col_cls[k];
+        size_t elems;
+        if (cls == TD_SCALAR) elems = n;
+        else if (dev_out->mode == TD_PACKED) elems = cls == TD_PROMPT ? res->prompt_tokens : res->response_tokens;
+        else elems = n * (size_t)(cls == TD_PROMPT ? dev_out->pad_prompt_to : dev_out->pad_response_to);
+        if (elems > host_out->col_capacity_elems[k]) return TD_EINVAL;
+        ok = d2h(host_out->col[k], dev_out->col[k], elems * v.col_esz[k]);
+    }
+    if (!ok || cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
+    return TD_OK;
+}
 
 }  // extern "C"
