@@ -166,6 +166,42 @@ int td_get(td_dock *dock, uint32_t consumer, uint32_t max_samples, const td_get_
            void *stream);
 size_t td_get_scratch_bytes(const td_dock *dock);
 
+/* Several columns in one call, as a worker that sends a whole record does (prompt and response
+ * ids together, say): the items are stored as if td_put had been called on each in array order,
+ * with three kernel launches for up to eight items instead of three per item.  Every field of
+ * an item means what the td_put argument of the same name means. */
+typedef struct {
+    uint32_t column, k;
+    const int32_t *d_indices;
+    const int32_t *d_cu;
+    const void *d_data;
+    uint64_t data_elems;
+} td_put_item;
+int td_put_many(td_dock *dock, const td_put_item *items, uint32_t n_items, void *stream);
+
+/* Many gets served by one call.  Each worker state has its own controller and a step serves
+ * several of them, each in several micro-batches; a plan fixes the list of requests (consumer,
+ * max_samples, output buffers) once and td_get_many then serves all of them with three kernel
+ * launches.  Requests that name the same consumer are served in array order: the result is the
+ * one td_get would give when called on each request in turn, except that a group cut off by
+ * TD_ERR_OUT_TRUNCATED is not offered to the later requests of the same call.
+ *   td_plan_bytes   device bytes a plan of n_req requests needs (request table + scan scratch).
+ *   td_plan_create  checks the requests (host array; out.scratch is not used), uploads them into
+ *                   d_plan (device, 256-byte aligned, caller-owned, must outlive the plan) on
+ *                   `stream`.  n_req * n_columns must not exceed 4096.
+ *   td_get_many     enqueues the gets.  A plan must not be in flight twice at the same time;
+ *                   reusing it on one stream, call after call, is the intended use. */
+typedef struct {
+    uint32_t consumer, max_samples;
+    td_get_out out;
+} td_get_req;
+typedef struct td_plan td_plan;
+size_t td_plan_bytes(const td_dock *dock, uint32_t n_req);
+int td_plan_create(td_dock *dock, const td_get_req *reqs, uint32_t n_req, void *d_plan,
+                   size_t plan_bytes, void *stream, td_plan **out);
+int td_plan_destroy(td_plan *plan);
+int td_get_many(td_dock *dock, td_plan *plan, void *stream);
+
 /* One buffer serves one RL iteration: forget every table, bitmap and counter; payload bytes
  * and capacities stay. */
 int td_reset(td_dock *dock, void *stream);

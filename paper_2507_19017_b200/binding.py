@@ -29,7 +29,8 @@ ELEM_SIZE = {I32: 4, F32: 4, BF16: 2}
 EXPORTS = ["td_query_workspace", "td_create", "td_destroy", "td_put", "td_get",
            "td_get_scratch_bytes", "td_reset", "td_status", "td_debug_table",
            "td_launch_count", "td_strerror", "td_kernel_timing", "td_kernel_timing_read",
-           "td_put_host_stage_bytes", "td_put_host", "td_get_host"]
+           "td_put_host_stage_bytes", "td_put_host", "td_get_host", "td_put_many",
+           "td_plan_bytes", "td_plan_create", "td_plan_destroy", "td_get_many"]
 
 
 class TdColumn(C.Structure):
@@ -62,6 +63,15 @@ class TdGetOut(C.Structure):
                 ("cu_seq", C.c_void_p), ("col", C.c_void_p * 32),
                 ("col_capacity_elems", C.c_uint64 * 32), ("advantages", C.c_void_p),
                 ("result", C.c_void_p), ("scratch", C.c_void_p), ("scratch_bytes", C.c_uint64)]
+
+
+class TdPutItem(C.Structure):
+    _fields_ = [("column", C.c_uint32), ("k", C.c_uint32), ("d_indices", C.c_void_p),
+                ("d_cu", C.c_void_p), ("d_data", C.c_void_p), ("data_elems", C.c_uint64)]
+
+
+class TdGetReq(C.Structure):
+    _fields_ = [("consumer", C.c_uint32), ("max_samples", C.c_uint32), ("out", TdGetOut)]
 
 
 class TdStats(C.Structure):
@@ -129,6 +139,16 @@ def lib():
         L.td_put_host.argtypes = [vp, u32, vp, u32, vp, vp, u64, vp, C.c_size_t, vp]
         L.td_get_host.restype = C.c_int
         L.td_get_host.argtypes = [vp, u32, u32, C.POINTER(TdGetOut), C.POINTER(TdGetOut), vp]
+        L.td_put_many.restype = C.c_int
+        L.td_put_many.argtypes = [vp, C.POINTER(TdPutItem), u32, vp]
+        L.td_plan_bytes.restype = C.c_size_t
+        L.td_plan_bytes.argtypes = [vp, u32]
+        L.td_plan_create.restype = C.c_int
+        L.td_plan_create.argtypes = [vp, C.POINTER(TdGetReq), u32, vp, C.c_size_t, vp, C.POINTER(vp)]
+        L.td_plan_destroy.restype = C.c_int
+        L.td_plan_destroy.argtypes = [vp]
+        L.td_get_many.restype = C.c_int
+        L.td_get_many.argtypes = [vp, vp, vp]
         _lib = L
     return _lib
 
@@ -264,6 +284,36 @@ class HostGetBuffers:
         return total
 
 
+class Plan:
+    """A fixed list of gets (one GetBuffers each) that td_get_many serves in one call."""
+
+    def __init__(self, dock: "Dock", bufs: Sequence[GetBuffers], stream=None):
+        import torch
+        self.dock, self.bufs = dock, list(bufs)
+        n = len(self.bufs)
+        reqs = (TdGetReq * n)()
+        for j, b in enumerate(self.bufs):
+            reqs[j].consumer, reqs[j].max_samples = b.consumer, b.max_samples
+            reqs[j].out = b.struct
+        self.nbytes = lib().td_plan_bytes(dock.handle, n)
+        self.memory = torch.empty(self.nbytes, dtype=torch.uint8, device=dock.device)
+        h = C.c_void_p()
+        _check("td_plan_create", lib().td_plan_create(dock.handle, reqs, n, self.memory.data_ptr(),
+                                                      self.nbytes, _stream_ptr(stream), C.byref(h)))
+        self.handle = h
+
+    def close(self):
+        if getattr(self, "handle", None):
+            lib().td_plan_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
 class Dock:
     """A transfer dock living in one torch-allocated workspace on `device`."""
 
@@ -302,6 +352,20 @@ class Dock:
         _check("td_put", lib().td_put(self.handle, column, indices.data_ptr(), k,
                                       cu.data_ptr() if cu is not None else None,
                                       data.data_ptr(), data.numel(), _stream_ptr(stream)))
+
+    def put_many(self, items: Sequence[Tuple], stream=None):
+        """items: (column, indices, cu or None, data) device tensors, stored in this order."""
+        arr = (TdPutItem * len(items))()
+        for j, (column, indices, cu, data) in enumerate(items):
+            arr[j] = TdPutItem(column, indices.numel(), indices.data_ptr(),
+                               cu.data_ptr() if cu is not None else None, data.data_ptr(), data.numel())
+        _check("td_put_many", lib().td_put_many(self.handle, arr, len(items), _stream_ptr(stream)))
+
+    def plan(self, bufs: Sequence[GetBuffers], stream=None) -> "Plan":
+        return Plan(self, bufs, stream)
+
+    def get_many(self, plan: "Plan", stream=None):
+        _check("td_get_many", lib().td_get_many(self.handle, plan.handle, _stream_ptr(stream)))
 
     def get(self, bufs: GetBuffers, stream=None, max_samples: Optional[int] = None):
         _check("td_get", lib().td_get(self.handle, bufs.consumer,

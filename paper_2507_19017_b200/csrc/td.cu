@@ -220,31 +220,99 @@ int td_reset(td_dock *d, void *stream) {
     return TD_OK;
 }
 
+namespace {
+
+// One launch group: alloc (if any ragged item), scatter, publish.  Items are taken in order;
+// a column appears at most once per group, so that duplicate detection sees earlier items.
+int put_group(td_dock *d, const PutBatch &b, cudaStream_t st) {
+    const DockView &v = d->dv;
+    uint64_t ragged_bytes = 0, entries = 0;
+    for (uint32_t i = 0; i < b.n_items; ++i) {
+        entries += b.item[i].k;
+        if (v.col_cls[b.item[i].column] != TD_SCALAR)
+            ragged_bytes += b.item[i].data_elems * v.col_esz[b.item[i].column] + kSpanBytes;
+    }
+    if (entries == 0) return TD_OK;
+    if (entries >= (1ull << 32)) return TD_EINVAL;
+    if (ragged_bytes) {
+        if (launch(d, put_alloc_kernel, dim3(1), dim3(kAllocThreads), put_alloc_smem_bytes(v.S), st, v, b) != cudaSuccess)
+            return TD_ECUDA;
+        uint64_t blocks = ragged_bytes / kSpanBytes;
+        const uint64_t max_blocks = (uint64_t)d->sm_count * 4;
+        if (blocks > max_blocks) blocks = max_blocks;
+        if (blocks == 0) blocks = 1;
+        if (launch_timed(d, 0, put_scatter_kernel, dim3((uint32_t)blocks), dim3(kSpanThreads), 0, st, v, b) != cudaSuccess)
+            return TD_ECUDA;
+    }
+    if (launch(d, put_publish_kernel, dim3((uint32_t)((entries + 255) / 256)), dim3(256), 0, st, v, b) != cudaSuccess)
+        return TD_ECUDA;
+    return TD_OK;
+}
+
+bool valid_put_item(const td_dock *d, const td_put_item &it) {
+    if (it.column >= d->dv.ncol) return false;
+    if (it.k == 0) return true;
+    if (!it.d_indices || (!it.d_data && it.data_elems)) return false;
+    if (d->dv.col_cls[it.column] != TD_SCALAR && !it.d_cu) return false;
+    return it.data_elems < (1ull << 31);                 // cu is int32
+}
+
+uint32_t gather_blocks(const td_dock *d, uint64_t room_bytes) {
+    uint64_t blocks = room_bytes / kSpanBytes + 1;
+    const uint64_t max_blocks = (uint64_t)d->sm_count * 4;
+    if (blocks > max_blocks) blocks = max_blocks;
+    return (uint32_t)blocks;
+}
+
+uint64_t room_bytes_of(const DockView &v, uint32_t consumer, uint32_t max_samples, const td_get_out &out) {
+    uint64_t bytes = 0;
+    for (uint32_t k = 0; k < v.ncol; ++k)
+        if (((v.outm[consumer] >> k) & 1u) && out.col[k]) {
+            uint64_t room = out.col_capacity_elems[k];
+            if (v.col_cls[k] == TD_SCALAR && room > max_samples) room = max_samples;
+            bytes += room * v.col_esz[k] + kSpanBytes;
+        }
+    return bytes;
+}
+
+int check_get_out(const DockView &v, uint32_t consumer, uint32_t max_samples, const td_get_out *out) {
+    if (!out || consumer >= v.ncons) return TD_EINVAL;
+    if (max_samples / v.N == 0) return TD_EINVAL;
+    if (!out->indices || !out->cu_prompt || !out->cu_response || !out->result) return TD_EINVAL;
+    if (out->mode != TD_PACKED && out->mode != TD_PADDED) return TD_EINVAL;
+    if ((v.cflags[consumer] & TD_F_ADVANTAGE) && !out->advantages) return TD_EINVAL;
+    return TD_OK;
+}
+
+}  // namespace
+
+int td_put_many(td_dock *d, const td_put_item *items, uint32_t n_items, void *stream) {
+    if (!d || (n_items && !items)) return TD_EINVAL;
+    for (uint32_t i = 0; i < n_items; ++i)
+        if (!valid_put_item(d, items[i])) return TD_EINVAL;
+    cudaStream_t st = (cudaStream_t)stream;
+    PutBatch b;
+    std::memset(&b, 0, sizeof(b));
+    uint32_t seen = 0;
+    for (uint32_t i = 0; i < n_items; ++i) {
+        const td_put_item &it = items[i];
+        if (it.k == 0) continue;
+        if (b.n_items == kMaxPutItems || (seen >> it.column) & 1u) {
+            const int rc = put_group(d, b, st);
+            if (rc != TD_OK) return rc;
+            b.n_items = 0; seen = 0;
+        }
+        b.item[b.n_items++] = PutArgs{it.column, it.k, it.d_indices, it.d_cu,
+                                      static_cast<const uint8_t *>(it.d_data), it.data_elems};
+        seen |= 1u << it.column;
+    }
+    return b.n_items ? put_group(d, b, st) : TD_OK;
+}
+
 int td_put(td_dock *d, uint32_t column, const int32_t *d_indices, uint32_t k, const int32_t *d_cu,
            const void *d_data, uint64_t data_elems, void *stream) {
-    if (!d || column >= d->dv.ncol) return TD_EINVAL;
-    if (k == 0) return TD_OK;
-    if (!d_indices || (!d_data && data_elems)) return TD_EINVAL;
-    const uint32_t cls = d->dv.col_cls[column];
-    if (cls != TD_SCALAR && !d_cu) return TD_EINVAL;
-    if (data_elems >= (1ull << 31)) return TD_EINVAL;       // cu is int32
-    cudaStream_t st = (cudaStream_t)stream;
-    PutArgs a{column, k, d_indices, d_cu, static_cast<const uint8_t *>(d_data), data_elems};
-    if (cls == TD_SCALAR) {
-        if (launch(d, put_scalar_kernel, dim3((k + 255) / 256), dim3(256), 0, st, d->dv, a) != cudaSuccess) return TD_ECUDA;
-        return TD_OK;
-    }
-    if (launch(d, put_alloc_kernel, dim3(1), dim3(kAllocThreads), put_alloc_smem_bytes(d->dv.S), st, d->dv, a) != cudaSuccess)
-        return TD_ECUDA;
-    const uint64_t bytes = data_elems * d->dv.col_esz[column];
-    const uint64_t chunks = (bytes + kWarpChunkBytes - 1) / kWarpChunkBytes;
-    uint64_t blocks = (chunks + kCopyWarps - 1) / kCopyWarps;
-    const uint64_t max_blocks = (uint64_t)d->sm_count * 8;
-    if (blocks > max_blocks) blocks = max_blocks;
-    if (blocks == 0) blocks = 1;
-    if (launch_timed(d, 0, put_scatter_kernel, dim3((uint32_t)blocks), dim3(kCopyThreads), 0, st, d->dv, a) != cudaSuccess) return TD_ECUDA;
-    if (launch(d, put_publish_kernel, dim3((k + 255) / 256), dim3(256), 0, st, d->dv, a) != cudaSuccess) return TD_ECUDA;
-    return TD_OK;
+    const td_put_item it{column, k, d_indices, d_cu, d_data, data_elems};
+    return td_put_many(d, &it, 1, stream);
 }
 
 size_t td_get_scratch_bytes(const td_dock *d) {
@@ -252,17 +320,15 @@ size_t td_get_scratch_bytes(const td_dock *d) {
 }
 
 int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out *out, void *stream) {
-    if (!d || !out || consumer >= d->dv.ncons) return TD_EINVAL;
+    if (!d) return TD_EINVAL;
     const DockView &v = d->dv;
-    const uint32_t m = max_samples / v.N;
-    if (m == 0) return TD_EINVAL;
-    if (!out->indices || !out->cu_prompt || !out->cu_response || !out->result) return TD_EINVAL;
-    if (out->mode != TD_PACKED && out->mode != TD_PADDED) return TD_EINVAL;
-    if ((v.cflags[consumer] & TD_F_ADVANTAGE) && !out->advantages) return TD_EINVAL;
+    const int chk = check_get_out(v, consumer, max_samples, out);
+    if (chk != TD_OK) return chk;
     if (!out->scratch || (reinterpret_cast<uintptr_t>(out->scratch) & 15u) ||
         out->scratch_bytes < sel_scratch_bytes(v.G))
         return TD_EWORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
+    const uint32_t m = max_samples / v.N;
 
     GetInline one;
     std::memset(&one, 0, sizeof(one));
@@ -280,20 +346,107 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     if (launch(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
-    // gather grid from the room the caller supplied
-    uint64_t bytes = 0;
-    for (uint32_t k = 0; k < v.ncol; ++k)
-        if (((v.outm[consumer] >> k) & 1u) && out->col[k]) {
-            uint64_t room = out->col_capacity_elems[k];
-            if (v.col_cls[k] == TD_SCALAR && room > max_samples) room = max_samples;
-            bytes += room * v.col_esz[k] + kGatherChunkBytes;
+    const uint32_t blocks = gather_blocks(d, room_bytes_of(v, consumer, max_samples, *out));
+    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kSpanThreads), 0, st, v, one,
+                     (const GetReq *)nullptr, 1u) != cudaSuccess) return TD_ECUDA;
+    return TD_OK;
+}
+
+// ---- plans: many gets served by one call ----
+struct td_plan {
+    td_dock *dock;
+    uint32_t n_req, n_slots;
+    GetReq *d_reqs;
+    ConsumerSlot *d_slots;
+    uint64_t room_bytes;
+    std::vector<uint8_t> host_image;      // what was uploaded; kept until the plan dies
+};
+
+size_t td_plan_bytes(const td_dock *d, uint32_t n_req) {
+    if (!d || n_req == 0) return 0;
+    const size_t slots = d->dv.ncons;
+    return align_up_sz((size_t)n_req * sizeof(GetReq), 256) + align_up_sz(slots * sizeof(ConsumerSlot), 256) +
+           slots * align_up_sz(sel_scratch_bytes(d->dv.G), 256);
+}
+
+int td_plan_create(td_dock *d, const td_get_req *reqs, uint32_t n_req, void *d_plan, size_t plan_bytes,
+                   void *stream, td_plan **out) {
+    if (!d || !reqs || !out || n_req == 0) return TD_EINVAL;
+    const DockView &v = d->dv;
+    if ((uint64_t)n_req * v.ncol > (uint64_t)kMaxJobs) return TD_EINVAL;
+    if (!d_plan || (reinterpret_cast<uintptr_t>(d_plan) & 255u) || plan_bytes < td_plan_bytes(d, n_req))
+        return TD_EWORKSPACE;
+    for (uint32_t q = 0; q < n_req; ++q) {
+        const int chk = check_get_out(v, reqs[q].consumer, reqs[q].max_samples, &reqs[q].out);
+        if (chk != TD_OK) return chk;
+    }
+    td_plan *p = new (std::nothrow) td_plan();
+    if (!p) return TD_EINVAL;
+    p->dock = d; p->n_req = n_req;
+    const size_t off_slots = align_up_sz((size_t)n_req * sizeof(GetReq), 256);
+    const size_t off_scratch = off_slots + align_up_sz((size_t)v.ncons * sizeof(ConsumerSlot), 256);
+    const size_t scratch_each = align_up_sz(sel_scratch_bytes(v.G), 256);
+    uint8_t *base = static_cast<uint8_t *>(d_plan);
+    p->d_reqs = reinterpret_cast<GetReq *>(base);
+    p->d_slots = reinterpret_cast<ConsumerSlot *>(base + off_slots);
+    p->host_image.assign(off_scratch, 0);
+    GetReq *hr = reinterpret_cast<GetReq *>(p->host_image.data());
+    ConsumerSlot *hs = reinterpret_cast<ConsumerSlot *>(p->host_image.data() + off_slots);
+    // consumer slots in order of first appearance; requests of one consumer share its candidates
+    int slot_of[32];
+    for (int &x : slot_of) x = -1;
+    uint32_t n_slots = 0;
+    uint64_t room = 0;
+    for (uint32_t q = 0; q < n_req; ++q) {
+        const uint32_t c = reqs[q].consumer;
+        if (slot_of[c] < 0) {
+            slot_of[c] = (int)n_slots;
+            hs[n_slots].consumer = c; hs[n_slots].max_groups = 0;
+            hs[n_slots].scratch = base + off_scratch + (size_t)n_slots * scratch_each;
+            ++n_slots;
         }
-    uint64_t blocks = (bytes / kGatherChunkBytes + kGatherWarps - 1) / kGatherWarps;
-    const uint64_t max_blocks = (uint64_t)d->sm_count * 8;
-    if (blocks > max_blocks) blocks = max_blocks;
-    if (blocks == 0) blocks = 1;
-    if (launch_timed(d, 1, get_gather_kernel, dim3((uint32_t)blocks), dim3(kGatherThreads), 0, st, v, one,
-               (const GetReq *)nullptr, 1u) != cudaSuccess) return TD_ECUDA;
+        ConsumerSlot &cs = hs[slot_of[c]];
+        const uint32_t m = reqs[q].max_samples / v.N;
+        hr[q].out = reqs[q].out;
+        hr[q].consumer = c;
+        hr[q].rank_base = cs.max_groups;
+        hr[q].max_groups = m;
+        hr[q].cslot = (uint32_t)slot_of[c];
+        const uint64_t sum = (uint64_t)cs.max_groups + m;
+        cs.max_groups = sum > v.G ? v.G : (uint32_t)sum;
+        if (hr[q].rank_base > v.G) hr[q].rank_base = v.G;
+        room += room_bytes_of(v, c, reqs[q].max_samples, reqs[q].out);
+    }
+    p->n_slots = n_slots;
+    p->room_bytes = room;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (cudaMemsetAsync(base + off_scratch, 0, (size_t)v.ncons * scratch_each, st) != cudaSuccess ||
+        cudaMemcpyAsync(base, p->host_image.data(), off_scratch, cudaMemcpyHostToDevice, st) != cudaSuccess) {
+        delete p;
+        return TD_ECUDA;
+    }
+    *out = p;
+    return TD_OK;
+}
+
+int td_plan_destroy(td_plan *p) {
+    delete p;
+    return TD_OK;
+}
+
+int td_get_many(td_dock *d, td_plan *p, void *stream) {
+    if (!d || !p || p->dock != d) return TD_EINVAL;
+    const DockView &v = d->dv;
+    cudaStream_t st = (cudaStream_t)stream;
+    GetInline none;
+    std::memset(&none, 0, sizeof(none));
+    const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
+    if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), p->n_slots), dim3(kSelThreads), 0, st, v, none,
+               (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
+    if (launch(d, get_finalize_kernel, dim3(p->n_req), dim3(kFinThreads), 0, st, v, none, (const GetReq *)p->d_reqs,
+               (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
+    if (launch_timed(d, 1, get_gather_kernel, dim3(gather_blocks(d, p->room_bytes)), dim3(kSpanThreads), 0, st, v, none,
+                     (const GetReq *)p->d_reqs, p->n_req) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 

@@ -221,15 +221,70 @@ __device__ __forceinline__ void warp_fill(uint8_t *dst, uint64_t nbytes, uint32_
     }
 }
 
-// first index i in [0, count] with a[i] > x, minus one: the row containing element x,
-// skipping rows of length zero (a is a non-decreasing prefix array with a[0] = 0).
-__device__ __forceinline__ uint32_t row_of(const int32_t *a, uint32_t count, int64_t x) {
-    uint32_t lo = 0, hi = count;        // invariant: a[lo] <= x, a[hi] > x (hi = count: total > x)
-    while (hi - lo > 1) {
-        uint32_t mid = (lo + hi) >> 1;
-        if ((int64_t)a[mid] <= x) lo = mid; else hi = mid;
+// --------------------------------------------------------------------------------------------
+// Span copy.  The packed side of a ragged copy (the source of a put, the destination of a
+// packed get) is cut into spans of kSpanBytes; one CTA serves one span at a time:
+//   1. all threads together find the row the span starts in (a k-ary search of cu with one
+//      probe per thread and round, instead of a dependent bisection per warp);
+//   2. one thread per row resolves where that row lives on the other side (index -> tables);
+//   3. each warp copies its kWarpBytes slice of the span, piece by piece, from the row
+//      descriptors now in shared memory.
+// This keeps every dependent metadata lookup off the warps' critical path and leaves the
+// copy itself as wide aligned vector traffic.
+// --------------------------------------------------------------------------------------------
+constexpr int kSpanThreads = 256;
+constexpr int kSpanWarps = kSpanThreads / 32;
+constexpr uint32_t kWarpBytes = 4096;
+constexpr uint32_t kSpanBytes = kWarpBytes * kSpanWarps;
+
+struct RowDesc {
+    uint64_t lo, hi;          // byte range of the row on the packed side
+    uint8_t *other;           // start of the row on the other side, nullptr = skip the row
+};
+
+// Largest i in [0, rows) with cu[i] <= x (the row holding element x, rows of length zero
+// skipped); 0 when even cu[0] > x.  Every thread of the CTA must call it; all get the answer.
+__device__ __forceinline__ uint32_t block_find_row(const int32_t *cu, uint32_t rows, int64_t x) {
+    uint32_t lo = 0, len = rows;
+    while (len > 1) {
+        const uint32_t stride = (len + kSpanThreads - 1) / kSpanThreads;
+        const uint64_t probe = (uint64_t)threadIdx.x * stride;
+        const bool ok = probe < len && (int64_t)cu[lo + probe] <= x;
+        int cnt = __syncthreads_count(ok);          // ok holds for a prefix of the threads
+        if (cnt < 1) cnt = 1;
+        const uint32_t step = (uint32_t)(cnt - 1) * stride;
+        lo += step;
+        len = min(stride, len - step);
     }
     return lo;
+}
+
+// First descriptor in d[0, n) whose hi exceeds x (hi is non-decreasing); n if none.
+__device__ __forceinline__ uint32_t first_desc_after(const RowDesc *d, uint32_t n, uint64_t x) {
+    uint32_t lo = 0, hi = n;
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if (d[mid].hi > x) hi = mid; else lo = mid + 1;
+    }
+    return lo;
+}
+
+// Step 3 for one warp: copy the parts of the described rows that fall inside [w_lo, w_hi) of
+// the packed side.  kToPacked: the packed side is the destination (get), else the source (put).
+template <bool kToPacked>
+__device__ __forceinline__ void warp_copy_rows(const RowDesc *d, uint32_t n, uint64_t w_lo, uint64_t w_hi,
+                                               uint8_t *packed, uint32_t esz, uint32_t lane,
+                                               const uint8_t *src_lo, const uint8_t *src_hi) {
+    for (uint32_t r = first_desc_after(d, n, w_lo); r < n; ++r) {
+        const uint64_t rlo = d[r].lo;
+        if (rlo >= w_hi) break;
+        uint8_t *other = d[r].other;
+        if (other == nullptr) continue;
+        const uint64_t lo = max(rlo, w_lo), hi = min(d[r].hi, w_hi);
+        if (hi <= lo) continue;
+        if (kToPacked) warp_copy(packed + lo, other + (lo - rlo), hi - lo, esz, lane, src_lo, src_hi);
+        else warp_copy(other + (lo - rlo), packed + lo, hi - lo, esz, lane, src_lo, src_hi);
+    }
 }
 
 }  // namespace td

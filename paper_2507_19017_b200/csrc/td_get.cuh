@@ -10,10 +10,7 @@ namespace td {
 constexpr int kSelThreads = 256;            // one thread per group; a tile is 256 groups
 constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kFinThreads = 256;
-constexpr int kGatherThreads = 256;
-constexpr int kGatherWarps = kGatherThreads / 32;
-constexpr uint32_t kGatherChunkBytes = 4096;   // output bytes one warp produces per step
-constexpr int kMaxJobs = 2048;              // (request, column) pairs one gather launch serves
+constexpr int kMaxJobs = 4096;              // (request, column) pairs one gather launch serves
 
 // Tile descriptor of the single-pass scan: [63:32] launch sequence number, [31:30] state,
 // [29:0] count.  A descriptor whose sequence number is not the launch's is "not written yet",
@@ -348,69 +345,75 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
 }
 
 // ---------------------------------------------------------------------------------------------
-// Gather.  Persistent grid.  Every (request, wanted column) is a job whose output space is cut
-// into warp chunks of kGatherChunkBytes; warps stride over the chunks of all jobs, so the
-// work is balanced over bytes whatever the mix of row lengths.
+// Gather.  Persistent grid.  Every (request, column) pair is a job; the output space of each
+// job is cut into spans of kSpanBytes and CTAs stride over the spans of all jobs, so the work
+// is balanced over bytes whatever the mix of requests and row lengths (see "Span copy" in
+// td_device.cuh).
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(kGatherThreads)
+__device__ __forceinline__ uint64_t job_bytes(const DockView &dv, const GetReq &rq, uint32_t k) {
+    const td_get_out &out = rq.out;
+    if (!((dv.outm[rq.consumer] >> k) & 1u) || out.col[k] == nullptr) return 0;
+    const td_result *res = out.result;
+    const uint32_t cls = dv.col_cls[k], esz = dv.col_esz[k];
+    const uint64_t n_s = res->n_samples;
+    if (cls == TD_SCALAR) return n_s * esz;
+    if (out.mode == TD_PACKED) return (cls == TD_PROMPT ? res->prompt_tokens : res->response_tokens) * esz;
+    return n_s * (uint64_t)(cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to) * esz;
+}
+
+__global__ void __launch_bounds__(kSpanThreads, 4)
 get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
                   const GetReq *reqs_dev, const uint32_t n_req) {
     const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
-    __shared__ uint64_t job_end[kMaxJobs];          // inclusive prefix of chunks per job
-    __shared__ uint16_t job_req[kMaxJobs];
-    __shared__ uint8_t job_col[kMaxJobs];
-    __shared__ uint32_t s_njobs;
-    const uint32_t tid = threadIdx.x, lane = tid & 31;
+    __shared__ RowDesc desc[kSpanThreads];
+    __shared__ uint32_t job_end[kMaxJobs];          // inclusive prefix of spans, jobs = [request][column]
+    __shared__ uint32_t s_wsum[kSpanWarps];
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t ncol = dv.ncol;
+    const uint32_t njobs = n_req * ncol;
 
-    // job table (every CTA builds the same one)
-    if (tid == 0) {
-        uint32_t nj = 0; uint64_t acc = 0;
-        for (uint32_t q = 0; q < n_req; ++q) {
-            const td_get_out &out = reqs[q].out;
-            const td_result res = *out.result;
-            const uint32_t outm = dv.outm[reqs[q].consumer];
-            for (uint32_t k = 0; k < dv.ncol && nj < kMaxJobs; ++k) {
-                if (!((outm >> k) & 1u) || out.col[k] == nullptr) continue;
-                const uint32_t cls = dv.col_cls[k], esz = dv.col_esz[k];
-                uint64_t bytes;
-                if (cls == TD_SCALAR) bytes = (uint64_t)res.n_samples * esz;
-                else if (out.mode == TD_PACKED)
-                    bytes = (cls == TD_PROMPT ? res.prompt_tokens : res.response_tokens) * esz;
-                else
-                    bytes = (uint64_t)res.n_samples * (cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to) * esz;
-                if (bytes == 0) continue;
-                acc += (bytes + kGatherChunkBytes - 1) / kGatherChunkBytes;
-                job_end[nj] = acc; job_req[nj] = (uint16_t)q; job_col[nj] = (uint8_t)k;
-                ++nj;
-            }
+    // job table: each thread sizes a contiguous run of jobs, then one block scan
+    {
+        const uint32_t per = (njobs + kSpanThreads - 1) / kSpanThreads;
+        const uint32_t j0 = tid * per, j1 = min(j0 + per, njobs);
+        uint32_t local = 0;
+        for (uint32_t j = j0; j < j1; ++j) {
+            const uint64_t b = job_bytes(dv, reqs[j / ncol], j % ncol);
+            local += (uint32_t)((b + kSpanBytes - 1) / kSpanBytes);
+            job_end[j] = local;                       // inclusive within the thread's run
         }
-        s_njobs = nj;
+        uint32_t inc = local;
+        #pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const uint32_t t = __shfl_up_sync(kFullMask, inc, d);
+            if ((int)lane >= d) inc += t;
+        }
+        if (lane == 31) s_wsum[warp] = inc;
+        __syncthreads();
+        uint32_t before = inc - local;
+        for (uint32_t w = 0; w < warp; ++w) before += s_wsum[w];
+        for (uint32_t j = j0; j < j1; ++j) job_end[j] += before;
+        __syncthreads();
     }
-    __syncthreads();
-    const uint32_t njobs = s_njobs;
-    if (njobs == 0) return;
-    const uint64_t n_chunks = job_end[njobs - 1];
-    const uint64_t warp0 = (uint64_t)blockIdx.x * kGatherWarps + (tid >> 5);
-    const uint64_t stride = (uint64_t)gridDim.x * kGatherWarps;
+    const uint32_t n_spans = njobs ? job_end[njobs - 1] : 0;
 
-    for (uint64_t ch = warp0; ch < n_chunks; ch += stride) {
-        // job of this chunk: first j with job_end[j] > ch
+    for (uint32_t sp = blockIdx.x; sp < n_spans; sp += gridDim.x) {
+        // job of this span: first j with job_end[j] > sp
         uint32_t jlo = 0, jhi = njobs - 1;
-        while (jlo < jhi) { const uint32_t m = (jlo + jhi) >> 1; if (job_end[m] > ch) jhi = m; else jlo = m + 1; }
+        while (jlo < jhi) { const uint32_t m = (jlo + jhi) >> 1; if (job_end[m] > sp) jhi = m; else jlo = m + 1; }
         const uint32_t j = jlo;
-        const uint64_t local = ch - (j ? job_end[j - 1] : 0);
-        const GetReq &rq = reqs[job_req[j]];
+        const GetReq &rq = reqs[j / ncol];
         const td_get_out &out = rq.out;
-        const uint32_t k = job_col[j];
+        const uint32_t k = j % ncol;
         const uint32_t cls = dv.col_cls[k], esz = dv.col_esz[k];
         const uint32_t n_s = out.result->n_samples;
         uint8_t *dst0 = reinterpret_cast<uint8_t *>(out.col[k]);
-        const uint8_t *base = dv.colbase[k];
-        const uint64_t b0 = local * kGatherChunkBytes;
+        uint8_t *base = dv.colbase[k];
+        const uint64_t b0 = (uint64_t)(sp - (j ? job_end[j - 1] : 0)) * kSpanBytes;
 
         if (cls == TD_SCALAR) {
-            const uint64_t e0 = b0 / esz, e1 = min((b0 + kGatherChunkBytes) / esz, (uint64_t)n_s);
-            for (uint64_t e = e0 + lane; e < e1; e += 32) {
+            const uint64_t e0 = b0 / esz, e1 = min((b0 + kSpanBytes) / esz, (uint64_t)n_s);
+            for (uint64_t e = e0 + tid; e < e1; e += kSpanThreads) {
                 const int32_t s = out.indices[e];
                 if (esz == 4) reinterpret_cast<uint32_t *>(dst0)[e] = reinterpret_cast<const uint32_t *>(base)[s];
                 else reinterpret_cast<uint16_t *>(dst0)[e] = reinterpret_cast<const uint16_t *>(base)[s];
@@ -420,43 +423,56 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
         const uint64_t cap = dv.cap[cls];
         const uint8_t *src_lo = base, *src_hi = base + (uint64_t)dv.S * cap * esz;
         const long long *offt = dv.off[cls];
-        if (out.mode == TD_PACKED) {
-            const int32_t *cu = cls == TD_PROMPT ? out.cu_prompt : out.cu_response;
-            const uint64_t total = (uint64_t)(int64_t)cu[n_s] * esz;
-            const uint64_t b1 = min(b0 + (uint64_t)kGatherChunkBytes, total);
-            for (uint32_t i = row_of(cu, n_s, (int64_t)(b0 / esz)); i < n_s; ++i) {
-                const uint64_t row_lo = (uint64_t)(int64_t)cu[i] * esz;
-                if (row_lo >= b1) break;
-                const uint64_t row_hi = (uint64_t)(int64_t)cu[i + 1] * esz;
-                const uint64_t lo = max(row_lo, b0), hi = min(row_hi, b1);
-                if (hi <= lo) continue;
-                const uint32_t s = (uint32_t)out.indices[i];
-                const uint8_t *src = base + ((uint64_t)shard_of(dv, s) * cap + (uint64_t)offt[s]) * esz + (lo - row_lo);
-                warp_copy(dst0 + lo, src, hi - lo, esz, lane, src_lo, src_hi);
-            }
-        } else {
-            const uint32_t W = cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to;
-            const int32_t *lent = dv.len[cls];
-            const uint64_t row_bytes = (uint64_t)W * esz;
-            const uint64_t total = (uint64_t)n_s * row_bytes;
-            const uint64_t b1 = min(b0 + (uint64_t)kGatherChunkBytes, total);
-            for (uint64_t i = b0 / row_bytes; i < n_s; ++i) {
-                const uint64_t row_lo = i * row_bytes;
-                if (row_lo >= b1) break;
-                const uint32_t s = (uint32_t)out.indices[i];
-                const int32_t l = lent[s];
-                const uint64_t valid_hi = row_lo + (uint64_t)(l > 0 ? l : 0) * esz;
-                const uint64_t lo = max(row_lo, b0), hi = min(row_lo + row_bytes, b1);
-                // payload part
-                const uint64_t phi = min(hi, valid_hi);
-                if (phi > lo) {
-                    const uint8_t *src = base + ((uint64_t)shard_of(dv, s) * cap + (uint64_t)offt[s]) * esz + (lo - row_lo);
-                    warp_copy(dst0 + lo, src, phi - lo, esz, lane, src_lo, src_hi);
+        const bool packed = out.mode == TD_PACKED;
+        const int32_t *cu = cls == TD_PROMPT ? out.cu_prompt : out.cu_response;
+        const uint32_t W = cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to;
+        const uint64_t row_bytes = (uint64_t)W * esz;
+        const uint64_t total = packed ? (uint64_t)(int64_t)cu[n_s] * esz : (uint64_t)n_s * row_bytes;
+        const uint64_t b1 = min(b0 + (uint64_t)kSpanBytes, total);
+        const uint64_t w_lo = b0 + (uint64_t)warp * kWarpBytes;
+        const uint64_t w_hi = min(w_lo + (uint64_t)kWarpBytes, b1);
+
+        uint32_t r0 = packed ? block_find_row(cu, n_s, (int64_t)(b0 / esz)) : (uint32_t)(b0 / row_bytes);
+        for (;;) {
+            const uint32_t i = r0 + tid;
+            bool in_span = false;
+            RowDesc d; d.lo = 0; d.hi = 0; d.other = nullptr;
+            if (i < n_s) {
+                const uint64_t rlo = packed ? (uint64_t)(int64_t)cu[i] * esz : (uint64_t)i * row_bytes;
+                in_span = rlo < b1;
+                if (in_span) {
+                    const uint32_t s = (uint32_t)out.indices[i];
+                    uint64_t len_b;
+                    if (packed) len_b = (uint64_t)(int64_t)cu[i + 1] * esz - rlo;
+                    else { const int32_t l = dv.len[cls][s]; len_b = (uint64_t)(l > 0 ? l : 0) * esz; }
+                    const long long off = offt[s];
+                    d.lo = rlo; d.hi = rlo + len_b;
+                    d.other = off >= 0 ? base + ((uint64_t)shard_of(dv, s) * cap + (uint64_t)off) * esz : nullptr;
                 }
-                // padding part
-                const uint64_t plo = max(lo, valid_hi);
-                if (hi > plo) warp_fill(dst0 + plo, hi - plo, dv.col_pad[k], esz, lane);
             }
+            desc[tid] = d;
+            const uint32_t n_rows = (uint32_t)__syncthreads_count(in_span);
+            if (w_lo < w_hi) {
+                if (packed) {
+                    warp_copy_rows<true>(desc, n_rows, w_lo, w_hi, dst0, esz, lane, src_lo, src_hi);
+                } else {
+                    // fixed-width rows: payload part, then the pad pattern up to the row's end
+                    for (uint32_t r = (uint32_t)(max(w_lo / row_bytes, (uint64_t)r0) - r0); r < n_rows; ++r) {
+                        const uint64_t rlo = desc[r].lo;
+                        if (rlo >= w_hi) break;
+                        const uint64_t valid_hi = desc[r].hi, rhi = rlo + row_bytes;
+                        const uint64_t lo = max(rlo, w_lo), hi = min(rhi, w_hi);
+                        const uint64_t phi = min(hi, valid_hi);
+                        if (phi > lo && desc[r].other)
+                            warp_copy(dst0 + lo, desc[r].other + (lo - rlo), phi - lo, esz, lane, src_lo, src_hi);
+                        const uint64_t plo = max(lo, valid_hi);
+                        if (hi > plo) warp_fill(dst0 + plo, hi - plo, dv.col_pad[k], esz, lane);
+                    }
+                }
+            }
+            __syncthreads();
+            if (n_rows < kSpanThreads) break;
+            r0 += kSpanThreads;
         }
     }
 }

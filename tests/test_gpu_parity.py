@@ -150,6 +150,99 @@ def test_many_tiles_look_back(G):
     assert batches[0][1].n_samples == 2200
 
 
+# ------------------------------------------------------------------- batched calls
+def _many_vs_serial(G, w, mode=td.PACKED):
+    """All columns in one td_put_many, all gets of the schedule in one td_get_many; the oracle
+    runs the same calls one by one."""
+    o = H.make_oracle(w)
+    g = G.GpuDock(w)
+    pad_p, pad_r = (w.pad_prompt_to, w.pad_response_to) if mode == td.PADDED else (0, 0)
+    items, keep = [], []
+    for op in w.ops:
+        if op.kind == "put":
+            cu, data = w.pack(op.column, op.indices)
+            o.put(op.column, op.indices, cu, data)
+            t = (op.column, G.to_device(np.ascontiguousarray(op.indices, np.int32), g.device),
+                 G.to_device(cu, g.device) if cu is not None else None, G.to_device(data, g.device))
+            items.append(t)
+    g.dock.put_many(items)
+    G.assert_state_equal(g, o, ctx="after put_many")
+    gets = [op for op in w.ops if op.kind == "get"]
+    bufs = [g.buffers(op.consumer, op.max_samples, mode, pad_p, pad_r, key=j) for j, op in enumerate(gets)]
+    plan = g.dock.plan(bufs)
+    g.dock.get_many(plan)
+    for j, op in enumerate(gets):
+        want = o.get(op.consumer, op.max_samples, mode, pad_p, pad_r)
+        G.assert_batch_equal(g.read(bufs[j]), want, f"request {j}")
+    G.assert_state_equal(g, o, ctx="after get_many")
+    G.assert_stats_equal(g, o, "many")
+    # the same plan again: everything is consumed, every request comes back empty
+    g.dock.get_many(plan)
+    assert all(g.read(b).n_samples == 0 for b in bufs)
+    return g, o, plan, bufs
+
+
+def test_put_many_get_many_small(G):
+    w = wl.make_custom("many", 24, 3, 4, prompt_len=(1, 70), response=("uniform", 0, 200), vocab=50000,
+                       micro_batch=9, seed=31, with_entropy=True, schedule="bulk")
+    _many_vs_serial(G, w)
+    _many_vs_serial(G, w, mode=td.PADDED)
+
+
+@pytest.mark.parametrize("cid", [2, 3])
+def test_put_many_get_many_full_size(G, cid):
+    _many_vs_serial(G, wl.make_config(cid))
+
+
+def test_get_many_partial_readiness_and_reuse(G):
+    """A plan that asks for more than is ready: early requests are filled, later ones come back
+    short or empty; after more puts the same plan serves the rest."""
+    w = wl.make_custom("many2", 20, 2, 2, prompt_len=(1, 30), response=("uniform", 1, 60), vocab=500,
+                       micro_batch=8, seed=32, schedule="bulk")
+    o = H.make_oracle(w)
+    g = G.GpuDock(w)
+    first = np.arange(0, 22, dtype=np.int32)          # 11 groups
+    rest = np.arange(22, w.n, dtype=np.int32)
+    for idx in (first,):
+        for c in range(len(w.columns)):
+            cu, data = w.pack(c, idx)
+            o.put(c, idx, cu, data); g.put(c, idx, cu, data)
+    gets = [op for op in w.ops if op.kind == "get"]
+    bufs = [g.buffers(op.consumer, op.max_samples, key=j) for j, op in enumerate(gets)]
+    plan = g.dock.plan(bufs)
+    g.dock.get_many(plan)
+    served = 0
+    for j, op in enumerate(gets):
+        want = o.get(op.consumer, op.max_samples)
+        G.assert_batch_equal(g.read(bufs[j]), want, f"round 1 request {j}")
+        served += want.n_samples
+    assert served == 22 * len(w.consumers)
+    for c in range(len(w.columns)):
+        cu, data = w.pack(c, rest)
+        o.put(c, rest, cu, data); g.put(c, rest, cu, data)
+    g.dock.get_many(plan)
+    for j, op in enumerate(gets):
+        G.assert_batch_equal(g.read(bufs[j]), o.get(op.consumer, op.max_samples), f"round 2 request {j}")
+    G.assert_state_equal(g, o, ctx="many2")
+
+
+def test_put_many_same_column_twice_and_errors(G):
+    w = wl.make_custom("many3", 8, 2, 2, prompt_len=(1, 30), response=("uniform", 1, 60), vocab=500,
+                       micro_batch=8, seed=33, schedule="none")
+    o = H.make_oracle(w)
+    g = G.GpuDock(w)
+    rid = w.column_index("response_ids")
+    a, b = np.array([0, 1, 2, 3], np.int32), np.array([3, 4, 5, 99], np.int32)
+    items = []
+    for idx in (a, b):
+        cu, data = w.pack(rid, np.clip(idx, 0, w.n - 1))
+        o.put(rid, idx, cu, data)
+        items.append((rid, G.to_device(idx, g.device), G.to_device(cu, g.device), G.to_device(data, g.device)))
+    g.dock.put_many(items)
+    G.assert_state_equal(g, o, ctx="same column twice")
+    G.assert_stats_equal(g, o, "same column twice")
+
+
 # ----------------------------------------------------------------------------- error paths
 def test_put_errors_are_counted_and_skipped(G):
     w = wl.make_custom("err", 8, 4, 2, prompt_len=(3, 40), response=("uniform", 1, 90), vocab=1000,
