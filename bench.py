@@ -38,6 +38,9 @@ def parse_args():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--api", default="many", choices=["many", "single"],
+                    help="many: one td_put_many and one td_get_many per step; single: one td_put per "
+                         "column and one td_get per micro-batch")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU-oracle time budget")
     return ap.parse_args()
 
@@ -132,8 +135,9 @@ def algorithmic_bytes(w):
 class GpuStep:
     """Device-resident inputs and per-get output buffers of one step, and the step itself."""
 
-    def __init__(self, w, device_index: int):
+    def __init__(self, w, device_index: int, api: str = "many"):
         import torch
+        self.api = api
         from paper_2507_19017_b200 import binding as td
         from paper_2507_19017_b200 import workloads as wl
         self.torch, self.td, self.w = torch, td, w
@@ -167,6 +171,7 @@ class GpuStep:
                                  prompt_tokens_cap=int(lp[:m].sum(dtype=np.int64)),
                                  response_tokens_cap=int(lr[:m].sum(dtype=np.int64)))
             self.gets.append(bufs)
+        self.plan = self.dock.plan(self.gets) if api == "many" else None
         self.flush_buf = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=self.dev)
         self.stage = None
         self.host_gets = None
@@ -182,12 +187,18 @@ class GpuStep:
 
     def put_phase(self):
         self.dock.reset()
-        for col, idx, cu, data in self.puts:
-            self.dock.put(col, idx, cu, data)
+        if self.api == "many":
+            self.dock.put_many(self.puts)
+        else:
+            for col, idx, cu, data in self.puts:
+                self.dock.put(col, idx, cu, data)
 
     def drain_phase(self):
-        for bufs in self.gets:
-            self.dock.get(bufs)
+        if self.api == "many":
+            self.dock.get_many(self.plan)
+        else:
+            for bufs in self.gets:
+                self.dock.get(bufs)
 
     def timed_step(self):
         """Returns (put_ms, drain_ms) measured with CUDA events on the current stream."""
@@ -332,7 +343,9 @@ def main():
         torch.cuda.set_device(local_rank)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    step = GpuStep(w, local_rank)
+    step = GpuStep(w, local_rank, args.api)
+    config["api"] = ("td_put_many + td_get_many (one call each per step)" if args.api == "many"
+                     else "td_put per column + td_get per micro-batch")
     peak, peak_kind = load_peaks()
     put_bytes, put_ragged_bytes, get_bytes = algorithmic_bytes(w)
 
