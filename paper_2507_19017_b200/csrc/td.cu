@@ -222,6 +222,17 @@ int td_reset(td_dock *d, void *stream) {
 
 namespace {
 
+// Grid and chunk size of a copy launch that may move up to room_bytes on the packed side.
+uint32_t copy_grid(const td_dock *d, uint64_t room_bytes, uint32_t *chunk_bytes) {
+    const uint64_t max_blocks = (uint64_t)d->sm_count * kCopyBlocksPerSM;
+    const uint32_t chunk = pick_chunk_bytes(room_bytes, max_blocks * kCopyWarps);
+    uint64_t blocks = (room_bytes / chunk + kCopyWarps) / kCopyWarps;
+    if (blocks > max_blocks) blocks = max_blocks;
+    if (blocks == 0) blocks = 1;
+    *chunk_bytes = chunk;
+    return (uint32_t)blocks;
+}
+
 // One launch group: alloc (if any ragged item), scatter, publish.  Items are taken in order;
 // a column appears at most once per group, so that duplicate detection sees earlier items.
 int put_group(td_dock *d, const PutBatch &b, cudaStream_t st) {
@@ -230,18 +241,16 @@ int put_group(td_dock *d, const PutBatch &b, cudaStream_t st) {
     for (uint32_t i = 0; i < b.n_items; ++i) {
         entries += b.item[i].k;
         if (v.col_cls[b.item[i].column] != TD_SCALAR)
-            ragged_bytes += b.item[i].data_elems * v.col_esz[b.item[i].column] + kSpanBytes;
+            ragged_bytes += b.item[i].data_elems * v.col_esz[b.item[i].column] + kMinChunkBytes;
     }
     if (entries == 0) return TD_OK;
     if (entries >= (1ull << 32)) return TD_EINVAL;
     if (ragged_bytes) {
         if (launch(d, put_alloc_kernel, dim3(1), dim3(kAllocThreads), put_alloc_smem_bytes(v.S), st, v, b) != cudaSuccess)
             return TD_ECUDA;
-        uint64_t blocks = ragged_bytes / kSpanBytes;
-        const uint64_t max_blocks = (uint64_t)d->sm_count * 4;
-        if (blocks > max_blocks) blocks = max_blocks;
-        if (blocks == 0) blocks = 1;
-        if (launch_timed(d, 0, put_scatter_kernel, dim3((uint32_t)blocks), dim3(kSpanThreads), 0, st, v, b) != cudaSuccess)
+        uint32_t chunk = 0;
+        const uint32_t blocks = copy_grid(d, ragged_bytes, &chunk);
+        if (launch_timed(d, 0, put_scatter_kernel, dim3(blocks), dim3(kCopyThreads), 0, st, v, b, chunk) != cudaSuccess)
             return TD_ECUDA;
     }
     if (launch(d, put_publish_kernel, dim3((uint32_t)((entries + 255) / 256)), dim3(256), 0, st, v, b) != cudaSuccess)
@@ -257,12 +266,6 @@ bool valid_put_item(const td_dock *d, const td_put_item &it) {
     return it.data_elems < (1ull << 31);                 // cu is int32
 }
 
-uint32_t gather_blocks(const td_dock *d, uint64_t room_bytes) {
-    uint64_t blocks = room_bytes / kSpanBytes + 1;
-    const uint64_t max_blocks = (uint64_t)d->sm_count * 4;
-    if (blocks > max_blocks) blocks = max_blocks;
-    return (uint32_t)blocks;
-}
 
 uint64_t room_bytes_of(const DockView &v, uint32_t consumer, uint32_t max_samples, const td_get_out &out) {
     uint64_t bytes = 0;
@@ -270,7 +273,7 @@ uint64_t room_bytes_of(const DockView &v, uint32_t consumer, uint32_t max_sample
         if (((v.outm[consumer] >> k) & 1u) && out.col[k]) {
             uint64_t room = out.col_capacity_elems[k];
             if (v.col_cls[k] == TD_SCALAR && room > max_samples) room = max_samples;
-            bytes += room * v.col_esz[k] + kSpanBytes;
+            bytes += room * v.col_esz[k] + kMinChunkBytes;
         }
     return bytes;
 }
@@ -346,9 +349,10 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     if (launch(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
-    const uint32_t blocks = gather_blocks(d, room_bytes_of(v, consumer, max_samples, *out));
-    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kSpanThreads), 0, st, v, one,
-                     (const GetReq *)nullptr, 1u) != cudaSuccess) return TD_ECUDA;
+    uint32_t chunk = 0;
+    const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out), &chunk);
+    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), 0, st, v, one,
+                     (const GetReq *)nullptr, 1u, chunk) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 
@@ -445,8 +449,10 @@ int td_get_many(td_dock *d, td_plan *p, void *stream) {
                (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
     if (launch(d, get_finalize_kernel, dim3(p->n_req), dim3(kFinThreads), 0, st, v, none, (const GetReq *)p->d_reqs,
                (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
-    if (launch_timed(d, 1, get_gather_kernel, dim3(gather_blocks(d, p->room_bytes)), dim3(kSpanThreads), 0, st, v, none,
-                     (const GetReq *)p->d_reqs, p->n_req) != cudaSuccess) return TD_ECUDA;
+    uint32_t chunk = 0;
+    const uint32_t blocks = copy_grid(d, p->room_bytes, &chunk);
+    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), 0, st, v, none,
+                     (const GetReq *)p->d_reqs, p->n_req, chunk) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 

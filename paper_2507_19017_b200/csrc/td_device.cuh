@@ -141,15 +141,11 @@ __device__ __forceinline__ void copy_body_shifted(uint4 *dst, const uint8_t *src
     }
     if (v_hi <= v_lo) return;
     uint32_t v = v_lo + lane;
-    for (; v + 96 < v_hi; v += 128) {
+    for (; v + 32 < v_hi; v += 64) {
         uint4 a0 = ld_stream(S + v),      b0 = ld_stream(S + v + 1);
         uint4 a1 = ld_stream(S + v + 32), b1 = ld_stream(S + v + 33);
-        uint4 a2 = ld_stream(S + v + 64), b2 = ld_stream(S + v + 65);
-        uint4 a3 = ld_stream(S + v + 96), b3 = ld_stream(S + v + 97);
         st_stream(dst + v,      shift_window<WSH>(a0, b0, bsh));
         st_stream(dst + v + 32, shift_window<WSH>(a1, b1, bsh));
-        st_stream(dst + v + 64, shift_window<WSH>(a2, b2, bsh));
-        st_stream(dst + v + 96, shift_window<WSH>(a3, b3, bsh));
     }
     for (; v < v_hi; v += 32) {
         uint4 a = ld_stream(S + v), b = ld_stream(S + v + 1);
@@ -222,68 +218,92 @@ __device__ __forceinline__ void warp_fill(uint8_t *dst, uint64_t nbytes, uint32_
 }
 
 // --------------------------------------------------------------------------------------------
-// Span copy.  The packed side of a ragged copy (the source of a put, the destination of a
-// packed get) is cut into spans of kSpanBytes; one CTA serves one span at a time:
-//   1. all threads together find the row the span starts in (a k-ary search of cu with one
-//      probe per thread and round, instead of a dependent bisection per warp);
-//   2. one thread per row resolves where that row lives on the other side (index -> tables);
-//   3. each warp copies its kWarpBytes slice of the span, piece by piece, from the row
-//      descriptors now in shared memory.
-// This keeps every dependent metadata lookup off the warps' critical path and leaves the
-// copy itself as wide aligned vector traffic.
+// Chunked ragged copy.  The packed side of a ragged copy (the source of a put, the destination
+// of a packed get) is cut into chunks of a launch-chosen size; warps stride over the chunks
+// and never wait for one another.  Per chunk a warp
+//   1. finds the row the chunk starts in with a 32-ary search of cu (one probe per lane and
+//      round instead of a dependent bisection),
+//   2. lets lane l resolve row r0 + l: its byte range on the packed side and where the row
+//      lives on the other side (index -> tables), all lanes' lookups in flight together,
+//   3. walks the rows, broadcasting each descriptor by shuffle, and copies the pieces that
+//      fall inside the chunk as wide aligned vector traffic.
+// With many resident warps per SM the metadata latency of one warp hides behind the copies of
+// the others; there is no block-wide barrier on the path.
 // --------------------------------------------------------------------------------------------
-constexpr int kSpanThreads = 256;
-constexpr int kSpanWarps = kSpanThreads / 32;
-constexpr uint32_t kWarpBytes = 4096;
-constexpr uint32_t kSpanBytes = kWarpBytes * kSpanWarps;
+constexpr int kCopyThreads = 256;
+constexpr int kCopyWarps = kCopyThreads / 32;
+constexpr uint32_t kMinChunkBytes = 1024, kMaxChunkBytes = 16384;
+constexpr int kCopyBlocksPerSM = 6;          // resident CTAs per SM the copy kernels are built for
 
-struct RowDesc {
-    uint64_t lo, hi;          // byte range of the row on the packed side
-    uint8_t *other;           // start of the row on the other side, nullptr = skip the row
-};
+// Chunk size for a launch that may move up to room_bytes with n_warps resident warps: aim at
+// eight chunks per warp, a power of two within [kMinChunkBytes, kMaxChunkBytes].
+static inline uint32_t pick_chunk_bytes(uint64_t room_bytes, uint64_t n_warps) {
+    uint64_t want = room_bytes / (n_warps * 8 + 1);
+    uint32_t c = kMinChunkBytes;
+    while (c < kMaxChunkBytes && c < want) c <<= 1;
+    return c;
+}
 
 // Largest i in [0, rows) with cu[i] <= x (the row holding element x, rows of length zero
-// skipped); 0 when even cu[0] > x.  Every thread of the CTA must call it; all get the answer.
-__device__ __forceinline__ uint32_t block_find_row(const int32_t *cu, uint32_t rows, int64_t x) {
+// skipped); 0 when even cu[0] > x.  Warp-cooperative; all lanes get the answer.
+__device__ __forceinline__ uint32_t warp_find_row(const int32_t *cu, uint32_t rows, int64_t x, uint32_t lane) {
     uint32_t lo = 0, len = rows;
     while (len > 1) {
-        const uint32_t stride = (len + kSpanThreads - 1) / kSpanThreads;
-        const uint64_t probe = (uint64_t)threadIdx.x * stride;
-        const bool ok = probe < len && (int64_t)cu[lo + probe] <= x;
-        int cnt = __syncthreads_count(ok);          // ok holds for a prefix of the threads
+        const uint32_t stride = (len + 31u) >> 5;
+        const uint64_t probe = (uint64_t)lane * stride;
+        const bool ok = probe < len && (int64_t)__ldg(cu + lo + probe) <= x;
+        uint32_t cnt = __popc(__ballot_sync(kFullMask, ok));     // ok holds for a prefix of the lanes
         if (cnt < 1) cnt = 1;
-        const uint32_t step = (uint32_t)(cnt - 1) * stride;
+        const uint32_t step = (cnt - 1u) * stride;
         lo += step;
         len = min(stride, len - step);
     }
     return lo;
 }
 
-// First descriptor in d[0, n) whose hi exceeds x (hi is non-decreasing); n if none.
-__device__ __forceinline__ uint32_t first_desc_after(const RowDesc *d, uint32_t n, uint64_t x) {
-    uint32_t lo = 0, hi = n;
-    while (lo < hi) {
-        const uint32_t mid = (lo + hi) >> 1;
-        if (d[mid].hi > x) hi = mid; else lo = mid + 1;
-    }
-    return lo;
+__device__ __forceinline__ uint64_t shfl_u64(uint64_t v, uint32_t src) {
+    const uint32_t lo = __shfl_sync(kFullMask, (uint32_t)v, src);
+    const uint32_t hi = __shfl_sync(kFullMask, (uint32_t)(v >> 32), src);
+    return ((uint64_t)hi << 32) | lo;
 }
 
-// Step 3 for one warp: copy the parts of the described rows that fall inside [w_lo, w_hi) of
-// the packed side.  kToPacked: the packed side is the destination (get), else the source (put).
-template <bool kToPacked>
-__device__ __forceinline__ void warp_copy_rows(const RowDesc *d, uint32_t n, uint64_t w_lo, uint64_t w_hi,
-                                               uint8_t *packed, uint32_t esz, uint32_t lane,
-                                               const uint8_t *src_lo, const uint8_t *src_hi) {
-    for (uint32_t r = first_desc_after(d, n, w_lo); r < n; ++r) {
-        const uint64_t rlo = d[r].lo;
-        if (rlo >= w_hi) break;
-        uint8_t *other = d[r].other;
-        if (other == nullptr) continue;
-        const uint64_t lo = max(rlo, w_lo), hi = min(d[r].hi, w_hi);
-        if (hi <= lo) continue;
-        if (kToPacked) warp_copy(packed + lo, other + (lo - rlo), hi - lo, esz, lane, src_lo, src_hi);
-        else warp_copy(other + (lo - rlo), packed + lo, hi - lo, esz, lane, src_lo, src_hi);
+// Steps 2 and 3 for one chunk [b0, b1) of a packed side described by cu[0..rows].
+// resolve(i) returns where row i starts on the other side, or nullptr to skip the row; it is
+// called by one lane per row.  kToPacked: the packed side is the destination (get), else the
+// source (put).
+template <bool kToPacked, typename Resolve>
+__device__ __forceinline__ void warp_copy_chunk(const int32_t *cu, uint32_t rows, uint64_t b0, uint64_t b1,
+                                                uint8_t *packed, uint32_t esz, uint32_t lane,
+                                                const uint8_t *src_lo, const uint8_t *src_hi, Resolve resolve) {
+    uint32_t r0 = warp_find_row(cu, rows, (int64_t)(b0 / esz), lane);
+    for (;;) {
+        const uint32_t i = r0 + lane;
+        bool in = false;
+        uint64_t rlo = 0, rhi = 0;
+        uint8_t *other = nullptr;
+        if (i < rows) {
+            const int64_t c0 = __ldg(cu + i);
+            rlo = (uint64_t)c0 * esz;
+            in = c0 >= 0 && rlo < b1;
+            if (in) {
+                const int64_t c1 = __ldg(cu + i + 1);
+                rhi = c1 > c0 ? (uint64_t)c1 * esz : rlo;
+                other = rhi > b0 ? resolve(i, c0, c1) : nullptr;
+            }
+        }
+        // rows inside the chunk form a prefix of the lanes
+        const uint32_t n_rows = (uint32_t)__ffs(~__ballot_sync(kFullMask, in)) - 1u;   // 32 when all lanes are in
+        const uint32_t n_here = n_rows > 32u ? 32u : n_rows;
+        for (uint32_t r = 0; r < n_here; ++r) {
+            const uint64_t lo_r = shfl_u64(rlo, r), hi_r = shfl_u64(rhi, r);
+            uint8_t *o = reinterpret_cast<uint8_t *>(shfl_u64(reinterpret_cast<uint64_t>(other), r));
+            const uint64_t lo = max(lo_r, b0), hi = min(hi_r, b1);
+            if (o == nullptr || hi <= lo) continue;
+            if (kToPacked) warp_copy(packed + lo, o + (lo - lo_r), hi - lo, esz, lane, src_lo, src_hi);
+            else warp_copy(o + (lo - lo_r), packed + lo, hi - lo, esz, lane, src_lo, src_hi);
+        }
+        if (n_here < 32u) break;
+        r0 += 32u;
     }
 }
 

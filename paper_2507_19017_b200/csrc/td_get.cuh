@@ -346,8 +346,8 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
 
 // ---------------------------------------------------------------------------------------------
 // Gather.  Persistent grid.  Every (request, column) pair is a job; the output space of each
-// job is cut into spans of kSpanBytes and CTAs stride over the spans of all jobs, so the work
-// is balanced over bytes whatever the mix of requests and row lengths (see "Span copy" in
+// job is cut into chunks and warps stride over the chunks of all jobs, so the work is balanced
+// over bytes whatever the mix of requests and row lengths (see "Chunked ragged copy" in
 // td_device.cuh).
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint64_t job_bytes(const DockView &dv, const GetReq &rq, uint32_t k) {
@@ -361,25 +361,24 @@ __device__ __forceinline__ uint64_t job_bytes(const DockView &dv, const GetReq &
     return n_s * (uint64_t)(cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to) * esz;
 }
 
-__global__ void __launch_bounds__(kSpanThreads, 4)
+__global__ void __launch_bounds__(kCopyThreads, 6)
 get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
-                  const GetReq *reqs_dev, const uint32_t n_req) {
+                  const GetReq *reqs_dev, const uint32_t n_req, const uint32_t chunk_bytes) {
     const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
-    __shared__ RowDesc desc[kSpanThreads];
-    __shared__ uint32_t job_end[kMaxJobs];          // inclusive prefix of spans, jobs = [request][column]
-    __shared__ uint32_t s_wsum[kSpanWarps];
+    __shared__ uint32_t job_end[kMaxJobs];          // inclusive prefix of chunks, jobs = [request][column]
+    __shared__ uint32_t s_wsum[kCopyWarps];
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t ncol = dv.ncol;
     const uint32_t njobs = n_req * ncol;
 
     // job table: each thread sizes a contiguous run of jobs, then one block scan
     {
-        const uint32_t per = (njobs + kSpanThreads - 1) / kSpanThreads;
-        const uint32_t j0 = tid * per, j1 = min(j0 + per, njobs);
+        const uint32_t per = (njobs + kCopyThreads - 1) / kCopyThreads;
+        const uint32_t j0 = min(tid * per, njobs), j1 = min(j0 + per, njobs);
         uint32_t local = 0;
         for (uint32_t j = j0; j < j1; ++j) {
             const uint64_t b = job_bytes(dv, reqs[j / ncol], j % ncol);
-            local += (uint32_t)((b + kSpanBytes - 1) / kSpanBytes);
+            local += (uint32_t)((b + chunk_bytes - 1) / chunk_bytes);
             job_end[j] = local;                       // inclusive within the thread's run
         }
         uint32_t inc = local;
@@ -395,12 +394,14 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
         for (uint32_t j = j0; j < j1; ++j) job_end[j] += before;
         __syncthreads();
     }
-    const uint32_t n_spans = njobs ? job_end[njobs - 1] : 0;
+    const uint32_t n_chunks = njobs ? job_end[njobs - 1] : 0;
+    const uint32_t warp0 = blockIdx.x * kCopyWarps + warp;
+    const uint32_t stride = gridDim.x * kCopyWarps;
 
-    for (uint32_t sp = blockIdx.x; sp < n_spans; sp += gridDim.x) {
-        // job of this span: first j with job_end[j] > sp
+    for (uint32_t ch = warp0; ch < n_chunks; ch += stride) {
+        // job of this chunk: first j with job_end[j] > ch
         uint32_t jlo = 0, jhi = njobs - 1;
-        while (jlo < jhi) { const uint32_t m = (jlo + jhi) >> 1; if (job_end[m] > sp) jhi = m; else jlo = m + 1; }
+        while (jlo < jhi) { const uint32_t m = (jlo + jhi) >> 1; if (job_end[m] > ch) jhi = m; else jlo = m + 1; }
         const uint32_t j = jlo;
         const GetReq &rq = reqs[j / ncol];
         const td_get_out &out = rq.out;
@@ -409,12 +410,13 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
         const uint32_t n_s = out.result->n_samples;
         uint8_t *dst0 = reinterpret_cast<uint8_t *>(out.col[k]);
         uint8_t *base = dv.colbase[k];
-        const uint64_t b0 = (uint64_t)(sp - (j ? job_end[j - 1] : 0)) * kSpanBytes;
+        const int32_t *indices = out.indices;
+        const uint64_t b0 = (uint64_t)(ch - (j ? job_end[j - 1] : 0)) * chunk_bytes;
 
         if (cls == TD_SCALAR) {
-            const uint64_t e0 = b0 / esz, e1 = min((b0 + kSpanBytes) / esz, (uint64_t)n_s);
-            for (uint64_t e = e0 + tid; e < e1; e += kSpanThreads) {
-                const int32_t s = out.indices[e];
+            const uint64_t e0 = b0 / esz, e1 = min((b0 + chunk_bytes) / esz, (uint64_t)n_s);
+            for (uint64_t e = e0 + lane; e < e1; e += 32) {
+                const int32_t s = __ldg(indices + e);
                 if (esz == 4) reinterpret_cast<uint32_t *>(dst0)[e] = reinterpret_cast<const uint32_t *>(base)[s];
                 else reinterpret_cast<uint16_t *>(dst0)[e] = reinterpret_cast<const uint16_t *>(base)[s];
             }
@@ -423,56 +425,44 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
         const uint64_t cap = dv.cap[cls];
         const uint8_t *src_lo = base, *src_hi = base + (uint64_t)dv.S * cap * esz;
         const long long *offt = dv.off[cls];
-        const bool packed = out.mode == TD_PACKED;
-        const int32_t *cu = cls == TD_PROMPT ? out.cu_prompt : out.cu_response;
-        const uint32_t W = cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to;
-        const uint64_t row_bytes = (uint64_t)W * esz;
-        const uint64_t total = packed ? (uint64_t)(int64_t)cu[n_s] * esz : (uint64_t)n_s * row_bytes;
-        const uint64_t b1 = min(b0 + (uint64_t)kSpanBytes, total);
-        const uint64_t w_lo = b0 + (uint64_t)warp * kWarpBytes;
-        const uint64_t w_hi = min(w_lo + (uint64_t)kWarpBytes, b1);
-
-        uint32_t r0 = packed ? block_find_row(cu, n_s, (int64_t)(b0 / esz)) : (uint32_t)(b0 / row_bytes);
-        for (;;) {
-            const uint32_t i = r0 + tid;
-            bool in_span = false;
-            RowDesc d; d.lo = 0; d.hi = 0; d.other = nullptr;
-            if (i < n_s) {
-                const uint64_t rlo = packed ? (uint64_t)(int64_t)cu[i] * esz : (uint64_t)i * row_bytes;
-                in_span = rlo < b1;
-                if (in_span) {
-                    const uint32_t s = (uint32_t)out.indices[i];
-                    uint64_t len_b;
-                    if (packed) len_b = (uint64_t)(int64_t)cu[i + 1] * esz - rlo;
-                    else { const int32_t l = dv.len[cls][s]; len_b = (uint64_t)(l > 0 ? l : 0) * esz; }
-                    const long long off = offt[s];
-                    d.lo = rlo; d.hi = rlo + len_b;
-                    d.other = off >= 0 ? base + ((uint64_t)shard_of(dv, s) * cap + (uint64_t)off) * esz : nullptr;
+        auto row_src = [&](uint32_t i) -> uint8_t * {
+            const uint32_t s = (uint32_t)__ldg(indices + i);
+            const long long off = offt[s];
+            return off >= 0 ? base + ((uint64_t)shard_of(dv, s) * cap + (uint64_t)off) * esz : nullptr;
+        };
+        if (out.mode == TD_PACKED) {
+            const int32_t *cu = cls == TD_PROMPT ? out.cu_prompt : out.cu_response;
+            const uint64_t total = (uint64_t)(int64_t)__ldg(cu + n_s) * esz;
+            const uint64_t b1 = min(b0 + (uint64_t)chunk_bytes, total);
+            warp_copy_chunk<true>(cu, n_s, b0, b1, dst0, esz, lane, src_lo, src_hi,
+                                  [&](uint32_t i, int64_t, int64_t) -> uint8_t * { return row_src(i); });
+        } else {
+            // fixed-width rows: payload part, then the pad pattern up to the row's end
+            const uint32_t W = cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to;
+            const uint64_t row_bytes = (uint64_t)W * esz;
+            const uint64_t b1 = min(b0 + (uint64_t)chunk_bytes, (uint64_t)n_s * row_bytes);
+            const int32_t *lent = dv.len[cls];
+            for (uint64_t r0 = b0 / row_bytes; r0 < n_s && r0 * row_bytes < b1; r0 += 32) {
+                const uint64_t i = r0 + lane;
+                uint64_t valid = 0;
+                uint8_t *src = nullptr;
+                if (i < n_s && i * row_bytes < b1) {
+                    const int32_t l = lent[(uint32_t)__ldg(indices + i)];
+                    valid = (uint64_t)(l > 0 ? l : 0) * esz;
+                    src = row_src((uint32_t)i);
+                }
+                for (uint32_t r = 0; r < 32; ++r) {
+                    const uint64_t rlo = (r0 + r) * row_bytes;
+                    if (r0 + r >= n_s || rlo >= b1) break;
+                    const uint64_t valid_hi = rlo + shfl_u64(valid, r);
+                    uint8_t *o = reinterpret_cast<uint8_t *>(shfl_u64(reinterpret_cast<uint64_t>(src), r));
+                    const uint64_t lo = max(rlo, b0), hi = min(rlo + row_bytes, b1);
+                    const uint64_t phi = min(hi, valid_hi);
+                    if (phi > lo && o) warp_copy(dst0 + lo, o + (lo - rlo), phi - lo, esz, lane, src_lo, src_hi);
+                    const uint64_t plo = max(lo, valid_hi);
+                    if (hi > plo) warp_fill(dst0 + plo, hi - plo, dv.col_pad[k], esz, lane);
                 }
             }
-            desc[tid] = d;
-            const uint32_t n_rows = (uint32_t)__syncthreads_count(in_span);
-            if (w_lo < w_hi) {
-                if (packed) {
-                    warp_copy_rows<true>(desc, n_rows, w_lo, w_hi, dst0, esz, lane, src_lo, src_hi);
-                } else {
-                    // fixed-width rows: payload part, then the pad pattern up to the row's end
-                    for (uint32_t r = (uint32_t)(max(w_lo / row_bytes, (uint64_t)r0) - r0); r < n_rows; ++r) {
-                        const uint64_t rlo = desc[r].lo;
-                        if (rlo >= w_hi) break;
-                        const uint64_t valid_hi = desc[r].hi, rhi = rlo + row_bytes;
-                        const uint64_t lo = max(rlo, w_lo), hi = min(rhi, w_hi);
-                        const uint64_t phi = min(hi, valid_hi);
-                        if (phi > lo && desc[r].other)
-                            warp_copy(dst0 + lo, desc[r].other + (lo - rlo), phi - lo, esz, lane, src_lo, src_hi);
-                        const uint64_t plo = max(lo, valid_hi);
-                        if (hi > plo) warp_fill(dst0 + plo, hi - plo, dv.col_pad[k], esz, lane);
-                    }
-                }
-            }
-            __syncthreads();
-            if (n_rows < kSpanThreads) break;
-            r0 += kSpanThreads;
         }
     }
 }

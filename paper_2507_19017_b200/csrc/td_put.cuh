@@ -177,78 +177,52 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
     }
 }
 
-// Scatter.  The packed sources of the call's ragged items are cut into spans of kSpanBytes, so
-// that work is balanced over tokens rather than samples; CTAs stride over the spans of all
-// items (see "Span copy" in td_device.cuh).
-__global__ void __launch_bounds__(kSpanThreads, 4)
-put_scatter_kernel(const DockView dv, const PutBatch batch) {
-    __shared__ RowDesc desc[kSpanThreads];
-    __shared__ uint64_t item_end[kMaxPutItems];       // inclusive prefix of spans per item
-    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+// Scatter.  The packed sources of the call's ragged items are cut into chunks, so that work is
+// balanced over tokens rather than samples; warps stride over the chunks of all items (see
+// "Chunked ragged copy" in td_device.cuh).
+__global__ void __launch_bounds__(kCopyThreads, 6)
+put_scatter_kernel(const DockView dv, const PutBatch batch, const uint32_t chunk_bytes) {
+    __shared__ uint64_t item_end[kMaxPutItems];       // inclusive prefix of chunks per item
+    const uint32_t tid = threadIdx.x, lane = tid & 31;
 
     if (tid == 0) {
         uint64_t acc = 0;
         for (uint32_t it = 0; it < batch.n_items; ++it) {
             const PutArgs &a = batch.item[it];
-            uint64_t spans = 0;
+            uint64_t chunks = 0;
             if (dv.col_cls[a.column] != TD_SCALAR && a.k) {
                 const int64_t tot = a.cu[a.k];
                 if (tot > 0 && (uint64_t)tot <= a.data_elems)
-                    spans = ((uint64_t)tot * dv.col_esz[a.column] + kSpanBytes - 1) / kSpanBytes;
+                    chunks = ((uint64_t)tot * dv.col_esz[a.column] + chunk_bytes - 1) / chunk_bytes;
             }
-            acc += spans;
+            acc += chunks;
             item_end[it] = acc;
         }
     }
     __syncthreads();
-    const uint64_t n_spans = item_end[batch.n_items - 1];
+    const uint64_t n_chunks = item_end[batch.n_items - 1];
+    const uint64_t warp0 = (uint64_t)blockIdx.x * kCopyWarps + (tid >> 5);
+    const uint64_t stride = (uint64_t)gridDim.x * kCopyWarps;
 
-    for (uint64_t sp = blockIdx.x; sp < n_spans; sp += gridDim.x) {
+    for (uint64_t ch = warp0; ch < n_chunks; ch += stride) {
         uint32_t it = 0;
-        while (item_end[it] <= sp) ++it;
+        while (item_end[it] <= ch) ++it;
         const PutArgs &a = batch.item[it];
         const uint32_t L = dv.col_cls[a.column];
         const uint32_t esz = dv.col_esz[a.column];
         const uint32_t bit = 1u << a.column;
-        const uint64_t total_bytes = (uint64_t)(int64_t)a.cu[a.k] * esz;
-        const uint64_t b0 = (sp - (it ? item_end[it - 1] : 0)) * kSpanBytes;
-        const uint64_t b1 = min(b0 + (uint64_t)kSpanBytes, total_bytes);
-        const uint8_t *src_lo = a.data, *src_hi = a.data + a.data_elems * esz;
+        const uint64_t total_bytes = (uint64_t)(int64_t)__ldg(a.cu + a.k) * esz;
+        const uint64_t b0 = (ch - (it ? item_end[it - 1] : 0)) * chunk_bytes;
+        const uint64_t b1 = min(b0 + (uint64_t)chunk_bytes, total_bytes);
         uint8_t *arena = dv.colbase[a.column];
         const uint64_t cap = dv.cap[L];
-        const uint64_t w_lo = b0 + (uint64_t)warp * kWarpBytes;
-        const uint64_t w_hi = min(w_lo + (uint64_t)kWarpBytes, b1);
-
-        uint32_t r0 = block_find_row(a.cu, a.k, (int64_t)(b0 / esz));
-        for (;;) {
-            // one thread per row: where does it go?
-            const uint32_t i = r0 + tid;
-            bool in_span = false;
-            RowDesc d; d.lo = 0; d.hi = 0; d.other = nullptr;      // never leave a stale descriptor
-            if (i < a.k) {
-                const int64_t c0 = a.cu[i];
-                const uint64_t rlo = (uint64_t)c0 * esz;
-                in_span = c0 >= 0 && rlo < b1;
-                if (in_span) {
-                    d.lo = rlo; d.hi = rlo;
-                    int32_t s; int64_t l; long long off;
-                    if (put_entry_live(dv, a, i, L, bit, s, l, off)) {
-                        d.hi = rlo + (uint64_t)l * esz;
-                        d.other = arena + ((uint64_t)shard_of(dv, (uint32_t)s) * cap + (uint64_t)off) * esz;
-                    } else {
-                        const int64_t c1 = a.cu[i + 1];
-                        d.hi = c1 > c0 ? (uint64_t)c1 * esz : rlo;   // keeps hi monotone
-                    }
-                }
-            }
-            desc[tid] = d;
-            const uint32_t n_rows = (uint32_t)__syncthreads_count(in_span);
-            if (w_lo < w_hi)
-                warp_copy_rows<false>(desc, n_rows, w_lo, w_hi, const_cast<uint8_t *>(a.data), esz, lane, src_lo, src_hi);
-            __syncthreads();                       // desc is reused
-            if (n_rows < kSpanThreads) break;
-            r0 += kSpanThreads;
-        }
+        warp_copy_chunk<false>(a.cu, a.k, b0, b1, const_cast<uint8_t *>(a.data), esz, lane,
+                               a.data, a.data + a.data_elems * esz,
+                               [&](uint32_t i, int64_t, int64_t) -> uint8_t * {
+                                   int32_t s; int64_t l; long long off;
+                                   if (!put_entry_live(dv, a, i, L, bit, s, l, off)) return nullptr;
+                                   return arena + ((uint64_t)shard_of(dv, (uint32_t)s) * cap + (uint64_t)off) * esz;
+                               });
     }
 }
 
