@@ -55,7 +55,7 @@ def load_peaks():
 
 # --------------------------------------------------------------------------- clocks
 class ClockSampler:
-    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+    QUERY = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
@@ -66,7 +66,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.uuid}", f"--query-gpu={self.QUERY}",
-                 "--format=csv,noheader,nounits", "-lms", "100"],
+                 "--format=csv,noheader,nounits", "-lms", "20"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
             self.thread = threading.Thread(target=self._read, daemon=True)
             self.thread.start()
@@ -75,31 +75,45 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.time(), line.strip()))
 
-    def stop(self):
+    def stop(self, t_begin: float, t_end: float):
+        """Summary of the samples taken inside [t_begin, t_end] (the timed region); when the
+        region was too short to catch three, of everything sampled since start (warm-up and
+        timed region, both under the same load)."""
         if not self.proc:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
-        sm, mx, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
-            f = [x.strip() for x in ln.split(",")]
-            if len(f) < 9:
-                continue
-            try:
-                sm.append(float(f[1])); mx.append(float(f[2]))
-            except ValueError:
-                continue
-            for nm, val in zip(names, f[5:9]):
-                if val.lower().startswith("active"):
-                    reasons.add(nm)
-        return {"sm_mhz": statistics.median(sm) if sm else None,
-                "sm_max_mhz": max(mx) if mx else None, "samples": len(sm), "reasons": sorted(reasons)}
+
+        def summarise(lines):
+            sm, mx, reasons = [], [], set()
+            for _t, ln in lines:
+                f = [x.strip() for x in ln.split(",")]
+                if len(f) < 9:
+                    continue
+                try:
+                    sm.append(float(f[1])); mx.append(float(f[2]))
+                except ValueError:
+                    continue
+                for nm, val in zip(names, f[5:9]):
+                    if val.lower().startswith("active"):
+                        reasons.add(nm)
+            return sm, mx, reasons
+
+        inside = [(t, ln) for t, ln in self.lines if t_begin <= t <= t_end + 0.03]
+        window = "timed region"
+        sm, mx, reasons = summarise(inside)
+        if len(sm) < 3:
+            window = "warm-up and timed region"
+            sm, mx, reasons = summarise(self.lines)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "window": window, "reasons": sorted(reasons)}
 
 
 def gpu_id_for_smi(torch, local_rank: int) -> str:
@@ -349,6 +363,8 @@ def main():
     peak, peak_kind = load_peaks()
     put_bytes, put_ragged_bytes, get_bytes = algorithmic_bytes(w)
 
+    sampler = ClockSampler(gpu_id_for_smi(torch, local_rank))
+    sampler.start()
     for _ in range(max(args.warmup, 3)):
         step.timed_step()
     served_s, served_t = step.served()
@@ -359,17 +375,19 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    sampler = ClockSampler(gpu_id_for_smi(torch, local_rank))
     barrier()
-    sampler.start()
+    t_begin = time.time()
+    torch.cuda.cudart().cudaProfilerStart()        # lets a profiler capture the timed region only
     launches0 = step.dock.launch_count()
     put_ms, drain_ms = [], []
     for _ in range(args.steps):
         a, b = step.timed_step()
         put_ms.append(a); drain_ms.append(b)
     barrier()
+    torch.cuda.cudart().cudaProfilerStop()
+    t_end = time.time()
     launches = step.dock.launch_count() - launches0
-    clocks = sampler.stop()
+    clocks = sampler.stop(t_begin, t_end)
 
     mean_put, mean_drain = sum(put_ms) / len(put_ms), sum(drain_ms) / len(drain_ms)
     ms_per_step = mean_put + mean_drain

@@ -59,7 +59,8 @@ enum {
     TD_ERR_ARENA_FULL       = 1u << 3,  /* put: shard arena has no room for the row             */
     TD_ERR_OUT_TRUNCATED    = 1u << 4,  /* get: stopped before a group that would not fit       */
     TD_ERR_LOOKBACK_TIMEOUT = 1u << 5,  /* get: a scan tile gave up waiting; nothing returned   */
-    TD_ERR_BAD_LENGTH       = 1u << 6   /* put: cu not monotone or beyond data_elems            */
+    TD_ERR_BAD_LENGTH       = 1u << 6,  /* put: cu not monotone or beyond data_elems            */
+    TD_ERR_COPY_TIMEOUT     = 1u << 7   /* a staged copy did not land in time; plain loads used  */
 };
 
 typedef struct {

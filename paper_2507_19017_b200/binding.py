@@ -19,7 +19,7 @@ PACKED, PADDED = 0, 1
 F_ADVANTAGE = 1
 OK, EINVAL, EWORKSPACE, ECUDA = 0, -1, -2, -3
 ERR_OOB_INDEX, ERR_DUP_PUT, ERR_LEN_MISMATCH, ERR_ARENA_FULL = 1, 2, 4, 8
-ERR_OUT_TRUNCATED, ERR_LOOKBACK_TIMEOUT, ERR_BAD_LENGTH = 16, 32, 64
+ERR_OUT_TRUNCATED, ERR_LOOKBACK_TIMEOUT, ERR_BAD_LENGTH, ERR_COPY_TIMEOUT = 16, 32, 64, 128
 
 DTYPE_TAG = {"i32": I32, "f32": F32, "bf16": BF16}
 CLASS_TAG = {"scalar": SCALAR, "prompt": PROMPT, "response": RESPONSE}

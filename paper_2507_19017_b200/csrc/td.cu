@@ -36,6 +36,12 @@ std::atomic<uint32_t> g_seq{1};     // launch sequence numbers for scan scratch,
 inline size_t align_up_sz(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline uint32_t esize_of(int32_t dtype) { return dtype == TD_BF16 ? 2u : 4u; }
 
+// Dynamic shared memory of the copy kernels: the warps' stages and mbarriers, then (gather) the
+// block-scan scratch and the job table.
+constexpr size_t kStageSmem = (size_t)kCopyWarps * kStages * kStageBytes + (size_t)kCopyWarps * kStages * 8;
+size_t scatter_smem_bytes() { return kStageSmem; }
+size_t gather_smem_bytes(uint32_t njobs) { return kStageSmem + (size_t)kCopyWarps * 8 + (size_t)njobs * 8; }
+
 struct Layout {
     size_t status, len[3], off[3], cursor[3], claim, consumed, errword, counters, col[kMaxColumns], total;
     uint32_t claim_words, consumed_words;
@@ -156,6 +162,12 @@ int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **o
         cudaFuncSetAttribute(put_alloc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)alloc_smem) != cudaSuccess)
         return TD_ECUDA;
 
+    if (cudaFuncSetAttribute(put_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)scatter_smem_bytes()) != cudaSuccess ||
+        cudaFuncSetAttribute(get_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)gather_smem_bytes(kMaxJobs)) != cudaSuccess)
+        return TD_ECUDA;
+
     td_dock *d = new (std::nothrow) td_dock();
     if (!d) return TD_EINVAL;
     d->cfg = *cfg; d->cfg.columns = nullptr; d->cfg.consumers = nullptr;
@@ -168,6 +180,8 @@ int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **o
     v.G = cfg->n_prompts; v.N = cfg->n_per_group; v.S = cfg->n_shards; v.n = v.G * v.N;
     v.ncol = cfg->n_columns; v.ncons = cfg->n_consumers;
     v.prompts_per_shard = v.G / v.S;
+    v.div_shard = make_fastdiv(v.N * v.prompts_per_shard);
+    v.div_ncol = make_fastdiv(v.ncol);
     v.reward_col = cfg->reward_column;
     v.claim_words = L.claim_words; v.consumed_words = L.consumed_words;
     v.spin_limit = 1u << 20;
@@ -222,14 +236,13 @@ int td_reset(td_dock *d, void *stream) {
 
 namespace {
 
-// Grid and chunk size of a copy launch that may move up to room_bytes on the packed side.
-uint32_t copy_grid(const td_dock *d, uint64_t room_bytes, uint32_t *chunk_bytes) {
+// Grid of a copy launch that may move up to room_bytes on the packed side: one resident wave
+// at most, fewer CTAs when there is less than a minimum chunk per warp.
+uint32_t copy_grid(const td_dock *d, uint64_t room_bytes) {
     const uint64_t max_blocks = (uint64_t)d->sm_count * kCopyBlocksPerSM;
-    const uint32_t chunk = pick_chunk_bytes(room_bytes, max_blocks * kCopyWarps);
-    uint64_t blocks = (room_bytes / chunk + kCopyWarps) / kCopyWarps;
+    uint64_t blocks = (room_bytes / kMinChunkBytes + kCopyWarps) / kCopyWarps;
     if (blocks > max_blocks) blocks = max_blocks;
     if (blocks == 0) blocks = 1;
-    *chunk_bytes = chunk;
     return (uint32_t)blocks;
 }
 
@@ -248,9 +261,8 @@ int put_group(td_dock *d, const PutBatch &b, cudaStream_t st) {
     if (ragged_bytes) {
         if (launch(d, put_alloc_kernel, dim3(1), dim3(kAllocThreads), put_alloc_smem_bytes(v.S), st, v, b) != cudaSuccess)
             return TD_ECUDA;
-        uint32_t chunk = 0;
-        const uint32_t blocks = copy_grid(d, ragged_bytes, &chunk);
-        if (launch_timed(d, 0, put_scatter_kernel, dim3(blocks), dim3(kCopyThreads), 0, st, v, b, chunk) != cudaSuccess)
+        if (launch_timed(d, 0, put_scatter_kernel, dim3(copy_grid(d, ragged_bytes)), dim3(kCopyThreads),
+                         scatter_smem_bytes(), st, v, b) != cudaSuccess)
             return TD_ECUDA;
     }
     if (launch(d, put_publish_kernel, dim3((uint32_t)((entries + 255) / 256)), dim3(256), 0, st, v, b) != cudaSuccess)
@@ -349,10 +361,9 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     if (launch(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
-    uint32_t chunk = 0;
-    const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out), &chunk);
-    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), 0, st, v, one,
-                     (const GetReq *)nullptr, 1u, chunk) != cudaSuccess) return TD_ECUDA;
+    const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
+    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(v.ncol), st, v, one,
+                     (const GetReq *)nullptr, 1u) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 
@@ -449,10 +460,9 @@ int td_get_many(td_dock *d, td_plan *p, void *stream) {
                (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
     if (launch(d, get_finalize_kernel, dim3(p->n_req), dim3(kFinThreads), 0, st, v, none, (const GetReq *)p->d_reqs,
                (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
-    uint32_t chunk = 0;
-    const uint32_t blocks = copy_grid(d, p->room_bytes, &chunk);
-    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), 0, st, v, none,
-                     (const GetReq *)p->d_reqs, p->n_req, chunk) != cudaSuccess) return TD_ECUDA;
+    if (launch_timed(d, 1, get_gather_kernel, dim3(copy_grid(d, p->room_bytes)), dim3(kCopyThreads),
+                     gather_smem_bytes(p->n_req * v.ncol), st, v, none,
+                     (const GetReq *)p->d_reqs, p->n_req) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 

@@ -21,12 +21,30 @@ enum : int {
     CNT_TOTAL = 112
 };
 
+// Division by a run-time constant d through a multiply and a shift, exact for n < 2^31:
+// n / d = (umulhi(n, mul) + n) >> shr with shr = ceil(log2 d), mul = floor(2^32 (2^shr - d) / d) + 1
+// (mul = 0 when d is a power of two).
+struct FastDiv {
+    uint32_t mul, shr;
+};
+static inline FastDiv make_fastdiv(uint32_t d) {
+    uint32_t l = 0;
+    while ((1ull << l) < d) ++l;
+    const uint64_t m = (1ull << l) == d ? 0 : ((1ull << 32) * ((1ull << l) - d)) / d + 1;
+    return FastDiv{(uint32_t)m, l};
+}
+__device__ __forceinline__ uint32_t fast_div(uint32_t n, FastDiv f) {
+    return (__umulhi(n, f.mul) + n) >> f.shr;
+}
+
 // Everything a kernel needs to know about a dock; passed by value (constant bank).
 struct DockView {
     uint32_t G, N, S, n;
     uint32_t ncol, ncons;
     uint32_t prompts_per_shard;
     uint32_t reward_col;
+    FastDiv  div_shard;                     // by samples per shard = N * prompts_per_shard
+    FastDiv  div_ncol;                      // by ncol
     uint32_t claim_words, consumed_words;   // words per consumer
     uint32_t spin_limit;                    // polls before a look-back wait gives up
     uint32_t pad0;
@@ -49,8 +67,9 @@ struct DockView {
     uint8_t  col_cls[kMaxColumns];
 };
 
+// Warehouses hold contiguous blocks of whole prompts: shard(s) = (s / N) / (G / S).
 __device__ __forceinline__ uint32_t shard_of(const DockView &dv, uint32_t s) {
-    return (s / dv.N) / dv.prompts_per_shard;
+    return fast_div(s, dv.div_shard);
 }
 
 __device__ __forceinline__ uint64_t align_row(uint64_t elems) {
@@ -95,7 +114,12 @@ __device__ __forceinline__ void copy_elems(uint8_t *dst, const uint8_t *src, uin
     }
 }
 
-__device__ __forceinline__ uint4 ld_stream(const uint4 *p) { return __ldcs(p); }
+// kSmem: the source is a shared-memory stage (plain load); else global memory read once (streaming load)
+template <bool kSmem>
+__device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
+    if (kSmem) return *p;
+    return __ldcs(p);
+}
 __device__ __forceinline__ void st_stream(uint4 *p, uint4 v) { __stcs(p, v); }
 
 // 16 source bytes starting `delta` bytes into the 32-byte window (a, b); delta in 2..14, even.
@@ -124,7 +148,7 @@ __device__ __forceinline__ uint4 load_window_slow(const uint8_t *p, uint32_t esz
     return r;
 }
 
-template <int WSH>
+template <int WSH, bool kSmem>
 __device__ __forceinline__ void copy_body_shifted(uint4 *dst, const uint8_t *src, uint32_t nvec,
                                                   uint32_t delta, uint32_t esz, uint32_t lane,
                                                   const uint8_t *src_lo, const uint8_t *src_hi) {
@@ -142,17 +166,18 @@ __device__ __forceinline__ void copy_body_shifted(uint4 *dst, const uint8_t *src
     if (v_hi <= v_lo) return;
     uint32_t v = v_lo + lane;
     for (; v + 32 < v_hi; v += 64) {
-        uint4 a0 = ld_stream(S + v),      b0 = ld_stream(S + v + 1);
-        uint4 a1 = ld_stream(S + v + 32), b1 = ld_stream(S + v + 33);
+        uint4 a0 = ld_stream<kSmem>(S + v),      b0 = ld_stream<kSmem>(S + v + 1);
+        uint4 a1 = ld_stream<kSmem>(S + v + 32), b1 = ld_stream<kSmem>(S + v + 33);
         st_stream(dst + v,      shift_window<WSH>(a0, b0, bsh));
         st_stream(dst + v + 32, shift_window<WSH>(a1, b1, bsh));
     }
     for (; v < v_hi; v += 32) {
-        uint4 a = ld_stream(S + v), b = ld_stream(S + v + 1);
+        uint4 a = ld_stream<kSmem>(S + v), b = ld_stream<kSmem>(S + v + 1);
         st_stream(dst + v, shift_window<WSH>(a, b, bsh));
     }
 }
 
+template <bool kSmem = false>
 __device__ __forceinline__ void warp_copy(uint8_t *dst, const uint8_t *src, uint64_t nbytes,
                                           uint32_t esz, uint32_t lane,
                                           const uint8_t *src_lo, const uint8_t *src_hi) {
@@ -172,18 +197,18 @@ __device__ __forceinline__ void warp_copy(uint8_t *dst, const uint8_t *src, uint
             const uint4 *S = reinterpret_cast<const uint4 *>(src);
             uint32_t v = lane;
             for (; v + 96 < nvec; v += 128) {
-                uint4 a0 = ld_stream(S + v), a1 = ld_stream(S + v + 32);
-                uint4 a2 = ld_stream(S + v + 64), a3 = ld_stream(S + v + 96);
+                uint4 a0 = ld_stream<kSmem>(S + v), a1 = ld_stream<kSmem>(S + v + 32);
+                uint4 a2 = ld_stream<kSmem>(S + v + 64), a3 = ld_stream<kSmem>(S + v + 96);
                 st_stream(D + v, a0); st_stream(D + v + 32, a1);
                 st_stream(D + v + 64, a2); st_stream(D + v + 96, a3);
             }
-            for (; v < nvec; v += 32) st_stream(D + v, ld_stream(S + v));
+            for (; v < nvec; v += 32) st_stream(D + v, ld_stream<kSmem>(S + v));
         } else {
             switch (delta >> 2) {
-                case 0: copy_body_shifted<0>(D, src, nvec, delta, esz, lane, src_lo, src_hi); break;
-                case 1: copy_body_shifted<1>(D, src, nvec, delta, esz, lane, src_lo, src_hi); break;
-                case 2: copy_body_shifted<2>(D, src, nvec, delta, esz, lane, src_lo, src_hi); break;
-                default: copy_body_shifted<3>(D, src, nvec, delta, esz, lane, src_lo, src_hi); break;
+                case 0: copy_body_shifted<0, kSmem>(D, src, nvec, delta, esz, lane, src_lo, src_hi); break;
+                case 1: copy_body_shifted<1, kSmem>(D, src, nvec, delta, esz, lane, src_lo, src_hi); break;
+                case 2: copy_body_shifted<2, kSmem>(D, src, nvec, delta, esz, lane, src_lo, src_hi); break;
+                default: copy_body_shifted<3, kSmem>(D, src, nvec, delta, esz, lane, src_lo, src_hi); break;
             }
         }
     }
@@ -232,16 +257,36 @@ __device__ __forceinline__ void warp_fill(uint8_t *dst, uint64_t nbytes, uint32_
 // --------------------------------------------------------------------------------------------
 constexpr int kCopyThreads = 256;
 constexpr int kCopyWarps = kCopyThreads / 32;
-constexpr uint32_t kMinChunkBytes = 1024, kMaxChunkBytes = 16384;
-constexpr int kCopyBlocksPerSM = 6;          // resident CTAs per SM the copy kernels are built for
+#ifndef TD_COPY_BLOCKS_PER_SM
+#define TD_COPY_BLOCKS_PER_SM 3
+#endif
+#ifndef TD_CHUNK_TARGET_BYTES
+#define TD_CHUNK_TARGET_BYTES 32768
+#endif
+constexpr int kCopyBlocksPerSM = TD_COPY_BLOCKS_PER_SM;      // resident CTAs per SM the copy kernels are built for
+constexpr uint32_t kMinChunkBytes = 1024;                    // a warp is not given less than this
+constexpr uint32_t kChunkTargetBytes = TD_CHUNK_TARGET_BYTES;   // chunk size aimed at when there is plenty of work
 
-// Chunk size for a launch that may move up to room_bytes with n_warps resident warps: aim at
-// eight chunks per warp, a power of two within [kMinChunkBytes, kMaxChunkBytes].
-static inline uint32_t pick_chunk_bytes(uint64_t room_bytes, uint64_t n_warps) {
-    uint64_t want = room_bytes / (n_warps * 8 + 1);
-    uint32_t c = kMinChunkBytes;
-    while (c < kMaxChunkBytes && c < want) c <<= 1;
-    return c;
+// All jobs of a launch (columns of a put, (request, column) pairs of a get) are laid end to end
+// in one logical byte space, each job rounded up to 16 bytes.  The space is cut into chunks of
+// equal size, chosen on the device from the actual total so that every warp of the grid gets
+// the same whole number of chunks: balance over bytes is then exact whatever the mix of jobs
+// and row lengths, and no chunk is left half empty at a job's end.
+struct ChunkPlan {
+    uint64_t chunk_bytes;    // multiple of 16
+    uint64_t n_chunks;
+};
+__device__ __forceinline__ ChunkPlan plan_chunks(uint64_t total_bytes, uint64_t n_warps) {
+    ChunkPlan p;
+    const uint64_t per_warp = (total_bytes + n_warps - 1) / n_warps;
+    uint64_t rounds = (per_warp + kChunkTargetBytes / 2) / kChunkTargetBytes;
+    if (rounds < 1) rounds = 1;
+    uint64_t c = (total_bytes + n_warps * rounds - 1) / (n_warps * rounds);
+    c = (c + 15) & ~uint64_t(15);
+    if (c < kMinChunkBytes) c = kMinChunkBytes;
+    p.chunk_bytes = c;
+    p.n_chunks = (total_bytes + c - 1) / c;
+    return p;
 }
 
 // Largest i in [0, rows) with cu[i] <= x (the row holding element x, rows of length zero
@@ -267,6 +312,128 @@ __device__ __forceinline__ uint64_t shfl_u64(uint64_t v, uint32_t src) {
     return ((uint64_t)hi << 32) | lo;
 }
 
+__device__ __forceinline__ uint64_t shfl_up_u64(uint64_t v, int delta) {
+    const uint32_t lo = __shfl_up_sync(kFullMask, (uint32_t)v, delta);
+    const uint32_t hi = __shfl_up_sync(kFullMask, (uint32_t)(v >> 32), delta);
+    return ((uint64_t)hi << 32) | lo;
+}
+
+// --------------------------------------------------------------------------------------------
+// Asynchronous staging.  Each warp owns kStages shared-memory stages and one mbarrier per
+// stage.  A piece of a row is fetched with one bulk asynchronous copy (cp.async.bulk, global to
+// shared, completion counted in bytes on the stage's mbarrier) while the piece fetched before
+// it is written out from the other stage, so a warp keeps up to a stage of loads in flight
+// without holding a single register for them; the bytes in flight per SM are what a ragged
+// copy needs to cover HBM latency.  The bulk copy wants 16-byte aligned addresses and sizes:
+// the source window is widened to the enclosing 16-byte boundaries (rows in an arena start
+// aligned and are padded, so the window stays inside the arena) and the write-out shifts the
+// bytes into place.  Every wait on an mbarrier is bounded; a warp that gives up records the
+// error, falls back to plain loads and still drains its own copy before it returns.
+// --------------------------------------------------------------------------------------------
+constexpr int kStages = 2;
+constexpr uint32_t kStageBytes = 4096;
+constexpr uint32_t kPieceMax = kStageBytes - 16;      // payload of one bulk copy; the aligned window still fits
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile("{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+                 : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ void bulk_global_to_shared(uint32_t dst, const void *src, uint32_t bytes, uint32_t bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
+
+struct WarpPipe {
+    uint8_t *stage;            // this warp's kStages * kStageBytes bytes of shared memory
+    uint32_t bar;              // shared address of this warp's kStages mbarriers
+    uint32_t parity;           // bit s: phase the next wait on stage s looks for
+    uint32_t next;             // stage the next copy goes to
+    uint32_t spin_limit;
+    uint32_t failed;           // a wait ran out: plain loads from here on
+    bool pending;              // a copy is in flight and not yet written out
+    uint8_t *p_dst;
+    const uint8_t *p_src;
+    uint32_t p_n, p_pre, p_stage, p_esz;
+
+    __device__ __forceinline__ void init(uint8_t *stage_mem, unsigned long long *bars, uint32_t lane, uint32_t spin) {
+        stage = stage_mem; bar = smem_u32(bars); parity = 0; next = 0; spin_limit = spin; failed = 0; pending = false;
+        p_dst = nullptr; p_src = nullptr; p_n = p_pre = p_stage = 0; p_esz = 4;
+        if (lane == 0) {
+            for (int s = 0; s < kStages; ++s) mbar_init(bar + 8u * s, 1);
+            fence_mbar_init();
+        }
+        __syncwarp();
+    }
+
+    __device__ __forceinline__ bool wait_stage(uint32_t s) {
+        const uint32_t b = bar + 8u * s;
+        const uint32_t ph = (parity >> s) & 1u;
+        uint32_t polls = 0;
+        bool ok = mbar_try_wait(b, ph);
+        while (!ok && ++polls < spin_limit) { __nanosleep(20); ok = mbar_try_wait(b, ph); }
+        if (ok) parity ^= 1u << s;
+        return ok;
+    }
+
+    // write the pending piece out of its stage; if the wait runs out, copy it with plain loads
+    __device__ __forceinline__ void drain(uint32_t lane) {
+        if (!pending) return;
+        pending = false;
+        if (wait_stage(p_stage)) {
+            const uint8_t *s0 = stage + (size_t)p_stage * kStageBytes;
+            warp_copy<true>(p_dst, s0 + p_pre, p_n, p_esz, lane, s0, s0 + kStageBytes);
+        } else {
+            failed |= 1u | (2u << p_stage);                // stage p_stage still has a copy in flight
+            warp_copy(p_dst, p_src, p_n, p_esz, lane, p_src, p_src + p_n);
+        }
+    }
+
+    // before the warp returns: nothing of its own may still be landing in shared memory
+    __device__ __forceinline__ uint32_t finish(uint32_t lane) {
+        drain(lane);
+        for (uint32_t s = 0; s < (uint32_t)kStages; ++s)
+            if (failed & (2u << s)) wait_stage(s);
+        return failed;
+    }
+
+    // copy n bytes from src to dst through the stages (element-aligned, any length)
+    __device__ __forceinline__ void push(uint8_t *dst, const uint8_t *src, uint64_t n, uint32_t esz, uint32_t lane,
+                                         const uint8_t *src_lo, const uint8_t *src_hi) {
+        while (n > 0) {
+            const uint32_t m = n > kPieceMax ? kPieceMax : (uint32_t)n;
+            const uint32_t pre = (uint32_t)(reinterpret_cast<uintptr_t>(src) & 15u);
+            const uint8_t *win = src - pre;
+            const uint32_t size = (pre + m + 15u) & ~15u;
+            if (failed || m < 64u || win < src_lo || win + size > src_hi) {
+                warp_copy(dst, src, m, esz, lane, src_lo, src_hi);       // short, at a buffer edge, or after a failure
+            } else {
+                const uint32_t s = next;
+                __syncwarp();                                            // every lane is done reading stage s
+                if (lane == 0) {
+                    fence_proxy_async();
+                    mbar_expect_tx(bar + 8u * s, size);
+                    bulk_global_to_shared(smem_u32(stage + (size_t)s * kStageBytes), win, size, bar + 8u * s);
+                }
+                drain(lane);                                             // the piece fetched before this one
+                pending = true; p_dst = dst; p_src = src; p_n = m; p_pre = pre; p_stage = s; p_esz = esz;
+                next = s ^ 1u;
+            }
+            dst += m; src += m; n -= m;
+        }
+    }
+};
+
 // Steps 2 and 3 for one chunk [b0, b1) of a packed side described by cu[0..rows].
 // resolve(i) returns where row i starts on the other side, or nullptr to skip the row; it is
 // called by one lane per row.  kToPacked: the packed side is the destination (get), else the
@@ -274,7 +441,8 @@ __device__ __forceinline__ uint64_t shfl_u64(uint64_t v, uint32_t src) {
 template <bool kToPacked, typename Resolve>
 __device__ __forceinline__ void warp_copy_chunk(const int32_t *cu, uint32_t rows, uint64_t b0, uint64_t b1,
                                                 uint8_t *packed, uint32_t esz, uint32_t lane,
-                                                const uint8_t *src_lo, const uint8_t *src_hi, Resolve resolve) {
+                                                const uint8_t *src_lo, const uint8_t *src_hi, WarpPipe &pipe,
+                                                Resolve resolve) {
     uint32_t r0 = warp_find_row(cu, rows, (int64_t)(b0 / esz), lane);
     for (;;) {
         const uint32_t i = r0 + lane;
@@ -299,8 +467,8 @@ __device__ __forceinline__ void warp_copy_chunk(const int32_t *cu, uint32_t rows
             uint8_t *o = reinterpret_cast<uint8_t *>(shfl_u64(reinterpret_cast<uint64_t>(other), r));
             const uint64_t lo = max(lo_r, b0), hi = min(hi_r, b1);
             if (o == nullptr || hi <= lo) continue;
-            if (kToPacked) warp_copy(packed + lo, o + (lo - lo_r), hi - lo, esz, lane, src_lo, src_hi);
-            else warp_copy(o + (lo - lo_r), packed + lo, hi - lo, esz, lane, src_lo, src_hi);
+            if (kToPacked) pipe.push(packed + lo, o + (lo - lo_r), hi - lo, esz, lane, src_lo, src_hi);
+            else pipe.push(o + (lo - lo_r), packed + lo, hi - lo, esz, lane, src_lo, src_hi);
         }
         if (n_here < 32u) break;
         r0 += 32u;

@@ -361,13 +361,18 @@ __device__ __forceinline__ uint64_t job_bytes(const DockView &dv, const GetReq &
     return n_s * (uint64_t)(cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to) * esz;
 }
 
-__global__ void __launch_bounds__(kCopyThreads, 6)
+__global__ void __launch_bounds__(kCopyThreads, kCopyBlocksPerSM)
 get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
-                  const GetReq *reqs_dev, const uint32_t n_req, const uint32_t chunk_bytes) {
+                  const GetReq *reqs_dev, const uint32_t n_req) {
     const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
-    __shared__ uint32_t job_end[kMaxJobs];          // inclusive prefix of chunks, jobs = [request][column]
-    __shared__ uint32_t s_wsum[kCopyWarps];
+    extern __shared__ __align__(128) uint8_t gather_smem[];
+    uint8_t *stages = gather_smem;                                           // [warps][stages][kStageBytes]
+    unsigned long long *bars = reinterpret_cast<unsigned long long *>(stages + kCopyWarps * kStages * kStageBytes);
+    uint64_t *s_wsum = reinterpret_cast<uint64_t *>(bars + kCopyWarps * kStages);
+    uint64_t *job_end = s_wsum + kCopyWarps;        // [n_req * ncol] inclusive prefix of bytes (16-byte padded)
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    WarpPipe pipe;
+    pipe.init(stages + (size_t)warp * kStages * kStageBytes, bars + warp * kStages, lane, dv.spin_limit);
     const uint32_t ncol = dv.ncol;
     const uint32_t njobs = n_req * ncol;
 
@@ -375,96 +380,106 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
     {
         const uint32_t per = (njobs + kCopyThreads - 1) / kCopyThreads;
         const uint32_t j0 = min(tid * per, njobs), j1 = min(j0 + per, njobs);
-        uint32_t local = 0;
+        uint64_t local = 0;
         for (uint32_t j = j0; j < j1; ++j) {
-            const uint64_t b = job_bytes(dv, reqs[j / ncol], j % ncol);
-            local += (uint32_t)((b + chunk_bytes - 1) / chunk_bytes);
+            const uint32_t q = fast_div(j, dv.div_ncol);
+            local += (job_bytes(dv, reqs[q], j - q * ncol) + 15) & ~uint64_t(15);
             job_end[j] = local;                       // inclusive within the thread's run
         }
-        uint32_t inc = local;
+        uint64_t inc = local;
         #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
-            const uint32_t t = __shfl_up_sync(kFullMask, inc, d);
+            const uint64_t t = shfl_up_u64(inc, d);
             if ((int)lane >= d) inc += t;
         }
         if (lane == 31) s_wsum[warp] = inc;
         __syncthreads();
-        uint32_t before = inc - local;
+        uint64_t before = inc - local;
         for (uint32_t w = 0; w < warp; ++w) before += s_wsum[w];
         for (uint32_t j = j0; j < j1; ++j) job_end[j] += before;
         __syncthreads();
     }
-    const uint32_t n_chunks = njobs ? job_end[njobs - 1] : 0;
-    const uint32_t warp0 = blockIdx.x * kCopyWarps + warp;
-    const uint32_t stride = gridDim.x * kCopyWarps;
+    const uint64_t total_all = njobs ? job_end[njobs - 1] : 0;
+    const uint64_t n_warps = (uint64_t)gridDim.x * kCopyWarps;
+    const ChunkPlan plan = plan_chunks(total_all, n_warps);
+    const uint64_t warp0 = (uint64_t)blockIdx.x * kCopyWarps + warp;
 
-    for (uint32_t ch = warp0; ch < n_chunks; ch += stride) {
-        // job of this chunk: first j with job_end[j] > ch
-        uint32_t jlo = 0, jhi = njobs - 1;
-        while (jlo < jhi) { const uint32_t m = (jlo + jhi) >> 1; if (job_end[m] > ch) jhi = m; else jlo = m + 1; }
-        const uint32_t j = jlo;
-        const GetReq &rq = reqs[j / ncol];
-        const td_get_out &out = rq.out;
-        const uint32_t k = j % ncol;
-        const uint32_t cls = dv.col_cls[k], esz = dv.col_esz[k];
-        const uint32_t n_s = out.result->n_samples;
-        uint8_t *dst0 = reinterpret_cast<uint8_t *>(out.col[k]);
-        uint8_t *base = dv.colbase[k];
-        const int32_t *indices = out.indices;
-        const uint64_t b0 = (uint64_t)(ch - (j ? job_end[j - 1] : 0)) * chunk_bytes;
+    for (uint64_t ch = warp0; ch < plan.n_chunks; ch += n_warps) {
+        uint64_t g0 = ch * plan.chunk_bytes;
+        const uint64_t g1 = min(g0 + plan.chunk_bytes, total_all);
+        // first job that reaches beyond g0
+        uint32_t j = 0;
+        { uint32_t jhi = njobs - 1; while (j < jhi) { const uint32_t m = (j + jhi) >> 1; if (job_end[m] > g0) jhi = m; else j = m + 1; } }
+        for (; g0 < g1; ++j) {
+            const uint64_t start = j ? job_end[j - 1] : 0;
+            const uint64_t b0 = g0 - start;
+            g0 = min(g1, job_end[j]);
+            if (job_end[j] == start) continue;        // empty job
+            const uint32_t q = fast_div(j, dv.div_ncol);
+            const uint32_t k = j - q * ncol;
+            const GetReq &rq = reqs[q];
+            const td_get_out &out = rq.out;
+            const uint32_t cls = dv.col_cls[k], esz = dv.col_esz[k];
+            const uint32_t n_s = out.result->n_samples;
+            uint8_t *dst0 = reinterpret_cast<uint8_t *>(out.col[k]);
+            uint8_t *base = dv.colbase[k];
+            const int32_t *indices = out.indices;
+            const uint64_t b1_raw = g0 - start;          // end of this warp's part of the job, padded space
 
-        if (cls == TD_SCALAR) {
-            const uint64_t e0 = b0 / esz, e1 = min((b0 + chunk_bytes) / esz, (uint64_t)n_s);
-            for (uint64_t e = e0 + lane; e < e1; e += 32) {
-                const int32_t s = __ldg(indices + e);
-                if (esz == 4) reinterpret_cast<uint32_t *>(dst0)[e] = reinterpret_cast<const uint32_t *>(base)[s];
-                else reinterpret_cast<uint16_t *>(dst0)[e] = reinterpret_cast<const uint16_t *>(base)[s];
-            }
-            continue;
-        }
-        const uint64_t cap = dv.cap[cls];
-        const uint8_t *src_lo = base, *src_hi = base + (uint64_t)dv.S * cap * esz;
-        const long long *offt = dv.off[cls];
-        auto row_src = [&](uint32_t i) -> uint8_t * {
-            const uint32_t s = (uint32_t)__ldg(indices + i);
-            const long long off = offt[s];
-            return off >= 0 ? base + ((uint64_t)shard_of(dv, s) * cap + (uint64_t)off) * esz : nullptr;
-        };
-        if (out.mode == TD_PACKED) {
-            const int32_t *cu = cls == TD_PROMPT ? out.cu_prompt : out.cu_response;
-            const uint64_t total = (uint64_t)(int64_t)__ldg(cu + n_s) * esz;
-            const uint64_t b1 = min(b0 + (uint64_t)chunk_bytes, total);
-            warp_copy_chunk<true>(cu, n_s, b0, b1, dst0, esz, lane, src_lo, src_hi,
-                                  [&](uint32_t i, int64_t, int64_t) -> uint8_t * { return row_src(i); });
-        } else {
-            // fixed-width rows: payload part, then the pad pattern up to the row's end
-            const uint32_t W = cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to;
-            const uint64_t row_bytes = (uint64_t)W * esz;
-            const uint64_t b1 = min(b0 + (uint64_t)chunk_bytes, (uint64_t)n_s * row_bytes);
-            const int32_t *lent = dv.len[cls];
-            for (uint64_t r0 = b0 / row_bytes; r0 < n_s && r0 * row_bytes < b1; r0 += 32) {
-                const uint64_t i = r0 + lane;
-                uint64_t valid = 0;
-                uint8_t *src = nullptr;
-                if (i < n_s && i * row_bytes < b1) {
-                    const int32_t l = lent[(uint32_t)__ldg(indices + i)];
-                    valid = (uint64_t)(l > 0 ? l : 0) * esz;
-                    src = row_src((uint32_t)i);
+            if (cls == TD_SCALAR) {
+                const uint64_t e0 = b0 / esz, e1 = min(b1_raw / esz, (uint64_t)n_s);
+                for (uint64_t e = e0 + lane; e < e1; e += 32) {
+                    const int32_t s = __ldg(indices + e);
+                    if (esz == 4) reinterpret_cast<uint32_t *>(dst0)[e] = reinterpret_cast<const uint32_t *>(base)[s];
+                    else reinterpret_cast<uint16_t *>(dst0)[e] = reinterpret_cast<const uint16_t *>(base)[s];
                 }
-                for (uint32_t r = 0; r < 32; ++r) {
-                    const uint64_t rlo = (r0 + r) * row_bytes;
-                    if (r0 + r >= n_s || rlo >= b1) break;
-                    const uint64_t valid_hi = rlo + shfl_u64(valid, r);
-                    uint8_t *o = reinterpret_cast<uint8_t *>(shfl_u64(reinterpret_cast<uint64_t>(src), r));
-                    const uint64_t lo = max(rlo, b0), hi = min(rlo + row_bytes, b1);
-                    const uint64_t phi = min(hi, valid_hi);
-                    if (phi > lo && o) warp_copy(dst0 + lo, o + (lo - rlo), phi - lo, esz, lane, src_lo, src_hi);
-                    const uint64_t plo = max(lo, valid_hi);
-                    if (hi > plo) warp_fill(dst0 + plo, hi - plo, dv.col_pad[k], esz, lane);
+                continue;
+            }
+            const uint64_t cap = dv.cap[cls];
+            const uint8_t *src_lo = base, *src_hi = base + (uint64_t)dv.S * cap * esz;
+            const long long *offt = dv.off[cls];
+            auto row_src = [&](uint32_t i) -> uint8_t * {
+                const uint32_t s = (uint32_t)__ldg(indices + i);
+                const long long off = offt[s];
+                return off >= 0 ? base + ((uint64_t)shard_of(dv, s) * cap + (uint64_t)off) * esz : nullptr;
+            };
+            if (out.mode == TD_PACKED) {
+                const int32_t *cu = cls == TD_PROMPT ? out.cu_prompt : out.cu_response;
+                const uint64_t b1 = min(b1_raw, (uint64_t)(int64_t)__ldg(cu + n_s) * esz);
+                if (b1 <= b0) continue;
+                warp_copy_chunk<true>(cu, n_s, b0, b1, dst0, esz, lane, src_lo, src_hi, pipe,
+                                      [&](uint32_t i, int64_t, int64_t) -> uint8_t * { return row_src(i); });
+            } else {
+                // fixed-width rows: payload part, then the pad pattern up to the row's end
+                const uint32_t W = cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to;
+                const uint64_t row_bytes = (uint64_t)W * esz;
+                const uint64_t b1 = min(b1_raw, (uint64_t)n_s * row_bytes);
+                const int32_t *lent = dv.len[cls];
+                for (uint64_t r0 = b0 / row_bytes; r0 < n_s && r0 * row_bytes < b1; r0 += 32) {
+                    const uint64_t i = r0 + lane;
+                    uint64_t valid = 0;
+                    uint8_t *src = nullptr;
+                    if (i < n_s && i * row_bytes < b1) {
+                        const int32_t l = lent[(uint32_t)__ldg(indices + i)];
+                        valid = (uint64_t)(l > 0 ? l : 0) * esz;
+                        src = row_src((uint32_t)i);
+                    }
+                    for (uint32_t r = 0; r < 32; ++r) {
+                        const uint64_t rlo = (r0 + r) * row_bytes;
+                        if (r0 + r >= n_s || rlo >= b1) break;
+                        const uint64_t valid_hi = rlo + shfl_u64(valid, r);
+                        uint8_t *o = reinterpret_cast<uint8_t *>(shfl_u64(reinterpret_cast<uint64_t>(src), r));
+                        const uint64_t lo = max(rlo, b0), hi = min(rlo + row_bytes, b1);
+                        const uint64_t phi = min(hi, valid_hi);
+                        if (phi > lo && o) pipe.push(dst0 + lo, o + (lo - rlo), phi - lo, esz, lane, src_lo, src_hi);
+                        const uint64_t plo = max(lo, valid_hi);
+                        if (hi > plo) warp_fill(dst0 + plo, hi - plo, dv.col_pad[k], esz, lane);
+                    }
                 }
             }
         }
     }
+    if (pipe.finish(lane) && lane == 0) flag_error(dv, TD_ERR_COPY_TIMEOUT, CNT_TIMEOUT);
 }
 
 // Reset: every table, bitmap and counter back to the empty state; payload untouched.

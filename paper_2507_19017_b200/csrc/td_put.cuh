@@ -177,53 +177,72 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
     }
 }
 
-// Scatter.  The packed sources of the call's ragged items are cut into chunks, so that work is
-// balanced over tokens rather than samples; warps stride over the chunks of all items (see
-// "Chunked ragged copy" in td_device.cuh).
-__global__ void __launch_bounds__(kCopyThreads, 6)
-put_scatter_kernel(const DockView dv, const PutBatch batch, const uint32_t chunk_bytes) {
-    __shared__ uint64_t item_end[kMaxPutItems];       // inclusive prefix of chunks per item
+// Scatter.  The packed sources of the call's ragged items, laid end to end, are cut into equal
+// chunks, so that work is balanced over tokens rather than samples; warps stride over the
+// chunks (see "Chunked ragged copy" in td_device.cuh).
+__global__ void __launch_bounds__(kCopyThreads, kCopyBlocksPerSM)
+put_scatter_kernel(const DockView dv, const PutBatch batch) {
+    __shared__ uint64_t item_end[kMaxPutItems];       // inclusive prefix of bytes (16-byte padded) per item
+    extern __shared__ __align__(128) uint8_t scatter_smem[];
+    uint8_t *stages = scatter_smem;                                          // [warps][stages][kStageBytes]
+    unsigned long long *bars = reinterpret_cast<unsigned long long *>(stages + kCopyWarps * kStages * kStageBytes);
     const uint32_t tid = threadIdx.x, lane = tid & 31;
+    WarpPipe pipe;
+    pipe.init(stages + (size_t)(tid >> 5) * kStages * kStageBytes, bars + (tid >> 5) * kStages, lane, dv.spin_limit);
 
     if (tid == 0) {
         uint64_t acc = 0;
         for (uint32_t it = 0; it < batch.n_items; ++it) {
             const PutArgs &a = batch.item[it];
-            uint64_t chunks = 0;
+            uint64_t bytes = 0;
             if (dv.col_cls[a.column] != TD_SCALAR && a.k) {
                 const int64_t tot = a.cu[a.k];
-                if (tot > 0 && (uint64_t)tot <= a.data_elems)
-                    chunks = ((uint64_t)tot * dv.col_esz[a.column] + chunk_bytes - 1) / chunk_bytes;
+                if (tot > 0 && (uint64_t)tot <= a.data_elems) bytes = (uint64_t)tot * dv.col_esz[a.column];
             }
-            acc += chunks;
+            acc += (bytes + 15) & ~uint64_t(15);
             item_end[it] = acc;
         }
     }
     __syncthreads();
-    const uint64_t n_chunks = item_end[batch.n_items - 1];
+    const uint64_t n_warps = (uint64_t)gridDim.x * kCopyWarps;
+    const ChunkPlan plan = plan_chunks(item_end[batch.n_items - 1], n_warps);
     const uint64_t warp0 = (uint64_t)blockIdx.x * kCopyWarps + (tid >> 5);
-    const uint64_t stride = (uint64_t)gridDim.x * kCopyWarps;
 
-    for (uint64_t ch = warp0; ch < n_chunks; ch += stride) {
+    for (uint64_t ch = warp0; ch < plan.n_chunks; ch += n_warps) {
+        uint64_t g0 = ch * plan.chunk_bytes;
+        const uint64_t g1 = min(g0 + plan.chunk_bytes, item_end[batch.n_items - 1]);
         uint32_t it = 0;
-        while (item_end[it] <= ch) ++it;
-        const PutArgs &a = batch.item[it];
-        const uint32_t L = dv.col_cls[a.column];
-        const uint32_t esz = dv.col_esz[a.column];
-        const uint32_t bit = 1u << a.column;
-        const uint64_t total_bytes = (uint64_t)(int64_t)__ldg(a.cu + a.k) * esz;
-        const uint64_t b0 = (ch - (it ? item_end[it - 1] : 0)) * chunk_bytes;
-        const uint64_t b1 = min(b0 + (uint64_t)chunk_bytes, total_bytes);
-        uint8_t *arena = dv.colbase[a.column];
-        const uint64_t cap = dv.cap[L];
-        warp_copy_chunk<false>(a.cu, a.k, b0, b1, const_cast<uint8_t *>(a.data), esz, lane,
-                               a.data, a.data + a.data_elems * esz,
-                               [&](uint32_t i, int64_t, int64_t) -> uint8_t * {
-                                   int32_t s; int64_t l; long long off;
-                                   if (!put_entry_live(dv, a, i, L, bit, s, l, off)) return nullptr;
-                                   return arena + ((uint64_t)shard_of(dv, (uint32_t)s) * cap + (uint64_t)off) * esz;
-                               });
+        while (item_end[it] <= g0) ++it;
+        for (; g0 < g1; ++it) {
+            const uint64_t start = it ? item_end[it - 1] : 0;
+            const PutArgs &a = batch.item[it];
+            const uint32_t L = dv.col_cls[a.column];
+            const uint32_t esz = dv.col_esz[a.column];
+            const uint32_t bit = 1u << a.column;
+            const uint64_t b0 = g0 - start;
+            g0 = min(g1, item_end[it]);
+            if (L == TD_SCALAR || a.k == 0) continue;
+            const uint64_t total_bytes = (uint64_t)(int64_t)__ldg(a.cu + a.k) * esz;
+            const uint64_t b1 = min(g0 - start, total_bytes);
+            if (b1 <= b0) continue;
+            uint8_t *arena = dv.colbase[a.column];
+            const uint64_t cap = dv.cap[L];
+            warp_copy_chunk<false>(a.cu, a.k, b0, b1, const_cast<uint8_t *>(a.data), esz, lane,
+                                   a.data, a.data + a.data_elems * esz, pipe,
+                                   [&](uint32_t i, int64_t c0, int64_t c1) -> uint8_t * {
+                                       // the row is live if the alloc kernel accepted it
+                                       const int32_t s = a.idx[i];
+                                       if (s < 0 || (uint32_t)s >= dv.n) return nullptr;
+                                       if (dv.status[s] & bit) return nullptr;
+                                       if (c1 < c0 || (uint64_t)c1 > a.data_elems) return nullptr;
+                                       if ((int64_t)dv.len[L][s] != c1 - c0) return nullptr;
+                                       const long long off = dv.off[L][s];
+                                       if (off < 0) return nullptr;
+                                       return arena + ((uint64_t)shard_of(dv, (uint32_t)s) * cap + (uint64_t)off) * esz;
+                                   });
+        }
     }
+    if (pipe.finish(lane) && lane == 0) flag_error(dv, TD_ERR_COPY_TIMEOUT, CNT_TIMEOUT);
 }
 
 // Publish.  Runs after the scatter kernel has finished, so every payload byte of the call is
