@@ -130,6 +130,23 @@ def gpu_id_for_smi(torch, local_rank: int) -> str:
     return str(local_rank)
 
 
+# --------------------------------------------------------------------------- multi-rank glue
+def max_over_ranks(dist, values, device):
+    """Element-wise maximum of `values` over all ranks (identity without a process group).
+    Docks on different ranks are independent: the only exchange is this reduction of timings."""
+    if dist is None:
+        return list(values)
+    import torch
+    t = torch.tensor(list(values), device=device, dtype=torch.float64)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def whole_job_rate(world: int, units_per_rank: int, seconds: float) -> float:
+    """Weak scaling: every rank dispatches units_per_rank in the slowest rank's time."""
+    return world * units_per_rank / seconds
+
+
 # --------------------------------------------------------------------------- workload glue
 def algorithmic_bytes(w):
     """Bytes the method must move per step: every put row read and written once, every served
@@ -391,11 +408,8 @@ def main():
 
     mean_put, mean_drain = sum(put_ms) / len(put_ms), sum(drain_ms) / len(drain_ms)
     ms_per_step = mean_put + mean_drain
-    if dist is not None:
-        t = torch.tensor([ms_per_step, mean_put, mean_drain], device=step.dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        ms_per_step, mean_put, mean_drain = t.tolist()
-    value = world * n_dispatch / (ms_per_step * 1e-3)
+    ms_per_step, mean_put, mean_drain = max_over_ranks(dist, [ms_per_step, mean_put, mean_drain], step.dev)
+    value = whole_job_rate(world, n_dispatch, ms_per_step * 1e-3)
 
     # per-kernel pass: event pairs around every launch of the two copy kernels
     step.dock.kernel_timing(True)
@@ -421,11 +435,8 @@ def main():
     e2e = None
     if not args.no_e2e:
         e2e_s, d2h = step.run_e2e(min(args.steps, 5), 1)
-        if dist is not None:
-            t = torch.tensor([e2e_s], device=step.dev, dtype=torch.float64)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            e2e_s = t.item()
-        e2e = {"value": world * n_dispatch / e2e_s, "unit": "samples/s", "ms_per_step": e2e_s * 1e3,
+        e2e_s, = max_over_ranks(dist, [e2e_s], step.dev)
+        e2e = {"value": whole_job_rate(world, n_dispatch, e2e_s), "unit": "samples/s", "ms_per_step": e2e_s * 1e3,
                "h2d_bytes_per_step": step.h2d_bytes, "d2h_bytes_per_step": d2h}
 
     if rank != 0:
