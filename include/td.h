@@ -48,7 +48,8 @@ typedef enum {
     TD_OK = 0,
     TD_EINVAL = -1,       /* bad argument                                   */
     TD_EWORKSPACE = -2,   /* workspace or scratch too small or misaligned   */
-    TD_ECUDA = -3         /* a CUDA runtime call failed (no device, ...)    */
+    TD_ECUDA = -3,        /* a CUDA runtime call failed (no device, ...)    */
+    TD_ETOOLARGE = -4     /* td_get_static: the dock exceeds its fixed scratch */
 } td_error;
 
 /* device-detected conditions */
@@ -166,6 +167,28 @@ int td_put(td_dock *dock, uint32_t column, const int32_t *d_indices, uint32_t k,
 int td_get(td_dock *dock, uint32_t consumer, uint32_t max_samples, const td_get_out *out,
            void *stream);
 size_t td_get_scratch_bytes(const td_dock *dock);
+
+/* td_get for callers that cannot provide scratch memory.  (The paper has no counterpart: this
+ * is a convenience of this library.)  Some code that wants to serve a batch may not allocate
+ * device memory at all: a step running inside a serving loop whose memory pool is frozen, a
+ * plug-in that is handed nothing but its input and output buffers, a process whose memory
+ * budget is already committed.  td_get asks such a caller for td_get_scratch_bytes() of
+ * zero-filled device memory it does not have.  td_get_static does the same get with the scan
+ * scratch kept in a fixed array inside the library (about 65 KB, held by every GPU that loads
+ * the library until the process exits); out->scratch and out->scratch_bytes are ignored, every
+ * other field of `out` means what it means for td_get, and the results are the same.
+ *   - Limit: docks of at most 16384 prompts (G); a larger dock gets TD_ETOOLARGE and nothing
+ *     is enqueued.
+ *   - The call allocates and frees nothing.  Its first call on a device looks the array's device
+ *     address up (once per device; a host-side query, no allocation); make that first call
+ *     outside any stream capture.
+ *   - All calls share the one array, which still holds the previous call's contents; the words
+ *     that must start at zero are cleared on `stream` before the scan.  Two td_get_static calls
+ *     that overlap on the GPU (different streams, no ordering between them) race on it and may
+ *     return nothing or report TD_ERR_LOOKBACK_TIMEOUT; order them, or use td_get with separate
+ *     scratch for concurrent gets. */
+int td_get_static(td_dock *dock, uint32_t consumer, uint32_t max_samples, const td_get_out *out,
+                  void *stream);
 
 /* Several columns in one call, as a worker that sends a whole record does (prompt and response
  * ids together, say): the items are stored as if td_put had been called on each in array order,

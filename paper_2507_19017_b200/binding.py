@@ -17,7 +17,7 @@ I32, F32, BF16 = 0, 1, 2
 SCALAR, PROMPT, RESPONSE = 0, 1, 2
 PACKED, PADDED = 0, 1
 F_ADVANTAGE = 1
-OK, EINVAL, EWORKSPACE, ECUDA = 0, -1, -2, -3
+OK, EINVAL, EWORKSPACE, ECUDA, ETOOLARGE = 0, -1, -2, -3, -4
 ERR_OOB_INDEX, ERR_DUP_PUT, ERR_LEN_MISMATCH, ERR_ARENA_FULL = 1, 2, 4, 8
 ERR_OUT_TRUNCATED, ERR_LOOKBACK_TIMEOUT, ERR_BAD_LENGTH, ERR_COPY_TIMEOUT = 16, 32, 64, 128
 
@@ -30,7 +30,7 @@ EXPORTS = ["td_query_workspace", "td_create", "td_destroy", "td_put", "td_get",
            "td_get_scratch_bytes", "td_reset", "td_status", "td_debug_table",
            "td_launch_count", "td_strerror", "td_kernel_timing", "td_kernel_timing_read",
            "td_put_host_stage_bytes", "td_put_host", "td_get_host", "td_put_many",
-           "td_plan_bytes", "td_plan_create", "td_plan_destroy", "td_get_many"]
+           "td_plan_bytes", "td_plan_create", "td_plan_destroy", "td_get_many", "td_get_static"]
 
 
 class TdColumn(C.Structure):
@@ -149,6 +149,8 @@ def lib():
         L.td_plan_destroy.argtypes = [vp]
         L.td_get_many.restype = C.c_int
         L.td_get_many.argtypes = [vp, vp, vp]
+        L.td_get_static.restype = C.c_int
+        L.td_get_static.argtypes = [vp, u32, u32, C.POINTER(TdGetOut), vp]
         _lib = L
     return _lib
 
@@ -371,6 +373,12 @@ class Dock:
         _check("td_get", lib().td_get(self.handle, bufs.consumer,
                                       bufs.max_samples if max_samples is None else max_samples,
                                       C.byref(bufs.struct), _stream_ptr(stream)))
+
+    def get_static(self, bufs: GetBuffers, stream=None):
+        """The same get with the scan scratch inside the library (no scratch buffer needed;
+        docks of at most 16384 prompts; calls must not overlap on the GPU)."""
+        _check("td_get_static", lib().td_get_static(self.handle, bufs.consumer, bufs.max_samples,
+                                                    C.byref(bufs.struct), _stream_ptr(stream)))
 
     def reset(self, stream=None):
         _check("td_reset", lib().td_reset(self.handle, _stream_ptr(stream)))

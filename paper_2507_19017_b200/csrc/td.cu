@@ -140,6 +140,7 @@ const char *td_strerror(int code) {
         case TD_EINVAL: return "invalid argument";
         case TD_EWORKSPACE: return "workspace or scratch too small or misaligned";
         case TD_ECUDA: return "CUDA runtime call failed";
+        case TD_ETOOLARGE: return "dock has more prompts than the fixed-scratch get supports";
         default: return "unknown error";
     }
 }
@@ -355,6 +356,81 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
     one.cs.consumer = consumer;
     one.cs.max_groups = one.req.max_groups;
     one.cs.scratch = out->scratch;
+    const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
+
+    if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
+               (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
+    if (launch(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
+               (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
+    const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
+    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(v.ncol), st, v, one,
+                     (const GetReq *)nullptr, 1u) != cudaSuccess) return TD_ECUDA;
+    return TD_OK;
+}
+
+// ---- a get whose scan scratch is a fixed array inside the library ----
+// For callers that have nowhere to take scratch memory from: code running where device memory
+// may not be allocated (inside a serving loop with a frozen memory pool, in a plug-in that was
+// handed only its input and output buffers, under a memory budget that is already spent).
+// td_get makes such a caller supply td_get_scratch_bytes() of zero-filled device memory; this
+// variant keeps that scratch in the array below instead, which every device that loads the
+// library holds (kStaticScratchBytes, about 65 KB) until the process exits.
+constexpr uint32_t kStaticMaxGroups = 16384;          // docks with more prompts are refused
+constexpr size_t kStaticScratchBytes = (((2 + (kStaticMaxGroups + kSelThreads - 1) / kSelThreads) * 8 +
+                                         (size_t)kStaticMaxGroups * 4) + 15) & ~size_t(15);
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+namespace {
+constexpr int kMaxDevices = 64;
+std::mutex g_static_mu;
+void *g_static_ptr[kMaxDevices] = {};                 // device address of g_static_scratch, per device
+
+// In host code the array's name is only a handle: the device address has to be asked for, once
+// per device, with that device current.
+int static_scratch_address(int device, void **out) {
+    if (device < 0 || device >= kMaxDevices) return TD_EINVAL;
+    std::lock_guard<std::mutex> lk(g_static_mu);
+    if (!g_static_ptr[device]) {
+        int cur = -1;
+        if (cudaGetDevice(&cur) != cudaSuccess) return TD_ECUDA;
+        if (cur != device && cudaSetDevice(device) != cudaSuccess) return TD_ECUDA;
+        void *p = nullptr;
+        const cudaError_t rc = cudaGetSymbolAddress(&p, g_static_scratch);
+        if (cur != device) cudaSetDevice(cur);
+        if (rc != cudaSuccess || !p) return TD_ECUDA;
+        g_static_ptr[device] = p;
+    }
+    *out = g_static_ptr[device];
+    return TD_OK;
+}
+}  // namespace
+
+int td_get_static(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out *out, void *stream) {
+    if (!d) return TD_EINVAL;
+    const DockView &v = d->dv;
+    const int chk = check_get_out(v, consumer, max_samples, out);
+    if (chk != TD_OK) return chk;
+    if (v.G > kStaticMaxGroups || sel_scratch_bytes(v.G) > kStaticScratchBytes) return TD_ETOOLARGE;
+    void *scratch = nullptr;
+    const int rc = static_scratch_address(d->device, &scratch);
+    if (rc != TD_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    // The array still holds what the last call left.  The scan tags what it writes with the
+    // call's sequence number, but the ticket and the tile descriptors are cleared all the same,
+    // so that nothing here depends on what ran before.
+    if (cudaMemsetAsync(scratch, 0, (2 + (size_t)sel_tiles(v.G)) * 8, st) != cudaSuccess) return TD_ECUDA;
+    const uint32_t m = max_samples / v.N;
+
+    GetInline one;
+    std::memset(&one, 0, sizeof(one));
+    one.req.out = *out;
+    one.req.consumer = consumer;
+    one.req.max_groups = m < v.G ? m : v.G;
+    one.req.rank_base = 0;
+    one.req.cslot = 0;
+    one.cs.consumer = consumer;
+    one.cs.max_groups = one.req.max_groups;
+    one.cs.scratch = scratch;
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
 
     if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
