@@ -116,6 +116,64 @@ class ClockSampler:
                 "samples": len(sm), "window": window, "reasons": sorted(reasons)}
 
 
+class NvmlSampler:
+    """Reads SM clock and clock-event reasons through NVML every 2 ms from a thread (read-only
+    queries): nvidia-smi's own loop is too slow for a timed region of a few milliseconds."""
+    REASONS = {0x4: "sw_power_cap", 0x8: "hw_slowdown", 0x20: "sw_thermal_slowdown",
+               0x40: "hw_thermal_slowdown", 0x80: "hw_power_brake_slowdown"}
+
+    def __init__(self, uuid: str):
+        import pynvml
+        self.nv = pynvml
+        pynvml.nvmlInit()
+        self.h = pynvml.nvmlDeviceGetHandleByUUID(uuid.encode() if isinstance(uuid, str) else uuid)
+        self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        self.samples, self.stop_flag, self.thread = [], threading.Event(), None
+
+    def _loop(self):
+        nv = self.nv
+        get_reasons = getattr(nv, "nvmlDeviceGetCurrentClocksEventReasons", None) or \
+            nv.nvmlDeviceGetCurrentClocksThrottleReasons
+        while not self.stop_flag.is_set():
+            try:
+                self.samples.append((time.time(), float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)),
+                                     int(get_reasons(self.h))))
+            except Exception:
+                pass
+            time.sleep(0.002)
+
+    def start(self):
+        self.thread = threading.Thread(target=self._loop, daemon=True)
+        self.thread.start()
+
+    def stop(self, t_begin: float, t_end: float):
+        self.stop_flag.set()
+        if self.thread:
+            self.thread.join(timeout=2)
+        inside = [s for s in self.samples if t_begin <= s[0] <= t_end]
+        window = "timed region"
+        if len(inside) < 3:
+            inside, window = self.samples, "warm-up and timed region"
+        reasons = set()
+        for _t, _mhz, bits in inside:
+            for bit, name in self.REASONS.items():
+                if bits & bit:
+                    reasons.add(name)
+        sm = [s[1] for s in inside]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": self.max_mhz,
+                "samples": len(sm), "window": window, "source": "nvml", "reasons": sorted(reasons)}
+
+
+def make_sampler(torch, local_rank: int):
+    gpu_id = gpu_id_for_smi(torch, local_rank)
+    if gpu_id.startswith("GPU-"):
+        try:
+            return NvmlSampler(gpu_id)
+        except Exception:
+            pass
+    return ClockSampler(gpu_id)
+
+
 def gpu_id_for_smi(torch, local_rank: int) -> str:
     """The id nvidia-smi knows this process's device by: its UUID when listed, else its index."""
     try:
@@ -380,7 +438,7 @@ def main():
     peak, peak_kind = load_peaks()
     put_bytes, put_ragged_bytes, get_bytes = algorithmic_bytes(w)
 
-    sampler = ClockSampler(gpu_id_for_smi(torch, local_rank))
+    sampler = make_sampler(torch, local_rank)
     sampler.start()
     for _ in range(max(args.warmup, 3)):
         step.timed_step()
