@@ -10,7 +10,7 @@ _ROOT = os.path.dirname(_HERE)
 CSRC = os.path.join(_HERE, "csrc")
 LIB_PATH = os.path.join(_HERE, "libtd.so")
 SOURCES = ["td.cu"]
-HEADERS = ["td_device.cuh", "td_put.cuh", "td_get.cuh"]
+HEADERS = ["td_device.cuh", "td_alloc.cuh", "td_put.cuh", "td_get.cuh"]
 
 NVCC_FLAGS = [
     "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",

@@ -106,12 +106,31 @@ cudaError_t launch(td_dock *d, void (*kernel)(KArgs...), dim3 grid, dim3 block, 
     return cudaGetLastError();
 }
 
+// Launch of a kernel that may be brought on before the kernel ahead of it in the stream has
+// finished (programmatic dependent launch); the kernel itself waits, with griddep_wait(), before
+// it touches that kernel's results.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_dep(td_dock *d, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                       cudaStream_t st, Args &&...args) {
+#ifdef TD_NO_PDL
+    return launch(d, kernel, grid, block, smem, st, std::forward<Args>(args)...);
+#endif
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    d->launches.fetch_add(1, std::memory_order_relaxed);
+    return cudaLaunchKernelEx(&cfg, kernel, KArgs(std::forward<Args>(args))...);
+}
+
 // Launch bracketed by a pair of events on the same stream while timing is switched on.
 template <typename... KArgs, typename... Args>
 cudaError_t launch_timed(td_dock *d, int which, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
                          cudaStream_t st, Args &&...args) {
     if (!d->timing.load(std::memory_order_relaxed))
-        return launch(d, kernel, grid, block, smem, st, std::forward<Args>(args)...);
+        return launch_dep(d, kernel, grid, block, smem, st, std::forward<Args>(args)...);
     cudaEvent_t e0, e1;
     if (cudaEventCreate(&e0) != cudaSuccess || cudaEventCreate(&e1) != cudaSuccess) return cudaErrorUnknown;
     cudaEventRecord(e0, st);
@@ -159,8 +178,7 @@ int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **o
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess) return TD_ECUDA;
     const size_t alloc_smem = put_alloc_smem_bytes(cfg->n_shards);
-    if (alloc_smem > 48 * 1024 &&
-        cudaFuncSetAttribute(put_alloc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)alloc_smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(put_alloc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)alloc_smem) != cudaSuccess)
         return TD_ECUDA;
 
     if (cudaFuncSetAttribute(put_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -260,13 +278,13 @@ int put_group(td_dock *d, const PutBatch &b, cudaStream_t st) {
     if (entries == 0) return TD_OK;
     if (entries >= (1ull << 32)) return TD_EINVAL;
     if (ragged_bytes) {
-        if (launch(d, put_alloc_kernel, dim3(1), dim3(kAllocThreads), put_alloc_smem_bytes(v.S), st, v, b) != cudaSuccess)
+        if (launch(d, put_alloc_kernel, dim3(2), dim3(kAllocThreads), put_alloc_smem_bytes(v.S), st, v, b) != cudaSuccess)
             return TD_ECUDA;
         if (launch_timed(d, 0, put_scatter_kernel, dim3(copy_grid(d, ragged_bytes)), dim3(kCopyThreads),
                          scatter_smem_bytes(), st, v, b) != cudaSuccess)
             return TD_ECUDA;
     }
-    if (launch(d, put_publish_kernel, dim3((uint32_t)((entries + 255) / 256)), dim3(256), 0, st, v, b) != cudaSuccess)
+    if (launch_dep(d, put_publish_kernel, dim3((uint32_t)((entries + 255) / 256)), dim3(256), 0, st, v, b) != cudaSuccess)
         return TD_ECUDA;
     return TD_OK;
 }
@@ -360,7 +378,7 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
 
     if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
-    if (launch(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
+    if (launch_dep(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
     if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(v.ncol), st, v, one,
@@ -435,7 +453,7 @@ int td_get_static(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_
 
     if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
-    if (launch(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
+    if (launch_dep(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
     if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(v.ncol), st, v, one,
@@ -534,7 +552,7 @@ int td_get_many(td_dock *d, td_plan *p, void *stream) {
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
     if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), p->n_slots), dim3(kSelThreads), 0, st, v, none,
                (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
-    if (launch(d, get_finalize_kernel, dim3(p->n_req), dim3(kFinThreads), 0, st, v, none, (const GetReq *)p->d_reqs,
+    if (launch_dep(d, get_finalize_kernel, dim3(p->n_req), dim3(kFinThreads), 0, st, v, none, (const GetReq *)p->d_reqs,
                (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
     if (launch_timed(d, 1, get_gather_kernel, dim3(copy_grid(d, p->room_bytes)), dim3(kCopyThreads),
                      gather_smem_bytes(p->n_req * v.ncol), st, v, none,

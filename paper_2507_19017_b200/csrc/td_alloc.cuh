@@ -1,0 +1,224 @@
+// td_put, first kernel: reserve the rows of a put in the shard arenas.
+// Workflow step 2 of "Distributed Transfer Dock Strategy" (a worker sends real data to the
+// warehouses): before payload can move, every row needs its place.
+#pragma once
+
+#include "td_device.cuh"
+
+namespace td {
+
+constexpr int kAllocThreads = 1024;
+constexpr int kAllocWarps = kAllocThreads / 32;
+constexpr int kAllocPer = 4;                                   // entries per thread and pass
+constexpr int kAllocPass = kAllocThreads * kAllocPer;          // entries per pass
+constexpr int kMaxPutItems = 8;                                // columns one put launch can carry
+constexpr uint32_t kNotAllocating = 0xffffffffu;
+
+struct PutArgs {
+    uint32_t column, k;
+    const int32_t *idx;
+    const int32_t *cu;
+    const uint8_t *data;
+    uint64_t data_elems;
+};
+struct PutBatch {                              // the columns of one call, in call order
+    uint32_t n_items;
+    uint32_t pad;
+    PutArgs item[kMaxPutItems];
+};
+
+static inline size_t put_alloc_smem_bytes(uint32_t S) {
+    return (size_t)(kAllocWarps + 2) * S * sizeof(unsigned long long);
+}
+
+// Ordered exclusive prefix of `room` over the lanes that allocate in the same shard, and that
+// shard's sum over the warp.  leader: the first allocating lane of its shard.
+__device__ __forceinline__ void warp_shard_prefix(bool alloc, uint32_t sh, uint32_t room, uint32_t lane,
+                                                  unsigned long long &pre, unsigned long long &wsum, bool &leader) {
+    pre = 0; wsum = 0; leader = false;
+    const uint32_t mask = __ballot_sync(kFullMask, alloc);
+    if (mask == 0) return;
+    const uint32_t first = (uint32_t)__ffs(mask) - 1u;
+    // usual case: every allocating lane of the warp is in one shard -> one shuffle scan
+    const uint32_t first_sh = __shfl_sync(kFullMask, sh, first);      // every lane takes part
+    const uint32_t key = alloc ? sh : first_sh;
+    int same;
+    __match_all_sync(kFullMask, key, &same);
+    if (same) {
+        unsigned long long inc = alloc ? room : 0u;
+        #pragma unroll
+        for (int d = 1; d < 32; d <<= 1) {
+            const unsigned long long t = shfl_up_u64(inc, d);
+            if ((int)lane >= d) inc += t;
+        }
+        wsum = shfl_u64(inc, 31);
+        pre = inc - (alloc ? room : 0u);
+        leader = alloc && lane == first;
+        return;
+    }
+    const uint32_t k2 = alloc ? sh : kNotAllocating;
+    leader = alloc;
+    #pragma unroll 8
+    for (uint32_t j = 0; j < 32; ++j) {
+        const uint32_t kj = __shfl_sync(kFullMask, k2, j);
+        const uint32_t rj = __shfl_sync(kFullMask, room, j);
+        if (alloc && kj == k2) {
+            wsum += rj;
+            if (j < lane) { pre += rj; leader = false; }
+        }
+    }
+}
+
+// Alloc.  grid = 2: CTA 0 serves the prompt-length items of the call, CTA 1 the response-length
+// ones (the two classes share no table), each class's items one after the other, in passes of
+// kAllocPass entries in call order.  Per pass:
+//   1. every thread validates kAllocPer entries and settles with a CAS on len[] which of them
+//      are first arrivals of their length class, i.e. reserve a row;
+//   2. round by round (kAllocThreads entries each) an ordered per-shard exclusive scan of the
+//      row sizes (warp shuffles, then the warps' sums through shared memory) gives every new
+//      row the place, relative to the pass, a sequential walk would have given it;
+//   3. one atomicAdd per shard reserves the pass's space; rows are placed behind it.
+// A pass without a first arrival (a later column of a class whose rows exist) ends after 1.
+// A pass that would overflow a shard is replayed by one thread, entry by entry, so that only
+// the rows without room are refused.
+__global__ void __launch_bounds__(kAllocThreads)
+put_alloc_kernel(const DockView dv, const PutBatch batch) {
+    extern __shared__ unsigned long long smem_u64[];
+    const uint32_t S = dv.S;
+    unsigned long long *tot = smem_u64;                            // [kAllocWarps][S]
+    unsigned long long *s_run = tot + (size_t)kAllocWarps * S;     // [S] space asked so far in this pass
+    unsigned long long *s_start = s_run + S;                       // [S] where the pass's space begins
+    __shared__ int32_t e_s[kAllocPass];
+    __shared__ uint32_t e_room[kAllocPass];
+    __shared__ uint32_t s_overflow;
+
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const uint32_t L = blockIdx.x + 1;                             // TD_PROMPT or TD_RESPONSE
+    griddep_launch_dependents();                                   // the scatter may set itself up meanwhile
+    const uint64_t cap = dv.cap[L];
+    uint32_t n_oob = 0, n_dup = 0, n_bad = 0, n_mis = 0, n_full = 0;
+
+    for (uint32_t it = 0; it < batch.n_items; ++it) {
+        const PutArgs &a = batch.item[it];
+        if (dv.col_cls[a.column] != L) continue;
+        const uint32_t bit = 1u << a.column;
+        for (uint32_t base = 0; base < a.k; base += kAllocPass) {
+            // 1. validate, CAS
+            int32_t s[kAllocPer];
+            uint32_t room[kAllocPer], sh[kAllocPer];
+            bool alloc[kAllocPer];
+            bool any = false;
+            #pragma unroll
+            for (int j = 0; j < kAllocPer; ++j) {
+                const uint32_t i = base + j * kAllocThreads + tid;
+                alloc[j] = false; s[j] = -1; room[j] = 0; sh[j] = 0;
+                if (i < a.k) {
+                    s[j] = a.idx[i];
+                    if (s[j] < 0 || (uint32_t)s[j] >= dv.n) { ++n_oob; }
+                    else if (dv.status[s[j]] & bit) { ++n_dup; }
+                    else {
+                        const int64_t c0 = a.cu[i], c1 = a.cu[i + 1];
+                        const int64_t l = c1 - c0;
+                        if (l < 0 || c0 < 0 || (uint64_t)c1 > a.data_elems) { ++n_bad; }
+                        else {
+                            const int32_t old = atomicCAS(&dv.len[L][s[j]], -1, (int32_t)l);
+                            if (old == -1) {
+                                alloc[j] = true;
+                                room[j] = (uint32_t)align_row((uint64_t)l);
+                                sh[j] = shard_of(dv, (uint32_t)s[j]);
+                            } else if (old != (int32_t)l) { ++n_mis; }
+                        }
+                    }
+                }
+                e_s[j * kAllocThreads + tid] = s[j];
+                e_room[j * kAllocThreads + tid] = alloc[j] ? room[j] : kNotAllocating;
+                any |= alloc[j];
+            }
+            for (uint32_t k2 = tid; k2 < S; k2 += kAllocThreads) s_run[k2] = 0;
+            if (tid == 0) s_overflow = 0;
+            if (!__syncthreads_or(any)) continue;                 // no first arrival in this pass
+
+            // 2. relative places, round by round
+            unsigned long long rel[kAllocPer];
+            #pragma unroll
+            for (int j = 0; j < kAllocPer; ++j) {
+                rel[j] = 0;
+                if (base + (uint32_t)j * kAllocThreads >= a.k) break;     // uniform
+                for (uint32_t q = tid; q < kAllocWarps * S; q += kAllocThreads) tot[q] = 0;
+                unsigned long long pre, wsum;
+                bool leader;
+                warp_shard_prefix(alloc[j], sh[j], room[j], lane, pre, wsum, leader);
+                __syncthreads();
+                if (leader) tot[warp * S + sh[j]] = wsum;
+                __syncthreads();
+                for (uint32_t k2 = warp; k2 < S; k2 += kAllocWarps) {
+                    const unsigned long long v = tot[lane * S + k2];
+                    unsigned long long inc = v;
+                    #pragma unroll
+                    for (int d = 1; d < 32; d <<= 1) {
+                        const unsigned long long t = shfl_up_u64(inc, d);
+                        if ((int)lane >= d) inc += t;
+                    }
+                    const unsigned long long run = s_run[k2];
+                    tot[lane * S + k2] = run + inc - v;
+                    __syncwarp();
+                    if (lane == 31) s_run[k2] = run + inc;
+                }
+                __syncthreads();
+                if (alloc[j]) rel[j] = tot[warp * S + sh[j]] + pre;
+                __syncthreads();
+            }
+
+            // 3. reserve the pass's space, place the rows
+            for (uint32_t k2 = tid; k2 < S; k2 += kAllocThreads) {
+                // rows of length zero still get a place: the cursor as it stands
+                const unsigned long long start = atomicAdd(&dv.cursor[L][k2], s_run[k2]);
+                if (start + s_run[k2] > cap) s_overflow = 1;
+                s_start[k2] = start;
+            }
+            __syncthreads();
+            if (!s_overflow) {
+                #pragma unroll
+                for (int j = 0; j < kAllocPer; ++j)
+                    if (alloc[j]) dv.off[L][s[j]] = (long long)(s_start[sh[j]] + rel[j]);
+            } else {
+                // hand the pass's reservations back, then replay the pass in call order
+                for (uint32_t k2 = tid; k2 < S; k2 += kAllocThreads)
+                    atomicAdd(&dv.cursor[L][k2], 0ull - s_run[k2]);
+                __syncthreads();
+                if (tid == 0) {
+                    const uint32_t n_here = min((uint32_t)kAllocPass, a.k - base);
+                    for (uint32_t t = 0; t < n_here; ++t) {
+                        const uint32_t r = e_room[t];
+                        if (r == kNotAllocating) continue;
+                        const int32_t ss = e_s[t];
+                        const uint32_t k2 = shard_of(dv, (uint32_t)ss);
+                        const unsigned long long start = atomicAdd(&dv.cursor[L][k2], (unsigned long long)r);
+                        if (start + r > cap) {
+                            atomicAdd(&dv.cursor[L][k2], 0ull - (unsigned long long)r);
+                            atomicExch(&dv.len[L][ss], -1);
+                            ++n_full;
+                        } else {
+                            dv.off[L][ss] = (long long)start;
+                        }
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+    n_oob = __reduce_add_sync(kFullMask, n_oob);
+    n_dup = __reduce_add_sync(kFullMask, n_dup);
+    n_bad = __reduce_add_sync(kFullMask, n_bad);
+    n_mis = __reduce_add_sync(kFullMask, n_mis);
+    n_full = __reduce_add_sync(kFullMask, n_full);
+    if (lane == 0) {
+        if (n_oob) flag_error(dv, TD_ERR_OOB_INDEX, CNT_OOB, n_oob);
+        if (n_dup) flag_error(dv, TD_ERR_DUP_PUT, CNT_DUP, n_dup);
+        if (n_bad) flag_error(dv, TD_ERR_BAD_LENGTH, CNT_BADLEN, n_bad);
+        if (n_mis) flag_error(dv, TD_ERR_LEN_MISMATCH, CNT_MISMATCH, n_mis);
+        if (n_full) flag_error(dv, TD_ERR_ARENA_FULL, CNT_FULL, n_full);
+    }
+}
+
+}  // namespace td

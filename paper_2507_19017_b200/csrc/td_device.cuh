@@ -90,6 +90,15 @@ __device__ __forceinline__ void st_release_u64(unsigned long long *p, unsigned l
     asm volatile("st.release.gpu.global.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 
+// Programmatic dependent launch: the kernels of one call are chained so that the next one is
+// launched, and runs its prologue, while the previous one is still finishing.  A kernel calls
+// griddep_wait() before it touches anything the kernel before it in the stream wrote (the wait
+// returns when that kernel has completed and its writes are visible; without the launch
+// attribute it returns at once), and griddep_launch_dependents() as soon as the next kernel
+// may be brought on.
+__device__ __forceinline__ void griddep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void griddep_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __device__ __forceinline__ void flag_error(const DockView &dv, uint32_t bit, int counter, uint32_t count = 1) {
     atomicOr(dv.errword, bit);
     atomicAdd(&dv.counters[counter], (unsigned long long)count);

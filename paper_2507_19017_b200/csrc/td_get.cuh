@@ -82,6 +82,7 @@ get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     __shared__ uint32_t s_tile, s_excl, s_failed;
     __shared__ uint32_t s_warp[kSelWarps];
+    griddep_launch_dependents();
 
     if (tid == 0) {
         // ticket word = seq << 32 | tiles started; sequence numbers only grow
@@ -218,6 +219,8 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     const uint32_t tid = threadIdx.x;
     __shared__ uint64_t sh_a[kFinThreads / 32], sh_b[kFinThreads / 32];
     __shared__ uint32_t s_first_over;
+    griddep_launch_dependents();
+    griddep_wait();                                    // the scan's candidate list is complete
 
     // how many groups were ready, from the last tile's inclusive prefix
     const unsigned long long last = sc.desc[sel_tiles(dv.G) - 1];
@@ -373,6 +376,7 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     WarpPipe pipe;
     pipe.init(stages + (size_t)warp * kStages * kStageBytes, bars + warp * kStages, lane, dv.spin_limit);
+    griddep_wait();                                    // indices, cu_seqlens and result blocks are complete
     const uint32_t ncol = dv.ncol;
     const uint32_t njobs = n_req * ncol;
 

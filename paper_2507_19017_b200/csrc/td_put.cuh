@@ -3,27 +3,10 @@
 // the warehouses, then the warehouse state becomes visible to every controller.
 #pragma once
 
+#include "td_alloc.cuh"
 #include "td_device.cuh"
 
 namespace td {
-
-constexpr int kAllocThreads = 1024;
-constexpr int kAllocWarps = kAllocThreads / 32;
-constexpr int kMaxPutItems = 8;                // columns one put launch can carry
-constexpr uint32_t kNotAllocating = 0xffffffffu;
-
-struct PutArgs {
-    uint32_t column, k;
-    const int32_t *idx;
-    const int32_t *cu;
-    const uint8_t *data;
-    uint64_t data_elems;
-};
-struct PutBatch {                              // the columns of one call, in call order
-    uint32_t n_items;
-    uint32_t pad;
-    PutArgs item[kMaxPutItems];
-};
 
 // Is entry i of this item a row that the alloc kernel accepted?  Recomputed from the tables by
 // the scatter and publish kernels, so that a put needs no scratch memory of its own.
@@ -43,140 +26,6 @@ __device__ __forceinline__ bool put_entry_live(const DockView &dv, const PutArgs
     return true;
 }
 
-static inline size_t put_alloc_smem_bytes(uint32_t S) {
-    return (size_t)(kAllocWarps + 2) * S * sizeof(unsigned long long);
-}
-
-// Alloc.  One CTA walks the ragged items of the call one after the other, each in rounds of
-// kAllocThreads entries in call order.  Per round: validate, decide who reserves a row (first
-// arrival of the length class, settled by a CAS on len), then an ordered per-shard exclusive
-// scan of the row sizes gives every new row the offset a sequential walk would have given it.
-// A round that would overflow a shard is replayed by one thread, entry by entry, so that only
-// the rows without room are refused.
-__global__ void __launch_bounds__(kAllocThreads)
-put_alloc_kernel(const DockView dv, const PutBatch batch) {
-    extern __shared__ unsigned long long smem_u64[];
-    const uint32_t S = dv.S;
-    unsigned long long *tot = smem_u64;                            // [kAllocWarps][S]
-    unsigned long long *s_total = tot + (size_t)kAllocWarps * S;   // [S] row space asked per shard
-    unsigned long long *s_start = s_total + S;                     // [S] where the round's space begins
-    __shared__ int32_t e_s[kAllocThreads];
-    __shared__ uint32_t e_room[kAllocThreads];
-    __shared__ uint32_t s_overflow;
-
-    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    uint32_t n_oob = 0, n_dup = 0, n_bad = 0, n_mis = 0, n_full = 0;
-
-    for (uint32_t it = 0; it < batch.n_items; ++it) {
-        const PutArgs &a = batch.item[it];
-        const uint32_t L = dv.col_cls[a.column];
-        if (L == TD_SCALAR) continue;
-        const uint32_t bit = 1u << a.column;
-        const uint64_t cap = dv.cap[L];
-        for (uint32_t base = 0; base < a.k; base += kAllocThreads) {
-            for (uint32_t j = tid; j < kAllocWarps * S; j += kAllocThreads) tot[j] = 0;
-            if (tid == 0) s_overflow = 0;
-            const uint32_t i = base + tid;
-            bool alloc = false;
-            int32_t s = -1;
-            uint32_t room = 0, sh = 0;
-            if (i < a.k) {
-                s = a.idx[i];
-                if (s < 0 || (uint32_t)s >= dv.n) { ++n_oob; }
-                else if (dv.status[s] & bit) { ++n_dup; }
-                else {
-                    const int64_t c0 = a.cu[i], c1 = a.cu[i + 1];
-                    const int64_t l = c1 - c0;
-                    if (l < 0 || c0 < 0 || (uint64_t)c1 > a.data_elems) { ++n_bad; }
-                    else {
-                        const int32_t old = atomicCAS(&dv.len[L][s], -1, (int32_t)l);
-                        if (old == -1) {
-                            alloc = true;
-                            room = (uint32_t)align_row((uint64_t)l);
-                            sh = shard_of(dv, (uint32_t)s);
-                        } else if (old != (int32_t)l) { ++n_mis; }
-                    }
-                }
-            }
-            e_s[tid] = s;
-            e_room[tid] = alloc ? room : kNotAllocating;
-            // ordered exclusive prefix per shard inside the warp
-            const uint32_t key = alloc ? sh : kNotAllocating;
-            unsigned long long pre = 0, wsum = 0;
-            bool leader = alloc;
-            #pragma unroll 8
-            for (uint32_t j = 0; j < 32; ++j) {
-                const uint32_t kj = __shfl_sync(kFullMask, key, j);
-                const uint32_t rj = __shfl_sync(kFullMask, room, j);
-                if (alloc && kj == key) {
-                    wsum += rj;
-                    if (j < lane) { pre += rj; leader = false; }
-                }
-            }
-            __syncthreads();                                   // tot zeroed, e_* written
-            if (leader) tot[warp * S + sh] = wsum;
-            __syncthreads();
-            // per shard: exclusive scan of the warps' sums in warp order, then reserve
-            for (uint32_t key2 = warp; key2 < S; key2 += kAllocWarps) {
-                const unsigned long long v = tot[lane * S + key2];
-                unsigned long long inc = v;
-                #pragma unroll
-                for (int d = 1; d < 32; d <<= 1) {
-                    const unsigned long long t = __shfl_up_sync(kFullMask, inc, d);
-                    if ((int)lane >= d) inc += t;
-                }
-                tot[lane * S + key2] = inc - v;
-                if (lane == 31) {
-                    s_total[key2] = inc;
-                    // rows of length zero still get a place: the cursor as it stands
-                    const unsigned long long start = atomicAdd(&dv.cursor[L][key2], inc);
-                    if (start + inc > cap) s_overflow = 1;
-                    s_start[key2] = start;
-                }
-            }
-            __syncthreads();
-            if (!s_overflow) {
-                if (alloc) dv.off[L][s] = (long long)(s_start[sh] + tot[warp * S + sh] + pre);
-            } else {
-                // hand the round's reservations back, then replay the round in call order
-                for (uint32_t key2 = tid; key2 < S; key2 += kAllocThreads)
-                    atomicAdd(&dv.cursor[L][key2], 0ull - s_total[key2]);
-                __syncthreads();
-                if (tid == 0) {
-                    for (uint32_t t = 0; t < kAllocThreads; ++t) {
-                        const uint32_t r = e_room[t];
-                        if (r == kNotAllocating) continue;
-                        const int32_t ss = e_s[t];
-                        const uint32_t key2 = shard_of(dv, (uint32_t)ss);
-                        const unsigned long long start = atomicAdd(&dv.cursor[L][key2], (unsigned long long)r);
-                        if (start + r > cap) {
-                            atomicAdd(&dv.cursor[L][key2], 0ull - (unsigned long long)r);
-                            atomicExch(&dv.len[L][ss], -1);
-                            ++n_full;
-                        } else {
-                            dv.off[L][ss] = (long long)start;
-                        }
-                    }
-                }
-            }
-            __syncthreads();
-        }
-        __threadfence_block();
-    }
-    n_oob = __reduce_add_sync(kFullMask, n_oob);
-    n_dup = __reduce_add_sync(kFullMask, n_dup);
-    n_bad = __reduce_add_sync(kFullMask, n_bad);
-    n_mis = __reduce_add_sync(kFullMask, n_mis);
-    n_full = __reduce_add_sync(kFullMask, n_full);
-    if (lane == 0) {
-        if (n_oob) flag_error(dv, TD_ERR_OOB_INDEX, CNT_OOB, n_oob);
-        if (n_dup) flag_error(dv, TD_ERR_DUP_PUT, CNT_DUP, n_dup);
-        if (n_bad) flag_error(dv, TD_ERR_BAD_LENGTH, CNT_BADLEN, n_bad);
-        if (n_mis) flag_error(dv, TD_ERR_LEN_MISMATCH, CNT_MISMATCH, n_mis);
-        if (n_full) flag_error(dv, TD_ERR_ARENA_FULL, CNT_FULL, n_full);
-    }
-}
-
 // Scatter.  The packed sources of the call's ragged items, laid end to end, are cut into equal
 // chunks, so that work is balanced over tokens rather than samples; warps stride over the
 // chunks (see "Chunked ragged copy" in td_device.cuh).
@@ -189,6 +38,8 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
     const uint32_t tid = threadIdx.x, lane = tid & 31;
     WarpPipe pipe;
     pipe.init(stages + (size_t)(tid >> 5) * kStages * kStageBytes, bars + (tid >> 5) * kStages, lane, dv.spin_limit);
+    griddep_launch_dependents();
+    griddep_wait();                                    // the alloc kernel's tables are complete
 
     if (tid == 0) {
         uint64_t acc = 0;
@@ -250,6 +101,7 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
 // that acquire it.  A scalar item needs no scatter: its element is stored here, then published.
 __global__ void __launch_bounds__(256)
 put_publish_kernel(const DockView dv, const PutBatch batch) {
+    griddep_wait();                                    // every payload byte of the call is in place
     uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     uint32_t it = 0;
     while (it < batch.n_items && i >= batch.item[it].k) { i -= batch.item[it].k; ++it; }

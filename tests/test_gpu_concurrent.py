@@ -3,6 +3,7 @@ own stream while consumer threads poll td_get on theirs.  Several outcomes are v
 checks are the invariants every outcome must satisfy, plus bit parity of every batch's payload,
 cu_seqlens and advantages with what the oracle gathers for the same indices."""
 import threading
+import time
 
 import numpy as np
 import pytest
@@ -57,7 +58,9 @@ def run_concurrent(G, w, consumer_threads):
                 pc, rc = g.token_caps(w.micro_batch)
                 bufs = td.GetBuffers(g.dock, c, w.micro_batch, prompt_tokens_cap=pc, response_tokens_cap=rc)
                 idle = 0
+                deadline = time.time() + 120
                 while True:
+                    assert time.time() < deadline, "consumer did not finish in time"
                     g.dock.get(bufs, stream=s)
                     b = g.read(bufs, stream=s)
                     assert b.status == 0
@@ -82,7 +85,7 @@ def run_concurrent(G, w, consumer_threads):
     for t in threads:
         t.start()
     for t in threads:
-        t.join(timeout=600)
+        t.join(timeout=150)
     assert not any(t.is_alive() for t in threads), "a thread did not finish"
     if errors:
         raise errors[0]

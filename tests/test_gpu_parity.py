@@ -287,6 +287,27 @@ def test_arena_full_refuses_only_rows_without_room(G):
     assert g.dock.status().error_word == td.ERR_ARENA_FULL
 
 
+def test_one_put_of_many_passes_in_random_order(G):
+    """One call carrying 9000 rows in shuffled order over 12 shards: several allocation passes,
+    warps whose rows fall into different shards, and - with a tight arena - an overflow that
+    only shows up in a late pass.  Offsets must still be those of a walk in call order."""
+    w = wl.make_custom("passes", 3000, 3, 12, prompt_len=(0, 9), response=("uniform", 0, 40), vocab=999,
+                       micro_batch=9000, seed=61, with_entropy=True, schedule="none")
+    order = np.random.default_rng(3).permutation(w.n).astype(np.int32)
+    for tight in (False, True):
+        room = (w.len_response.reshape(w.S, -1).astype(np.int64) + 7) // 8 * 8
+        cap = int(room.sum(axis=1).min() * 0.9 // 8 * 8) if tight else None
+        o = H.make_oracle(w, response_cap=cap)
+        g = G.GpuDock(w, response_cap=cap)
+        for c in (w.column_index("response_ids"), w.column_index("prompt_ids"), w.column_index("entropy")):
+            cu, data = w.pack(c, order)
+            o.put(c, order, cu, data)
+            g.put(c, order, cu, data)
+        G.assert_state_equal(g, o, ctx=f"tight={tight}")
+        G.assert_stats_equal(g, o, f"tight={tight}")
+        assert (o.stats().n_arena_full > 0) == tight
+
+
 def test_output_capacity_truncation_matches(G):
     w = wl.make_custom("trunc", 8, 2, 2, prompt_len=(3, 40), response=("uniform", 1, 90), vocab=1000,
                        micro_batch=16, seed=7, schedule="none")
