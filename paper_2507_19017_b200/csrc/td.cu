@@ -38,7 +38,7 @@ inline uint32_t esize_of(int32_t dtype) { return dtype == TD_BF16 ? 2u : 4u; }
 
 // Dynamic shared memory of the copy kernels: the warps' stages and mbarriers, then (gather) the
 // block-scan scratch and the job table.
-constexpr size_t kStageSmem = (size_t)kCopyWarps * kStages * kStageBytes + (size_t)kCopyWarps * kStages * 8;
+constexpr size_t kStageSmem = (size_t)kCopyWarps * kPipeSmemPerWarp;
 size_t scatter_smem_bytes() { return kStageSmem; }
 size_t gather_smem_bytes(uint32_t njobs) { return kStageSmem + (size_t)kCopyWarps * 8 + (size_t)njobs * 8; }
 

@@ -186,8 +186,11 @@ __device__ __forceinline__ void copy_body_shifted(uint4 *dst, const uint8_t *src
     }
 }
 
+#ifndef TD_COPY_INLINE
+#define TD_COPY_INLINE __forceinline__
+#endif
 template <bool kSmem = false>
-__device__ __forceinline__ void warp_copy(uint8_t *dst, const uint8_t *src, uint64_t nbytes,
+__device__ TD_COPY_INLINE void warp_copy(uint8_t *dst, const uint8_t *src, uint64_t nbytes,
                                           uint32_t esz, uint32_t lane,
                                           const uint8_t *src_lo, const uint8_t *src_hi) {
     if (nbytes == 0) return;
@@ -264,10 +267,13 @@ __device__ __forceinline__ void warp_fill(uint8_t *dst, uint64_t nbytes, uint32_
 // With many resident warps per SM the metadata latency of one warp hides behind the copies of
 // the others; there is no block-wide barrier on the path.
 // --------------------------------------------------------------------------------------------
-constexpr int kCopyThreads = 256;
+#ifndef TD_COPY_THREADS
+#define TD_COPY_THREADS 256
+#endif
+constexpr int kCopyThreads = TD_COPY_THREADS;
 constexpr int kCopyWarps = kCopyThreads / 32;
 #ifndef TD_COPY_BLOCKS_PER_SM
-#define TD_COPY_BLOCKS_PER_SM 3
+#define TD_COPY_BLOCKS_PER_SM 2
 #endif
 #ifndef TD_CHUNK_TARGET_BYTES
 #define TD_CHUNK_TARGET_BYTES 32768
@@ -328,20 +334,30 @@ __device__ __forceinline__ uint64_t shfl_up_u64(uint64_t v, int delta) {
 }
 
 // --------------------------------------------------------------------------------------------
-// Asynchronous staging.  Each warp owns kStages shared-memory stages and one mbarrier per
-// stage.  A piece of a row is fetched with one bulk asynchronous copy (cp.async.bulk, global to
-// shared, completion counted in bytes on the stage's mbarrier) while the piece fetched before
-// it is written out from the other stage, so a warp keeps up to a stage of loads in flight
-// without holding a single register for them; the bytes in flight per SM are what a ragged
-// copy needs to cover HBM latency.  The bulk copy wants 16-byte aligned addresses and sizes:
+// Asynchronous staging.  Each warp owns a ring of kStages shared-memory stages with one
+// mbarrier and one descriptor each.  A piece of a row is fetched with one bulk asynchronous
+// copy (cp.async.bulk, global to shared, completion counted in bytes on the stage's mbarrier);
+// a piece is written out to its destination only when the ring is full and its stage is
+// needed again, so a warp keeps kStages copies in flight without holding a single register
+// for them; the bytes in flight per SM are what a ragged copy needs to cover HBM latency,
+// whatever the row lengths.  The bulk copy wants 16-byte aligned addresses and sizes:
 // the source window is widened to the enclosing 16-byte boundaries (rows in an arena start
 // aligned and are padded, so the window stays inside the arena) and the write-out shifts the
 // bytes into place.  Every wait on an mbarrier is bounded; a warp that gives up records the
 // error, falls back to plain loads and still drains its own copy before it returns.
 // --------------------------------------------------------------------------------------------
-constexpr int kStages = 2;
-constexpr uint32_t kStageBytes = 4096;
+#ifndef TD_STAGES
+#define TD_STAGES 2
+#endif
+#ifndef TD_STAGE_BYTES
+#define TD_STAGE_BYTES 6144
+#endif
+constexpr int kStages = TD_STAGES;
+constexpr uint32_t kStageBytes = TD_STAGE_BYTES;
 constexpr uint32_t kPieceMax = kStageBytes - 16;      // payload of one bulk copy; the aligned window still fits
+// stages, descriptors, mbarriers of one warp; rounded so that every warp's stages start 128-byte aligned
+constexpr size_t kPipeSmemPerWarp = (((size_t)kStages * (kStageBytes + 32 + 8)) + 127) & ~size_t(127);
+static_assert(kStageBytes % 16 == 0 && kPipeSmemPerWarp % 128 == 0, "bulk copies need 16-byte aligned stages");
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
@@ -363,21 +379,29 @@ __device__ __forceinline__ void bulk_global_to_shared(uint32_t dst, const void *
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 
+struct PieceDesc {             // one copy in flight, kept beside its stage in shared memory
+    uint8_t *dst;
+    const uint8_t *src;
+    uint32_t n;                // payload bytes
+    uint32_t pre;              // payload starts this many bytes into the stage (source misalignment)
+    uint32_t esz;
+    uint32_t pad;
+};
+
 struct WarpPipe {
     uint8_t *stage;            // this warp's kStages * kStageBytes bytes of shared memory
+    PieceDesc *desc;           // kStages descriptors
     uint32_t bar;              // shared address of this warp's kStages mbarriers
     uint32_t parity;           // bit s: phase the next wait on stage s looks for
-    uint32_t next;             // stage the next copy goes to
+    uint32_t head, tail;       // copies issued / written out so far; stage of copy i is i % kStages
     uint32_t spin_limit;
-    uint32_t failed;           // a wait ran out: plain loads from here on
-    bool pending;              // a copy is in flight and not yet written out
-    uint8_t *p_dst;
-    const uint8_t *p_src;
-    uint32_t p_n, p_pre, p_stage, p_esz;
+    uint32_t failed;           // bit 0: a wait ran out, plain loads from here on; bit 1 + s: stage s may still be landing
 
-    __device__ __forceinline__ void init(uint8_t *stage_mem, unsigned long long *bars, uint32_t lane, uint32_t spin) {
-        stage = stage_mem; bar = smem_u32(bars); parity = 0; next = 0; spin_limit = spin; failed = 0; pending = false;
-        p_dst = nullptr; p_src = nullptr; p_n = p_pre = p_stage = 0; p_esz = 4;
+    __device__ __forceinline__ void init(uint8_t *mem, uint32_t lane, uint32_t spin) {
+        stage = mem;
+        desc = reinterpret_cast<PieceDesc *>(mem + (size_t)kStages * kStageBytes);
+        bar = smem_u32(desc + kStages);
+        parity = 0; head = 0; tail = 0; spin_limit = spin; failed = 0;
         if (lane == 0) {
             for (int s = 0; s < kStages; ++s) mbar_init(bar + 8u * s, 1);
             fence_mbar_init();
@@ -395,22 +419,24 @@ struct WarpPipe {
         return ok;
     }
 
-    // write the pending piece out of its stage; if the wait runs out, copy it with plain loads
-    __device__ __forceinline__ void drain(uint32_t lane) {
-        if (!pending) return;
-        pending = false;
-        if (wait_stage(p_stage)) {
-            const uint8_t *s0 = stage + (size_t)p_stage * kStageBytes;
-            warp_copy<true>(p_dst, s0 + p_pre, p_n, p_esz, lane, s0, s0 + kStageBytes);
+    // write the oldest copy in flight out of its stage; if its wait runs out, redo it with plain loads
+    __device__ __forceinline__ void drain_one(uint32_t lane) {
+        const uint32_t s = tail % kStages;
+        ++tail;
+        __syncwarp();                                          // lane 0's descriptor is visible
+        const PieceDesc d = desc[s];
+        const uint8_t *s0 = stage + (size_t)s * kStageBytes;
+        if (wait_stage(s)) {
+            warp_copy<true>(d.dst, s0 + d.pre, d.n, d.esz, lane, s0, s0 + kStageBytes);
         } else {
-            failed |= 1u | (2u << p_stage);                // stage p_stage still has a copy in flight
-            warp_copy(p_dst, p_src, p_n, p_esz, lane, p_src, p_src + p_n);
+            failed |= 1u | (2u << s);
+            warp_copy(d.dst, d.src, d.n, d.esz, lane, d.src, d.src + d.n);
         }
     }
 
-    // before the warp returns: nothing of its own may still be landing in shared memory
+    // before the warp returns: everything written out, nothing of its own still landing
     __device__ __forceinline__ uint32_t finish(uint32_t lane) {
-        drain(lane);
+        while (tail != head) drain_one(lane);
         for (uint32_t s = 0; s < (uint32_t)kStages; ++s)
             if (failed & (2u << s)) wait_stage(s);
         return failed;
@@ -427,16 +453,17 @@ struct WarpPipe {
             if (failed || m < 64u || win < src_lo || win + size > src_hi) {
                 warp_copy(dst, src, m, esz, lane, src_lo, src_hi);       // short, at a buffer edge, or after a failure
             } else {
-                const uint32_t s = next;
+                if (head - tail == (uint32_t)kStages) drain_one(lane);   // every stage busy: free the oldest
+                const uint32_t s = head % kStages;
+                ++head;
                 __syncwarp();                                            // every lane is done reading stage s
                 if (lane == 0) {
+                    PieceDesc d; d.dst = dst; d.src = src; d.n = m; d.pre = pre; d.esz = esz; d.pad = 0;
+                    desc[s] = d;
                     fence_proxy_async();
                     mbar_expect_tx(bar + 8u * s, size);
                     bulk_global_to_shared(smem_u32(stage + (size_t)s * kStageBytes), win, size, bar + 8u * s);
                 }
-                drain(lane);                                             // the piece fetched before this one
-                pending = true; p_dst = dst; p_src = src; p_n = m; p_pre = pre; p_stage = s; p_esz = esz;
-                next = s ^ 1u;
             }
             dst += m; src += m; n -= m;
         }

@@ -369,25 +369,33 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
                   const GetReq *reqs_dev, const uint32_t n_req) {
     const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
     extern __shared__ __align__(128) uint8_t gather_smem[];
-    uint8_t *stages = gather_smem;                                           // [warps][stages][kStageBytes]
-    unsigned long long *bars = reinterpret_cast<unsigned long long *>(stages + kCopyWarps * kStages * kStageBytes);
-    uint64_t *s_wsum = reinterpret_cast<uint64_t *>(bars + kCopyWarps * kStages);
+    uint64_t *s_wsum = reinterpret_cast<uint64_t *>(gather_smem + (size_t)kCopyWarps * kPipeSmemPerWarp);
     uint64_t *job_end = s_wsum + kCopyWarps;        // [n_req * ncol] inclusive prefix of bytes (16-byte padded)
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     WarpPipe pipe;
-    pipe.init(stages + (size_t)warp * kStages * kStageBytes, bars + warp * kStages, lane, dv.spin_limit);
+    pipe.init(gather_smem + (size_t)warp * kPipeSmemPerWarp, lane, dv.spin_limit);
     griddep_wait();                                    // indices, cu_seqlens and result blocks are complete
     const uint32_t ncol = dv.ncol;
     const uint32_t njobs = n_req * ncol;
 
-    // job table: each thread sizes a contiguous run of jobs, then one block scan
+    // job table: sizes first (strided over the threads, so the dependent loads behind each
+    // size - request, result block - are all in flight together), then one block scan in which
+    // each thread owns a contiguous run
     {
         const uint32_t per = (njobs + kCopyThreads - 1) / kCopyThreads;
+        #pragma unroll 4
+        for (uint32_t i = 0; i < per; ++i) {
+            const uint32_t j = i * kCopyThreads + tid;
+            if (j < njobs) {
+                const uint32_t q = fast_div(j, dv.div_ncol);
+                job_end[j] = (job_bytes(dv, reqs[q], j - q * ncol) + 15) & ~uint64_t(15);
+            }
+        }
+        __syncthreads();
         const uint32_t j0 = min(tid * per, njobs), j1 = min(j0 + per, njobs);
         uint64_t local = 0;
         for (uint32_t j = j0; j < j1; ++j) {
-            const uint32_t q = fast_div(j, dv.div_ncol);
-            local += (job_bytes(dv, reqs[q], j - q * ncol) + 15) & ~uint64_t(15);
+            local += job_end[j];
             job_end[j] = local;                       // inclusive within the thread's run
         }
         uint64_t inc = local;

@@ -33,11 +33,9 @@ __global__ void __launch_bounds__(kCopyThreads, kCopyBlocksPerSM)
 put_scatter_kernel(const DockView dv, const PutBatch batch) {
     __shared__ uint64_t item_end[kMaxPutItems];       // inclusive prefix of bytes (16-byte padded) per item
     extern __shared__ __align__(128) uint8_t scatter_smem[];
-    uint8_t *stages = scatter_smem;                                          // [warps][stages][kStageBytes]
-    unsigned long long *bars = reinterpret_cast<unsigned long long *>(stages + kCopyWarps * kStages * kStageBytes);
     const uint32_t tid = threadIdx.x, lane = tid & 31;
-    WarpPipe pipe;
-    pipe.init(stages + (size_t)(tid >> 5) * kStages * kStageBytes, bars + (tid >> 5) * kStages, lane, dv.spin_limit);
+    WarpPipe pipe;                                                           // [warps][kPipeSmemPerWarp]
+    pipe.init(scatter_smem + (size_t)(tid >> 5) * kPipeSmemPerWarp, lane, dv.spin_limit);
     griddep_launch_dependents();
     griddep_wait();                                    // the alloc kernel's tables are complete
 
