@@ -378,11 +378,13 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
 
     if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
+    // word 1 of the scan scratch is the gather's chunk counter
+    unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
     if (launch_dep(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
-               (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
+               (const ConsumerSlot *)nullptr, seq, counter, (uint64_t *)nullptr) != cudaSuccess) return TD_ECUDA;
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
     if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(v.ncol), st, v, one,
-                     (const GetReq *)nullptr, 1u) != cudaSuccess) return TD_ECUDA;
+                     (const GetReq *)nullptr, 1u, counter, (const uint64_t *)nullptr) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 
@@ -453,11 +455,13 @@ int td_get_static(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_
 
     if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
+    // word 1 of the scan scratch is the gather's chunk counter
+    unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
     if (launch_dep(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
-               (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
+               (const ConsumerSlot *)nullptr, seq, counter, (uint64_t *)nullptr) != cudaSuccess) return TD_ECUDA;
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
     if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(v.ncol), st, v, one,
-                     (const GetReq *)nullptr, 1u) != cudaSuccess) return TD_ECUDA;
+                     (const GetReq *)nullptr, 1u, counter, (const uint64_t *)nullptr) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 
@@ -468,6 +472,8 @@ struct td_plan {
     GetReq *d_reqs;
     ConsumerSlot *d_slots;
     uint64_t room_bytes;
+    unsigned long long *d_counter;        // the gather's chunk counter: word 1 of slot 0's scan scratch
+    uint64_t *d_job_sizes;                // [n_req][n_columns] output bytes, written by the finalize kernel
     std::vector<uint8_t> host_image;      // what was uploaded; kept until the plan dies
 };
 
@@ -475,7 +481,8 @@ size_t td_plan_bytes(const td_dock *d, uint32_t n_req) {
     if (!d || n_req == 0) return 0;
     const size_t slots = d->dv.ncons;
     return align_up_sz((size_t)n_req * sizeof(GetReq), 256) + align_up_sz(slots * sizeof(ConsumerSlot), 256) +
-           slots * align_up_sz(sel_scratch_bytes(d->dv.G), 256);
+           slots * align_up_sz(sel_scratch_bytes(d->dv.G), 256) +
+           align_up_sz((size_t)n_req * d->dv.ncol * sizeof(uint64_t), 256);
 }
 
 int td_plan_create(td_dock *d, const td_get_req *reqs, uint32_t n_req, void *d_plan, size_t plan_bytes,
@@ -527,6 +534,8 @@ int td_plan_create(td_dock *d, const td_get_req *reqs, uint32_t n_req, void *d_p
         room += room_bytes_of(v, c, reqs[q].max_samples, reqs[q].out);
     }
     p->n_slots = n_slots;
+    p->d_counter = reinterpret_cast<unsigned long long *>(base + off_scratch) + 1;
+    p->d_job_sizes = reinterpret_cast<uint64_t *>(base + off_scratch + (size_t)v.ncons * scratch_each);
     p->room_bytes = room;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(base + off_scratch, 0, (size_t)v.ncons * scratch_each, st) != cudaSuccess ||
@@ -553,10 +562,10 @@ int td_get_many(td_dock *d, td_plan *p, void *stream) {
     if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), p->n_slots), dim3(kSelThreads), 0, st, v, none,
                (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
     if (launch_dep(d, get_finalize_kernel, dim3(p->n_req), dim3(kFinThreads), 0, st, v, none, (const GetReq *)p->d_reqs,
-               (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
+               (const ConsumerSlot *)p->d_slots, seq, p->d_counter, p->d_job_sizes) != cudaSuccess) return TD_ECUDA;
     if (launch_timed(d, 1, get_gather_kernel, dim3(copy_grid(d, p->room_bytes)), dim3(kCopyThreads),
                      gather_smem_bytes(p->n_req * v.ncol), st, v, none,
-                     (const GetReq *)p->d_reqs, p->n_req) != cudaSuccess) return TD_ECUDA;
+                     (const GetReq *)p->d_reqs, p->n_req, p->d_counter, (const uint64_t *)p->d_job_sizes) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 

@@ -304,6 +304,25 @@ __device__ __forceinline__ ChunkPlan plan_chunks(uint64_t total_bytes, uint64_t 
     return p;
 }
 
+// Chunks for a launch whose warps fetch them from a shared counter: about TD_DYN_CHUNKS_PER_WARP per
+// warp, between 16 KB and 32 KB each.
+#ifndef TD_DYN_CHUNKS_PER_WARP
+#define TD_DYN_CHUNKS_PER_WARP 2
+#endif
+__device__ __forceinline__ ChunkPlan plan_chunks_dynamic(uint64_t total_bytes, uint64_t n_warps) {
+    ChunkPlan p;
+    uint64_t c = total_bytes / (n_warps * TD_DYN_CHUNKS_PER_WARP);
+    c = (c + 15) & ~uint64_t(15);
+#ifndef TD_DYN_MIN_CHUNK
+#define TD_DYN_MIN_CHUNK 16384
+#endif
+    if (c < TD_DYN_MIN_CHUNK) c = TD_DYN_MIN_CHUNK;
+    if (c > 32768) c = 32768;
+    p.chunk_bytes = c;
+    p.n_chunks = (total_bytes + c - 1) / c;
+    return p;
+}
+
 // Largest i in [0, rows) with cu[i] <= x (the row holding element x, rows of length zero
 // skipped); 0 when even cu[0] > x.  Warp-cooperative; all lanes get the answer.
 __device__ __forceinline__ uint32_t warp_find_row(const int32_t *cu, uint32_t rows, int64_t x, uint32_t lane) {

@@ -206,9 +206,21 @@ __device__ __forceinline__ uint64_t block_scan_incl_2(uint64_t a, uint64_t b, ui
     return a + oa;
 }
 
+// Output bytes of column k of a request that serves n_s samples with these token totals.
+__device__ __forceinline__ uint64_t job_bytes_of(const DockView &dv, const GetReq &rq, uint32_t k,
+                                                 uint64_t n_s, uint64_t prompt_tokens, uint64_t response_tokens) {
+    const td_get_out &out = rq.out;
+    if (!((dv.outm[rq.consumer] >> k) & 1u) || out.col[k] == nullptr) return 0;
+    const uint32_t cls = dv.col_cls[k], esz = dv.col_esz[k];
+    if (cls == TD_SCALAR) return n_s * esz;
+    if (out.mode == TD_PACKED) return (cls == TD_PROMPT ? prompt_tokens : response_tokens) * esz;
+    return n_s * (uint64_t)(cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to) * esz;
+}
+
 __global__ void __launch_bounds__(kFinThreads)
 get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
-                    const GetReq *reqs_dev, const ConsumerSlot *slots_dev, const uint32_t seq) {
+                    const GetReq *reqs_dev, const ConsumerSlot *slots_dev, const uint32_t seq,
+                    unsigned long long *work_counter, uint64_t *job_sizes) {
     const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
     const ConsumerSlot *slots = slots_dev ? slots_dev : &one.cs;
     const GetReq &rq = reqs[blockIdx.x];
@@ -221,6 +233,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     __shared__ uint32_t s_first_over;
     griddep_launch_dependents();
     griddep_wait();                                    // the scan's candidate list is complete
+    if (blockIdx.x == 0 && threadIdx.x == 0) *work_counter = 0;     // the gather hands out its chunks from zero
 
     // how many groups were ready, from the last tile's inclusive prefix
     const unsigned long long last = sc.desc[sel_tiles(dv.G) - 1];
@@ -345,6 +358,11 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
         atomicAdd(&dv.counters[CNT_GOT_SAMPLES + c], (unsigned long long)n_s);
         atomicAdd(&dv.counters[CNT_GOT_TOKENS + c], (unsigned long long)(r.prompt_tokens + r.response_tokens));
     }
+    // the gather's job table: this request's output bytes per column, padded to 16
+    if (job_sizes && tid < dv.ncol)
+        job_sizes[(size_t)blockIdx.x * dv.ncol + tid] =
+            (job_bytes_of(dv, rq, tid, n_s, (uint64_t)(int64_t)out.cu_prompt[n_s],
+                          (uint64_t)(int64_t)out.cu_response[n_s]) + 15) & ~uint64_t(15);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -354,19 +372,14 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
 // td_device.cuh).
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ uint64_t job_bytes(const DockView &dv, const GetReq &rq, uint32_t k) {
-    const td_get_out &out = rq.out;
-    if (!((dv.outm[rq.consumer] >> k) & 1u) || out.col[k] == nullptr) return 0;
-    const td_result *res = out.result;
-    const uint32_t cls = dv.col_cls[k], esz = dv.col_esz[k];
-    const uint64_t n_s = res->n_samples;
-    if (cls == TD_SCALAR) return n_s * esz;
-    if (out.mode == TD_PACKED) return (cls == TD_PROMPT ? res->prompt_tokens : res->response_tokens) * esz;
-    return n_s * (uint64_t)(cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to) * esz;
+    const td_result *res = rq.out.result;
+    return job_bytes_of(dv, rq, k, res->n_samples, res->prompt_tokens, res->response_tokens);
 }
 
 __global__ void __launch_bounds__(kCopyThreads, kCopyBlocksPerSM)
 get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
-                  const GetReq *reqs_dev, const uint32_t n_req) {
+                  const GetReq *reqs_dev, const uint32_t n_req, unsigned long long *work_counter,
+                  const uint64_t *job_sizes) {
     const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
     extern __shared__ __align__(128) uint8_t gather_smem[];
     uint64_t *s_wsum = reinterpret_cast<uint64_t *>(gather_smem + (size_t)kCopyWarps * kPipeSmemPerWarp);
@@ -387,8 +400,12 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
         for (uint32_t i = 0; i < per; ++i) {
             const uint32_t j = i * kCopyThreads + tid;
             if (j < njobs) {
-                const uint32_t q = fast_div(j, dv.div_ncol);
-                job_end[j] = (job_bytes(dv, reqs[q], j - q * ncol) + 15) & ~uint64_t(15);
+                if (job_sizes) {
+                    job_end[j] = job_sizes[j];                 // written by the finalize kernel
+                } else {
+                    const uint32_t q = fast_div(j, dv.div_ncol);
+                    job_end[j] = (job_bytes(dv, reqs[q], j - q * ncol) + 15) & ~uint64_t(15);
+                }
             }
         }
         __syncthreads();
@@ -413,10 +430,16 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
     }
     const uint64_t total_all = njobs ? job_end[njobs - 1] : 0;
     const uint64_t n_warps = (uint64_t)gridDim.x * kCopyWarps;
-    const ChunkPlan plan = plan_chunks(total_all, n_warps);
-    const uint64_t warp0 = (uint64_t)blockIdx.x * kCopyWarps + warp;
+    // Chunks are handed out by a counter in scratch memory (zeroed by the finalize kernel): equal
+    // bytes are not equal time when one chunk holds a few long rows and another many short ones.
+    const ChunkPlan plan = plan_chunks_dynamic(total_all, n_warps);
+    unsigned long long ch = 0;
+    if (lane == 0) ch = atomicAdd(work_counter, 1ull);
+    ch = shfl_u64(ch, 0);
 
-    for (uint64_t ch = warp0; ch < plan.n_chunks; ch += n_warps) {
+    while (ch < plan.n_chunks) {
+        unsigned long long next = 0;
+        if (lane == 0) next = atomicAdd(work_counter, 1ull);       // in flight while this chunk is copied
         uint64_t g0 = ch * plan.chunk_bytes;
         const uint64_t g1 = min(g0 + plan.chunk_bytes, total_all);
         // first job that reaches beyond g0
@@ -490,6 +513,7 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
                 }
             }
         }
+        ch = shfl_u64(next, 0);
     }
     if (pipe.finish(lane) && lane == 0) flag_error(dv, TD_ERR_COPY_TIMEOUT, CNT_TIMEOUT);
 }

@@ -189,7 +189,7 @@ def test_put_many_get_many_small(G):
     _many_vs_serial(G, w, mode=td.PADDED)
 
 
-@pytest.mark.parametrize("cid", [2, 3])
+@pytest.mark.parametrize("cid", [2, 3, 5])
 def test_put_many_get_many_full_size(G, cid):
     _many_vs_serial(G, wl.make_config(cid))
 
