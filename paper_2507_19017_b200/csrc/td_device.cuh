@@ -105,127 +105,45 @@ __device__ __forceinline__ void flag_error(const DockView &dv, uint32_t bit, int
 }
 
 // --------------------------------------------------------------------------------------------
-// Warp-cooperative copy of nbytes from src to dst.  Both are aligned to the element size
-// (2 or 4 bytes) and nbytes is a multiple of it; nothing else is assumed.  Stores are issued
-// as aligned 16-byte vectors; the source stream is read as aligned 16-byte vectors too and
-// shifted into place when the two sides disagree modulo 16.  [src_lo, src_hi) bounds the
-// buffer the source lies in: an aligned source vector that would reach outside it is
-// assembled from element loads instead.
+// Warp-cooperative copy of n bytes from src to dst.  Both addresses and n are multiples of the
+// element size (2 or 4 bytes); nothing else is assumed.  Stores are 16-byte vectors aligned on
+// dst, each fed by four 32-bit loads (eight 16-bit loads when the two sides differ by an odd
+// number of half words) at whatever alignment the source has; head and tail move half words.
+// It reads exactly the bytes it copies, and src may be shared memory (a stage) or global
+// memory.  Kept small on purpose: it is inlined into the copy kernels' inner loops, and their
+// instruction footprint showed up as fetch stalls.
 // --------------------------------------------------------------------------------------------
-__device__ __forceinline__ void copy_elems(uint8_t *dst, const uint8_t *src, uint32_t count,
-                                           uint32_t esz, uint32_t lane) {
-    // count < 32 elements
-    if (lane < count) {
-        if (esz == 4)
-            reinterpret_cast<uint32_t *>(dst)[lane] = reinterpret_cast<const uint32_t *>(src)[lane];
-        else
-            reinterpret_cast<uint16_t *>(dst)[lane] = reinterpret_cast<const uint16_t *>(src)[lane];
-    }
-}
-
-// kSmem: the source is a shared-memory stage (plain load); else global memory read once (streaming load)
-template <bool kSmem>
-__device__ __forceinline__ uint4 ld_stream(const uint4 *p) {
-    if (kSmem) return *p;
-    return __ldcs(p);
-}
-__device__ __forceinline__ void st_stream(uint4 *p, uint4 v) { __stcs(p, v); }
-
-// 16 source bytes starting `delta` bytes into the 32-byte window (a, b); delta in 2..14, even.
-template <int WSH>
-__device__ __forceinline__ uint4 shift_window(const uint4 &a, const uint4 &b, uint32_t bsh) {
-    const uint32_t w[8] = {a.x, a.y, a.z, a.w, b.x, b.y, b.z, b.w};
-    uint4 r;
-    r.x = __funnelshift_r(w[WSH + 0], w[WSH + 1], bsh);
-    r.y = __funnelshift_r(w[WSH + 1], w[WSH + 2], bsh);
-    r.z = __funnelshift_r(w[WSH + 2], w[WSH + 3], bsh);
-    r.w = __funnelshift_r(w[WSH + 3], w[(WSH + 4) & 7], bsh);   // w[WSH+4] is only used when bsh > 0
-    return r;
-}
-
-__device__ __forceinline__ uint4 load_window_slow(const uint8_t *p, uint32_t esz) {
-    // 16 bytes from an element-aligned address, element by element
-    uint4 r;
-    if (esz == 4) {
-        const uint32_t *q = reinterpret_cast<const uint32_t *>(p);
-        r.x = q[0]; r.y = q[1]; r.z = q[2]; r.w = q[3];
-    } else {
-        const uint16_t *q = reinterpret_cast<const uint16_t *>(p);
-        r.x = q[0] | (uint32_t(q[1]) << 16); r.y = q[2] | (uint32_t(q[3]) << 16);
-        r.z = q[4] | (uint32_t(q[5]) << 16); r.w = q[6] | (uint32_t(q[7]) << 16);
-    }
-    return r;
-}
-
-template <int WSH, bool kSmem>
-__device__ __forceinline__ void copy_body_shifted(uint4 *dst, const uint8_t *src, uint32_t nvec,
-                                                  uint32_t delta, uint32_t esz, uint32_t lane,
-                                                  const uint8_t *src_lo, const uint8_t *src_hi) {
-    const uint4 *S = reinterpret_cast<const uint4 *>(src - delta);
-    const uint32_t bsh = (delta & 3u) * 8u;
-    // vectors whose 32-byte window lies inside [src_lo, src_hi)
-    uint32_t v_lo = 0, v_hi = nvec;
-    if (reinterpret_cast<const uint8_t *>(S) < src_lo) v_lo = 1;
-    if (reinterpret_cast<const uint8_t *>(S + nvec + 1) > src_hi) v_hi = nvec - 1;
-    if (lane == 0) {
-        if (v_lo == 1) st_stream(dst, load_window_slow(src, esz));
-        if (v_hi != nvec && nvec >= 1 && !(v_lo == 1 && nvec == 1))
-            st_stream(dst + (nvec - 1), load_window_slow(src + 16ull * (nvec - 1), esz));
-    }
-    if (v_hi <= v_lo) return;
-    uint32_t v = v_lo + lane;
-    for (; v + 32 < v_hi; v += 64) {
-        uint4 a0 = ld_stream<kSmem>(S + v),      b0 = ld_stream<kSmem>(S + v + 1);
-        uint4 a1 = ld_stream<kSmem>(S + v + 32), b1 = ld_stream<kSmem>(S + v + 33);
-        st_stream(dst + v,      shift_window<WSH>(a0, b0, bsh));
-        st_stream(dst + v + 32, shift_window<WSH>(a1, b1, bsh));
-    }
-    for (; v < v_hi; v += 32) {
-        uint4 a = ld_stream<kSmem>(S + v), b = ld_stream<kSmem>(S + v + 1);
-        st_stream(dst + v, shift_window<WSH>(a, b, bsh));
-    }
-}
-
-#ifndef TD_COPY_INLINE
-#define TD_COPY_INLINE __forceinline__
-#endif
-template <bool kSmem = false>
-__device__ TD_COPY_INLINE void warp_copy(uint8_t *dst, const uint8_t *src, uint64_t nbytes,
-                                          uint32_t esz, uint32_t lane,
-                                          const uint8_t *src_lo, const uint8_t *src_hi) {
-    if (nbytes == 0) return;
-    // head: bring dst to a 16-byte boundary
+__device__ __forceinline__ void warp_copy(uint8_t *dst, const uint8_t *src, uint32_t n, uint32_t lane) {
     uint32_t head = (16u - (uint32_t)(reinterpret_cast<uintptr_t>(dst) & 15u)) & 15u;
-    if (head > nbytes) head = (uint32_t)nbytes;
-    if (head) {
-        copy_elems(dst, src, head / esz, esz, lane);
-        dst += head; src += head; nbytes -= head;
-    }
-    const uint32_t nvec = (uint32_t)(nbytes >> 4);
-    const uint32_t delta = (uint32_t)(reinterpret_cast<uintptr_t>(src) & 15u);
-    if (nvec) {
-        uint4 *D = reinterpret_cast<uint4 *>(dst);
-        if (delta == 0) {
-            const uint4 *S = reinterpret_cast<const uint4 *>(src);
-            uint32_t v = lane;
-            for (; v + 96 < nvec; v += 128) {
-                uint4 a0 = ld_stream<kSmem>(S + v), a1 = ld_stream<kSmem>(S + v + 32);
-                uint4 a2 = ld_stream<kSmem>(S + v + 64), a3 = ld_stream<kSmem>(S + v + 96);
-                st_stream(D + v, a0); st_stream(D + v + 32, a1);
-                st_stream(D + v + 64, a2); st_stream(D + v + 96, a3);
-            }
-            for (; v < nvec; v += 32) st_stream(D + v, ld_stream<kSmem>(S + v));
-        } else {
-            switch (delta >> 2) {
-                case 0: copy_body_shifted<0, kSmem>(D, src, nvec, delta, esz, lane, src_lo, src_hi); break;
-                case 1: copy_body_shifted<1, kSmem>(D, src, nvec, delta, esz, lane, src_lo, src_hi); break;
-                case 2: copy_body_shifted<2, kSmem>(D, src, nvec, delta, esz, lane, src_lo, src_hi); break;
-                default: copy_body_shifted<3, kSmem>(D, src, nvec, delta, esz, lane, src_lo, src_hi); break;
-            }
+    if (head > n) head = n;
+    if (lane < (head >> 1)) reinterpret_cast<uint16_t *>(dst)[lane] = reinterpret_cast<const uint16_t *>(src)[lane];
+    dst += head; src += head; n -= head;
+    const uint32_t nvec = n >> 4;
+    uint4 *D = reinterpret_cast<uint4 *>(dst);
+    if ((reinterpret_cast<uintptr_t>(src) & 3u) == 0) {
+        const uint32_t *S = reinterpret_cast<const uint32_t *>(src);
+        uint32_t v = lane;
+        for (; v + 32 < nvec; v += 64) {
+            const uint32_t *p = S + 4u * v, *q = p + 128;
+            const uint4 a = make_uint4(p[0], p[1], p[2], p[3]);
+            const uint4 b = make_uint4(q[0], q[1], q[2], q[3]);
+            __stcs(D + v, a); __stcs(D + v + 32, b);
+        }
+        for (; v < nvec; v += 32) {
+            const uint32_t *p = S + 4u * v;
+            __stcs(D + v, make_uint4(p[0], p[1], p[2], p[3]));
+        }
+    } else {
+        const uint16_t *S = reinterpret_cast<const uint16_t *>(src);
+        for (uint32_t v = lane; v < nvec; v += 32) {
+            const uint16_t *p = S + 8u * v;
+            __stcs(D + v, make_uint4(p[0] | ((uint32_t)p[1] << 16), p[2] | ((uint32_t)p[3] << 16),
+                                     p[4] | ((uint32_t)p[5] << 16), p[6] | ((uint32_t)p[7] << 16)));
         }
     }
-    const uint32_t tail = (uint32_t)(nbytes & 15u);
-    if (tail) copy_elems(dst + 16ull * nvec, src + 16ull * nvec, tail / esz, esz, lane);
+    const uint32_t tail = n & 15u;
+    if (lane < (tail >> 1))
+        reinterpret_cast<uint16_t *>(dst + (nvec << 4))[lane] = reinterpret_cast<const uint16_t *>(src + (nvec << 4))[lane];
 }
 
 // Warp-cooperative fill of nbytes at dst (element aligned) with the element pattern `bits`.
@@ -245,7 +163,7 @@ __device__ __forceinline__ void warp_fill(uint8_t *dst, uint64_t nbytes, uint32_
     const uint64_t nvec = nbytes >> 4;
     uint4 *D = reinterpret_cast<uint4 *>(dst);
     const uint4 val = make_uint4(word, word, word, word);
-    for (uint64_t v = lane; v < nvec; v += 32) st_stream(D + v, val);
+    for (uint64_t v = lane; v < nvec; v += 32) __stcs(D + v, val);
     const uint32_t tail = (uint32_t)(nbytes & 15u);
     if (tail && lane < tail / esz) {
         uint8_t *t = dst + 16ull * nvec;
@@ -446,10 +364,10 @@ struct WarpPipe {
         const PieceDesc d = desc[s];
         const uint8_t *s0 = stage + (size_t)s * kStageBytes;
         if (wait_stage(s)) {
-            warp_copy<true>(d.dst, s0 + d.pre, d.n, d.esz, lane, s0, s0 + kStageBytes);
+            warp_copy(d.dst, s0 + d.pre, d.n, lane);
         } else {
             failed |= 1u | (2u << s);
-            warp_copy(d.dst, d.src, d.n, d.esz, lane, d.src, d.src + d.n);
+            warp_copy(d.dst, d.src, d.n, lane);
         }
     }
 
@@ -470,7 +388,7 @@ struct WarpPipe {
             const uint8_t *win = src - pre;
             const uint32_t size = (pre + m + 15u) & ~15u;
             if (failed || m < 64u || win < src_lo || win + size > src_hi) {
-                warp_copy(dst, src, m, esz, lane, src_lo, src_hi);       // short, at a buffer edge, or after a failure
+                warp_copy(dst, src, m, lane);                            // short, at a buffer edge, or after a failure
             } else {
                 if (head - tail == (uint32_t)kStages) drain_one(lane);   // every stage busy: free the oldest
                 const uint32_t s = head % kStages;
