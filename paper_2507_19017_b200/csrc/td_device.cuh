@@ -362,13 +362,12 @@ struct WarpPipe {
         ++tail;
         __syncwarp();                                          // lane 0's descriptor is visible
         const PieceDesc d = desc[s];
-        const uint8_t *s0 = stage + (size_t)s * kStageBytes;
-        if (wait_stage(s)) {
-            warp_copy(d.dst, s0 + d.pre, d.n, lane);
-        } else {
+        const uint8_t *from = stage + (size_t)s * kStageBytes + d.pre;
+        if (!wait_stage(s)) {                                  // never seen; the piece is read again, directly
             failed |= 1u | (2u << s);
-            warp_copy(d.dst, d.src, d.n, lane);
+            from = d.src;
         }
+        warp_copy(d.dst, from, d.n, lane);
     }
 
     // before the warp returns: everything written out, nothing of its own still landing
