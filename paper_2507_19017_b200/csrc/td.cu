@@ -40,7 +40,9 @@ inline uint32_t esize_of(int32_t dtype) { return dtype == TD_BF16 ? 2u : 4u; }
 // block-scan scratch and the job table.
 constexpr size_t kStageSmem = (size_t)kCopyWarps * kPipeSmemPerWarp;
 size_t scatter_smem_bytes() { return kStageSmem; }
-size_t gather_smem_bytes(uint32_t njobs) { return kStageSmem + (size_t)kCopyWarps * 8 + (size_t)njobs * 8; }
+size_t gather_smem_bytes(uint32_t n_req, uint32_t ncol) {
+    return kStageSmem + (size_t)kCopyWarps * 8 + (size_t)n_req * ncol * 8 + (size_t)n_req * 4;
+}
 
 struct Layout {
     size_t status, len[3], off[3], cursor[3], claim, consumed, errword, counters, col[kMaxColumns], total;
@@ -53,7 +55,8 @@ bool valid_config(const td_config *c) {
     if (c->n_prompts == 0 || c->n_per_group == 0 || c->n_shards == 0 || c->n_shards > 256) return false;
     if (c->n_prompts % c->n_shards) return false;
     if (c->n_columns == 0 || c->n_columns > 32 || c->n_consumers == 0 || c->n_consumers > 32) return false;
-    if ((uint64_t)c->n_prompts * c->n_per_group >= (1ull << 30)) return false;
+    if ((uint64_t)c->n_prompts * c->n_per_group >= (1ull << 28)) return false;   // a row count fits 28 bits
+
     for (uint32_t k = 0; k < c->n_columns; ++k) {
         const td_column &col = c->columns[k];
         if (col.dtype < TD_I32 || col.dtype > TD_BF16) return false;
@@ -184,7 +187,7 @@ int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **o
     if (cudaFuncSetAttribute(put_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)scatter_smem_bytes()) != cudaSuccess ||
         cudaFuncSetAttribute(get_gather_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             (int)gather_smem_bytes(kMaxJobs)) != cudaSuccess)
+                             (int)gather_smem_bytes(kMaxJobs, 1)) != cudaSuccess)
         return TD_ECUDA;
 
     td_dock *d = new (std::nothrow) td_dock();
@@ -381,10 +384,10 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
     if (launch_dep(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
-               (const ConsumerSlot *)nullptr, seq, counter, (uint64_t *)nullptr) != cudaSuccess) return TD_ECUDA;
+               (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr) != cudaSuccess) return TD_ECUDA;
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
-    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(v.ncol), st, v, one,
-                     (const GetReq *)nullptr, 1u, counter, (const uint64_t *)nullptr) != cudaSuccess) return TD_ECUDA;
+    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, v.ncol), st, v, one,
+                     (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 
@@ -458,10 +461,10 @@ int td_get_static(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
     if (launch_dep(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
-               (const ConsumerSlot *)nullptr, seq, counter, (uint64_t *)nullptr) != cudaSuccess) return TD_ECUDA;
+               (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr) != cudaSuccess) return TD_ECUDA;
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
-    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(v.ncol), st, v, one,
-                     (const GetReq *)nullptr, 1u, counter, (const uint64_t *)nullptr) != cudaSuccess) return TD_ECUDA;
+    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, v.ncol), st, v, one,
+                     (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 
@@ -473,7 +476,7 @@ struct td_plan {
     ConsumerSlot *d_slots;
     uint64_t room_bytes;
     unsigned long long *d_counter;        // the gather's chunk counter: word 1 of slot 0's scan scratch
-    uint64_t *d_job_sizes;                // [n_req][n_columns] output bytes, written by the finalize kernel
+    JobSize *d_job_sizes;                 // [n_req][n_columns] output bytes and rows, written by the finalize kernel
     std::vector<uint8_t> host_image;      // what was uploaded; kept until the plan dies
 };
 
@@ -482,7 +485,7 @@ size_t td_plan_bytes(const td_dock *d, uint32_t n_req) {
     const size_t slots = d->dv.ncons;
     return align_up_sz((size_t)n_req * sizeof(GetReq), 256) + align_up_sz(slots * sizeof(ConsumerSlot), 256) +
            slots * align_up_sz(sel_scratch_bytes(d->dv.G), 256) +
-           align_up_sz((size_t)n_req * d->dv.ncol * sizeof(uint64_t), 256);
+           align_up_sz((size_t)n_req * d->dv.ncol * sizeof(JobSize), 256);
 }
 
 int td_plan_create(td_dock *d, const td_get_req *reqs, uint32_t n_req, void *d_plan, size_t plan_bytes,
@@ -535,7 +538,7 @@ int td_plan_create(td_dock *d, const td_get_req *reqs, uint32_t n_req, void *d_p
     }
     p->n_slots = n_slots;
     p->d_counter = reinterpret_cast<unsigned long long *>(base + off_scratch) + 1;
-    p->d_job_sizes = reinterpret_cast<uint64_t *>(base + off_scratch + (size_t)v.ncons * scratch_each);
+    p->d_job_sizes = reinterpret_cast<JobSize *>(base + off_scratch + (size_t)v.ncons * scratch_each);
     p->room_bytes = room;
     cudaStream_t st = (cudaStream_t)stream;
     if (cudaMemsetAsync(base + off_scratch, 0, (size_t)v.ncons * scratch_each, st) != cudaSuccess ||
@@ -564,8 +567,8 @@ int td_get_many(td_dock *d, td_plan *p, void *stream) {
     if (launch_dep(d, get_finalize_kernel, dim3(p->n_req), dim3(kFinThreads), 0, st, v, none, (const GetReq *)p->d_reqs,
                (const ConsumerSlot *)p->d_slots, seq, p->d_counter, p->d_job_sizes) != cudaSuccess) return TD_ECUDA;
     if (launch_timed(d, 1, get_gather_kernel, dim3(copy_grid(d, p->room_bytes)), dim3(kCopyThreads),
-                     gather_smem_bytes(p->n_req * v.ncol), st, v, none,
-                     (const GetReq *)p->d_reqs, p->n_req, p->d_counter, (const uint64_t *)p->d_job_sizes) != cudaSuccess) return TD_ECUDA;
+                     gather_smem_bytes(p->n_req, v.ncol), st, v, none,
+                     (const GetReq *)p->d_reqs, p->n_req, p->d_counter, (const JobSize *)p->d_job_sizes) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 

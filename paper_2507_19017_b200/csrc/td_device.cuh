@@ -113,7 +113,7 @@ __device__ __forceinline__ void flag_error(const DockView &dv, uint32_t bit, int
 // memory.  Kept small on purpose: it is inlined into the copy kernels' inner loops, and their
 // instruction footprint showed up as fetch stalls.
 // --------------------------------------------------------------------------------------------
-__device__ __forceinline__ void warp_copy(uint8_t *dst, const uint8_t *src, uint32_t n, uint32_t lane) {
+__device__ __noinline__ void warp_copy(uint8_t *dst, const uint8_t *src, uint32_t n, uint32_t lane) {
     uint32_t head = (16u - (uint32_t)(reinterpret_cast<uintptr_t>(dst) & 15u)) & 15u;
     if (head > n) head = n;
     if (lane < (head >> 1)) reinterpret_cast<uint16_t *>(dst)[lane] = reinterpret_cast<const uint16_t *>(src)[lane];
@@ -144,6 +144,52 @@ __device__ __forceinline__ void warp_copy(uint8_t *dst, const uint8_t *src, uint
     const uint32_t tail = n & 15u;
     if (lane < (tail >> 1))
         reinterpret_cast<uint16_t *>(dst + (nvec << 4))[lane] = reinterpret_cast<const uint16_t *>(src + (nvec << 4))[lane];
+}
+
+// The same copy with the source in shared memory, given as a shared-window address: the loads
+// are ld.shared instead of generic loads that find out at run time which memory they address.
+__device__ __forceinline__ uint32_t lds_u32(uint32_t a) {
+    uint32_t v;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t lds_u16(uint32_t a) {
+    uint16_t v;
+    asm volatile("ld.shared.u16 %0, [%1];" : "=h"(v) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint4 lds_4x32(uint32_t a) {
+    uint4 v;
+    asm volatile("ld.shared.u32 %0, [%4];\n\tld.shared.u32 %1, [%4+4];\n\tld.shared.u32 %2, [%4+8];\n\tld.shared.u32 %3, [%4+12];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "r"(a));
+    return v;
+}
+__device__ __forceinline__ uint32_t smem_u32(const void *p);
+__device__ __forceinline__ void warp_copy_from_shared(uint8_t *dst, uint32_t src, uint32_t n, uint32_t lane) {
+    uint32_t head = (16u - (uint32_t)(reinterpret_cast<uintptr_t>(dst) & 15u)) & 15u;
+    if (head > n) head = n;
+    if (lane < (head >> 1)) reinterpret_cast<uint16_t *>(dst)[lane] = (uint16_t)lds_u16(src + 2u * lane);
+    dst += head; src += head; n -= head;
+    const uint32_t nvec = n >> 4;
+    uint4 *D = reinterpret_cast<uint4 *>(dst);
+    if ((src & 3u) == 0) {
+        uint32_t v = lane;
+        for (; v + 32 < nvec; v += 64) {
+            const uint4 a = lds_4x32(src + 16u * v);
+            const uint4 b = lds_4x32(src + 16u * v + 512u);
+            __stcs(D + v, a); __stcs(D + v + 32, b);
+        }
+        for (; v < nvec; v += 32) __stcs(D + v, lds_4x32(src + 16u * v));
+    } else {
+        for (uint32_t v = lane; v < nvec; v += 32) {
+            const uint32_t p = src + 16u * v;
+            __stcs(D + v, make_uint4(lds_u16(p) | (lds_u16(p + 2) << 16), lds_u16(p + 4) | (lds_u16(p + 6) << 16),
+                                     lds_u16(p + 8) | (lds_u16(p + 10) << 16), lds_u16(p + 12) | (lds_u16(p + 14) << 16)));
+        }
+    }
+    const uint32_t tail = n & 15u;
+    if (lane < (tail >> 1))
+        reinterpret_cast<uint16_t *>(dst + (nvec << 4))[lane] = (uint16_t)lds_u16(src + (nvec << 4) + 2u * lane);
 }
 
 // Warp-cooperative fill of nbytes at dst (element aligned) with the element pattern `bits`.
@@ -243,9 +289,14 @@ __device__ __forceinline__ ChunkPlan plan_chunks_dynamic(uint64_t total_bytes, u
 
 // Largest i in [0, rows) with cu[i] <= x (the row holding element x, rows of length zero
 // skipped); 0 when even cu[0] > x.  Warp-cooperative; all lanes get the answer.
-__device__ __forceinline__ uint32_t warp_find_row(const int32_t *cu, uint32_t rows, int64_t x, uint32_t lane) {
+// Every load of a round is independent of the others, and the last round covers up to 256
+// entries (eight per lane), so a table of up to 256 rows costs one memory round trip, one of up
+// to 8192 rows two.  `along`, when given, is an array indexed like cu that the caller reads
+// next (sample indices): its lines are prefetched into L1 beside the last round's loads.
+__device__ __forceinline__ uint32_t warp_find_row(const int32_t *cu, uint32_t rows, int64_t x, uint32_t lane,
+                                                  const int32_t *along = nullptr) {
     uint32_t lo = 0, len = rows;
-    while (len > 1) {
+    while (len > 256u) {
         const uint32_t stride = (len + 31u) >> 5;
         const uint64_t probe = (uint64_t)lane * stride;
         const bool ok = probe < len && (int64_t)__ldg(cu + lo + probe) <= x;
@@ -255,7 +306,15 @@ __device__ __forceinline__ uint32_t warp_find_row(const int32_t *cu, uint32_t ro
         lo += step;
         len = min(stride, len - step);
     }
-    return lo;
+    const uint32_t per = (len + 31u) >> 5;                       // entries per lane, at most 8
+    const uint32_t e0 = lane * per;
+    if (along && e0 < len) asm volatile("prefetch.global.L1 [%0];" ::"l"(along + lo + e0));
+    uint32_t cnt = 0;
+    #pragma unroll
+    for (uint32_t t = 0; t < 8u; ++t)
+        if (t < per && e0 + t < len && (int64_t)__ldg(cu + lo + e0 + t) <= x) ++cnt;
+    cnt = __reduce_add_sync(kFullMask, cnt);                     // entries <= x form a prefix of the table
+    return lo + (cnt ? cnt - 1u : 0u);
 }
 
 __device__ __forceinline__ uint64_t shfl_u64(uint64_t v, uint32_t src) {
@@ -362,12 +421,12 @@ struct WarpPipe {
         ++tail;
         __syncwarp();                                          // lane 0's descriptor is visible
         const PieceDesc d = desc[s];
-        const uint8_t *from = stage + (size_t)s * kStageBytes + d.pre;
-        if (!wait_stage(s)) {                                  // never seen; the piece is read again, directly
+        if (wait_stage(s)) {
+            warp_copy_from_shared(d.dst, smem_u32(stage) + s * kStageBytes + d.pre, d.n, lane);
+        } else {                                               // never seen; the piece is read again, directly
             failed |= 1u | (2u << s);
-            from = d.src;
+            warp_copy(d.dst, d.src, d.n, lane);
         }
-        warp_copy(d.dst, from, d.n, lane);
     }
 
     // before the warp returns: everything written out, nothing of its own still landing
@@ -408,14 +467,14 @@ struct WarpPipe {
 
 // Steps 2 and 3 for one chunk [b0, b1) of a packed side described by cu[0..rows].
 // resolve(i) returns where row i starts on the other side, or nullptr to skip the row; it is
-// called by one lane per row.  kToPacked: the packed side is the destination (get), else the
-// source (put).
+// called by one lane per row; `along` is the index array it reads (prefetched by the row
+// search).  kToPacked: the packed side is the destination (get), else the source (put).
 template <bool kToPacked, typename Resolve>
 __device__ __forceinline__ void warp_copy_chunk(const int32_t *cu, uint32_t rows, uint64_t b0, uint64_t b1,
                                                 uint8_t *packed, uint32_t esz, uint32_t lane,
                                                 const uint8_t *src_lo, const uint8_t *src_hi, WarpPipe &pipe,
-                                                Resolve resolve) {
-    uint32_t r0 = warp_find_row(cu, rows, (int64_t)(b0 / esz), lane);
+                                                const int32_t *along, Resolve resolve) {
+    uint32_t r0 = warp_find_row(cu, rows, (int64_t)(b0 / esz), lane, along);
     for (;;) {
         const uint32_t i = r0 + lane;
         bool in = false;

@@ -217,10 +217,17 @@ __device__ __forceinline__ uint64_t job_bytes_of(const DockView &dv, const GetRe
     return n_s * (uint64_t)(cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to) * esz;
 }
 
+// What the gather needs to know about a (request, column) pair before it touches the request.
+struct JobSize {
+    uint64_t bytes;       // output bytes of the column (not padded)
+    uint32_t rows;        // samples served
+    uint32_t pad;
+};
+
 __global__ void __launch_bounds__(kFinThreads)
 get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
                     const GetReq *reqs_dev, const ConsumerSlot *slots_dev, const uint32_t seq,
-                    unsigned long long *work_counter, uint64_t *job_sizes) {
+                    unsigned long long *work_counter, JobSize *job_sizes) {
     const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
     const ConsumerSlot *slots = slots_dev ? slots_dev : &one.cs;
     const GetReq &rq = reqs[blockIdx.x];
@@ -358,11 +365,14 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
         atomicAdd(&dv.counters[CNT_GOT_SAMPLES + c], (unsigned long long)n_s);
         atomicAdd(&dv.counters[CNT_GOT_TOKENS + c], (unsigned long long)(r.prompt_tokens + r.response_tokens));
     }
-    // the gather's job table: this request's output bytes per column, padded to 16
-    if (job_sizes && tid < dv.ncol)
-        job_sizes[(size_t)blockIdx.x * dv.ncol + tid] =
-            (job_bytes_of(dv, rq, tid, n_s, (uint64_t)(int64_t)out.cu_prompt[n_s],
-                          (uint64_t)(int64_t)out.cu_response[n_s]) + 15) & ~uint64_t(15);
+    // the gather's job table: this request's output bytes per column and its row count
+    if (job_sizes && tid < dv.ncol) {
+        JobSize js;
+        js.bytes = job_bytes_of(dv, rq, tid, n_s, (uint64_t)(int64_t)out.cu_prompt[n_s],
+                                (uint64_t)(int64_t)out.cu_response[n_s]);
+        js.rows = n_s; js.pad = 0;
+        job_sizes[(size_t)blockIdx.x * dv.ncol + tid] = js;
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -371,19 +381,26 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
 // over bytes whatever the mix of requests and row lengths (see "Chunked ragged copy" in
 // td_device.cuh).
 // ---------------------------------------------------------------------------------------------
-__device__ __forceinline__ uint64_t job_bytes(const DockView &dv, const GetReq &rq, uint32_t k) {
+__device__ __forceinline__ JobSize job_size(const DockView &dv, const GetReq &rq, uint32_t k) {
     const td_result *res = rq.out.result;
-    return job_bytes_of(dv, rq, k, res->n_samples, res->prompt_tokens, res->response_tokens);
+    JobSize js;
+    js.rows = res->n_samples; js.pad = 0;
+    js.bytes = job_bytes_of(dv, rq, k, js.rows, res->prompt_tokens, res->response_tokens);
+    return js;
 }
 
 __global__ void __launch_bounds__(kCopyThreads, kCopyBlocksPerSM)
 get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
                   const GetReq *reqs_dev, const uint32_t n_req, unsigned long long *work_counter,
-                  const uint64_t *job_sizes) {
+                  const JobSize *job_sizes) {
     const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
     extern __shared__ __align__(128) uint8_t gather_smem[];
     uint64_t *s_wsum = reinterpret_cast<uint64_t *>(gather_smem + (size_t)kCopyWarps * kPipeSmemPerWarp);
-    uint64_t *job_end = s_wsum + kCopyWarps;        // [n_req * ncol] inclusive prefix of bytes (16-byte padded)
+    // [n_req * ncol] inclusive prefix of the jobs' bytes, each job padded to 16; the low four
+    // bits hold the padding behind the job.  With this and the rows served per request in
+    // shared memory, a chunk's warp needs neither the result block nor the last cu entry.
+    uint64_t *job_end = s_wsum + kCopyWarps;
+    uint32_t *req_rows = reinterpret_cast<uint32_t *>(job_end + n_req * dv.ncol);    // [n_req]
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     WarpPipe pipe;
     pipe.init(gather_smem + (size_t)warp * kPipeSmemPerWarp, lane, dv.spin_limit);
@@ -400,20 +417,25 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
         for (uint32_t i = 0; i < per; ++i) {
             const uint32_t j = i * kCopyThreads + tid;
             if (j < njobs) {
+                JobSize js;
                 if (job_sizes) {
-                    job_end[j] = job_sizes[j];                 // written by the finalize kernel
+                    js = job_sizes[j];                         // written by the finalize kernel
                 } else {
                     const uint32_t q = fast_div(j, dv.div_ncol);
-                    job_end[j] = (job_bytes(dv, reqs[q], j - q * ncol) + 15) & ~uint64_t(15);
+                    js = job_size(dv, reqs[q], j - q * ncol);
                 }
+                job_end[j] = js.bytes;
+                const uint32_t q = fast_div(j, dv.div_ncol);
+                if (j == q * ncol) req_rows[q] = js.rows;
             }
         }
         __syncthreads();
         const uint32_t j0 = min(tid * per, njobs), j1 = min(j0 + per, njobs);
         uint64_t local = 0;
         for (uint32_t j = j0; j < j1; ++j) {
-            local += job_end[j];
-            job_end[j] = local;                       // inclusive within the thread's run
+            const uint64_t bytes = job_end[j], padded = (bytes + 15) & ~uint64_t(15);
+            local += padded;
+            job_end[j] = local | (padded - bytes);    // inclusive within the thread's run; padding in the low bits
         }
         uint64_t inc = local;
         #pragma unroll
@@ -428,34 +450,35 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
         for (uint32_t j = j0; j < j1; ++j) job_end[j] += before;
         __syncthreads();
     }
-    const uint64_t total_all = njobs ? job_end[njobs - 1] : 0;
+    const uint64_t total_all = njobs ? job_end[njobs - 1] & ~uint64_t(15) : 0;
     const uint64_t n_warps = (uint64_t)gridDim.x * kCopyWarps;
-    // Chunks are handed out by a counter in scratch memory (zeroed by the finalize kernel): equal
-    // bytes are not equal time when one chunk holds a few long rows and another many short ones.
+    // A warp starts on the chunk of its own number; the chunks after the first n_warps are
+    // handed out by a counter in scratch memory (zeroed by the finalize kernel): equal bytes are
+    // not equal time when one chunk holds a few long rows and another many short ones.
     const ChunkPlan plan = plan_chunks_dynamic(total_all, n_warps);
-    unsigned long long ch = 0;
-    if (lane == 0) ch = atomicAdd(work_counter, 1ull);
-    ch = shfl_u64(ch, 0);
+    unsigned long long ch = (uint64_t)blockIdx.x * kCopyWarps + warp;
 
     while (ch < plan.n_chunks) {
         unsigned long long next = 0;
-        if (lane == 0) next = atomicAdd(work_counter, 1ull);       // in flight while this chunk is copied
+        if (lane == 0) next = n_warps + atomicAdd(work_counter, 1ull);   // in flight while this chunk is copied
         uint64_t g0 = ch * plan.chunk_bytes;
         const uint64_t g1 = min(g0 + plan.chunk_bytes, total_all);
         // first job that reaches beyond g0
         uint32_t j = 0;
-        { uint32_t jhi = njobs - 1; while (j < jhi) { const uint32_t m = (j + jhi) >> 1; if (job_end[m] > g0) jhi = m; else j = m + 1; } }
+        { uint32_t jhi = njobs - 1; while (j < jhi) { const uint32_t m = (j + jhi) >> 1; if ((job_end[m] & ~uint64_t(15)) > g0) jhi = m; else j = m + 1; } }
         for (; g0 < g1; ++j) {
-            const uint64_t start = j ? job_end[j - 1] : 0;
+            const uint64_t start = j ? job_end[j - 1] & ~uint64_t(15) : 0;
+            const uint64_t end = job_end[j] & ~uint64_t(15);
             const uint64_t b0 = g0 - start;
-            g0 = min(g1, job_end[j]);
-            if (job_end[j] == start) continue;        // empty job
+            g0 = min(g1, end);
+            if (end == start) continue;               // empty job
             const uint32_t q = fast_div(j, dv.div_ncol);
             const uint32_t k = j - q * ncol;
             const GetReq &rq = reqs[q];
             const td_get_out &out = rq.out;
             const uint32_t cls = dv.col_cls[k], esz = dv.col_esz[k];
-            const uint32_t n_s = out.result->n_samples;
+            const uint32_t n_s = req_rows[q];
+            const uint64_t job_exact = end - start - (job_end[j] & 15u);
             uint8_t *dst0 = reinterpret_cast<uint8_t *>(out.col[k]);
             uint8_t *base = dv.colbase[k];
             const int32_t *indices = out.indices;
@@ -480,9 +503,9 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
             };
             if (out.mode == TD_PACKED) {
                 const int32_t *cu = cls == TD_PROMPT ? out.cu_prompt : out.cu_response;
-                const uint64_t b1 = min(b1_raw, (uint64_t)(int64_t)__ldg(cu + n_s) * esz);
+                const uint64_t b1 = min(b1_raw, job_exact);
                 if (b1 <= b0) continue;
-                warp_copy_chunk<true>(cu, n_s, b0, b1, dst0, esz, lane, src_lo, src_hi, pipe,
+                warp_copy_chunk<true>(cu, n_s, b0, b1, dst0, esz, lane, src_lo, src_hi, pipe, indices,
                                       [&](uint32_t i, int64_t, int64_t) -> uint8_t * { return row_src(i); });
             } else {
                 // fixed-width rows: payload part, then the pad pattern up to the row's end

@@ -32,6 +32,7 @@ __device__ __forceinline__ bool put_entry_live(const DockView &dv, const PutArgs
 __global__ void __launch_bounds__(kCopyThreads, kCopyBlocksPerSM)
 put_scatter_kernel(const DockView dv, const PutBatch batch) {
     __shared__ uint64_t item_end[kMaxPutItems];       // inclusive prefix of bytes (16-byte padded) per item
+    __shared__ uint64_t item_bytes[kMaxPutItems];     // packed bytes of each ragged item (0: nothing to copy)
     extern __shared__ __align__(128) uint8_t scatter_smem[];
     const uint32_t tid = threadIdx.x, lane = tid & 31;
     WarpPipe pipe;                                                           // [warps][kPipeSmemPerWarp]
@@ -39,16 +40,20 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
     griddep_launch_dependents();
     griddep_wait();                                    // the alloc kernel's tables are complete
 
+    if (tid < batch.n_items) {                         // one thread per item: the totals load side by side
+        const PutArgs &a = batch.item[tid];
+        uint64_t bytes = 0;
+        if (dv.col_cls[a.column] != TD_SCALAR && a.k) {
+            const int64_t tot = a.cu[a.k];
+            if (tot > 0 && (uint64_t)tot <= a.data_elems) bytes = (uint64_t)tot * dv.col_esz[a.column];
+        }
+        item_bytes[tid] = bytes;
+    }
+    __syncthreads();
     if (tid == 0) {
         uint64_t acc = 0;
         for (uint32_t it = 0; it < batch.n_items; ++it) {
-            const PutArgs &a = batch.item[it];
-            uint64_t bytes = 0;
-            if (dv.col_cls[a.column] != TD_SCALAR && a.k) {
-                const int64_t tot = a.cu[a.k];
-                if (tot > 0 && (uint64_t)tot <= a.data_elems) bytes = (uint64_t)tot * dv.col_esz[a.column];
-            }
-            acc += (bytes + 15) & ~uint64_t(15);
+            acc += (item_bytes[it] + 15) & ~uint64_t(15);
             item_end[it] = acc;
         }
     }
@@ -71,13 +76,12 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
             const uint64_t b0 = g0 - start;
             g0 = min(g1, item_end[it]);
             if (L == TD_SCALAR || a.k == 0) continue;
-            const uint64_t total_bytes = (uint64_t)(int64_t)__ldg(a.cu + a.k) * esz;
-            const uint64_t b1 = min(g0 - start, total_bytes);
+            const uint64_t b1 = min(g0 - start, item_bytes[it]);
             if (b1 <= b0) continue;
             uint8_t *arena = dv.colbase[a.column];
             const uint64_t cap = dv.cap[L];
             warp_copy_chunk<false>(a.cu, a.k, b0, b1, const_cast<uint8_t *>(a.data), esz, lane,
-                                   a.data, a.data + a.data_elems * esz, pipe,
+                                   a.data, a.data + a.data_elems * esz, pipe, a.idx,
                                    [&](uint32_t i, int64_t c0, int64_t c1) -> uint8_t * {
                                        // the row is live if the alloc kernel accepted it
                                        const int32_t s = a.idx[i];
