@@ -27,6 +27,9 @@ import numpy as np
 
 METRIC = "td_put+td_get samples/s dispatched"
 L2_FLUSH_BYTES = 256 << 20
+# DRAM bytes (read + write) of one launch, from the ncu capture summarised under profiles/ for
+# the kernels as built; (config, kernel) pairs without a capture report null.
+NCU_TRAFFIC = {(2, "get_gather"): 79_977_216, (2, "put_scatter"): 45_300_224}
 
 
 def parse_args():
@@ -487,7 +490,8 @@ def main():
         k["GBps"] = k["bytes_per_launch"] / (k["avg_ms"] * 1e-3) / 1e9 if k["avg_ms"] > 0 else 0.0
     dom = "get_gather" if ms_ga >= ms_sc else "put_scatter"
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kern[dom]["GBps"], "peak": peak, "unit": "GB/s",
-                "frac": kern[dom]["GBps"] / peak, "traffic": None, "peak_kind": peak_kind,
+                "frac": kern[dom]["GBps"] / peak, "traffic": NCU_TRAFFIC.get((args.config, dom)),
+                "peak_kind": peak_kind,
                 "bytes_per_launch": kern[dom]["bytes_per_launch"], "avg_launch_ms": kern[dom]["avg_ms"]}
 
     e2e = None

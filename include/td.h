@@ -81,7 +81,7 @@ typedef struct {
 
 typedef struct {
     uint32_t n_prompts;    /* G */
-    uint32_t n_per_group;  /* N; sample s = prompt * N + response, group = s / N; G * N < 2^28 */
+    uint32_t n_per_group;  /* N; sample s = prompt * N + response, group = s / N; G * N < 2^30 */
     uint32_t n_shards;     /* S warehouses, 1..256, must divide G; shard(s) = (s / N) / (G / S) */
     uint32_t n_columns;    const td_column   *columns;     /* 1..32, host array */
     uint32_t n_consumers;  const td_consumer *consumers;   /* 1..32, host array */

@@ -55,8 +55,7 @@ bool valid_config(const td_config *c) {
     if (c->n_prompts == 0 || c->n_per_group == 0 || c->n_shards == 0 || c->n_shards > 256) return false;
     if (c->n_prompts % c->n_shards) return false;
     if (c->n_columns == 0 || c->n_columns > 32 || c->n_consumers == 0 || c->n_consumers > 32) return false;
-    if ((uint64_t)c->n_prompts * c->n_per_group >= (1ull << 28)) return false;   // a row count fits 28 bits
-
+    if ((uint64_t)c->n_prompts * c->n_per_group >= (1ull << 30)) return false;
     for (uint32_t k = 0; k < c->n_columns; ++k) {
         const td_column &col = c->columns[k];
         if (col.dtype < TD_I32 || col.dtype > TD_BF16) return false;
