@@ -331,12 +331,12 @@ __device__ __forceinline__ uint64_t shfl_up_u64(uint64_t v, int delta) {
 
 // --------------------------------------------------------------------------------------------
 // Asynchronous staging.  Each warp owns a ring of kStages shared-memory stages with one
-// mbarrier and one descriptor each.  A piece of a row is fetched with one bulk asynchronous
-// copy (cp.async.bulk, global to shared, completion counted in bytes on the stage's mbarrier);
-// a piece is written out to its destination only when the ring is full and its stage is
-// needed again, so a warp keeps kStages copies in flight without holding a single register
-// for them; the bytes in flight per SM are what a ragged copy needs to cover HBM latency,
-// whatever the row lengths.  The bulk copy wants 16-byte aligned addresses and sizes:
+// mbarrier each.  A piece of a row is fetched with one bulk asynchronous copy (cp.async.bulk,
+// global to shared, completion counted in bytes on the stage's mbarrier); a piece is written
+// out to its destination only when the ring is full and its stage is needed again, so a warp
+// keeps kStages copies in flight, described by three warp-uniform registers each; the bytes
+// in flight per SM are what a ragged copy needs to cover HBM latency, whatever the row
+// lengths.  The bulk copy wants 16-byte aligned addresses and sizes:
 // the source window is widened to the enclosing 16-byte boundaries (rows in an arena start
 // aligned and are padded, so the window stays inside the arena) and the write-out shifts the
 // bytes into place.  Every wait on an mbarrier is bounded; a warp that gives up records the
@@ -351,8 +351,8 @@ __device__ __forceinline__ uint64_t shfl_up_u64(uint64_t v, int delta) {
 constexpr int kStages = TD_STAGES;
 constexpr uint32_t kStageBytes = TD_STAGE_BYTES;
 constexpr uint32_t kPieceMax = kStageBytes - 16;      // payload of one bulk copy; the aligned window still fits
-// stages, descriptors, mbarriers of one warp; rounded so that every warp's stages start 128-byte aligned
-constexpr size_t kPipeSmemPerWarp = (((size_t)kStages * (kStageBytes + 32 + 8)) + 127) & ~size_t(127);
+// stages and mbarriers of one warp; rounded so that every warp's stages start 128-byte aligned
+constexpr size_t kPipeSmemPerWarp = (((size_t)kStages * (kStageBytes + 8)) + 127) & ~size_t(127);
 static_assert(kStageBytes % 16 == 0 && kPipeSmemPerWarp % 128 == 0, "bulk copies need 16-byte aligned stages");
 
 __device__ __forceinline__ uint32_t smem_u32(const void *p) { return (uint32_t)__cvta_generic_to_shared(p); }
@@ -375,29 +375,25 @@ __device__ __forceinline__ void bulk_global_to_shared(uint32_t dst, const void *
 __device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 __device__ __forceinline__ void fence_mbar_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 
-struct PieceDesc {             // one copy in flight, kept beside its stage in shared memory
-    uint8_t *dst;
-    const uint8_t *src;
-    uint32_t n;                // payload bytes
-    uint32_t pre;              // payload starts this many bytes into the stage (source misalignment)
-    uint32_t esz;
-    uint32_t pad;
-};
-
 struct WarpPipe {
-    uint8_t *stage;            // this warp's kStages * kStageBytes bytes of shared memory
-    PieceDesc *desc;           // kStages descriptors
-    uint32_t bar;              // shared address of this warp's kStages mbarriers
+    uint32_t stage;            // shared-window address of this warp's kStages * kStageBytes bytes
+    uint32_t bar;              // shared-window address of this warp's kStages mbarriers
     uint32_t parity;           // bit s: phase the next wait on stage s looks for
     uint32_t head, tail;       // copies issued / written out so far; stage of copy i is i % kStages
     uint32_t spin_limit;
     uint32_t failed;           // bit 0: a wait ran out, plain loads from here on; bit 1 + s: stage s may still be landing
+    // the piece in flight in stage s (every lane holds the same values): destination, source
+    // (the payload starts (source & 15) bytes into the stage), payload bytes
+    uint8_t *p_dst[kStages];
+    const uint8_t *p_src[kStages];
+    uint32_t p_n[kStages];
 
     __device__ __forceinline__ void init(uint8_t *mem, uint32_t lane, uint32_t spin) {
-        stage = mem;
-        desc = reinterpret_cast<PieceDesc *>(mem + (size_t)kStages * kStageBytes);
-        bar = smem_u32(desc + kStages);
+        stage = smem_u32(mem);
+        bar = stage + (uint32_t)kStages * kStageBytes;
         parity = 0; head = 0; tail = 0; spin_limit = spin; failed = 0;
+        #pragma unroll
+        for (int s = 0; s < kStages; ++s) { p_dst[s] = nullptr; p_src[s] = nullptr; p_n[s] = 0; }
         if (lane == 0) {
             for (int s = 0; s < kStages; ++s) mbar_init(bar + 8u * s, 1);
             fence_mbar_init();
@@ -419,13 +415,17 @@ struct WarpPipe {
     __device__ __forceinline__ void drain_one(uint32_t lane) {
         const uint32_t s = tail % kStages;
         ++tail;
-        __syncwarp();                                          // lane 0's descriptor is visible
-        const PieceDesc d = desc[s];
+        uint8_t *dst = p_dst[0];
+        const uint8_t *src = p_src[0];
+        uint32_t n = p_n[0];
+        #pragma unroll
+        for (int i = 1; i < kStages; ++i)
+            if (s == (uint32_t)i) { dst = p_dst[i]; src = p_src[i]; n = p_n[i]; }
         if (wait_stage(s)) {
-            warp_copy_from_shared(d.dst, smem_u32(stage) + s * kStageBytes + d.pre, d.n, lane);
+            warp_copy_from_shared(dst, stage + s * kStageBytes + ((uint32_t)reinterpret_cast<uintptr_t>(src) & 15u), n, lane);
         } else {                                               // never seen; the piece is read again, directly
             failed |= 1u | (2u << s);
-            warp_copy(d.dst, d.src, d.n, lane);
+            warp_copy(dst, src, n, lane);
         }
     }
 
@@ -437,27 +437,33 @@ struct WarpPipe {
         return failed;
     }
 
-    // copy n bytes from src to dst through the stages (element-aligned, any length)
-    __device__ __forceinline__ void push(uint8_t *dst, const uint8_t *src, uint64_t n, uint32_t esz, uint32_t lane,
+    // Copy n bytes from src to dst through the stages (element-aligned, any length).  The bulk
+    // copy reads the 16-byte aligned window around a piece; with kCheckWindow the window is
+    // tested against [src_lo, src_hi) and a piece whose window would leave it is copied with
+    // plain loads.  Arena rows start aligned and are padded to 16 bytes, so a get needs no test.
+    template <bool kCheckWindow>
+    __device__ __forceinline__ void push(uint8_t *dst, const uint8_t *src, uint32_t n, uint32_t lane,
                                          const uint8_t *src_lo, const uint8_t *src_hi) {
         while (n > 0) {
-            const uint32_t m = n > kPieceMax ? kPieceMax : (uint32_t)n;
+            const uint32_t m = n > kPieceMax ? kPieceMax : n;
             const uint32_t pre = (uint32_t)(reinterpret_cast<uintptr_t>(src) & 15u);
-            const uint8_t *win = src - pre;
             const uint32_t size = (pre + m + 15u) & ~15u;
-            if (failed || m < 64u || win < src_lo || win + size > src_hi) {
-                warp_copy(dst, src, m, lane);                            // short, at a buffer edge, or after a failure
+            bool direct = failed || m < 64u;                             // after a failure, or too short to stage
+            if (kCheckWindow) direct = direct || src - pre < src_lo || src - pre + size > src_hi;
+            if (direct) {
+                warp_copy(dst, src, m, lane);
             } else {
                 if (head - tail == (uint32_t)kStages) drain_one(lane);   // every stage busy: free the oldest
                 const uint32_t s = head % kStages;
                 ++head;
+                #pragma unroll
+                for (int i = 0; i < kStages; ++i)
+                    if (s == (uint32_t)i) { p_dst[i] = dst; p_src[i] = src; p_n[i] = m; }
                 __syncwarp();                                            // every lane is done reading stage s
                 if (lane == 0) {
-                    PieceDesc d; d.dst = dst; d.src = src; d.n = m; d.pre = pre; d.esz = esz; d.pad = 0;
-                    desc[s] = d;
                     fence_proxy_async();
                     mbar_expect_tx(bar + 8u * s, size);
-                    bulk_global_to_shared(smem_u32(stage + (size_t)s * kStageBytes), win, size, bar + 8u * s);
+                    bulk_global_to_shared(stage + s * kStageBytes, src - pre, size, bar + 8u * s);
                 }
             }
             dst += m; src += m; n -= m;
@@ -465,43 +471,51 @@ struct WarpPipe {
     }
 };
 
-// Steps 2 and 3 for one chunk [b0, b1) of a packed side described by cu[0..rows].
-// resolve(i) returns where row i starts on the other side, or nullptr to skip the row; it is
-// called by one lane per row; `along` is the index array it reads (prefetched by the row
-// search).  kToPacked: the packed side is the destination (get), else the source (put).
+// Steps 2 and 3 for one chunk [b0, b1) of a packed side described by cu[0..rows] (a chunk is
+// shorter than 4 GB).  resolve(i) returns where row i starts on the other side, or nullptr to
+// skip the row; it is called by one lane per row; `along` is the index array it reads
+// (prefetched by the row search).  kToPacked: the packed side is the destination (get), else
+// the source (put, whose source window is tested against the caller's buffer).
 template <bool kToPacked, typename Resolve>
 __device__ __forceinline__ void warp_copy_chunk(const int32_t *cu, uint32_t rows, uint64_t b0, uint64_t b1,
                                                 uint8_t *packed, uint32_t esz, uint32_t lane,
                                                 const uint8_t *src_lo, const uint8_t *src_hi, WarpPipe &pipe,
                                                 const int32_t *along, Resolve resolve) {
     uint32_t r0 = warp_find_row(cu, rows, (int64_t)(b0 / esz), lane, along);
+    uint8_t *chunk0 = packed + b0;
     for (;;) {
+        // lane l: the part of row r0 + l that falls inside the chunk, as (offset from b0, bytes,
+        // address on the other side); bytes = 0 when there is nothing to copy
         const uint32_t i = r0 + lane;
         bool in = false;
-        uint64_t rlo = 0, rhi = 0;
+        uint32_t off = 0, len = 0;
         uint8_t *other = nullptr;
         if (i < rows) {
             const int64_t c0 = __ldg(cu + i);
-            rlo = (uint64_t)c0 * esz;
+            const uint64_t rlo = (uint64_t)c0 * esz;
             in = c0 >= 0 && rlo < b1;
             if (in) {
                 const int64_t c1 = __ldg(cu + i + 1);
-                rhi = c1 > c0 ? (uint64_t)c1 * esz : rlo;
-                other = rhi > b0 ? resolve(i, c0, c1) : nullptr;
+                const uint64_t rhi = c1 > c0 ? (uint64_t)c1 * esz : rlo;
+                const uint64_t lo = max(rlo, b0), hi = min(rhi, b1);
+                if (hi > lo) {
+                    uint8_t *row = resolve(i, c0, c1);
+                    if (row) { other = row + (lo - rlo); off = (uint32_t)(lo - b0); len = (uint32_t)(hi - lo); }
+                }
             }
         }
         // rows inside the chunk form a prefix of the lanes
         const uint32_t n_rows = (uint32_t)__ffs(~__ballot_sync(kFullMask, in)) - 1u;   // 32 when all lanes are in
-        const uint32_t n_here = n_rows > 32u ? 32u : n_rows;
-        for (uint32_t r = 0; r < n_here; ++r) {
-            const uint64_t lo_r = shfl_u64(rlo, r), hi_r = shfl_u64(rhi, r);
+        uint32_t todo = __ballot_sync(kFullMask, len != 0);
+        while (todo) {
+            const uint32_t r = (uint32_t)__ffs(todo) - 1u;
+            todo &= todo - 1u;
+            const uint32_t off_r = __shfl_sync(kFullMask, off, r), len_r = __shfl_sync(kFullMask, len, r);
             uint8_t *o = reinterpret_cast<uint8_t *>(shfl_u64(reinterpret_cast<uint64_t>(other), r));
-            const uint64_t lo = max(lo_r, b0), hi = min(hi_r, b1);
-            if (o == nullptr || hi <= lo) continue;
-            if (kToPacked) pipe.push(packed + lo, o + (lo - lo_r), hi - lo, esz, lane, src_lo, src_hi);
-            else pipe.push(o + (lo - lo_r), packed + lo, hi - lo, esz, lane, src_lo, src_hi);
+            if (kToPacked) pipe.template push<false>(chunk0 + off_r, o, len_r, lane, src_lo, src_hi);
+            else pipe.template push<true>(o, chunk0 + off_r, len_r, lane, src_lo, src_hi);
         }
-        if (n_here < 32u) break;
+        if (n_rows < 32u) break;
         r0 += 32u;
     }
 }

@@ -529,7 +529,8 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
                         uint8_t *o = reinterpret_cast<uint8_t *>(shfl_u64(reinterpret_cast<uint64_t>(src), r));
                         const uint64_t lo = max(rlo, b0), hi = min(rlo + row_bytes, b1);
                         const uint64_t phi = min(hi, valid_hi);
-                        if (phi > lo && o) pipe.push(dst0 + lo, o + (lo - rlo), phi - lo, esz, lane, src_lo, src_hi);
+                        if (phi > lo && o)
+                            pipe.push<false>(dst0 + lo, o + (lo - rlo), (uint32_t)(phi - lo), lane, src_lo, src_hi);
                         const uint64_t plo = max(lo, valid_hi);
                         if (hi > plo) warp_fill(dst0 + plo, hi - plo, dv.col_pad[k], esz, lane);
                     }
