@@ -106,48 +106,26 @@ __device__ __forceinline__ void flag_error(const DockView &dv, uint32_t bit, int
 
 // --------------------------------------------------------------------------------------------
 // Warp-cooperative copy of n bytes from src to dst.  Both addresses and n are multiples of the
-// element size (2 or 4 bytes); nothing else is assumed.  Stores are 16-byte vectors aligned on
-// dst, each fed by four 32-bit loads (eight 16-bit loads when the two sides differ by an odd
-// number of half words) at whatever alignment the source has; head and tail move half words.
-// It reads exactly the bytes it copies, and src may be shared memory (a stage) or global
-// memory.  Kept small on purpose: it is inlined into the copy kernels' inner loops, and their
-// instruction footprint showed up as fetch stalls.
+// element size (2 or 4 bytes); nothing else is assumed.  Two forms.  warp_copy is the plain one,
+// word by word (half words when anything is odd), reading exactly the bytes it copies: it
+// serves pieces too short to stage, pieces at the edge of a caller's buffer and the path after
+// a failed wait, and is as small as it can be, because the instruction footprint of the copy
+// kernels showed up in their speed.  warp_copy_from_shared is the one the data goes through:
+// the source is a stage in shared memory, given as a shared-window address; stores are
+// 16-byte vectors aligned on dst, each fed by four ld.shared.u32 (eight ld.shared.u16 when
+// the two sides differ by an odd number of half words) at whatever phase the source has;
+// head and tail move half words.
 // --------------------------------------------------------------------------------------------
 __device__ __noinline__ void warp_copy(uint8_t *dst, const uint8_t *src, uint32_t n, uint32_t lane) {
-    uint32_t head = (16u - (uint32_t)(reinterpret_cast<uintptr_t>(dst) & 15u)) & 15u;
-    if (head > n) head = n;
-    if (lane < (head >> 1)) reinterpret_cast<uint16_t *>(dst)[lane] = reinterpret_cast<const uint16_t *>(src)[lane];
-    dst += head; src += head; n -= head;
-    const uint32_t nvec = n >> 4;
-    uint4 *D = reinterpret_cast<uint4 *>(dst);
-    if ((reinterpret_cast<uintptr_t>(src) & 3u) == 0) {
-        const uint32_t *S = reinterpret_cast<const uint32_t *>(src);
-        uint32_t v = lane;
-        for (; v + 32 < nvec; v += 64) {
-            const uint32_t *p = S + 4u * v, *q = p + 128;
-            const uint4 a = make_uint4(p[0], p[1], p[2], p[3]);
-            const uint4 b = make_uint4(q[0], q[1], q[2], q[3]);
-            __stcs(D + v, a); __stcs(D + v + 32, b);
-        }
-        for (; v < nvec; v += 32) {
-            const uint32_t *p = S + 4u * v;
-            __stcs(D + v, make_uint4(p[0], p[1], p[2], p[3]));
-        }
+    if (((reinterpret_cast<uintptr_t>(dst) | reinterpret_cast<uintptr_t>(src) | n) & 3u) == 0) {
+        for (uint32_t i = lane; i < (n >> 2); i += 32)
+            reinterpret_cast<uint32_t *>(dst)[i] = reinterpret_cast<const uint32_t *>(src)[i];
     } else {
-        const uint16_t *S = reinterpret_cast<const uint16_t *>(src);
-        for (uint32_t v = lane; v < nvec; v += 32) {
-            const uint16_t *p = S + 8u * v;
-            __stcs(D + v, make_uint4(p[0] | ((uint32_t)p[1] << 16), p[2] | ((uint32_t)p[3] << 16),
-                                     p[4] | ((uint32_t)p[5] << 16), p[6] | ((uint32_t)p[7] << 16)));
-        }
+        for (uint32_t i = lane; i < (n >> 1); i += 32)
+            reinterpret_cast<uint16_t *>(dst)[i] = reinterpret_cast<const uint16_t *>(src)[i];
     }
-    const uint32_t tail = n & 15u;
-    if (lane < (tail >> 1))
-        reinterpret_cast<uint16_t *>(dst + (nvec << 4))[lane] = reinterpret_cast<const uint16_t *>(src + (nvec << 4))[lane];
 }
 
-// The same copy with the source in shared memory, given as a shared-window address: the loads
-// are ld.shared instead of generic loads that find out at run time which memory they address.
 __device__ __forceinline__ uint32_t lds_u32(uint32_t a) {
     uint32_t v;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(v) : "r"(a));
@@ -173,14 +151,10 @@ __device__ __forceinline__ void warp_copy_from_shared(uint8_t *dst, uint32_t src
     const uint32_t nvec = n >> 4;
     uint4 *D = reinterpret_cast<uint4 *>(dst);
     if ((src & 3u) == 0) {
-        uint32_t v = lane;
-        for (; v + 32 < nvec; v += 64) {
-            const uint4 a = lds_4x32(src + 16u * v);
-            const uint4 b = lds_4x32(src + 16u * v + 512u);
-            __stcs(D + v, a); __stcs(D + v + 32, b);
-        }
-        for (; v < nvec; v += 32) __stcs(D + v, lds_4x32(src + 16u * v));
+        #pragma unroll 1                       // unrolled versions were measured slower
+        for (uint32_t v = lane; v < nvec; v += 32) __stcs(D + v, lds_4x32(src + 16u * v));
     } else {
+        #pragma unroll 1
         for (uint32_t v = lane; v < nvec; v += 32) {
             const uint32_t p = src + 16u * v;
             __stcs(D + v, make_uint4(lds_u16(p) | (lds_u16(p + 2) << 16), lds_u16(p + 4) | (lds_u16(p + 6) << 16),
@@ -445,11 +419,23 @@ struct WarpPipe {
     __device__ __forceinline__ void push(uint8_t *dst, const uint8_t *src, uint32_t n, uint32_t lane,
                                          const uint8_t *src_lo, const uint8_t *src_hi) {
         while (n > 0) {
-            const uint32_t m = n > kPieceMax ? kPieceMax : n;
+            uint32_t m = n > kPieceMax ? kPieceMax : n;
             const uint32_t pre = (uint32_t)(reinterpret_cast<uintptr_t>(src) & 15u);
-            const uint32_t size = (pre + m + 15u) & ~15u;
             bool direct = failed || m < 64u;                             // after a failure, or too short to stage
-            if (kCheckWindow) direct = direct || src - pre < src_lo || src - pre + size > src_hi;
+            if (kCheckWindow && !direct) {
+                // a window that would leave the buffer: only the few bytes at that edge go the
+                // plain way, the piece is cut at the last 16-byte boundary inside the buffer
+                if (src - pre < src_lo) {
+                    m = min(m, 16u - pre);
+                    direct = true;
+                } else if (src - pre + ((pre + m + 15u) & ~15u) > src_hi) {
+                    const uintptr_t last = reinterpret_cast<uintptr_t>(src_hi) & ~uintptr_t(15);
+                    const uintptr_t at = reinterpret_cast<uintptr_t>(src);
+                    if (last > at && last - at >= 64u) m = (uint32_t)(last - at);
+                    else direct = true;                                  // fewer than 80 bytes are left
+                }
+            }
+            const uint32_t size = (pre + m + 15u) & ~15u;
             if (direct) {
                 warp_copy(dst, src, m, lane);
             } else {
