@@ -98,6 +98,18 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
     const uint64_t cap = dv.cap[L];
     uint32_t n_oob = 0, n_dup = 0, n_bad = 0, n_mis = 0, n_full = 0;
 
+    // The passes read the items' index and cu arrays one after the other, each read at the head
+    // of a chain of dependent accesses: ask for all of them now, one request per 128-byte line.
+    for (uint32_t it = 0; it < batch.n_items; ++it) {
+        const PutArgs &a = batch.item[it];
+        if (dv.col_cls[a.column] != L) continue;
+        const uint64_t bytes = (uint64_t)a.k * 4u;
+        for (uint64_t at = (uint64_t)tid * 128u; at < bytes; at += (uint64_t)kAllocThreads * 128u) {
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint8_t *>(a.idx) + at));
+            asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint8_t *>(a.cu) + at));
+        }
+    }
+
     for (uint32_t it = 0; it < batch.n_items; ++it) {
         const PutArgs &a = batch.item[it];
         if (dv.col_cls[a.column] != L) continue;
@@ -114,20 +126,25 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
                 alloc[j] = false; s[j] = -1; room[j] = 0; sh[j] = 0;
                 if (i < a.k) {
                     s[j] = a.idx[i];
+                    const int64_t c0 = a.cu[i], c1 = a.cu[i + 1];
+                    const int64_t l = c1 - c0;
                     if (s[j] < 0 || (uint32_t)s[j] >= dv.n) { ++n_oob; }
-                    else if (dv.status[s[j]] & bit) { ++n_dup; }
                     else {
-                        const int64_t c0 = a.cu[i], c1 = a.cu[i + 1];
-                        const int64_t l = c1 - c0;
-                        if (l < 0 || c0 < 0 || (uint64_t)c1 > a.data_elems) { ++n_bad; }
-                        else {
-                            const int32_t old = atomicCAS(&dv.len[L][s[j]], -1, (int32_t)l);
-                            if (old == -1) {
-                                alloc[j] = true;
-                                room[j] = (uint32_t)align_row((uint64_t)l);
-                                sh[j] = shard_of(dv, (uint32_t)s[j]);
-                            } else if (old != (int32_t)l) { ++n_mis; }
-                        }
+                        // The status word and the CAS travel side by side.  A column that is
+                        // already stored has its class's length set, so the CAS of a repeated
+                        // put changes nothing; it is then counted as a repeat, whatever its
+                        // length says.
+                        const bool bad = l < 0 || c0 < 0 || (uint64_t)c1 > a.data_elems;
+                        const uint32_t st = dv.status[s[j]];
+                        int32_t old = 0;
+                        if (!bad) old = atomicCAS(&dv.len[L][s[j]], -1, (int32_t)l);
+                        if (st & bit) { ++n_dup; }
+                        else if (bad) { ++n_bad; }
+                        else if (old == -1) {
+                            alloc[j] = true;
+                            room[j] = (uint32_t)align_row((uint64_t)l);
+                            sh[j] = shard_of(dv, (uint32_t)s[j]);
+                        } else if (old != (int32_t)l) { ++n_mis; }
                     }
                 }
                 e_s[j * kAllocThreads + tid] = s[j];

@@ -13,14 +13,17 @@ namespace td {
 __device__ __forceinline__ bool put_entry_live(const DockView &dv, const PutArgs &a, uint32_t i,
                                                uint32_t L, uint32_t bit, int32_t &s_out,
                                                int64_t &len_out, long long &off_out) {
+    // two rounds of loads: the entry, then the three table words behind its index
     const int32_t s = a.idx[i];
-    if (s < 0 || (uint32_t)s >= dv.n) return false;
-    if (dv.status[s] & bit) return false;
     const int64_t c0 = a.cu[i], c1 = a.cu[i + 1];
+    if (s < 0 || (uint32_t)s >= dv.n) return false;
+    const uint32_t st = dv.status[s];
+    const int32_t ln = dv.len[L][s];
+    const long long off = dv.off[L][s];
+    if (st & bit) return false;
     const int64_t l = c1 - c0;
     if (l < 0 || c0 < 0 || (uint64_t)c1 > a.data_elems) return false;
-    if ((int64_t)dv.len[L][s] != l) return false;
-    const long long off = dv.off[L][s];
+    if ((int64_t)ln != l) return false;
     if (off < 0) return false;
     s_out = s; len_out = l; off_out = off;
     return true;
@@ -86,10 +89,12 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
                                        // the row is live if the alloc kernel accepted it
                                        const int32_t s = a.idx[i];
                                        if (s < 0 || (uint32_t)s >= dv.n) return nullptr;
-                                       if (dv.status[s] & bit) return nullptr;
-                                       if (c1 < c0 || (uint64_t)c1 > a.data_elems) return nullptr;
-                                       if ((int64_t)dv.len[L][s] != c1 - c0) return nullptr;
+                                       const uint32_t st = dv.status[s];          // three loads side by side
+                                       const int32_t ln = dv.len[L][s];
                                        const long long off = dv.off[L][s];
+                                       if (st & bit) return nullptr;
+                                       if (c1 < c0 || (uint64_t)c1 > a.data_elems) return nullptr;
+                                       if ((int64_t)ln != c1 - c0) return nullptr;
                                        if (off < 0) return nullptr;
                                        return arena + ((uint64_t)shard_of(dv, (uint32_t)s) * cap + (uint64_t)off) * esz;
                                    });
