@@ -232,7 +232,12 @@ struct ChunkPlan {
 __device__ __forceinline__ ChunkPlan plan_chunks(uint64_t total_bytes, uint64_t n_warps) {
     ChunkPlan p;
     const uint64_t per_warp = (total_bytes + n_warps - 1) / n_warps;
-    uint64_t rounds = (per_warp + kChunkTargetBytes / 2) / kChunkTargetBytes;
+    // a warp with little to do takes it in two chunks from different parts of the space (rows
+    // of different kinds cost differently), down to 8 KB each
+    uint64_t target = per_warp / 2;
+    if (target < 8192u) target = 8192u;
+    if (target > kChunkTargetBytes) target = kChunkTargetBytes;
+    uint64_t rounds = (per_warp + target / 2) / target;
     if (rounds < 1) rounds = 1;
     uint64_t c = (total_bytes + n_warps * rounds - 1) / (n_warps * rounds);
     c = (c + 15) & ~uint64_t(15);
