@@ -266,19 +266,21 @@ __device__ __forceinline__ ChunkPlan plan_chunks_dynamic(uint64_t total_bytes, u
     return p;
 }
 
-// Largest i in [0, rows) with cu[i] <= x (the row holding element x, rows of length zero
-// skipped); 0 when even cu[0] > x.  Warp-cooperative; all lanes get the answer.
+// Largest i in [0, rows) with key(i) <= x (the row holding position x, rows of no extent
+// skipped); 0 when even key(0) > x.  Warp-cooperative; all lanes get the answer.
 // Every load of a round is independent of the others, and the last round covers up to 256
 // entries (eight per lane), so a table of up to 256 rows costs one memory round trip, one of up
 // to 8192 rows two.  `along`, when given, is an array indexed like cu that the caller reads
 // next (sample indices): its lines are prefetched into L1 beside the last round's loads.
-__device__ __forceinline__ uint32_t warp_find_row(const int32_t *cu, uint32_t rows, int64_t x, uint32_t lane,
-                                                  const int32_t *along = nullptr) {
+// The key of row e is where it starts in the chunked space: cu[e] * esz + e * row_cost.
+__device__ __forceinline__ uint32_t warp_find_row(const int32_t *cu, uint32_t rows, int64_t x, uint32_t esz,
+                                                  uint32_t row_cost, uint32_t lane, const int32_t *along = nullptr) {
     uint32_t lo = 0, len = rows;
     while (len > 256u) {
         const uint32_t stride = (len + 31u) >> 5;
         const uint64_t probe = (uint64_t)lane * stride;
-        const bool ok = probe < len && (int64_t)__ldg(cu + lo + probe) <= x;
+        const bool ok = probe < len &&
+                        (int64_t)__ldg(cu + lo + probe) * esz + (int64_t)(lo + probe) * row_cost <= x;
         uint32_t cnt = __popc(__ballot_sync(kFullMask, ok));     // ok holds for a prefix of the lanes
         if (cnt < 1) cnt = 1;
         const uint32_t step = (cnt - 1u) * stride;
@@ -291,7 +293,8 @@ __device__ __forceinline__ uint32_t warp_find_row(const int32_t *cu, uint32_t ro
     uint32_t cnt = 0;
     #pragma unroll
     for (uint32_t t = 0; t < 8u; ++t)
-        if (t < per && e0 + t < len && (int64_t)__ldg(cu + lo + e0 + t) <= x) ++cnt;
+        if (t < per && e0 + t < len &&
+            (int64_t)__ldg(cu + lo + e0 + t) * esz + (int64_t)(lo + e0 + t) * row_cost <= x) ++cnt;
     cnt = __reduce_add_sync(kFullMask, cnt);                     // entries <= x form a prefix of the table
     return lo + (cnt ? cnt - 1u : 0u);
 }
@@ -462,36 +465,51 @@ struct WarpPipe {
     }
 };
 
-// Steps 2 and 3 for one chunk [b0, b1) of a packed side described by cu[0..rows] (a chunk is
-// shorter than 4 GB).  resolve(i) returns where row i starts on the other side, or nullptr to
-// skip the row; it is called by one lane per row; `along` is the index array it reads
-// (prefetched by the row search).  kToPacked: the packed side is the destination (get), else
-// the source (put, whose source window is tested against the caller's buffer).
+// The space that is cut into chunks charges every row of a ragged job a fixed kRowCost on top
+// of its bytes, because that is what a row costs a warp (search, descriptor, a piece of its
+// own): row i of a job takes [cu[i] * esz + i * kRowCost, cu[i+1] * esz + (i+1) * kRowCost),
+// the fixed part first, its bytes behind it.  Chunks of equal size in this space take about
+// equal time whether they hold a few long rows or many short ones.
+#ifndef TD_ROW_COST
+#define TD_ROW_COST 6144
+#endif
+constexpr uint32_t kRowCost = TD_ROW_COST;
+static_assert(kRowCost % 16 == 0, "a job's extent stays a multiple of 16");
+
+// Steps 2 and 3 for one chunk [b0, b1) of that space (a chunk is shorter than 4 GB) of a packed
+// side described by cu[0..rows].  resolve(i) returns where row i starts on the other side, or
+// nullptr to skip the row; it is called by one lane per row; `along` is the index array it
+// reads (prefetched by the row search).  kToPacked: the packed side is the destination (get),
+// else the source (put, whose source window is tested against the caller's buffer).
 template <bool kToPacked, typename Resolve>
 __device__ __forceinline__ void warp_copy_chunk(const int32_t *cu, uint32_t rows, uint64_t b0, uint64_t b1,
                                                 uint8_t *packed, uint32_t esz, uint32_t lane,
                                                 const uint8_t *src_lo, const uint8_t *src_hi, WarpPipe &pipe,
                                                 const int32_t *along, Resolve resolve) {
-    uint32_t r0 = warp_find_row(cu, rows, (int64_t)(b0 / esz), lane, along);
-    uint8_t *chunk0 = packed + b0;
+    uint32_t r0 = warp_find_row(cu, rows, (int64_t)b0, esz, kRowCost, lane, along);
     for (;;) {
-        // lane l: the part of row r0 + l that falls inside the chunk, as (offset from b0, bytes,
-        // address on the other side); bytes = 0 when there is nothing to copy
+        // lane l: the part of row r0 + l that falls inside the chunk, as (address on the packed
+        // side, address on the other side, bytes); bytes = 0 when there is nothing to copy
         const uint32_t i = r0 + lane;
         bool in = false;
-        uint32_t off = 0, len = 0;
-        uint8_t *other = nullptr;
+        uint32_t len = 0;
+        uint8_t *mine = nullptr, *other = nullptr;
         if (i < rows) {
             const int64_t c0 = __ldg(cu + i);
-            const uint64_t rlo = (uint64_t)c0 * esz;
-            in = c0 >= 0 && rlo < b1;
+            const uint64_t row0 = (uint64_t)c0 * esz + (uint64_t)i * kRowCost;
+            in = c0 >= 0 && row0 < b1;
             if (in) {
                 const int64_t c1 = __ldg(cu + i + 1);
-                const uint64_t rhi = c1 > c0 ? (uint64_t)c1 * esz : rlo;
-                const uint64_t lo = max(rlo, b0), hi = min(rhi, b1);
+                const uint64_t dlo = row0 + kRowCost;                       // the row's bytes, in the chunked space
+                const uint64_t dhi = c1 > c0 ? dlo + (uint64_t)(c1 - c0) * esz : dlo;
+                const uint64_t lo = max(dlo, b0), hi = min(dhi, b1);
                 if (hi > lo) {
                     uint8_t *row = resolve(i, c0, c1);
-                    if (row) { other = row + (lo - rlo); off = (uint32_t)(lo - b0); len = (uint32_t)(hi - lo); }
+                    if (row) {
+                        other = row + (lo - dlo);
+                        mine = packed + (uint64_t)c0 * esz + (lo - dlo);
+                        len = (uint32_t)(hi - lo);
+                    }
                 }
             }
         }
@@ -501,10 +519,11 @@ __device__ __forceinline__ void warp_copy_chunk(const int32_t *cu, uint32_t rows
         while (todo) {
             const uint32_t r = (uint32_t)__ffs(todo) - 1u;
             todo &= todo - 1u;
-            const uint32_t off_r = __shfl_sync(kFullMask, off, r), len_r = __shfl_sync(kFullMask, len, r);
+            const uint32_t len_r = __shfl_sync(kFullMask, len, r);
+            uint8_t *p = reinterpret_cast<uint8_t *>(shfl_u64(reinterpret_cast<uint64_t>(mine), r));
             uint8_t *o = reinterpret_cast<uint8_t *>(shfl_u64(reinterpret_cast<uint64_t>(other), r));
-            if (kToPacked) pipe.template push<false>(chunk0 + off_r, o, len_r, lane, src_lo, src_hi);
-            else pipe.template push<true>(o, chunk0 + off_r, len_r, lane, src_lo, src_hi);
+            if (kToPacked) pipe.template push<false>(p, o, len_r, lane, src_lo, src_hi);
+            else pipe.template push<true>(o, p, len_r, lane, src_lo, src_hi);
         }
         if (n_rows < 32u) break;
         r0 += 32u;

@@ -221,8 +221,14 @@ __device__ __forceinline__ uint64_t job_bytes_of(const DockView &dv, const GetRe
 struct JobSize {
     uint64_t bytes;       // output bytes of the column (not padded)
     uint32_t rows;        // samples served
-    uint32_t pad;
+    uint32_t cost_rows;   // rows that are charged kRowCost in the chunked space: those of a packed ragged column
 };
+
+// Extent of a job in the space the gather cuts into chunks (see kRowCost).
+__device__ __forceinline__ uint32_t job_cost_rows(const DockView &dv, const GetReq &rq, uint32_t k,
+                                                  uint64_t bytes, uint32_t n_s) {
+    return (bytes != 0 && dv.col_cls[k] != TD_SCALAR && rq.out.mode == TD_PACKED) ? n_s : 0u;
+}
 
 __global__ void __launch_bounds__(kFinThreads)
 get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
@@ -370,22 +376,24 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
         JobSize js;
         js.bytes = job_bytes_of(dv, rq, tid, n_s, (uint64_t)(int64_t)out.cu_prompt[n_s],
                                 (uint64_t)(int64_t)out.cu_response[n_s]);
-        js.rows = n_s; js.pad = 0;
+        js.rows = n_s;
+        js.cost_rows = job_cost_rows(dv, rq, tid, js.bytes, n_s);
         job_sizes[(size_t)blockIdx.x * dv.ncol + tid] = js;
     }
 }
 
 // ---------------------------------------------------------------------------------------------
-// Gather.  Persistent grid.  Every (request, column) pair is a job; the output space of each
-// job is cut into chunks and warps stride over the chunks of all jobs, so the work is balanced
-// over bytes whatever the mix of requests and row lengths (see "Chunked ragged copy" in
-// td_device.cuh).
+// Gather.  Persistent grid.  Every (request, column) pair is a job; the jobs' extents (output
+// bytes, plus kRowCost per row of a packed ragged column) are laid end to end and cut into
+// chunks that warps take one after the other, so the work is balanced whatever the mix of
+// requests and row lengths (see "Chunked ragged copy" in td_device.cuh).
 // ---------------------------------------------------------------------------------------------
 __device__ __forceinline__ JobSize job_size(const DockView &dv, const GetReq &rq, uint32_t k) {
     const td_result *res = rq.out.result;
     JobSize js;
-    js.rows = res->n_samples; js.pad = 0;
+    js.rows = res->n_samples;
     js.bytes = job_bytes_of(dv, rq, k, js.rows, res->prompt_tokens, res->response_tokens);
+    js.cost_rows = job_cost_rows(dv, rq, k, js.bytes, js.rows);
     return js;
 }
 
@@ -396,7 +404,7 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
     const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
     extern __shared__ __align__(128) uint8_t gather_smem[];
     uint64_t *s_wsum = reinterpret_cast<uint64_t *>(gather_smem + (size_t)kCopyWarps * kPipeSmemPerWarp);
-    // [n_req * ncol] inclusive prefix of the jobs' bytes, each job padded to 16; the low four
+    // [n_req * ncol] inclusive prefix of the jobs' extents, each job padded to 16; the low four
     // bits hold the padding behind the job.  With this and the rows served per request in
     // shared memory, a chunk's warp needs neither the result block nor the last cu entry.
     uint64_t *job_end = s_wsum + kCopyWarps;
@@ -424,7 +432,7 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
                     const uint32_t q = fast_div(j, dv.div_ncol);
                     js = job_size(dv, reqs[q], j - q * ncol);
                 }
-                job_end[j] = js.bytes;
+                job_end[j] = js.bytes + (uint64_t)js.cost_rows * kRowCost;
                 const uint32_t q = fast_div(j, dv.div_ncol);
                 if (j == q * ncol) req_rows[q] = js.rows;
             }

@@ -29,13 +29,14 @@ __device__ __forceinline__ bool put_entry_live(const DockView &dv, const PutArgs
     return true;
 }
 
-// Scatter.  The packed sources of the call's ragged items, laid end to end, are cut into equal
-// chunks, so that work is balanced over tokens rather than samples; warps stride over the
-// chunks (see "Chunked ragged copy" in td_device.cuh).
+// Scatter.  The packed sources of the call's ragged items, laid end to end with every row
+// charged kRowCost on top of its bytes, are cut into equal chunks, so that work is balanced
+// over tokens and rows rather than samples; warps stride over the chunks (see "Chunked ragged
+// copy" in td_device.cuh).
 __global__ void __launch_bounds__(kCopyThreads, kCopyBlocksPerSM)
 put_scatter_kernel(const DockView dv, const PutBatch batch) {
-    __shared__ uint64_t item_end[kMaxPutItems];       // inclusive prefix of bytes (16-byte padded) per item
-    __shared__ uint64_t item_bytes[kMaxPutItems];     // packed bytes of each ragged item (0: nothing to copy)
+    __shared__ uint64_t item_end[kMaxPutItems];       // inclusive prefix of the items' extents (16-byte padded)
+    __shared__ uint64_t item_bytes[kMaxPutItems];     // extent of each ragged item: bytes + rows * kRowCost (0: nothing to copy)
     extern __shared__ __align__(128) uint8_t scatter_smem[];
     const uint32_t tid = threadIdx.x, lane = tid & 31;
     WarpPipe pipe;                                                           // [warps][kPipeSmemPerWarp]
@@ -48,7 +49,8 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
         uint64_t bytes = 0;
         if (dv.col_cls[a.column] != TD_SCALAR && a.k) {
             const int64_t tot = a.cu[a.k];
-            if (tot > 0 && (uint64_t)tot <= a.data_elems) bytes = (uint64_t)tot * dv.col_esz[a.column];
+            if (tot > 0 && (uint64_t)tot <= a.data_elems)
+                bytes = (uint64_t)tot * dv.col_esz[a.column] + (uint64_t)a.k * kRowCost;
         }
         item_bytes[tid] = bytes;
     }
