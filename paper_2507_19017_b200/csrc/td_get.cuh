@@ -100,16 +100,28 @@ get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
     const uint32_t tile = s_tile;
     const uint32_t g = tile * kSelThreads + tid;
 
+    // The claim word and the group's N status words are read with relaxed loads, all in flight
+    // together (four words per load when N allows), and one fence behind them makes the set an
+    // acquire: a status bit seen here was published after its payload, and the gather that
+    // follows in this stream reads that payload.
     bool ready = false;
     if (g < dv.G) {
-        const uint32_t cw = ld_acquire_u32(&claim[g >> 5]);
-        if (!((cw >> (g & 31)) & 1u)) {
-            ready = true;
-            const uint32_t *st = dv.status + (size_t)g * dv.N;
-            for (uint32_t j = 0; j < dv.N; ++j)
-                if ((ld_acquire_u32(st + j) & need) != need) { ready = false; break; }
+        const uint32_t cw = ld_relaxed_u32(&claim[g >> 5]);
+        const uint32_t *st = dv.status + (size_t)g * dv.N;
+        uint32_t all = need;
+        if ((dv.N & 3u) == 0) {
+            #pragma unroll 8
+            for (uint32_t j = 0; j < dv.N; j += 4) {
+                const uint4 w = ld_relaxed_u32x4(st + j);
+                all &= w.x & w.y & w.z & w.w;
+            }
+        } else {
+            #pragma unroll 4
+            for (uint32_t j = 0; j < dv.N; ++j) all &= ld_relaxed_u32(st + j);
         }
+        ready = !((cw >> (g & 31)) & 1u) && all == need;
     }
+    __threadfence();
     const uint32_t ballot = __ballot_sync(kFullMask, ready);
     const uint32_t in_warp = __popc(ballot & ((1u << lane) - 1u));
     if (lane == 0) s_warp[warp] = __popc(ballot);
@@ -348,15 +360,15 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     if ((dv.cflags[c] & TD_F_ADVANTAGE) && out.advantages) {
         const float *rew = reinterpret_cast<const float *>(dv.colbase[dv.reward_col]);
         for (uint32_t p = tid; p < n_grp; p += kFinThreads) {
-            const int32_t *ix = out.indices + (size_t)p * N;
+            const float *r = rew + out.indices[(size_t)p * N];       // a group's samples are consecutive
             double sum = 0.0;
-            for (uint32_t j = 0; j < N; ++j) sum += (double)rew[ix[j]];
+            for (uint32_t j = 0; j < N; ++j) sum += (double)r[j];
             const double mean = sum / (double)N;
             double ss = 0.0;
-            for (uint32_t j = 0; j < N; ++j) { const double d = (double)rew[ix[j]] - mean; ss += d * d; }
+            for (uint32_t j = 0; j < N; ++j) { const double d = (double)r[j] - mean; ss += d * d; }
             const double sd = sqrt(ss / (double)N);
             for (uint32_t j = 0; j < N; ++j)
-                out.advantages[(size_t)p * N + j] = (float)(((double)rew[ix[j]] - mean) / (sd + dv.eps));
+                out.advantages[(size_t)p * N + j] = (float)(((double)r[j] - mean) / (sd + dv.eps));
         }
     }
     __syncthreads();
