@@ -29,7 +29,7 @@ METRIC = "td_put+td_get samples/s dispatched"
 L2_FLUSH_BYTES = 256 << 20
 # DRAM bytes (read + write) of one launch, from the ncu capture summarised under profiles/ for
 # the kernels as built; (config, kernel) pairs without a capture report null.
-NCU_TRAFFIC = {(2, "get_gather"): 79_977_216, (2, "put_scatter"): 45_300_224}
+NCU_TRAFFIC = {(2, "get_gather"): 80_401_152, (2, "put_scatter"): 45_302_784}
 
 
 def parse_args():
