@@ -268,6 +268,23 @@ int td_put_host(td_dock *dock, uint32_t column, const int32_t *h_indices, uint32
 int td_get_host(td_dock *dock, uint32_t consumer, uint32_t max_samples, const td_get_out *dev_out,
                 const td_get_out *host_out, void *stream);
 
+/* The communication-volume model of "Distributed Transfer Dock Strategy", in bytes, for sizing a
+ * dock or a link (host arithmetic only; no device is touched):
+ *   cv        Eq. 1: what one actor-update request takes out of a centralized replay buffer,
+ *             G*N*B*(PL + n*SL + M);
+ *   tcv       Eq. 2: the total over the last three steps of the replay-buffer workflow,
+ *             G*N*B*(2*PL + 3*n*SL + 8*M)                         (Table 1 prints it in GB = 2^30 B);
+ *   tcv_dock  Eq. 4: the share of one of S warehouses when C controllers hold the metadata,
+ *             G*N*B*(2*PL + 3*n*SL + 8*(C+1)*M) / S               (a double: S need not divide).
+ * G prompts, N responses per prompt, PL / SL maximum prompt / response length, n response-length
+ * items and M scalars per sample, B bytes per element.  Any out pointer may be NULL.
+ * TD_EINVAL: NULL model, S = 0, or a product that does not fit 64 bits. */
+typedef struct {
+    uint64_t G, N, PL, n, SL, M, B;
+    uint64_t C, S;                     /* Eq. 4 only */
+} td_model;
+int td_model_bytes(const td_model *m, uint64_t *cv, uint64_t *tcv, double *tcv_dock);
+
 const char *td_strerror(int code);
 
 #ifdef __cplusplus

@@ -30,7 +30,12 @@ EXPORTS = ["td_query_workspace", "td_create", "td_destroy", "td_put", "td_get",
            "td_get_scratch_bytes", "td_reset", "td_status", "td_debug_table",
            "td_launch_count", "td_strerror", "td_kernel_timing", "td_kernel_timing_read",
            "td_put_host_stage_bytes", "td_put_host", "td_get_host", "td_put_many",
-           "td_plan_bytes", "td_plan_create", "td_plan_destroy", "td_get_many", "td_get_static"]
+           "td_plan_bytes", "td_plan_create", "td_plan_destroy", "td_get_many", "td_get_static",
+           "td_model_bytes"]
+
+
+class TdModel(C.Structure):
+    _fields_ = [(k, C.c_uint64) for k in ("G", "N", "PL", "n", "SL", "M", "B", "C", "S")]
 
 
 class TdColumn(C.Structure):
@@ -151,8 +156,18 @@ def lib():
         L.td_get_many.argtypes = [vp, vp, vp]
         L.td_get_static.restype = C.c_int
         L.td_get_static.argtypes = [vp, u32, u32, C.POINTER(TdGetOut), vp]
+        L.td_model_bytes.restype = C.c_int
+        L.td_model_bytes.argtypes = [C.POINTER(TdModel), C.POINTER(u64), C.POINTER(u64), C.POINTER(C.c_double)]
         _lib = L
     return _lib
+
+
+def model_bytes(G, N, PL, n, SL, M, B=4, C_=0, S=1):
+    """Eq. 1, Eq. 2 and Eq. 4 of the paper's volume model, in bytes: (cv, tcv, tcv_dock)."""
+    m = TdModel(G, N, PL, n, SL, M, B, C_, S)
+    cv, tcv, dock = C.c_uint64(), C.c_uint64(), C.c_double()
+    _check("td_model_bytes", lib().td_model_bytes(C.byref(m), C.byref(cv), C.byref(tcv), C.byref(dock)))
+    return cv.value, tcv.value, dock.value
 
 
 def _check(call: str, rc: int):

@@ -155,6 +155,37 @@ void drop_timing(td_dock *d) {
 
 extern "C" {
 
+// Eq. 1, Eq. 2 and Eq. 4 in exact integer arithmetic (128-bit intermediates, overflow = TD_EINVAL).
+int td_model_bytes(const td_model *m, uint64_t *cv, uint64_t *tcv, double *tcv_dock) {
+    if (!m) return TD_EINVAL;
+    typedef unsigned __int128 u128;
+    const u128 lim = (u128)1 << 64;
+    auto mul = [&](u128 a, u128 b, bool &ok) -> u128 {
+        if (a >= lim || b >= lim) { ok = false; return 0; }     // factors below 2^64: the product fits 128 bits
+        const u128 p = a * b;
+        if (p >= lim) ok = false;
+        return p;
+    };
+    bool ok = true;
+    const u128 samples = mul(mul(m->G, m->N, ok), m->B, ok);                 // G*N*B
+    const u128 resp = mul(m->n, m->SL, ok);                                   // n*SL
+    const u128 per1 = (u128)m->PL + resp + m->M;                              // Eq. 1 bracket
+    const u128 per2 = 2 * (u128)m->PL + 3 * resp + 8 * (u128)m->M;            // Eq. 2 bracket
+    const u128 v1 = mul(samples, per1, ok), v2 = mul(samples, per2, ok);
+    if (!ok) return TD_EINVAL;
+    if (cv) *cv = (uint64_t)v1;
+    if (tcv) *tcv = (uint64_t)v2;
+    if (tcv_dock) {
+        if (m->S == 0) return TD_EINVAL;
+        const u128 meta = mul(8 * ((u128)m->C + 1), m->M, ok);                // 8*(C+1)*M
+        const u128 per4 = 2 * (u128)m->PL + 3 * resp + meta;
+        const u128 v4 = mul(samples, per4, ok);
+        if (!ok) return TD_EINVAL;
+        *tcv_dock = (double)(uint64_t)v4 / (double)m->S;
+    }
+    return TD_OK;
+}
+
 const char *td_strerror(int code) {
     switch (code) {
         case TD_OK: return "ok";
