@@ -203,6 +203,29 @@ typedef struct {
 } td_put_item;
 int td_put_many(td_dock *dock, const td_put_item *items, uint32_t n_items, void *stream);
 
+/* Workflow steps 2 and 3 for a worker state that sends back what it computed from a batch it was
+ * just served (the reference model's log-probs, the reward, ...), which is how readiness cascades
+ * from generation through the inference states to the actor update (Fig. 1, Fig. 2): the samples
+ * are the ones the get returned, and their number is read from the get's result block on the
+ * device when the put executes, so the host neither waits for the get nor learns its size.
+ *   batch        the td_get_out of that get (host struct, device pointers): indices, cu_prompt,
+ *                cu_response and result are used and must stay valid until the put has executed;
+ *                the put must be ordered behind the get (same stream, or an event).
+ *   max_samples  upper bound of the batch size (the value given to the get).
+ *   items        host array; column `column` takes row i of the batch from d_data (device) at
+ *                element cu_<class>[i], i.e. rows packed in batch order exactly as a packed get
+ *                lays them out; a TD_SCALAR column takes element i.  data_elems bounds what is
+ *                read.
+ * Everything else is td_put_many's: rows are placed and checked the same way, and the same
+ * conditions are counted. */
+typedef struct {
+    uint32_t column, reserved;
+    const void *d_data;
+    uint64_t data_elems;
+} td_back_item;
+int td_put_back(td_dock *dock, const td_get_out *batch, uint32_t max_samples, const td_back_item *items,
+                uint32_t n_items, void *stream);
+
 /* Many gets served by one call.  Each worker state has its own controller and a step serves
  * several of them, each in several micro-batches; a plan fixes the list of requests (consumer,
  * max_samples, output buffers) once and td_get_many then serves all of them with three kernel

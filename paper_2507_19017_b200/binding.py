@@ -31,7 +31,7 @@ EXPORTS = ["td_query_workspace", "td_create", "td_destroy", "td_put", "td_get",
            "td_launch_count", "td_strerror", "td_kernel_timing", "td_kernel_timing_read",
            "td_put_host_stage_bytes", "td_put_host", "td_get_host", "td_put_many",
            "td_plan_bytes", "td_plan_create", "td_plan_destroy", "td_get_many", "td_get_static",
-           "td_model_bytes"]
+           "td_model_bytes", "td_put_back"]
 
 
 class TdModel(C.Structure):
@@ -73,6 +73,11 @@ class TdGetOut(C.Structure):
 class TdPutItem(C.Structure):
     _fields_ = [("column", C.c_uint32), ("k", C.c_uint32), ("d_indices", C.c_void_p),
                 ("d_cu", C.c_void_p), ("d_data", C.c_void_p), ("data_elems", C.c_uint64)]
+
+
+class TdBackItem(C.Structure):
+    _fields_ = [("column", C.c_uint32), ("reserved", C.c_uint32), ("d_data", C.c_void_p),
+                ("data_elems", C.c_uint64)]
 
 
 class TdGetReq(C.Structure):
@@ -146,6 +151,8 @@ def lib():
         L.td_get_host.argtypes = [vp, u32, u32, C.POINTER(TdGetOut), C.POINTER(TdGetOut), vp]
         L.td_put_many.restype = C.c_int
         L.td_put_many.argtypes = [vp, C.POINTER(TdPutItem), u32, vp]
+        L.td_put_back.restype = C.c_int
+        L.td_put_back.argtypes = [vp, C.POINTER(TdGetOut), u32, C.POINTER(TdBackItem), u32, vp]
         L.td_plan_bytes.restype = C.c_size_t
         L.td_plan_bytes.argtypes = [vp, u32]
         L.td_plan_create.restype = C.c_int
@@ -377,6 +384,15 @@ class Dock:
             arr[j] = TdPutItem(column, indices.numel(), indices.data_ptr(),
                                cu.data_ptr() if cu is not None else None, data.data_ptr(), data.numel())
         _check("td_put_many", lib().td_put_many(self.handle, arr, len(items), _stream_ptr(stream)))
+
+    def put_back(self, bufs: GetBuffers, items: Sequence[Tuple], stream=None):
+        """items: (column, data) device tensors holding the rows of the batch last served into
+        `bufs`, packed in batch order; the batch size is read on the device."""
+        arr = (TdBackItem * len(items))()
+        for j, (column, data) in enumerate(items):
+            arr[j] = TdBackItem(column, 0, data.data_ptr(), data.numel())
+        _check("td_put_back", lib().td_put_back(self.handle, C.byref(bufs.struct), bufs.max_samples,
+                                                arr, len(items), _stream_ptr(stream)))
 
     def plan(self, bufs: Sequence[GetBuffers], stream=None) -> "Plan":
         return Plan(self, bufs, stream)

@@ -353,27 +353,57 @@ int check_get_out(const DockView &v, uint32_t consumer, uint32_t max_samples, co
 
 }  // namespace
 
-int td_put_many(td_dock *d, const td_put_item *items, uint32_t n_items, void *stream) {
-    if (!d || (n_items && !items)) return TD_EINVAL;
-    for (uint32_t i = 0; i < n_items; ++i)
-        if (!valid_put_item(d, items[i])) return TD_EINVAL;
-    cudaStream_t st = (cudaStream_t)stream;
+namespace {
+// Items in call order, cut into launch groups of at most kMaxPutItems in which no column
+// appears twice.
+int put_items(td_dock *d, const PutArgs *items, uint32_t n_items, cudaStream_t st) {
     PutBatch b;
     std::memset(&b, 0, sizeof(b));
     uint32_t seen = 0;
     for (uint32_t i = 0; i < n_items; ++i) {
-        const td_put_item &it = items[i];
+        const PutArgs &it = items[i];
         if (it.k == 0) continue;
         if (b.n_items == kMaxPutItems || (seen >> it.column) & 1u) {
             const int rc = put_group(d, b, st);
             if (rc != TD_OK) return rc;
             b.n_items = 0; seen = 0;
         }
-        b.item[b.n_items++] = PutArgs{it.column, it.k, it.d_indices, it.d_cu,
-                                      static_cast<const uint8_t *>(it.d_data), it.data_elems};
+        b.item[b.n_items++] = it;
         seen |= 1u << it.column;
     }
     return b.n_items ? put_group(d, b, st) : TD_OK;
+}
+}  // namespace
+
+int td_put_many(td_dock *d, const td_put_item *items, uint32_t n_items, void *stream) {
+    if (!d || (n_items && !items)) return TD_EINVAL;
+    for (uint32_t i = 0; i < n_items; ++i)
+        if (!valid_put_item(d, items[i])) return TD_EINVAL;
+    std::vector<PutArgs> args(n_items);
+    for (uint32_t i = 0; i < n_items; ++i) {
+        const td_put_item &it = items[i];
+        args[i] = PutArgs{it.column, it.k, it.d_indices, it.d_cu, static_cast<const uint8_t *>(it.d_data),
+                          it.data_elems, nullptr};
+    }
+    return put_items(d, args.data(), n_items, (cudaStream_t)stream);
+}
+
+int td_put_back(td_dock *d, const td_get_out *batch, uint32_t max_samples, const td_back_item *items,
+                uint32_t n_items, void *stream) {
+    if (!d || !batch || (n_items && !items)) return TD_EINVAL;
+    if (!batch->indices || !batch->cu_prompt || !batch->cu_response || !batch->result) return TD_EINVAL;
+    if (max_samples == 0 || n_items == 0) return TD_OK;
+    const DockView &v = d->dv;
+    std::vector<PutArgs> args(n_items);
+    for (uint32_t i = 0; i < n_items; ++i) {
+        const td_back_item &it = items[i];
+        if (it.column >= v.ncol || (!it.d_data && it.data_elems) || it.data_elems >= (1ull << 31)) return TD_EINVAL;
+        const uint32_t cls = v.col_cls[it.column];
+        const int32_t *cu = cls == TD_PROMPT ? batch->cu_prompt : cls == TD_RESPONSE ? batch->cu_response : nullptr;
+        args[i] = PutArgs{it.column, max_samples, batch->indices, cu, static_cast<const uint8_t *>(it.d_data),
+                          it.data_elems, &batch->result->n_samples};
+    }
+    return put_items(d, args.data(), n_items, (cudaStream_t)stream);
 }
 
 int td_put(td_dock *d, uint32_t column, const int32_t *d_indices, uint32_t k, const int32_t *d_cu,

@@ -20,7 +20,13 @@ struct PutArgs {
     const int32_t *cu;
     const uint8_t *data;
     uint64_t data_elems;
+    const uint32_t *k_dev;                     // when set: the entry count, at most k, is read here on the device
 };
+// Entries of an item.  A worker that sends back what it computed from a batch does not know on
+// the host how many samples the get returned; the count then comes from the get's result block.
+__device__ __forceinline__ uint32_t item_k(const PutArgs &a) {
+    return a.k_dev ? min(a.k, *a.k_dev) : a.k;
+}
 struct PutBatch {                              // the columns of one call, in call order
     uint32_t n_items;
     uint32_t pad;
@@ -103,7 +109,7 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
     for (uint32_t it = 0; it < batch.n_items; ++it) {
         const PutArgs &a = batch.item[it];
         if (dv.col_cls[a.column] != L) continue;
-        const uint64_t bytes = (uint64_t)a.k * 4u;
+        const uint64_t bytes = (uint64_t)item_k(a) * 4u;
         for (uint64_t at = (uint64_t)tid * 128u; at < bytes; at += (uint64_t)kAllocThreads * 128u) {
             asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint8_t *>(a.idx) + at));
             asm volatile("prefetch.global.L2 [%0];" ::"l"(reinterpret_cast<const uint8_t *>(a.cu) + at));
@@ -114,7 +120,8 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
         const PutArgs &a = batch.item[it];
         if (dv.col_cls[a.column] != L) continue;
         const uint32_t bit = 1u << a.column;
-        for (uint32_t base = 0; base < a.k; base += kAllocPass) {
+        const uint32_t k = item_k(a);
+        for (uint32_t base = 0; base < k; base += kAllocPass) {
             // 1. validate, CAS
             int32_t s[kAllocPer];
             uint32_t room[kAllocPer], sh[kAllocPer];
@@ -124,7 +131,7 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
             for (int j = 0; j < kAllocPer; ++j) {
                 const uint32_t i = base + j * kAllocThreads + tid;
                 alloc[j] = false; s[j] = -1; room[j] = 0; sh[j] = 0;
-                if (i < a.k) {
+                if (i < k) {
                     s[j] = a.idx[i];
                     const int64_t c0 = a.cu[i], c1 = a.cu[i + 1];
                     const int64_t l = c1 - c0;
@@ -160,7 +167,7 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
             #pragma unroll
             for (int j = 0; j < kAllocPer; ++j) {
                 rel[j] = 0;
-                if (base + (uint32_t)j * kAllocThreads >= a.k) break;     // uniform
+                if (base + (uint32_t)j * kAllocThreads >= k) break;       // uniform
                 for (uint32_t q = tid; q < kAllocWarps * S; q += kAllocThreads) tot[q] = 0;
                 unsigned long long pre, wsum;
                 bool leader;
@@ -204,7 +211,7 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
                     atomicAdd(&dv.cursor[L][k2], 0ull - s_run[k2]);
                 __syncthreads();
                 if (tid == 0) {
-                    const uint32_t n_here = min((uint32_t)kAllocPass, a.k - base);
+                    const uint32_t n_here = min((uint32_t)kAllocPass, k - base);
                     for (uint32_t t = 0; t < n_here; ++t) {
                         const uint32_t r = e_room[t];
                         if (r == kNotAllocating) continue;

@@ -37,6 +37,7 @@ __global__ void __launch_bounds__(kCopyThreads, kCopyBlocksPerSM)
 put_scatter_kernel(const DockView dv, const PutBatch batch) {
     __shared__ uint64_t item_end[kMaxPutItems];       // inclusive prefix of the items' extents (16-byte padded)
     __shared__ uint64_t item_bytes[kMaxPutItems];     // extent of each ragged item: bytes + rows * kRowCost (0: nothing to copy)
+    __shared__ uint32_t item_rows[kMaxPutItems];      // entries of each item
     extern __shared__ __align__(128) uint8_t scatter_smem[];
     const uint32_t tid = threadIdx.x, lane = tid & 31;
     WarpPipe pipe;                                                           // [warps][kPipeSmemPerWarp]
@@ -46,13 +47,15 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
 
     if (tid < batch.n_items) {                         // one thread per item: the totals load side by side
         const PutArgs &a = batch.item[tid];
+        const uint32_t k = item_k(a);
         uint64_t bytes = 0;
-        if (dv.col_cls[a.column] != TD_SCALAR && a.k) {
-            const int64_t tot = a.cu[a.k];
+        if (dv.col_cls[a.column] != TD_SCALAR && k) {
+            const int64_t tot = a.cu[k];
             if (tot > 0 && (uint64_t)tot <= a.data_elems)
-                bytes = (uint64_t)tot * dv.col_esz[a.column] + (uint64_t)a.k * kRowCost;
+                bytes = (uint64_t)tot * dv.col_esz[a.column] + (uint64_t)k * kRowCost;
         }
         item_bytes[tid] = bytes;
+        item_rows[tid] = k;
     }
     __syncthreads();
     if (tid == 0) {
@@ -80,12 +83,12 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
             const uint32_t bit = 1u << a.column;
             const uint64_t b0 = g0 - start;
             g0 = min(g1, item_end[it]);
-            if (L == TD_SCALAR || a.k == 0) continue;
+            if (L == TD_SCALAR || item_rows[it] == 0) continue;
             const uint64_t b1 = min(g0 - start, item_bytes[it]);
             if (b1 <= b0) continue;
             uint8_t *arena = dv.colbase[a.column];
             const uint64_t cap = dv.cap[L];
-            warp_copy_chunk<false>(a.cu, a.k, b0, b1, const_cast<uint8_t *>(a.data), esz, lane,
+            warp_copy_chunk<false>(a.cu, item_rows[it], b0, b1, const_cast<uint8_t *>(a.data), esz, lane,
                                    a.data, a.data + a.data_elems * esz, pipe, a.idx,
                                    [&](uint32_t i, int64_t c0, int64_t c1) -> uint8_t * {
                                        // the row is live if the alloc kernel accepted it
@@ -113,7 +116,11 @@ put_publish_kernel(const DockView dv, const PutBatch batch) {
     griddep_wait();                                    // every payload byte of the call is in place
     uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     uint32_t it = 0;
-    while (it < batch.n_items && i >= batch.item[it].k) { i -= batch.item[it].k; ++it; }
+    for (; it < batch.n_items; ++it) {                 // grid slots are laid out by the items' largest counts
+        if (i < batch.item[it].k) break;
+        i -= batch.item[it].k;
+    }
+    if (it < batch.n_items && i >= item_k(batch.item[it])) it = batch.n_items;
     uint32_t ok = 0, n_oob = 0, n_dup = 0, n_bad = 0, column = 0;
     if (it < batch.n_items) {
         const PutArgs &a = batch.item[it];

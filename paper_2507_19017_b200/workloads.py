@@ -46,11 +46,12 @@ class ConsumerSpec:
 @dataclass
 class Op:
     """One call of a schedule: a put of `column` for `indices`, or a get."""
-    kind: str                         # "put" | "get"
+    kind: str                         # "put" | "get" | "put_back"
     column: int = -1                  # put: column number
     indices: Optional[np.ndarray] = None  # put: int32 sample indices, call order
     consumer: int = -1                # get: consumer number
     max_samples: int = 0              # get: micro-batch size
+    columns: Optional[List[int]] = None   # put_back: columns `consumer` sends back for the batch it got last
 
 
 @dataclass
@@ -71,6 +72,9 @@ class Workload:
     vocab: int
     seed: int
     ops: List[Op] = field(default_factory=list)
+    # cascade schedule: column -> what a worker state sends back for a batch, rows packed in batch
+    # order (row i of the batch at cu[i]); long enough for the largest micro-batch
+    pool: Dict[int, np.ndarray] = field(default_factory=dict)
 
     @property
     def n(self) -> int:
@@ -257,6 +261,61 @@ def _interleaved_ops(w: Workload, rng: np.random.Generator, lo: int, hi: int, po
     return ops
 
 
+# Which worker state produces which column in the cascade (Fig. 1: the inference states feed the
+# actor update): the reference model its log-probs, the reward state the reward, the actor's
+# inference pass the old log-probs (and the entropy, where the shape has it).
+CASCADE_PRODUCES = {"reference": ("ref_logprob",), "reward": ("reward",),
+                    "actor_inference": ("old_logprob", "entropy")}
+
+
+def _cascade_ops(w: Workload, rng: np.random.Generator, lo: int, hi: int, poll_every: int) -> List[Op]:
+    """The whole sample flow on one dock: generation puts prompt and response ids in shuffled
+    chunks; every `poll_every` puts each inference state takes a micro-batch and sends its
+    column back for exactly that batch, and the actor update takes what has become complete."""
+    gen = [w.column_index("prompt_ids"), w.column_index("response_ids")]
+    names = [c.name for c in w.columns]
+    produces = {ci: [w.column_index(nm) for nm in CASCADE_PRODUCES.get(k.name, ()) if nm in names]
+                for ci, k in enumerate(w.consumers)}
+    # the pools: seeded values of each produced column's type, sized for the largest micro-batch
+    top_r = int(np.sort(w.len_response)[::-1][:w.micro_batch].sum(dtype=np.int64))
+    for cols in produces.values():
+        for c in cols:
+            spec = w.columns[c]
+            m = w.micro_batch if spec.cls == SCALAR else top_r
+            if spec.name == "reward":
+                w.pool[c] = rng.standard_normal(m, dtype=np.float32)
+            elif spec.dtype == "bf16":
+                w.pool[c] = f32_to_bf16_bits(rng.random(m, dtype=np.float32) * np.float32(4.0))
+            else:
+                w.pool[c] = (rng.random(m, dtype=np.float32) * np.float32(10.0) - np.float32(10.0)).astype(np.float32)
+    puts: List[Op] = []
+    for c in gen:
+        for ch in _chunks(rng, rng.permutation(w.n), lo, hi):
+            puts.append(Op("put", column=c, indices=ch))
+    workers = [ci for ci, cols in produces.items() if cols]
+    updaters = [ci for ci, cols in produces.items() if not cols]
+
+    def poll(ops: List[Op], inference: bool = True):
+        if inference:
+            for ci in workers:
+                ops.append(Op("get", consumer=ci, max_samples=w.micro_batch))
+                ops.append(Op("put_back", consumer=ci, columns=produces[ci]))
+        for ci in updaters:
+            ops.append(Op("get", consumer=ci, max_samples=w.micro_batch))
+
+    ops: List[Op] = []
+    for j, i in enumerate(rng.permutation(len(puts))):
+        ops.append(puts[i])
+        if (j + 1) % poll_every == 0:
+            poll(ops)
+    rounds = -(-w.n // w.micro_batch)
+    for _ in range(rounds):
+        poll(ops)
+    for _ in range(rounds):
+        poll(ops, inference=False)
+    return ops
+
+
 def make_custom(name: str, G: int, N: int, S: int, *, prompt_len: Tuple[int, int],
                 response: Tuple, vocab: int, micro_batch: int, seed: int,
                 with_entropy: bool = False, schedule: str = "bulk",
@@ -287,6 +346,8 @@ def make_custom(name: str, G: int, N: int, S: int, *, prompt_len: Tuple[int, int
         w.ops = _random_order_ops(w, rng, *chunk)
     elif schedule == "interleaved":
         w.ops = _interleaved_ops(w, rng, chunk[0], chunk[1], poll_every)
+    elif schedule == "cascade":
+        w.ops = _cascade_ops(w, rng, chunk[0], chunk[1], poll_every)
     elif schedule == "none":
         w.ops = []
     else:

@@ -189,11 +189,26 @@ def replay_both(w: wl.Workload, mode: int = td.PACKED, check_state_every: int = 
     pad_p, pad_r = (w.pad_prompt_to, w.pad_response_to) if mode == td.PADDED else (0, 0)
     n_get = 0
     batches = []
+    last = {}
+    pool_dev = {c: to_device(a, g.device) for c, a in w.pool.items()}
     for j, op in enumerate(w.ops):
         if op.kind == "put":
             cu, data = w.pack(op.column, op.indices)
             o.put(op.column, op.indices, cu, data)
             g.put(op.column, op.indices, cu, data)
+        elif op.kind == "put_back":
+            # the get of this consumer was enqueued just before; nothing has synchronised since
+            want, bufs = last[op.consumer]
+            g.dock.put_back(bufs, [(c, pool_dev[c]) for c in op.columns])
+            H.oracle_put_back(w, o, want, op.columns)
+            assert_batch_equal(g.read(bufs), want, f"op {j} consumer {op.consumer} (after write-back)")
+        elif any(k.kind == "put_back" and k.consumer == op.consumer for k in w.ops[j + 1:j + 2]):
+            want = o.get(op.consumer, op.max_samples, mode, pad_p, pad_r)
+            bufs = g.buffers(op.consumer, op.max_samples, mode, pad_p, pad_r)
+            g.dock.get(bufs)                         # not read back before the write-back is enqueued
+            last[op.consumer] = (want, bufs)
+            batches.append((op.consumer, want))
+            n_get += 1
         else:
             if max_get_checks is not None and n_get >= max_get_checks:
                 continue

@@ -20,16 +20,40 @@ def make_oracle(w: wl.Workload, prompt_cap=None, response_cap=None, eps: float =
                           w.column_index("reward"), eps)
 
 
+def back_rows(w: wl.Workload, column: int, batch) -> tuple:
+    """What a worker state sends back for `batch`: (cu or None, data) cut from the workload's pool,
+    row i of the batch at cu[i]."""
+    k = batch.n_samples
+    cls = w.columns[column].cls
+    if cls == wl.SCALAR:
+        return None, w.pool[column][:k]
+    cu = batch.cu_prompt if cls == wl.PROMPT else batch.cu_response
+    return np.ascontiguousarray(cu[:k + 1], dtype=np.int32), w.pool[column][:int(cu[k])]
+
+
+def oracle_put_back(w: wl.Workload, dock: ora.OracleDock, batch, columns) -> None:
+    """The oracle's statement of a write-back: an ordinary put of the batch's samples."""
+    if batch.n_samples == 0:
+        return
+    for c in columns:
+        cu, data = back_rows(w, c, batch)
+        dock.put(c, batch.indices, cu, data)
+
+
 def replay_oracle(w: wl.Workload, dock: ora.OracleDock, mode: int = ora.PACKED) -> List:
     """Run w.ops in order; returns the list of batches of the get ops."""
     out = []
+    last = {}
     for op in w.ops:
         if op.kind == "put":
             cu, data = w.pack(op.column, op.indices)
             dock.put(op.column, op.indices, cu, data)
+        elif op.kind == "put_back":
+            oracle_put_back(w, dock, last[op.consumer], op.columns)
         else:
             out.append((op.consumer, dock.get(op.consumer, op.max_samples, mode,
                                               w.pad_prompt_to, w.pad_response_to)))
+            last[op.consumer] = out[-1][1]
     return out
 
 

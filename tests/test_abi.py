@@ -95,6 +95,7 @@ def test_create_reports_workspace_and_argument_errors_before_any_cuda_call(td):
     assert td.lib().td_put(None, 0, None, 1, None, None, 0, None) == td.EINVAL
     assert td.lib().td_get(None, 0, 8, None, None) == td.EINVAL
     assert td.lib().td_launch_count(None) == 0
+    assert td.lib().td_put_back(None, None, 8, None, 0, None) == td.EINVAL
 
 
 def test_create_fails_loudly_without_a_device(td):

@@ -76,6 +76,31 @@ def test_config4_interleaved_serialized(G):
 
 
 # --------------------------------------------------------------- shapes that stress the kernels
+def test_cascade_write_back_small(G):
+    """Generation puts, the inference states send their columns back for the batches they were
+    served (batch size read on the device, no host round trip), the actor update takes what is
+    complete: every get and the final state against the oracle."""
+    w = wl.make_custom("cascade-small", 24, 4, 3, prompt_len=(5, 70), response=("uniform", 1, 300),
+                       vocab=50000, micro_batch=8, seed=31, schedule="cascade", chunk=(1, 12),
+                       poll_every=3, with_entropy=True)
+    g, o, batches = G.replay_both(w, check_state_every=7)
+    upd = len(w.consumers) - 1
+    assert sum(b.n_samples for c, b in batches if c == upd) == w.n
+
+
+@pytest.mark.parametrize("cid", [2, 3])
+def test_cascade_write_back_full_size(G, cid):
+    base = wl.make_config(cid, schedule="none")
+    w = wl.make_custom(f"cascade-{cid}", base.G, base.N, base.S,
+                       prompt_len=(128, 1024) if cid == 2 else (256, 2048),
+                       response=("lognormal", 1500.0 if cid == 2 else 3000.0, 0.25, 4096 if cid == 2 else 16384),
+                       vocab=152064, micro_batch=base.micro_batch, seed=wl.BASE_SEED + 100 + cid,
+                       schedule="cascade", chunk=(16, 256), poll_every=6, with_entropy=cid == 3)
+    g, o, batches = G.replay_both(w, check_state_every=0, arenas=cid == 2)
+    upd = len(w.consumers) - 1
+    assert sum(b.n_samples for c, b in batches if c == upd) == w.n
+
+
 @pytest.mark.parametrize("N,Gp,S", [(1, 12, 3), (3, 10, 5), (5, 8, 2), (7, 6, 1), (32, 4, 4), (33, 3, 3)])
 def test_group_sizes_that_do_not_divide_a_warp(G, N, Gp, S):
     w = wl.make_custom("odd", Gp, N, S, prompt_len=(1, 70), response=("uniform", 0, 200), vocab=50000,
@@ -214,7 +239,7 @@ def test_get_many_partial_readiness_and_reuse(G):
     served = 0
     for j, op in enumerate(gets):
         want = o.get(op.consumer, op.max_samples)
-        G.assert_batch_equal(g.read(bufs[j]), want, f"round 1 request {j}")
+        G.assert_batch_equal(g.read(bufs[j]), want, f"first call, request {j}")
         served += want.n_samples
     assert served == 22 * len(w.consumers)
     for c in range(len(w.columns)):
@@ -222,7 +247,7 @@ def test_get_many_partial_readiness_and_reuse(G):
         o.put(c, rest, cu, data); g.put(c, rest, cu, data)
     g.dock.get_many(plan)
     for j, op in enumerate(gets):
-        G.assert_batch_equal(g.read(bufs[j]), o.get(op.consumer, op.max_samples), f"round 2 request {j}")
+        G.assert_batch_equal(g.read(bufs[j]), o.get(op.consumer, op.max_samples), f"second call, request {j}")
     G.assert_state_equal(g, o, ctx="many2")
 
 

@@ -361,3 +361,55 @@ def test_actor_update_get_moves_eq1_bytes_when_all_lengths_are_maximal():
     (_, b), = [x for x in H.replay_oracle(w, d) if x[0] == 3]
     nbytes = b.indices.nbytes + b.advantages.nbytes + sum(a.nbytes for a in b.columns.values())
     assert nbytes == pytest.approx(ora.cv(G, N, 4, PL, 3, SL, 3) * 1024 ** 3, rel=1e-12)
+
+
+# ---------------------------------------------------------------- cascade (write-back)
+def test_cascade_write_back_round_trip():
+    """The whole sample flow on one dock: inference states send a column back for the batch they
+    were served.  What the actor update finally receives is pinned without the oracle: the
+    test itself remembers which pool row went to which sample, from the batches' index lists
+    and the generator's lengths alone."""
+    w = small(schedule="cascade", G=12, N=3, S=3, poll_every=4, with_entropy=True, micro_batch=6)
+    d = H.make_oracle(w)
+    out = H.replay_oracle(w, d)
+    # rows each sample was sent, rebuilt from the batches
+    sent = {}
+    it = iter(out)
+    last = {}
+    for op in w.ops:
+        if op.kind == "get":
+            c, b = next(it)
+            last[c] = b
+        elif op.kind == "put_back":
+            b = last[op.consumer]
+            lens = w.len_response[b.indices] if b.n_samples else np.zeros(0, np.int32)
+            cu = np.concatenate([[0], np.cumsum(lens)])
+            for col in op.columns:
+                for i, s in enumerate(b.indices):
+                    if w.columns[col].cls == wl.SCALAR:
+                        sent[(col, int(s))] = w.pool[col][i:i + 1]
+                    else:
+                        sent[(col, int(s))] = w.pool[col][cu[i]:cu[i + 1]]
+    upd = len(w.consumers) - 1
+    seen = []
+    for c, b in out:
+        if c != upd:
+            continue
+        seen.extend(b.indices.tolist())
+        for col, spec in enumerate(w.columns):
+            if spec.name in ("prompt_ids", "response_ids"):
+                want = H.expected_packed(w, col, b.indices)
+            else:
+                parts = [sent[(col, int(s))] for s in b.indices]
+                want = np.concatenate(parts) if parts else np.zeros(0, w.pool[col].dtype)
+            assert H.bits_equal(b.columns[col], want), spec.name
+        # advantages from the rewards that were sent back, by numpy
+        rcol = w.column_index("reward")
+        for g in range(b.n_groups):
+            r = np.array([sent[(rcol, int(s))][0] for s in b.indices[g * w.N:(g + 1) * w.N]], dtype=np.float64)
+            want = (r - r.mean()) / (r.std() + 1e-6)
+            assert np.allclose(b.advantages[g * w.N:(g + 1) * w.N], want.astype(np.float32), rtol=1e-6, atol=1e-7)
+    assert sorted(seen) == list(range(w.n))
+    for c in range(len(w.consumers)):
+        assert sum(b.n_samples for cc, b in out if cc == c) == w.n
+    assert d.stats().error_word == 0
