@@ -171,6 +171,20 @@ static int wanted(const ora_dock *d, const ora_consumer *K, const ora_get_out *o
     return c < d->ncol && ((K->out_mask >> c) & 1u) && out->col[c] != NULL;
 }
 
+/* The fused stream joins a prompt-length and a response-length column of one element size, both
+ * among the consumer's output columns; its advantage twin needs the advantages. */
+static int seq_args_ok(const ora_dock *d, const ora_consumer *K, const ora_get_out *out) {
+    if (out->seq) {
+        uint32_t cp = out->seq_prompt_col, cr = out->seq_response_col;
+        if (cp >= d->ncol || cr >= d->ncol) return 0;
+        if (d->col[cp].cls != ORA_PROMPT || d->col[cr].cls != ORA_RESPONSE) return 0;
+        if (esize(d->col[cp].dtype) != esize(d->col[cr].dtype)) return 0;
+        if (!((K->out_mask >> cp) & 1u) || !((K->out_mask >> cr) & 1u)) return 0;
+    }
+    if (out->seq_advantages && !((K->flags & ORA_F_ADVANTAGE) && out->advantages)) return 0;
+    return 1;
+}
+
 /* Would `count` samples with these token totals and this longest row still fit
  * every buffer the caller supplied? */
 static int fits(const ora_dock *d, const ora_consumer *K, const ora_get_out *out,
@@ -189,6 +203,7 @@ static int fits(const ora_dock *d, const ora_consumer *K, const ora_get_out *out
             if (longest > W || count * (uint64_t)W > cap) return 0;
         }
     }
+    if ((out->seq || out->seq_advantages) && tokP + tokR > out->seq_capacity_elems) return 0;
     return 1;
 }
 
@@ -258,6 +273,31 @@ static void emit(const ora_dock *d, const ora_consumer *K, const int32_t *idx, u
                 out->advantages[g0 + j] = (float)(((double)rew[idx[g0 + j]] - mean) / (sd + d->eps));
         }
     }
+    /* Fused stream: what a varlen trainer reads directly.  Sample i occupies elements
+     * [cu_seq[i], cu_seq[i+1]): its prompt row, then its response row. */
+    if (out->seq || out->seq_advantages) {
+        const uint32_t cp = out->seq_prompt_col, cr = out->seq_response_col;
+        const size_t es = out->seq ? esize(d->col[cp].dtype) : 0;
+        size_t at = 0;
+        for (uint32_t i = 0; i < count; ++i) {
+            int32_t s = idx[i];
+            size_t lp = lenP[s] > 0 ? (size_t)lenP[s] : 0, lr = lenR[s] > 0 ? (size_t)lenR[s] : 0;
+            size_t sh = ora_shard_of(d, (uint32_t)s);
+            if (out->seq) {
+                const uint8_t *srcP = d->arena[cp] +
+                    (sh * d->cap[ORA_PROMPT] + (size_t)(d->off[ORA_PROMPT][s] > 0 ? d->off[ORA_PROMPT][s] : 0)) * es;
+                const uint8_t *srcR = d->arena[cr] +
+                    (sh * d->cap[ORA_RESPONSE] + (size_t)(d->off[ORA_RESPONSE][s] > 0 ? d->off[ORA_RESPONSE][s] : 0)) * es;
+                memcpy((uint8_t *)out->seq + at * es, srcP, lp * es);
+                memcpy((uint8_t *)out->seq + (at + lp) * es, srcR, lr * es);
+            }
+            if (out->seq_advantages) {
+                for (size_t j = 0; j < lp; ++j) out->seq_advantages[at + j] = 0.0f;
+                for (size_t j = 0; j < lr; ++j) out->seq_advantages[at + lp + j] = out->advantages[i];
+            }
+            at += lp + lr;
+        }
+    }
 }
 
 /*
@@ -272,6 +312,7 @@ int ora_get(ora_dock *d, uint32_t consumer, uint32_t max_samples, const ora_get_
     const uint32_t m = max_samples / d->N;
     if (m == 0) return -1;
     ora_consumer *K = &d->cons[consumer];
+    if (!seq_args_ok(d, K, out)) return -1;
     uint32_t taken = 0, status = 0;
     uint64_t tokP = 0, tokR = 0;
     uint32_t maxP = 0, maxR = 0;
@@ -319,6 +360,7 @@ int ora_gather(const ora_dock *d, uint32_t consumer, const int32_t *indices, uin
                const ora_get_out *out) {
     if (!d || !out || consumer >= d->ncons || (count && !indices)) return -1;
     const ora_consumer *K = &d->cons[consumer];
+    if (!seq_args_ok(d, K, out)) return -1;
     uint64_t tokP = 0, tokR = 0; uint32_t maxP = 0, maxR = 0;
     for (uint32_t i = 0; i < count; ++i) {
         int32_t s = indices[i];

@@ -80,6 +80,14 @@ typedef struct {
     uint64_t col_capacity_elems[32];
     float   *advantages;                 /* [max_samples] */
     ora_result *result;
+    /* Fused token stream, optional (seq == NULL and seq_advantages == NULL: not wanted): sample
+     * i's row of column seq_prompt_col followed by its row of column seq_response_col, at
+     * element cu_seq[i] of seq; seq_advantages has the same layout in float: 0 on the prompt
+     * tokens, the sample's advantage on its response tokens. */
+    uint32_t seq_prompt_col, seq_response_col;
+    void    *seq;
+    uint64_t seq_capacity_elems;         /* bounds both */
+    float   *seq_advantages;
 } ora_get_out;
 
 typedef struct {

@@ -65,7 +65,9 @@ class _GetOut(C.Structure):
                 ("indices", C.c_void_p), ("cu_prompt", C.c_void_p), ("cu_response", C.c_void_p),
                 ("cu_seq", C.c_void_p), ("col", C.c_void_p * 32),
                 ("col_capacity_elems", C.c_uint64 * 32), ("advantages", C.c_void_p),
-                ("result", C.POINTER(_Result))]
+                ("result", C.POINTER(_Result)),
+                ("seq_prompt_col", C.c_uint32), ("seq_response_col", C.c_uint32), ("seq", C.c_void_p),
+                ("seq_capacity_elems", C.c_uint64), ("seq_advantages", C.c_void_p)]
 
 
 class _Stats(C.Structure):
@@ -138,6 +140,8 @@ class Batch:
         self.cu_seq: np.ndarray = np.zeros(1, np.int32)
         self.columns: Dict[int, np.ndarray] = {}
         self.advantages: Optional[np.ndarray] = None
+        self.seq: Optional[np.ndarray] = None              # fused prompt+response stream, by cu_seq
+        self.seq_advantages: Optional[np.ndarray] = None   # same layout: 0 on prompt tokens, A on response tokens
 
 
 class OracleDock:
@@ -185,7 +189,7 @@ class OracleDock:
     # -- get / gather -----------------------------------------------------
     def _alloc(self, consumer: int, max_samples: int, mode: int, pad_p: int, pad_r: int,
                capacities: Optional[Dict[int, int]], want: Optional[Sequence[int]],
-               lens_bound: Sequence[int]):
+               lens_bound: Sequence[int], seq=None, seq_adv: bool = False, seq_cap: Optional[int] = None):
         need, outm, flags = self.consumers[consumer]
         res = _Result()
         go = _GetOut()
@@ -219,6 +223,16 @@ class OracleDock:
             adv = np.zeros(max_samples, np.float32)
             go.advantages = adv.ctypes.data
         go.result = C.pointer(res)
+        if seq is not None or seq_adv:
+            cap = int(seq_cap) if seq_cap is not None else int(lens_bound[1]) + int(lens_bound[2])
+            go.seq_capacity_elems = cap
+            if seq is not None:
+                go.seq_prompt_col, go.seq_response_col = seq
+                bufs["seq"] = np.zeros(max(cap, 1), NP_DTYPE[self.columns[seq[0]][0]])
+                go.seq = bufs["seq"].ctypes.data
+            if seq_adv:
+                bufs["seq_advantages"] = np.zeros(max(cap, 1), np.float32)
+                go.seq_advantages = bufs["seq_advantages"].ctypes.data
         return go, res, bufs, cols, adv
 
     def _finish(self, go, res, bufs, cols, adv, mode, pad_p, pad_r) -> Batch:
@@ -242,6 +256,11 @@ class OracleDock:
                 b.columns[c] = a[:tot].copy()
         if adv is not None:
             b.advantages = adv[:k].copy()
+        tot = int(b.prompt_tokens + b.response_tokens)
+        if "seq" in bufs:
+            b.seq = bufs["seq"][:tot].copy()
+        if "seq_advantages" in bufs:
+            b.seq_advantages = bufs["seq_advantages"][:tot].copy()
         return b
 
     def _bounds(self, max_samples: int) -> List[int]:
@@ -255,13 +274,17 @@ class OracleDock:
 
     def get(self, consumer: int, max_samples: int, mode: int = PACKED, pad_prompt_to: int = 0,
             pad_response_to: int = 0, capacities: Optional[Dict[int, int]] = None,
-            want: Optional[Sequence[int]] = None) -> Batch:
+            want: Optional[Sequence[int]] = None, seq=None, seq_adv: bool = False,
+            seq_cap: Optional[int] = None) -> Batch:
+        """seq = (prompt column, response column) asks for the fused token stream, seq_adv for
+        its advantage twin; seq_cap bounds both (default: room for the longest rows)."""
         ragged = [c for c, (_d, cls, _p) in enumerate(self.columns)
                   if cls != 0 and (self.consumers[consumer][1] >> c) & 1 and (want is None or c in want)]
         need_bound = mode == PACKED and any(capacities is None or c not in capacities for c in ragged)
+        need_bound = need_bound or ((seq is not None or seq_adv) and seq_cap is None)
         bound = self._bounds(max_samples) if need_bound else [0, 0, 0]
         go, res, bufs, cols, adv = self._alloc(consumer, max_samples, mode, pad_prompt_to,
-                                               pad_response_to, capacities, want, bound)
+                                               pad_response_to, capacities, want, bound, seq, seq_adv, seq_cap)
         rc = lib().ora_get(self._h, consumer, max_samples, C.byref(go))
         if rc != 0:
             raise ValueError("ora_get: bad argument")
@@ -286,14 +309,15 @@ class OracleDock:
                              cu.ctypes.data if cu is not None else None, data.ctypes.data)
 
     def gather(self, consumer: int, indices: np.ndarray, mode: int = PACKED, pad_prompt_to: int = 0,
-               pad_response_to: int = 0, want: Optional[Sequence[int]] = None) -> Batch:
+               pad_response_to: int = 0, want: Optional[Sequence[int]] = None, seq=None,
+               seq_adv: bool = False) -> Batch:
         idx = np.ascontiguousarray(indices, dtype=np.int32)
         k = len(idx)
         bound = [0, 0, 0]
         for cls in (1, 2):
             bound[cls] = int(np.maximum(self.lengths(cls)[idx], 0).sum(dtype=np.int64)) if k else 0
         go, res, bufs, cols, adv = self._alloc(consumer, max(k, 1), mode, pad_prompt_to,
-                                               pad_response_to, None, want, bound)
+                                               pad_response_to, None, want, bound, seq, seq_adv)
         rc = lib().ora_gather(self._h, consumer, idx.ctypes.data, k, C.byref(go))
         if rc != 0:
             raise ValueError("ora_gather: bad argument")

@@ -413,3 +413,63 @@ def test_cascade_write_back_round_trip():
     for c in range(len(w.consumers)):
         assert sum(b.n_samples for cc, b in out if cc == c) == w.n
     assert d.stats().error_word == 0
+
+
+# ---------------------------------------------------------------- fused token stream
+def _fill_bulk(w, d):
+    for c in range(len(w.columns)):
+        cu, data = w.pack(c, np.arange(w.n, dtype=np.int32))
+        d.put(c, np.arange(w.n), cu, data)
+
+
+def test_fused_stream_is_prompt_then_response_per_sample():
+    """seq equals, sample by sample, the generator's prompt row followed by its response row;
+    seq_advantages is 0 over the prompt and the sample's advantage (numpy z-score of its
+    group's rewards) over the response; cu_seq indexes both."""
+    w = small(schedule="none", G=6, N=3, S=2)
+    d = H.make_oracle(w)
+    _fill_bulk(w, d)
+    pc, rc = w.column_index("prompt_ids"), w.column_index("response_ids")
+    upd = len(w.consumers) - 1
+    b = d.get(upd, w.n, seq=(pc, rc), seq_adv=True)
+    assert b.n_samples == w.n
+    sp, sr = w.row_starts(wl.PROMPT), w.row_starts(wl.RESPONSE)
+    rew = w.data["reward"].astype(np.float64).reshape(w.G, w.N)
+    adv = ((rew - rew.mean(axis=1, keepdims=True)) / (rew.std(axis=1, keepdims=True) + 1e-6)).reshape(-1)
+    want_seq, want_adv = [], []
+    for s in range(w.n):
+        want_seq += [w.data["prompt_ids"][sp[s]:sp[s + 1]], w.data["response_ids"][sr[s]:sr[s + 1]]]
+        want_adv += [np.zeros(w.len_prompt[s], np.float32), np.full(w.len_response[s], adv[s], np.float32)]
+    assert np.array_equal(b.seq, np.concatenate(want_seq))
+    assert np.allclose(b.seq_advantages, np.concatenate(want_adv), rtol=1e-6, atol=1e-7)
+    assert np.array_equal(b.cu_seq, np.concatenate([[0], np.cumsum(w.len_prompt + w.len_response)]))
+    # the prompt part of the mask is exactly zero, and the response part repeats advantages[i]
+    for i in range(w.n):
+        a, m, e = b.cu_seq[i], b.cu_seq[i] + w.len_prompt[i], b.cu_seq[i + 1]
+        assert not b.seq_advantages[a:m].any()
+        assert (b.seq_advantages[m:e] == b.advantages[i]).all()
+
+
+def test_fused_stream_takes_float_columns_and_respects_capacity():
+    """Any prompt/response pair of one element size may be fused; a stream buffer that is too
+    small cuts the batch before the first group that does not fit, like any other column."""
+    cols = [("f32", "prompt", 0), ("f32", "response", 0), ("bf16", "response", 0), ("f32", "scalar", 0)]
+    d = ora.OracleDock(3, 2, 1, cols, [(0xF, 0xF, True)], 256, 256, 3)
+    lp, lr = np.array([3, 3, 5, 5, 2, 2]), np.array([4, 1, 0, 7, 6, 6])
+    rng = np.random.default_rng(3)
+    P, R = rng.random(lp.sum(), dtype=np.float32), rng.random(lr.sum(), dtype=np.float32)
+    idx = np.arange(6, dtype=np.int32)
+    cup, cur = np.concatenate([[0], np.cumsum(lp)]).astype(np.int32), np.concatenate([[0], np.cumsum(lr)]).astype(np.int32)
+    d.put(0, idx, cup, P); d.put(1, idx, cur, R)
+    d.put(2, idx, cur, np.zeros(lr.sum(), np.uint16)); d.put(3, idx, None, np.arange(6, dtype=np.float32))
+    with pytest.raises(ValueError):
+        d.get(0, 6, seq=(0, 2))                       # element sizes differ
+    with pytest.raises(ValueError):
+        d.get(0, 6, seq=(1, 0))                       # classes swapped
+    tot2 = int(lp[:4].sum() + lr[:4].sum())
+    b = d.get(0, 6, seq=(0, 1), seq_adv=True, seq_cap=tot2 + 3)     # room for two groups and a bit
+    assert b.n_groups == 2 and b.status & ora.ERR_OUT_TRUNC
+    want = np.concatenate([np.concatenate([P[cup[i]:cup[i + 1]], R[cur[i]:cur[i + 1]]]) for i in range(4)])
+    assert H.bits_equal(b.seq, want)
+    b2 = d.get(0, 6, seq=(0, 1), seq_cap=64)          # the group that was cut is still there
+    assert b2.n_groups == 1 and list(b2.indices) == [4, 5] and b2.status == 0
