@@ -119,6 +119,18 @@ typedef struct {
                                          this call while it is in flight; zero-filled once after
                                          allocation, never needs clearing afterwards       required */
     uint64_t scratch_bytes;
+    /* Fused token stream, optional (seq == NULL and seq_advantages == NULL: not wanted; a zeroed
+     * struct asks for neither).  What a varlen trainer reads directly: sample i's row of column
+     * seq_prompt_col (TD_PROMPT) followed by its row of column seq_response_col (TD_RESPONSE, same
+     * element size, both within the consumer's out_mask) at element cu_seq[i] of `seq`, in
+     * either output mode; cu_seq is then required.  seq_advantages (needs TD_F_ADVANTAGE) has the
+     * same layout in float: 0 on prompt tokens, the sample's advantage on its response tokens,
+     * i.e. advantage times loss mask.  seq_capacity_elems is the room behind each of the two; a
+     * group that would not fit ends the batch (TD_ERR_OUT_TRUNCATED). */
+    uint32_t seq_prompt_col, seq_response_col;
+    void    *seq;
+    uint64_t seq_capacity_elems;
+    float   *seq_advantages;
 } td_get_out;
 
 typedef struct {

@@ -67,7 +67,9 @@ class TdGetOut(C.Structure):
                 ("indices", C.c_void_p), ("cu_prompt", C.c_void_p), ("cu_response", C.c_void_p),
                 ("cu_seq", C.c_void_p), ("col", C.c_void_p * 32),
                 ("col_capacity_elems", C.c_uint64 * 32), ("advantages", C.c_void_p),
-                ("result", C.c_void_p), ("scratch", C.c_void_p), ("scratch_bytes", C.c_uint64)]
+                ("result", C.c_void_p), ("scratch", C.c_void_p), ("scratch_bytes", C.c_uint64),
+                ("seq_prompt_col", C.c_uint32), ("seq_response_col", C.c_uint32), ("seq", C.c_void_p),
+                ("seq_capacity_elems", C.c_uint64), ("seq_advantages", C.c_void_p)]
 
 
 class TdPutItem(C.Structure):
@@ -217,7 +219,10 @@ class GetBuffers:
     def __init__(self, dock: "Dock", consumer: int, max_samples: int, mode: int = PACKED,
                  pad_prompt_to: int = 0, pad_response_to: int = 0,
                  capacities: Optional[Dict[int, int]] = None, want: Optional[Sequence[int]] = None,
-                 prompt_tokens_cap: Optional[int] = None, response_tokens_cap: Optional[int] = None):
+                 prompt_tokens_cap: Optional[int] = None, response_tokens_cap: Optional[int] = None,
+                 seq: Optional[Tuple[int, int]] = None, seq_adv: bool = False, seq_cap: Optional[int] = None):
+        """seq = (prompt column, response column) adds the fused token stream, seq_adv its
+        advantage twin; seq_cap is the room behind each (default: both token caps together)."""
         import torch
         dev = dock.device
         self.dock, self.consumer, self.max_samples, self.mode = dock, consumer, max_samples, mode
@@ -260,6 +265,17 @@ class GetBuffers:
         go.advantages = self.advantages.data_ptr() if self.advantages is not None else None
         go.result = self.result.data_ptr()
         go.scratch, go.scratch_bytes = self.scratch.data_ptr(), self.scratch.numel()
+        self.seq = self.seq_advantages = None
+        if seq is not None or seq_adv:
+            cap = int(seq_cap) if seq_cap is not None else int(prompt_tokens_cap) + int(response_tokens_cap)
+            go.seq_capacity_elems = cap
+            if seq is not None:
+                go.seq_prompt_col, go.seq_response_col = seq
+                self.seq = torch.empty(max(cap, 1), dtype=tdt[dock.columns[seq[0]][0]], device=dev)
+                go.seq = self.seq.data_ptr()
+            if seq_adv:
+                self.seq_advantages = torch.empty(max(cap, 1), dtype=torch.float32, device=dev)
+                go.seq_advantages = self.seq_advantages.data_ptr()
         self.struct = go
 
     def read_result(self) -> TdResult:

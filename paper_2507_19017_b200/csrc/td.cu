@@ -40,8 +40,8 @@ inline uint32_t esize_of(int32_t dtype) { return dtype == TD_BF16 ? 2u : 4u; }
 // block-scan scratch and the job table.
 constexpr size_t kStageSmem = (size_t)kCopyWarps * kPipeSmemPerWarp;
 size_t scatter_smem_bytes() { return kStageSmem; }
-size_t gather_smem_bytes(uint32_t n_req, uint32_t ncol) {
-    return kStageSmem + (size_t)kCopyWarps * 8 + (size_t)n_req * ncol * 8 + (size_t)n_req * 4;
+size_t gather_smem_bytes(uint32_t n_req, uint32_t jobs_per_req) {
+    return kStageSmem + (size_t)kCopyWarps * 8 + (size_t)n_req * jobs_per_req * 8 + (size_t)n_req * 4;
 }
 
 struct Layout {
@@ -339,8 +339,13 @@ uint64_t room_bytes_of(const DockView &v, uint32_t consumer, uint32_t max_sample
             if (v.col_cls[k] == TD_SCALAR && room > max_samples) room = max_samples;
             bytes += room * v.col_esz[k] + kMinChunkBytes;
         }
+    if (out.seq) bytes += out.seq_capacity_elems * v.col_esz[out.seq_prompt_col] + kMinChunkBytes;
+    if (out.seq_advantages) bytes += out.seq_capacity_elems * 4u + kMinChunkBytes;
     return bytes;
 }
+
+bool wants_stream(const td_get_out &out) { return out.seq || out.seq_advantages; }
+uint32_t jobs_per_req(const DockView &v, bool stream) { return v.ncol + (stream ? kSeqJobs : 0u); }
 
 int check_get_out(const DockView &v, uint32_t consumer, uint32_t max_samples, const td_get_out *out) {
     if (!out || consumer >= v.ncons) return TD_EINVAL;
@@ -348,6 +353,14 @@ int check_get_out(const DockView &v, uint32_t consumer, uint32_t max_samples, co
     if (!out->indices || !out->cu_prompt || !out->cu_response || !out->result) return TD_EINVAL;
     if (out->mode != TD_PACKED && out->mode != TD_PADDED) return TD_EINVAL;
     if ((v.cflags[consumer] & TD_F_ADVANTAGE) && !out->advantages) return TD_EINVAL;
+    if (wants_stream(*out) && !out->cu_seq) return TD_EINVAL;
+    if (out->seq) {
+        const uint32_t cp = out->seq_prompt_col, cr = out->seq_response_col;
+        if (cp >= v.ncol || cr >= v.ncol) return TD_EINVAL;
+        if (v.col_cls[cp] != TD_PROMPT || v.col_cls[cr] != TD_RESPONSE || v.col_esz[cp] != v.col_esz[cr]) return TD_EINVAL;
+        if (!((v.outm[consumer] >> cp) & 1u) || !((v.outm[consumer] >> cr) & 1u)) return TD_EINVAL;
+    }
+    if (out->seq_advantages && !((v.cflags[consumer] & TD_F_ADVANTAGE) && out->advantages)) return TD_EINVAL;
     return TD_OK;
 }
 
@@ -438,16 +451,17 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
     one.cs.max_groups = one.req.max_groups;
     one.cs.scratch = out->scratch;
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
+    const uint32_t jpr = jobs_per_req(v, wants_stream(*out));
 
     if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
     if (launch_dep(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
-               (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr) != cudaSuccess) return TD_ECUDA;
+               (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr) != cudaSuccess) return TD_ECUDA;
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
-    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, v.ncol), st, v, one,
-                     (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr) != cudaSuccess) return TD_ECUDA;
+    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, jpr), st, v, one,
+                     (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr, jpr, make_fastdiv(jpr)) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 
@@ -515,16 +529,17 @@ int td_get_static(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_
     one.cs.max_groups = one.req.max_groups;
     one.cs.scratch = scratch;
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
+    const uint32_t jpr = jobs_per_req(v, wants_stream(*out));
 
     if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
     if (launch_dep(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
-               (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr) != cudaSuccess) return TD_ECUDA;
+               (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr) != cudaSuccess) return TD_ECUDA;
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
-    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, v.ncol), st, v, one,
-                     (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr) != cudaSuccess) return TD_ECUDA;
+    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, jpr), st, v, one,
+                     (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr, jpr, make_fastdiv(jpr)) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 
@@ -535,6 +550,7 @@ struct td_plan {
     GetReq *d_reqs;
     ConsumerSlot *d_slots;
     uint64_t room_bytes;
+    uint32_t jobs_per_req;                // columns, plus the stream's jobs when a request wants it
     unsigned long long *d_counter;        // the gather's chunk counter: word 1 of slot 0's scan scratch
     JobSize *d_job_sizes;                 // [n_req][n_columns] output bytes and rows, written by the finalize kernel
     std::vector<uint8_t> host_image;      // what was uploaded; kept until the plan dies
@@ -545,14 +561,17 @@ size_t td_plan_bytes(const td_dock *d, uint32_t n_req) {
     const size_t slots = d->dv.ncons;
     return align_up_sz((size_t)n_req * sizeof(GetReq), 256) + align_up_sz(slots * sizeof(ConsumerSlot), 256) +
            slots * align_up_sz(sel_scratch_bytes(d->dv.G), 256) +
-           align_up_sz((size_t)n_req * d->dv.ncol * sizeof(JobSize), 256);
+           align_up_sz((size_t)n_req * (d->dv.ncol + kSeqJobs) * sizeof(JobSize), 256);
 }
 
 int td_plan_create(td_dock *d, const td_get_req *reqs, uint32_t n_req, void *d_plan, size_t plan_bytes,
                    void *stream, td_plan **out) {
     if (!d || !reqs || !out || n_req == 0) return TD_EINVAL;
     const DockView &v = d->dv;
-    if ((uint64_t)n_req * v.ncol > (uint64_t)kMaxJobs) return TD_EINVAL;
+    bool stream_wanted = false;
+    for (uint32_t q = 0; q < n_req; ++q) stream_wanted |= wants_stream(reqs[q].out);
+    const uint32_t jpr = jobs_per_req(v, stream_wanted);
+    if ((uint64_t)n_req * jpr > (uint64_t)kMaxJobs) return TD_EINVAL;
     if (!d_plan || (reinterpret_cast<uintptr_t>(d_plan) & 255u) || plan_bytes < td_plan_bytes(d, n_req))
         return TD_EWORKSPACE;
     for (uint32_t q = 0; q < n_req; ++q) {
@@ -561,7 +580,7 @@ int td_plan_create(td_dock *d, const td_get_req *reqs, uint32_t n_req, void *d_p
     }
     td_plan *p = new (std::nothrow) td_plan();
     if (!p) return TD_EINVAL;
-    p->dock = d; p->n_req = n_req;
+    p->dock = d; p->n_req = n_req; p->jobs_per_req = jpr;
     const size_t off_slots = align_up_sz((size_t)n_req * sizeof(GetReq), 256);
     const size_t off_scratch = off_slots + align_up_sz((size_t)v.ncons * sizeof(ConsumerSlot), 256);
     const size_t scratch_each = align_up_sz(sel_scratch_bytes(v.G), 256);
@@ -625,10 +644,11 @@ int td_get_many(td_dock *d, td_plan *p, void *stream) {
     if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), p->n_slots), dim3(kSelThreads), 0, st, v, none,
                (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
     if (launch_dep(d, get_finalize_kernel, dim3(p->n_req), dim3(kFinThreads), 0, st, v, none, (const GetReq *)p->d_reqs,
-               (const ConsumerSlot *)p->d_slots, seq, p->d_counter, p->d_job_sizes) != cudaSuccess) return TD_ECUDA;
+               (const ConsumerSlot *)p->d_slots, seq, p->d_counter, p->d_job_sizes, p->jobs_per_req) != cudaSuccess) return TD_ECUDA;
     if (launch_timed(d, 1, get_gather_kernel, dim3(copy_grid(d, p->room_bytes)), dim3(kCopyThreads),
-                     gather_smem_bytes(p->n_req, v.ncol), st, v, none,
-                     (const GetReq *)p->d_reqs, p->n_req, p->d_counter, (const JobSize *)p->d_job_sizes) != cudaSuccess) return TD_ECUDA;
+                     gather_smem_bytes(p->n_req, p->jobs_per_req), st, v, none,
+                     (const GetReq *)p->d_reqs, p->n_req, p->d_counter, (const JobSize *)p->d_job_sizes,
+                     p->jobs_per_req, make_fastdiv(p->jobs_per_req)) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 
@@ -756,6 +776,16 @@ int td_get_host(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_ge
         else elems = n * (size_t)(cls == TD_PROMPT ? dev_out->pad_prompt_to : dev_out->pad_response_to);
         if (elems > host_out->col_capacity_elems[k]) return TD_EINVAL;
         ok = d2h(host_out->col[k], dev_out->col[k], elems * v.col_esz[k]);
+    }
+    if (ok && dev_out->seq && host_out->seq) {
+        const size_t elems = res->prompt_tokens + res->response_tokens;
+        if (elems > host_out->seq_capacity_elems) return TD_EINVAL;
+        ok = d2h(host_out->seq, dev_out->seq, elems * v.col_esz[dev_out->seq_prompt_col]);
+    }
+    if (ok && dev_out->seq_advantages && host_out->seq_advantages) {
+        const size_t elems = res->prompt_tokens + res->response_tokens;
+        if (elems > host_out->seq_capacity_elems) return TD_EINVAL;
+        ok = d2h(host_out->seq_advantages, dev_out->seq_advantages, elems * 4);
     }
     if (!ok || cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
     return TD_OK;

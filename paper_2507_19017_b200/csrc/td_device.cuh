@@ -492,11 +492,16 @@ static_assert(kRowCost % 16 == 0, "a job's extent stays a multiple of 16");
 // nullptr to skip the row; it is called by one lane per row; `along` is the index array it
 // reads (prefetched by the row search).  kToPacked: the packed side is the destination (get),
 // else the source (put, whose source window is tested against the caller's buffer).
+// seq_cu, when given, moves the rows on the packed side: row i then sits at element seq_cu[i]
+// (seq_tail false) or ends at element seq_cu[i + 1] (seq_tail true) instead of starting at
+// cu[i] - the two halves of a stream in which each sample's prompt row is followed by its
+// response row; cu still says how long the rows are and where they lie in the chunked space.
 template <bool kToPacked, typename Resolve>
 __device__ __forceinline__ void warp_copy_chunk(const int32_t *cu, uint32_t rows, uint64_t b0, uint64_t b1,
                                                 uint8_t *packed, uint32_t esz, uint32_t lane,
                                                 const uint8_t *src_lo, const uint8_t *src_hi, WarpPipe &pipe,
-                                                const int32_t *along, Resolve resolve) {
+                                                const int32_t *along, Resolve resolve,
+                                                const int32_t *seq_cu = nullptr, bool seq_tail = false) {
     uint32_t r0 = warp_find_row(cu, rows, (int64_t)b0, esz, kRowCost, lane, along);
     for (;;) {
         // lane l: the part of row r0 + l that falls inside the chunk, as (address on the packed
@@ -518,7 +523,10 @@ __device__ __forceinline__ void warp_copy_chunk(const int32_t *cu, uint32_t rows
                     uint8_t *row = resolve(i, c0, c1);
                     if (row) {
                         other = row + (lo - dlo);
-                        mine = packed + (uint64_t)c0 * esz + (lo - dlo);
+                        uint64_t at = (uint64_t)c0;
+                        if (seq_cu) at = seq_tail ? (uint64_t)((int64_t)__ldg(seq_cu + i + 1) - (c1 - c0))
+                                                  : (uint64_t)__ldg(seq_cu + i);
+                        mine = packed + at * esz + (lo - dlo);
                         len = (uint32_t)(hi - lo);
                     }
                 }

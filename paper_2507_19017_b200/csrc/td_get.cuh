@@ -11,6 +11,9 @@ constexpr int kSelThreads = 256;            // one thread per group; a tile is 2
 constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kFinThreads = 256;
 constexpr int kMaxJobs = 4096;              // (request, column) pairs one gather launch serves
+// A request that wants the fused token stream has three more jobs behind its columns: the
+// stream's prompt half, its response half, and the advantage twin.
+constexpr uint32_t kSeqJobs = 3;
 
 // Tile descriptor of the single-pass scan: [63:32] launch sequence number, [31:30] state,
 // [29:0] count.  A descriptor whose sequence number is not the launch's is "not written yet",
@@ -222,6 +225,12 @@ __device__ __forceinline__ uint64_t block_scan_incl_2(uint64_t a, uint64_t b, ui
 __device__ __forceinline__ uint64_t job_bytes_of(const DockView &dv, const GetReq &rq, uint32_t k,
                                                  uint64_t n_s, uint64_t prompt_tokens, uint64_t response_tokens) {
     const td_get_out &out = rq.out;
+    if (k >= dv.ncol) {
+        const uint32_t v = k - dv.ncol;
+        if (v == 2) return out.seq_advantages ? (prompt_tokens + response_tokens) * 4u : 0;
+        if (!out.seq) return 0;
+        return (v == 0 ? prompt_tokens : response_tokens) * dv.col_esz[out.seq_prompt_col];
+    }
     if (!((dv.outm[rq.consumer] >> k) & 1u) || out.col[k] == nullptr) return 0;
     const uint32_t cls = dv.col_cls[k], esz = dv.col_esz[k];
     if (cls == TD_SCALAR) return n_s * esz;
@@ -239,13 +248,14 @@ struct JobSize {
 // Extent of a job in the space the gather cuts into chunks (see kRowCost).
 __device__ __forceinline__ uint32_t job_cost_rows(const DockView &dv, const GetReq &rq, uint32_t k,
                                                   uint64_t bytes, uint32_t n_s) {
+    if (k >= dv.ncol) return (bytes != 0 && k - dv.ncol < 2u) ? n_s : 0u;      // the stream's halves are packed rows
     return (bytes != 0 && dv.col_cls[k] != TD_SCALAR && rq.out.mode == TD_PACKED) ? n_s : 0u;
 }
 
 __global__ void __launch_bounds__(kFinThreads)
 get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
                     const GetReq *reqs_dev, const ConsumerSlot *slots_dev, const uint32_t seq,
-                    unsigned long long *work_counter, JobSize *job_sizes) {
+                    unsigned long long *work_counter, JobSize *job_sizes, const uint32_t jobs_per_req) {
     const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
     const ConsumerSlot *slots = slots_dev ? slots_dev : &one.cs;
     const GetReq &rq = reqs[blockIdx.x];
@@ -308,6 +318,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
             room_rows = min(room_rows, W ? (uint64_t)(capk / W) : (uint64_t)0);
         }
     }
+    const uint64_t room_seq = (out.seq || out.seq_advantages) ? out.seq_capacity_elems : ~0ull;
     const bool padded = out.mode == TD_PADDED;
     bool want_p = false, want_r = false;
     for (uint32_t k = 0; k < dv.ncol; ++k)
@@ -335,6 +346,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
             if (!padded) over |= cp > room_tok[TD_PROMPT] || cr > room_tok[TD_RESPONSE];
             else over |= (uint64_t)(i + 1) > room_rows || (want_p && lp > out.pad_prompt_to) ||
                          (want_r && lr > out.pad_response_to);
+            over |= cp + cr > room_seq;
             if (over) atomicMin(&s_first_over, i);
         }
         carry_p += tp; carry_r += tr;
@@ -384,13 +396,13 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
         atomicAdd(&dv.counters[CNT_GOT_TOKENS + c], (unsigned long long)(r.prompt_tokens + r.response_tokens));
     }
     // the gather's job table: this request's output bytes per column and its row count
-    if (job_sizes && tid < dv.ncol) {
+    if (job_sizes && tid < jobs_per_req) {
         JobSize js;
         js.bytes = job_bytes_of(dv, rq, tid, n_s, (uint64_t)(int64_t)out.cu_prompt[n_s],
                                 (uint64_t)(int64_t)out.cu_response[n_s]);
         js.rows = n_s;
         js.cost_rows = job_cost_rows(dv, rq, tid, js.bytes, n_s);
-        job_sizes[(size_t)blockIdx.x * dv.ncol + tid] = js;
+        job_sizes[(size_t)blockIdx.x * jobs_per_req + tid] = js;
     }
 }
 
@@ -409,10 +421,47 @@ __device__ __forceinline__ JobSize job_size(const DockView &dv, const GetReq &rq
     return js;
 }
 
+// The advantage twin of the fused stream, bytes [b0, b1) of it: sample i's prompt tokens get 0,
+// its response tokens its advantage.  Lane l looks row r0 + l up, the warp fills row by row.
+__device__ __noinline__ void warp_fill_seq_advantages(const td_get_out &out, uint32_t n_s, uint64_t b0,
+                                                      uint64_t b1, uint32_t lane) {
+    if (b1 <= b0) return;
+    const int32_t *cs = out.cu_seq, *cp = out.cu_prompt;
+    uint8_t *dst = reinterpret_cast<uint8_t *>(out.seq_advantages);
+    uint32_t r0 = warp_find_row(cs, n_s, (int64_t)b0, 4u, 0u, lane);
+    for (;;) {
+        const uint32_t i = r0 + lane;
+        uint64_t lo = 0, mid = 0, hi = 0;
+        uint32_t bits = 0;
+        bool in = false;
+        if (i < n_s) {
+            lo = (uint64_t)__ldg(cs + i) * 4u;
+            in = lo < b1;
+            if (in) {
+                hi = (uint64_t)__ldg(cs + i + 1) * 4u;
+                mid = lo + (uint64_t)(__ldg(cp + i + 1) - __ldg(cp + i)) * 4u;
+                bits = __float_as_uint(out.advantages[i]);
+            }
+        }
+        const uint32_t inside = __ballot_sync(kFullMask, in);            // a prefix of the lanes
+        const uint32_t n_rows = (uint32_t)__popc(inside);
+        for (uint32_t r = 0; r < n_rows; ++r) {
+            const uint64_t rlo = shfl_u64(lo, r), rmid = shfl_u64(mid, r), rhi = shfl_u64(hi, r);
+            const uint32_t a = __shfl_sync(kFullMask, bits, r);
+            const uint64_t z0 = max(rlo, b0), z1 = min(rmid, b1);
+            if (z1 > z0) warp_fill(dst + z0, z1 - z0, 0u, 4u, lane);
+            const uint64_t a0 = max(rmid, b0), a1 = min(rhi, b1);
+            if (a1 > a0) warp_fill(dst + a0, a1 - a0, a, 4u, lane);
+        }
+        if (n_rows < 32u) break;
+        r0 += 32u;
+    }
+}
+
 __global__ void __launch_bounds__(kCopyThreads, kCopyBlocksPerSM)
 get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
                   const GetReq *reqs_dev, const uint32_t n_req, unsigned long long *work_counter,
-                  const JobSize *job_sizes) {
+                  const JobSize *job_sizes, const uint32_t jpr, const FastDiv div_jpr) {
     const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
     extern __shared__ __align__(128) uint8_t gather_smem[];
     uint64_t *s_wsum = reinterpret_cast<uint64_t *>(gather_smem + (size_t)kCopyWarps * kPipeSmemPerWarp);
@@ -420,13 +469,13 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
     // bits hold the padding behind the job.  With this and the rows served per request in
     // shared memory, a chunk's warp needs neither the result block nor the last cu entry.
     uint64_t *job_end = s_wsum + kCopyWarps;
-    uint32_t *req_rows = reinterpret_cast<uint32_t *>(job_end + n_req * dv.ncol);    // [n_req]
+    uint32_t *req_rows = reinterpret_cast<uint32_t *>(job_end + n_req * jpr);        // [n_req]
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     WarpPipe pipe;
     pipe.init(gather_smem + (size_t)warp * kPipeSmemPerWarp, lane, dv.spin_limit);
     griddep_wait();                                    // indices, cu_seqlens and result blocks are complete
-    const uint32_t ncol = dv.ncol;
-    const uint32_t njobs = n_req * ncol;
+    const uint32_t ncol = dv.ncol;                     // jpr = ncol, or ncol + kSeqJobs when a request wants the stream
+    const uint32_t njobs = n_req * jpr;
 
     // job table: sizes first (strided over the threads, so the dependent loads behind each
     // size - request, result block - are all in flight together), then one block scan in which
@@ -441,12 +490,12 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
                 if (job_sizes) {
                     js = job_sizes[j];                         // written by the finalize kernel
                 } else {
-                    const uint32_t q = fast_div(j, dv.div_ncol);
-                    js = job_size(dv, reqs[q], j - q * ncol);
+                    const uint32_t q = fast_div(j, div_jpr);
+                    js = job_size(dv, reqs[q], j - q * jpr);
                 }
                 job_end[j] = js.bytes + (uint64_t)js.cost_rows * kRowCost;
-                const uint32_t q = fast_div(j, dv.div_ncol);
-                if (j == q * ncol) req_rows[q] = js.rows;
+                const uint32_t q = fast_div(j, div_jpr);
+                if (j == q * jpr) req_rows[q] = js.rows;
             }
         }
         __syncthreads();
@@ -492,17 +541,31 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
             const uint64_t b0 = g0 - start;
             g0 = min(g1, end);
             if (end == start) continue;               // empty job
-            const uint32_t q = fast_div(j, dv.div_ncol);
-            const uint32_t k = j - q * ncol;
+            const uint32_t q = fast_div(j, div_jpr);
+            uint32_t k = j - q * jpr;
             const GetReq &rq = reqs[q];
             const td_get_out &out = rq.out;
-            const uint32_t cls = dv.col_cls[k], esz = dv.col_esz[k];
             const uint32_t n_s = req_rows[q];
             const uint64_t job_exact = end - start - (job_end[j] & 15u);
-            uint8_t *dst0 = reinterpret_cast<uint8_t *>(out.col[k]);
+            const uint64_t b1_raw = g0 - start;          // end of this warp's part of the job, padded space
+            uint8_t *dst0;
+            const int32_t *seq_cu = nullptr;             // set for the two halves of the fused stream
+            bool seq_tail = false;
+            if (k >= ncol) {
+                const uint32_t v = k - ncol;
+                if (v == 2) {
+                    warp_fill_seq_advantages(out, n_s, b0, min(b1_raw, job_exact), lane);
+                    continue;
+                }
+                k = v == 0 ? out.seq_prompt_col : out.seq_response_col;
+                seq_cu = out.cu_seq; seq_tail = v == 1;
+                dst0 = reinterpret_cast<uint8_t *>(out.seq);
+            } else {
+                dst0 = reinterpret_cast<uint8_t *>(out.col[k]);
+            }
+            const uint32_t cls = dv.col_cls[k], esz = dv.col_esz[k];
             uint8_t *base = dv.colbase[k];
             const int32_t *indices = out.indices;
-            const uint64_t b1_raw = g0 - start;          // end of this warp's part of the job, padded space
 
             if (cls == TD_SCALAR) {
                 const uint64_t e0 = b0 / esz, e1 = min(b1_raw / esz, (uint64_t)n_s);
@@ -521,12 +584,13 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
                 const long long off = offt[s];
                 return off >= 0 ? base + ((uint64_t)shard_of(dv, s) * cap + (uint64_t)off) * esz : nullptr;
             };
-            if (out.mode == TD_PACKED) {
+            if (out.mode == TD_PACKED || seq_cu) {
                 const int32_t *cu = cls == TD_PROMPT ? out.cu_prompt : out.cu_response;
                 const uint64_t b1 = min(b1_raw, job_exact);
                 if (b1 <= b0) continue;
                 warp_copy_chunk<true>(cu, n_s, b0, b1, dst0, esz, lane, src_lo, src_hi, pipe, indices,
-                                      [&](uint32_t i, int64_t, int64_t) -> uint8_t * { return row_src(i); });
+                                      [&](uint32_t i, int64_t, int64_t) -> uint8_t * { return row_src(i); },
+                                      seq_cu, seq_tail);
             } else {
                 // fixed-width rows: payload part, then the pad pattern up to the row's end
                 const uint32_t W = cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to;

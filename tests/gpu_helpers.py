@@ -62,18 +62,21 @@ class GpuDock:
         return p, r
 
     def buffers(self, consumer: int, max_samples: int, mode: int = td.PACKED, pad_p: int = 0,
-                pad_r: int = 0, capacities=None, want=None, key=None) -> td.GetBuffers:
+                pad_r: int = 0, capacities=None, want=None, key=None, seq=None, seq_adv=False,
+                seq_cap=None) -> td.GetBuffers:
         k = (consumer, max_samples, mode, pad_p, pad_r, key,
-             tuple(sorted(capacities.items())) if capacities else None, tuple(want) if want else None)
+             tuple(sorted(capacities.items())) if capacities else None, tuple(want) if want else None,
+             seq, seq_adv, seq_cap)
         if k not in self._bufs:
             pc, rc = self.token_caps(max_samples)
             self._bufs[k] = td.GetBuffers(self.dock, consumer, max_samples, mode, pad_p, pad_r,
-                                          capacities, want, pc, rc)
+                                          capacities, want, pc, rc, seq, seq_adv, seq_cap)
         return self._bufs[k]
 
     def get(self, consumer: int, max_samples: int, mode: int = td.PACKED, pad_p: int = 0, pad_r: int = 0,
-            capacities=None, want=None, stream=None, key=None) -> ora.Batch:
-        bufs = self.buffers(consumer, max_samples, mode, pad_p, pad_r, capacities, want, key)
+            capacities=None, want=None, stream=None, key=None, seq=None, seq_adv=False,
+            seq_cap=None) -> ora.Batch:
+        bufs = self.buffers(consumer, max_samples, mode, pad_p, pad_r, capacities, want, key, seq, seq_adv, seq_cap)
         self.dock.get(bufs, stream)
         return self.read(bufs, stream)
 
@@ -103,6 +106,11 @@ class GpuDock:
                 b.columns[c] = to_host(t[:tot])
         if bufs.advantages is not None:
             b.advantages = to_host(bufs.advantages[:k])
+        tot = int(b.prompt_tokens + b.response_tokens)
+        if bufs.seq is not None:
+            b.seq = to_host(bufs.seq[:tot])
+        if bufs.seq_advantages is not None:
+            b.seq_advantages = to_host(bufs.seq_advantages[:tot])
         return b
 
     # -- state ------------------------------------------------------------
@@ -129,6 +137,18 @@ def assert_batch_equal(got: ora.Batch, want: ora.Batch, ctx=""):
                            rtol=REL_TOL, atol=ABS_TOL), ctx
         # a zero-variance group must come out as exact zeros on both sides
         assert np.array_equal(got.advantages == 0.0, want.advantages == 0.0), ctx
+    assert (got.seq is None) == (want.seq is None) and (got.seq_advantages is None) == (want.seq_advantages is None), ctx
+    if want.seq is not None:
+        assert H.bits_equal(got.seq, want.seq), f"{ctx} fused stream"
+    if want.seq_advantages is not None:
+        assert np.allclose(got.seq_advantages.astype(np.float64), want.seq_advantages.astype(np.float64),
+                           rtol=REL_TOL, atol=ABS_TOL), f"{ctx} stream advantages"
+        # bit for bit the batch's own advantages over the response tokens, zero bits over the prompt
+        lp = np.diff(got.cu_prompt).astype(np.int64)
+        lr = np.diff(got.cu_response).astype(np.int64)
+        mine = np.repeat(np.stack([np.zeros_like(got.advantages), got.advantages], axis=1).reshape(-1),
+                         np.stack([lp, lr], axis=1).reshape(-1))
+        assert H.bits_equal(got.seq_advantages, mine.astype(np.float32)), f"{ctx} stream advantages layout"
 
 
 def _same(got: np.ndarray, want: np.ndarray, what: str):
@@ -180,8 +200,15 @@ def assert_stats_equal(g: GpuDock, o: ora.OracleDock, ctx=""):
         assert gs.got_tokens[c] == os_.got_tokens[c], f"{ctx} got_tokens[{c}]"
 
 
+def stream_args(w: wl.Workload, consumer: int) -> dict:
+    """Keyword arguments that ask for the fused id stream (and, for a consumer with advantages,
+    its advantage twin) on either side."""
+    return dict(seq=(w.column_index("prompt_ids"), w.column_index("response_ids")),
+                seq_adv=w.consumers[consumer].advantage)
+
+
 def replay_both(w: wl.Workload, mode: int = td.PACKED, check_state_every: int = 0,
-                max_get_checks: Optional[int] = None, arenas: bool = True):
+                max_get_checks: Optional[int] = None, arenas: bool = True, fused: bool = False):
     """Runs w.ops on the oracle and on the GPU in lock step, comparing every get; returns
     (gpu dock, oracle dock, batches)."""
     o = H.make_oracle(w)
@@ -212,8 +239,9 @@ def replay_both(w: wl.Workload, mode: int = td.PACKED, check_state_every: int = 
         else:
             if max_get_checks is not None and n_get >= max_get_checks:
                 continue
-            want = o.get(op.consumer, op.max_samples, mode, pad_p, pad_r)
-            got = g.get(op.consumer, op.max_samples, mode, pad_p, pad_r)
+            kw = stream_args(w, op.consumer) if fused else {}
+            want = o.get(op.consumer, op.max_samples, mode, pad_p, pad_r, **kw)
+            got = g.get(op.consumer, op.max_samples, mode, pad_p, pad_r, **kw)
             assert_batch_equal(got, want, f"op {j} consumer {op.consumer}")
             batches.append((op.consumer, want))
             n_get += 1

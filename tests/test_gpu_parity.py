@@ -176,7 +176,7 @@ def test_many_tiles_look_back(G):
 
 
 # ------------------------------------------------------------------- batched calls
-def _many_vs_serial(G, w, mode=td.PACKED):
+def _many_vs_serial(G, w, mode=td.PACKED, fused=False):
     """All columns in one td_put_many, all gets of the schedule in one td_get_many; the oracle
     runs the same calls one by one."""
     o = H.make_oracle(w)
@@ -193,11 +193,13 @@ def _many_vs_serial(G, w, mode=td.PACKED):
     g.dock.put_many(items)
     G.assert_state_equal(g, o, ctx="after put_many")
     gets = [op for op in w.ops if op.kind == "get"]
-    bufs = [g.buffers(op.consumer, op.max_samples, mode, pad_p, pad_r, key=j) for j, op in enumerate(gets)]
+    # fused: the actor update's requests ask for the token stream, the other consumers' do not
+    kws = [G.stream_args(w, op.consumer) if fused and w.consumers[op.consumer].advantage else {} for op in gets]
+    bufs = [g.buffers(op.consumer, op.max_samples, mode, pad_p, pad_r, key=j, **kws[j]) for j, op in enumerate(gets)]
     plan = g.dock.plan(bufs)
     g.dock.get_many(plan)
     for j, op in enumerate(gets):
-        want = o.get(op.consumer, op.max_samples, mode, pad_p, pad_r)
+        want = o.get(op.consumer, op.max_samples, mode, pad_p, pad_r, **kws[j])
         G.assert_batch_equal(g.read(bufs[j]), want, f"request {j}")
     G.assert_state_equal(g, o, ctx="after get_many")
     G.assert_stats_equal(g, o, "many")
@@ -217,6 +219,61 @@ def test_put_many_get_many_small(G):
 @pytest.mark.parametrize("cid", [2, 3, 5])
 def test_put_many_get_many_full_size(G, cid):
     _many_vs_serial(G, wl.make_config(cid))
+
+
+# ------------------------------------------------------------------- fused token stream
+def test_fused_stream_every_alignment(G):
+    """prompt row followed by response row at cu_seq, for every consumer, lengths 0..70 in every
+    order (zero-length prompts and responses included), packed and padded columns beside it."""
+    w = wl.make_custom("fuse", 64, 2, 4, prompt_len=(0, 37), response=("uniform", 0, 70), vocab=1 << 20,
+                       micro_batch=6, seed=41, with_entropy=True, schedule="random_order", chunk=(1, 7))
+    G.replay_both(w, fused=True)
+    G.replay_both(w, mode=td.PADDED, fused=True)
+    w2 = wl.make_custom("fuse2", 9, 7, 3, prompt_len=(1, 300), response=("uniform", 0, 5000), vocab=1 << 20,
+                        micro_batch=63, seed=42, schedule="bulk")
+    G.replay_both(w2, fused=True)
+
+
+def test_fused_stream_in_a_plan(G):
+    w = wl.make_custom("fuse3", 24, 3, 4, prompt_len=(1, 70), response=("uniform", 0, 200), vocab=50000,
+                       micro_batch=9, seed=43, with_entropy=True, schedule="bulk")
+    _many_vs_serial(G, w, fused=True)
+    _many_vs_serial(G, w, mode=td.PADDED, fused=True)
+
+
+@pytest.mark.parametrize("cid", [2, 3])
+def test_fused_stream_full_size(G, cid):
+    _many_vs_serial(G, wl.make_config(cid), fused=True)
+
+
+def test_fused_stream_of_a_float_pair_and_truncation(G):
+    """Any prompt/response pair of one element size can be fused; a stream buffer that is too
+    small ends the batch before the first group that does not fit and leaves it available."""
+    w = wl.make_custom("fuse4", 8, 2, 2, prompt_len=(3, 30), response=("uniform", 1, 60), vocab=500,
+                       micro_batch=16, seed=44, schedule="none")
+    o = H.make_oracle(w)
+    g = G.GpuDock(w)
+    idx = np.arange(w.n, dtype=np.int32)
+    for c in range(len(w.columns)):
+        cu, data = w.pack(c, idx)
+        o.put(c, idx, cu, data); g.put(c, idx, cu, data)
+    upd = len(w.consumers) - 1
+    pair = (w.column_index("prompt_ids"), w.column_index("old_logprob"))
+    room = int((w.len_prompt + w.len_response)[:6].sum()) + 5          # three groups and a bit
+    want = o.get(upd, 16, seq=pair, seq_adv=True, seq_cap=room)
+    got = g.get(upd, 16, seq=pair, seq_adv=True, seq_cap=room)
+    assert want.n_groups == 3 and want.status & td.ERR_OUT_TRUNCATED
+    G.assert_batch_equal(got, want, "truncated stream")
+    G.assert_batch_equal(g.get(upd, 16, seq=pair, seq_adv=True, key="rest"),
+                         o.get(upd, 16, seq=pair, seq_adv=True), "the rest")
+    G.assert_state_equal(g, o, ctx="fuse4")
+    # host-side refusals: classes swapped, element sizes differ, advantage twin without advantages
+    bad = g.buffers(0, 16, seq=(pair[1], pair[0]), key="bad")
+    with pytest.raises(td.TdError):
+        g.dock.get(bad)
+    bad2 = g.buffers(0, 16, seq_adv=True, key="bad2")
+    with pytest.raises(td.TdError):
+        g.dock.get(bad2)
 
 
 def test_get_many_partial_readiness_and_reuse(G):
