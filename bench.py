@@ -45,6 +45,13 @@ def parse_args():
                     help="many: one td_put_many and one td_get_many per step; single: one td_put per "
                          "column and one td_get per micro-batch")
     ap.add_argument("--cpu-seconds", type=float, default=10.0, help="CPU-oracle time budget")
+    ap.add_argument("--fused", action="store_true",
+                    help="the actor update's gets also ask for the fused prompt+response id stream and "
+                         "its per-token advantage twin")
+    ap.add_argument("--scenario", default="dispatch", choices=["dispatch", "cascade"],
+                    help="dispatch: put everything, then drain (the headline); cascade: generation puts in "
+                         "chunks, inference states get a micro-batch and send their column back for it "
+                         "(td_put_back, no host round trip), the actor update takes what is complete")
     return ap.parse_args()
 
 
@@ -227,7 +234,7 @@ def algorithmic_bytes(w):
 class GpuStep:
     """Device-resident inputs and per-get output buffers of one step, and the step itself."""
 
-    def __init__(self, w, device_index: int, api: str = "many"):
+    def __init__(self, w, device_index: int, api: str = "many", fused: bool = False):
         import torch
         self.api = api
         from paper_2507_19017_b200 import binding as td
@@ -259,9 +266,12 @@ class GpuStep:
             if op.kind != "get":
                 continue
             m = op.max_samples
+            stream = fused and w.consumers[op.consumer].advantage
             bufs = td.GetBuffers(self.dock, op.consumer, m, td.PACKED,
                                  prompt_tokens_cap=int(lp[:m].sum(dtype=np.int64)),
-                                 response_tokens_cap=int(lr[:m].sum(dtype=np.int64)))
+                                 response_tokens_cap=int(lr[:m].sum(dtype=np.int64)),
+                                 seq=(w.column_index("prompt_ids"), w.column_index("response_ids")) if stream else None,
+                                 seq_adv=stream)
             self.gets.append(bufs)
         self.plan = self.dock.plan(self.gets) if api == "many" else None
         self.flush_buf = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=self.dev)
@@ -349,6 +359,149 @@ class GpuStep:
         return (time.perf_counter() - t0) / steps, d2h
 
 
+class CascadeStep:
+    """The whole sample flow as one step: the schedule's generation puts, gets and write-backs
+    enqueued in order on one stream with no host synchronisation in between.  Each consumer
+    reuses one set of output buffers (a worker state has used its batch up by the time it asks
+    for the next)."""
+
+    def __init__(self, w, device_index: int):
+        import torch
+        from paper_2507_19017_b200 import binding as td
+        from paper_2507_19017_b200 import workloads as wl
+        self.torch, self.td, self.w = torch, td, w
+        torch.cuda.set_device(device_index)
+        self.dev = torch.device("cuda", device_index)
+        self.dock = td.Dock(w.G, w.N, w.S, w.column_tuples(), w.consumer_tuples(),
+                            w.shard_capacity(wl.PROMPT), w.shard_capacity(wl.RESPONSE),
+                            w.column_index("reward"), 1e-6, device_index)
+
+        def dev(a):
+            t = torch.from_numpy(np.ascontiguousarray(a).view(np.int16) if a.dtype == np.uint16 else np.ascontiguousarray(a))
+            return (t.view(torch.bfloat16) if a.dtype == np.uint16 else t).to(self.dev)
+
+        lp = np.sort(w.len_prompt)[::-1]
+        lr = np.sort(w.len_response)[::-1]
+        m = w.micro_batch
+        self.bufs = [td.GetBuffers(self.dock, c, m, td.PACKED, prompt_tokens_cap=int(lp[:m].sum(dtype=np.int64)),
+                                   response_tokens_cap=int(lr[:m].sum(dtype=np.int64)))
+                     for c in range(len(w.consumers))]
+        pool = {c: dev(a) for c, a in w.pool.items()}
+        self.calls = []
+        self.put_bytes = 0
+        for op in w.ops:
+            if op.kind == "put":
+                cu, data = w.pack(op.column, op.indices)
+                self.calls.append(("put", op.column, dev(np.ascontiguousarray(op.indices, np.int32)),
+                                   dev(cu) if cu is not None else None, dev(data)))
+                self.put_bytes += 2 * data.nbytes
+            elif op.kind == "get":
+                self.calls.append(("get", self.bufs[op.consumer]))
+            else:
+                self.calls.append(("back", self.bufs[op.consumer], [(c, pool[c]) for c in op.columns]))
+        self.flush_buf = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=self.dev)
+        # per-consumer totals are accumulated on the device from the result blocks
+        self.served_acc = torch.zeros(2, dtype=torch.int64, device=self.dev)
+
+    def run(self):
+        d = self.dock
+        d.reset()
+        for call in self.calls:
+            if call[0] == "put":
+                d.put(call[1], call[2], call[3], call[4])
+            elif call[0] == "get":
+                d.get(call[1])
+            else:
+                d.put_back(call[1], call[2])
+
+    def timed_step(self):
+        torch = self.torch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        self.flush_buf.zero_()
+        e0.record(); self.run(); e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
+
+    def served(self):
+        st = self.dock.status()
+        n_c = len(self.w.consumers)
+        return sum(st.got_samples[c] for c in range(n_c)), sum(st.got_tokens[c] for c in range(n_c))
+
+    def written_back(self):
+        st = self.dock.status()
+        return {self.w.columns[c].name: int(st.put_accepted[c]) for c in self.w.pool}
+
+
+def run_cascade(args, w, local_rank, world, dist, config):
+    """Times the cascade scenario and prints its JSON line (rank 0)."""
+    import torch
+    step = CascadeStep(w, local_rank)
+    peak, peak_kind = load_peaks()
+    sampler = make_sampler(torch, local_rank)
+    sampler.start()
+    for _ in range(max(args.warmup, 3)):
+        step.timed_step()
+    served_s, served_t = step.served()
+    n_dispatch = w.n * len(w.consumers)
+    assert served_s == n_dispatch, f"cascade served {served_s} of {n_dispatch} samples"
+    back = step.written_back()
+    assert all(v == w.n for v in back.values()), back
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    t_begin = time.time()
+    torch.cuda.cudart().cudaProfilerStart()
+    launches0 = step.dock.launch_count()
+    ms = [step.timed_step() for _ in range(args.steps)]
+    if dist is not None:
+        dist.barrier()
+    torch.cuda.synchronize()
+    torch.cuda.cudart().cudaProfilerStop()
+    t_end = time.time()
+    launches = step.dock.launch_count() - launches0
+    clocks = sampler.stop(t_begin, t_end)
+    ms_per_step, = max_over_ranks(dist, [sum(ms) / len(ms)], step.dev)
+    # algorithmic bytes: every stored row read and written once, every served row read and written once
+    _put, _ragged, get_bytes = algorithmic_bytes(w)
+    put_bytes = sum(2 * w.data[s.name].nbytes for s in w.columns)
+    step.dock.kernel_timing(True)
+    ksteps = min(args.steps, 3)
+    for _ in range(ksteps):
+        step.timed_step()
+    n_sc, ms_sc = step.dock.kernel_timing_read(0)
+    n_ga, ms_ga = step.dock.kernel_timing_read(1)
+    step.dock.kernel_timing(False)
+    ragged_put = sum(2 * w.data[s.name].nbytes for s in w.columns if s.cls != "scalar")
+    kern = {"put_scatter": {"launches_per_step": n_sc // ksteps, "avg_ms": ms_sc / max(n_sc, 1),
+                            "bytes_per_launch": ragged_put / max(n_sc // ksteps, 1)},
+            "get_gather": {"launches_per_step": n_ga // ksteps, "avg_ms": ms_ga / max(n_ga, 1),
+                           "bytes_per_launch": get_bytes / max(n_ga // ksteps, 1)}}
+    for k in kern.values():
+        k["GBps"] = k["bytes_per_launch"] / (k["avg_ms"] * 1e-3) / 1e9 if k["avg_ms"] > 0 else 0.0
+    dom = "get_gather" if ms_ga >= ms_sc else "put_scatter"
+    if int(os.environ.get("RANK", "0")) != 0:
+        return
+    calls = {k: sum(1 for c in step.calls if c[0] == k) for k in ("put", "get", "back")}
+    line = {
+        "metric": METRIC, "value": whole_job_rate(world, n_dispatch, ms_per_step * 1e-3), "unit": "samples/s",
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
+        "config": dict(config, scenario="cascade", calls_per_step=calls,
+                       api="td_put per generation chunk, td_get + td_put_back per micro-batch, one stream, no host sync",
+                       l2="flushed before each step (256 MiB write)"),
+        "tokens_per_s": world * served_t / (ms_per_step * 1e-3),
+        "step_GBps": (put_bytes + get_bytes) / (ms_per_step * 1e-3) / 1e9,
+        "kernels": kern,
+        "roofline": {"bound": "hbm", "kernel": dom, "achieved": kern[dom]["GBps"], "peak": peak, "unit": "GB/s",
+                     "frac": kern[dom]["GBps"] / peak, "traffic": None, "peak_kind": peak_kind,
+                     "bytes_per_launch": kern[dom]["bytes_per_launch"], "avg_launch_ms": kern[dom]["avg_ms"],
+                     "note": "average over many small launches: this scenario is bound by launch latency"},
+        "cpu_baseline": None, "e2e": None,
+        "gpu_launches": launches, "gpu_launches_per_step": launches // args.steps, "clocks": clocks,
+    }
+    print(json.dumps(line))
+
+
 # --------------------------------------------------------------------------- CPU oracle
 def time_oracle(w, budget_s: float):
     """The oracle as it stands, one thread, whole steps of the same workload until the time
@@ -397,7 +550,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
 
     from paper_2507_19017_b200 import workloads as wl
-    schedule = "bulk"
+    schedule = "bulk" if args.scenario == "dispatch" else "cascade"
     w = wl.make_config(args.config, seed=wl.BASE_SEED + args.config + 1000 * rank, schedule=schedule)
     config = {"workload": f"configs[{args.config - 1}] {w.name}", "G": w.G, "N": w.N, "S": w.S,
               "samples": w.n, "tokens": w.tokens_total(), "micro_batch": w.micro_batch,
@@ -435,11 +588,21 @@ def main():
         torch.cuda.set_device(local_rank)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
-    step = GpuStep(w, local_rank, args.api)
+    if args.scenario == "cascade":
+        run_cascade(args, w, local_rank, world, dist, config)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
+
+    step = GpuStep(w, local_rank, args.api, args.fused)
+    if args.fused:
+        config["fused_stream"] = "actor-update gets also write the prompt+response id stream and its advantage twin"
     config["api"] = ("td_put_many + td_get_many (one call each per step)" if args.api == "many"
                      else "td_put per column + td_get per micro-batch")
     peak, peak_kind = load_peaks()
     put_bytes, put_ragged_bytes, get_bytes = algorithmic_bytes(w)
+    if args.fused:       # the stream: both id columns read and written once more; the twin: one float written per token
+        get_bytes += 2 * (w.data["prompt_ids"].nbytes + w.data["response_ids"].nbytes) + 4 * w.tokens_total()
 
     sampler = make_sampler(torch, local_rank)
     sampler.start()

@@ -1,6 +1,7 @@
 // Host side of the C ABI declared in include/td.h: argument checks, workspace carving and
 // kernel launches.  No device memory is allocated here and nothing synchronises except
 // td_create (once) and td_status.
+#include <algorithm>
 #include <atomic>
 #include <cstdio>
 #include <cstring>
@@ -141,6 +142,17 @@ cudaError_t launch_timed(td_dock *d, int which, void (*kernel)(KArgs...), dim3 g
     std::lock_guard<std::mutex> lk(d->timing_mu);
     d->timing_ev[which].emplace_back(e0, e1);
     return rc;
+}
+
+// Finalize of a launch whose largest request may serve up to max_samples samples: one CTA per
+// request, a large block when a request is large (its scans then take a quarter of the rounds).
+template <typename... Args>
+cudaError_t launch_finalize(td_dock *d, uint32_t n_req, uint32_t max_samples, cudaStream_t st, Args &&...args) {
+    if (max_samples > kFinBigSamples)
+        return launch_dep(d, get_finalize_kernel<kFinThreadsBig>, dim3(n_req), dim3(kFinThreadsBig), 0, st,
+                          std::forward<Args>(args)...);
+    return launch_dep(d, get_finalize_kernel<kFinThreads>, dim3(n_req), dim3(kFinThreads), 0, st,
+                      std::forward<Args>(args)...);
 }
 
 void drop_timing(td_dock *d) {
@@ -457,7 +469,7 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
-    if (launch_dep(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
+    if (launch_finalize(d, 1u, one.req.max_groups * v.N, st, v, one, (const GetReq *)nullptr,
                (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr) != cudaSuccess) return TD_ECUDA;
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
     if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, jpr), st, v, one,
@@ -535,7 +547,7 @@ int td_get_static(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
-    if (launch_dep(d, get_finalize_kernel, dim3(1), dim3(kFinThreads), 0, st, v, one, (const GetReq *)nullptr,
+    if (launch_finalize(d, 1u, one.req.max_groups * v.N, st, v, one, (const GetReq *)nullptr,
                (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr) != cudaSuccess) return TD_ECUDA;
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
     if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, jpr), st, v, one,
@@ -551,6 +563,7 @@ struct td_plan {
     ConsumerSlot *d_slots;
     uint64_t room_bytes;
     uint32_t jobs_per_req;                // columns, plus the stream's jobs when a request wants it
+    uint32_t max_req_samples;             // the largest request, in samples
     unsigned long long *d_counter;        // the gather's chunk counter: word 1 of slot 0's scan scratch
     JobSize *d_job_sizes;                 // [n_req][n_columns] output bytes and rows, written by the finalize kernel
     std::vector<uint8_t> host_image;      // what was uploaded; kept until the plan dies
@@ -614,6 +627,7 @@ int td_plan_create(td_dock *d, const td_get_req *reqs, uint32_t n_req, void *d_p
         cs.max_groups = sum > v.G ? v.G : (uint32_t)sum;
         if (hr[q].rank_base > v.G) hr[q].rank_base = v.G;
         room += room_bytes_of(v, c, reqs[q].max_samples, reqs[q].out);
+        p->max_req_samples = std::max(p->max_req_samples, std::min(m, v.G) * v.N);
     }
     p->n_slots = n_slots;
     p->d_counter = reinterpret_cast<unsigned long long *>(base + off_scratch) + 1;
@@ -643,7 +657,7 @@ int td_get_many(td_dock *d, td_plan *p, void *stream) {
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
     if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), p->n_slots), dim3(kSelThreads), 0, st, v, none,
                (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
-    if (launch_dep(d, get_finalize_kernel, dim3(p->n_req), dim3(kFinThreads), 0, st, v, none, (const GetReq *)p->d_reqs,
+    if (launch_finalize(d, p->n_req, p->max_req_samples, st, v, none, (const GetReq *)p->d_reqs,
                (const ConsumerSlot *)p->d_slots, seq, p->d_counter, p->d_job_sizes, p->jobs_per_req) != cudaSuccess) return TD_ECUDA;
     if (launch_timed(d, 1, get_gather_kernel, dim3(copy_grid(d, p->room_bytes)), dim3(kCopyThreads),
                      gather_smem_bytes(p->n_req, p->jobs_per_req), st, v, none,

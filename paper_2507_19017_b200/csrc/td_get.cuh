@@ -9,7 +9,9 @@ namespace td {
 
 constexpr int kSelThreads = 256;            // one thread per group; a tile is 256 groups
 constexpr int kSelWarps = kSelThreads / 32;
-constexpr int kFinThreads = 256;
+constexpr int kFinThreads = 256;            // finalize: threads per request; kFinThreadsBig when a request is large
+constexpr int kFinThreadsBig = 1024;
+constexpr uint32_t kFinBigSamples = 1024;   // a request that may serve more samples than this gets the large block
 constexpr int kMaxJobs = 4096;              // (request, column) pairs one gather launch serves
 // A request that wants the fused token stream has three more jobs behind its columns: the
 // stream's prompt half, its response half, and the advantage twin.
@@ -198,6 +200,7 @@ get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
 // would not fit a supplied buffer (handing the cut groups back), sets the consumed bits,
 // computes the group-normalised advantages and writes the result block.
 // ---------------------------------------------------------------------------------------------
+template <int kThreads>
 __device__ __forceinline__ uint64_t block_scan_incl_2(uint64_t a, uint64_t b, uint64_t &out_b,
                                                       uint64_t *sh_a, uint64_t *sh_b,
                                                       uint64_t &tot_a, uint64_t &tot_b) {
@@ -213,7 +216,7 @@ __device__ __forceinline__ uint64_t block_scan_incl_2(uint64_t a, uint64_t b, ui
     __syncthreads();
     uint64_t oa = 0, ob = 0; tot_a = 0; tot_b = 0;
     #pragma unroll
-    for (int w = 0; w < kFinThreads / 32; ++w) {
+    for (int w = 0; w < kThreads / 32; ++w) {
         if (w < (int)warp) { oa += sh_a[w]; ob += sh_b[w]; }
         tot_a += sh_a[w]; tot_b += sh_b[w];
     }
@@ -245,6 +248,12 @@ struct JobSize {
     uint32_t cost_rows;   // rows that are charged kRowCost in the chunked space: those of a packed ragged column
 };
 
+// An element of a scalar column costs a warp two dependent loads and a store, far more than its
+// four bytes say: in the space the gather cuts into chunks it takes kScalarCost bytes, so that a
+// chunk never holds more than a few hundred of them.
+constexpr uint32_t kScalarCost = 64;
+static_assert(kScalarCost % 16 == 0, "a job's extent stays a multiple of 16");
+
 // Extent of a job in the space the gather cuts into chunks (see kRowCost).
 __device__ __forceinline__ uint32_t job_cost_rows(const DockView &dv, const GetReq &rq, uint32_t k,
                                                   uint64_t bytes, uint32_t n_s) {
@@ -252,7 +261,8 @@ __device__ __forceinline__ uint32_t job_cost_rows(const DockView &dv, const GetR
     return (bytes != 0 && dv.col_cls[k] != TD_SCALAR && rq.out.mode == TD_PACKED) ? n_s : 0u;
 }
 
-__global__ void __launch_bounds__(kFinThreads)
+template <int kThreads>
+__global__ void __launch_bounds__(kThreads)
 get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
                     const GetReq *reqs_dev, const ConsumerSlot *slots_dev, const uint32_t seq,
                     unsigned long long *work_counter, JobSize *job_sizes, const uint32_t jobs_per_req) {
@@ -264,7 +274,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     const SelScratch sc = sel_scratch(cs.scratch, dv.G);
     const uint32_t c = rq.consumer, N = dv.N;
     const uint32_t tid = threadIdx.x;
-    __shared__ uint64_t sh_a[kFinThreads / 32], sh_b[kFinThreads / 32];
+    __shared__ uint64_t sh_a[kThreads / 32], sh_b[kThreads / 32];
     __shared__ uint32_t s_first_over;
     griddep_launch_dependents();
     griddep_wait();                                    // the scan's candidate list is complete
@@ -282,12 +292,12 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
 
     // pass A: groups won, in order -> indices
     uint32_t n_grp = 0;
-    for (uint32_t base = 0; base < ncand; base += kFinThreads) {
+    for (uint32_t base = 0; base < ncand; base += kThreads) {
         const uint32_t r = base + tid;
         int32_t g = -1;
         if (r < ncand) g = sc.cand[lo + r];
         uint64_t dummy_b, ta, tb;
-        const uint64_t inc = block_scan_incl_2(g >= 0 ? 1u : 0u, 0, dummy_b, sh_a, sh_b, ta, tb);
+        const uint64_t inc = block_scan_incl_2<kThreads>(g >= 0 ? 1u : 0u, 0, dummy_b, sh_a, sh_b, ta, tb);
         if (g >= 0) {
             const uint32_t p = n_grp + (uint32_t)inc - 1u;
             for (uint32_t j = 0; j < N; ++j) out.indices[(size_t)p * N + j] = g * (int32_t)N + (int32_t)j;
@@ -327,7 +337,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
             want_r |= dv.col_cls[k] == TD_RESPONSE;
         }
     uint64_t carry_p = 0, carry_r = 0;
-    for (uint32_t base = 0; base < n_s; base += kFinThreads) {
+    for (uint32_t base = 0; base < n_s; base += kThreads) {
         const uint32_t i = base + tid;
         uint64_t lp = 0, lr = 0;
         if (i < n_s) {
@@ -336,7 +346,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
             lp = a > 0 ? (uint64_t)a : 0; lr = b > 0 ? (uint64_t)b : 0;
         }
         uint64_t ir, tp, tr;
-        const uint64_t ip = block_scan_incl_2(lp, lr, ir, sh_a, sh_b, tp, tr);
+        const uint64_t ip = block_scan_incl_2<kThreads>(lp, lr, ir, sh_a, sh_b, tp, tr);
         if (i < n_s) {
             const uint64_t cp = carry_p + ip, cr = carry_r + ir;
             out.cu_prompt[i + 1] = (int32_t)cp;
@@ -354,7 +364,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     __syncthreads();
     if (s_first_over != 0xffffffffu) {
         const uint32_t keep = s_first_over / N;
-        for (uint32_t p = keep + tid; p < n_grp; p += kFinThreads) {
+        for (uint32_t p = keep + tid; p < n_grp; p += kThreads) {
             const uint32_t g = (uint32_t)out.indices[(size_t)p * N] / N;
             atomicAnd(&dv.claim[(size_t)c * dv.claim_words + (g >> 5)], ~(1u << (g & 31)));
         }
@@ -364,14 +374,14 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     }
     // consumed bits
     uint32_t *consumed = dv.consumed + (size_t)c * dv.consumed_words;
-    for (uint32_t i = tid; i < n_s; i += kFinThreads) {
+    for (uint32_t i = tid; i < n_s; i += kThreads) {
         const uint32_t s = (uint32_t)out.indices[i];
         atomicOr(&consumed[s >> 5], 1u << (s & 31));
     }
     // group-normalised advantage, one thread per group, in double
     if ((dv.cflags[c] & TD_F_ADVANTAGE) && out.advantages) {
         const float *rew = reinterpret_cast<const float *>(dv.colbase[dv.reward_col]);
-        for (uint32_t p = tid; p < n_grp; p += kFinThreads) {
+        for (uint32_t p = tid; p < n_grp; p += kThreads) {
             const float *r = rew + out.indices[(size_t)p * N];       // a group's samples are consecutive
             double sum = 0.0;
             for (uint32_t j = 0; j < N; ++j) sum += (double)r[j];
@@ -493,9 +503,12 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
                     const uint32_t q = fast_div(j, div_jpr);
                     js = job_size(dv, reqs[q], j - q * jpr);
                 }
-                job_end[j] = js.bytes + (uint64_t)js.cost_rows * kRowCost;
                 const uint32_t q = fast_div(j, div_jpr);
-                if (j == q * jpr) req_rows[q] = js.rows;
+                const uint32_t k = j - q * jpr;
+                const bool scalar = k < ncol && dv.col_cls[k] == TD_SCALAR;
+                job_end[j] = scalar ? (js.bytes ? (uint64_t)js.rows * kScalarCost : 0)
+                                    : js.bytes + (uint64_t)js.cost_rows * kRowCost;
+                if (k == 0) req_rows[q] = js.rows;
             }
         }
         __syncthreads();
@@ -568,11 +581,25 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
             const int32_t *indices = out.indices;
 
             if (cls == TD_SCALAR) {
-                const uint64_t e0 = b0 / esz, e1 = min(b1_raw / esz, (uint64_t)n_s);
-                for (uint64_t e = e0 + lane; e < e1; e += 32) {
-                    const int32_t s = __ldg(indices + e);
-                    if (esz == 4) reinterpret_cast<uint32_t *>(dst0)[e] = reinterpret_cast<const uint32_t *>(base)[s];
-                    else reinterpret_cast<uint16_t *>(dst0)[e] = reinterpret_cast<const uint16_t *>(base)[s];
+                // element e belongs to the chunk that holds byte e * kScalarCost of the job; four
+                // elements per lane are looked up side by side
+                const uint32_t e0 = (uint32_t)((b0 + kScalarCost - 1) / kScalarCost);
+                const uint32_t e1 = (uint32_t)min((b1_raw + kScalarCost - 1) / kScalarCost, (uint64_t)n_s);
+                for (uint32_t e = e0 + lane; e < e1; e += 128) {
+                    int32_t s[4];
+                    uint32_t v[4];
+                    #pragma unroll
+                    for (int u = 0; u < 4; ++u) s[u] = e + 32u * u < e1 ? __ldg(indices + e + 32u * u) : -1;
+                    #pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        v[u] = s[u] < 0 ? 0u : esz == 4 ? reinterpret_cast<const uint32_t *>(base)[s[u]]
+                                                        : (uint32_t)reinterpret_cast<const uint16_t *>(base)[s[u]];
+                    #pragma unroll
+                    for (int u = 0; u < 4; ++u)
+                        if (s[u] >= 0) {
+                            if (esz == 4) reinterpret_cast<uint32_t *>(dst0)[e + 32u * u] = v[u];
+                            else reinterpret_cast<uint16_t *>(dst0)[e + 32u * u] = (uint16_t)v[u];
+                        }
                 }
                 continue;
             }

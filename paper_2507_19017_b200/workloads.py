@@ -368,9 +368,21 @@ CONFIG_NAMES = {
 
 def make_config(config_id: int, seed: Optional[int] = None, sigma: float = SIGMA_HEADLINE,
                 schedule: Optional[str] = None) -> Workload:
-    """The five benchmark shapes.  `schedule` overrides the default call order."""
+    """The five benchmark shapes.  `schedule` overrides the default call order ("cascade":
+    generation chunks of a quarter to four micro-batches, a poll every four puts)."""
     seed = BASE_SEED + config_id if seed is None else seed
     name = CONFIG_NAMES[config_id]
+    if schedule == "cascade":
+        base = make_config(config_id, seed, sigma, "none")
+        spec = {1: ((16, 64), ("uniform", 32, 256), 151936), 2: ((128, 1024), ("lognormal", 1500.0, sigma, 4096), 152064),
+                3: ((256, 2048), ("lognormal", 3000.0, sigma, 16384), 152064),
+                4: ((256, 2048), ("lognormal", 2500.0, sigma, 8192), 151936),
+                5: ((512, 4096), ("lognormal", 6000.0, sigma, 32768), 129280)}[config_id]
+        mb = base.micro_batch
+        return make_custom(name + "-cascade", base.G, base.N, base.S, prompt_len=spec[0], response=spec[1],
+                           vocab=spec[2], micro_batch=mb, seed=seed, with_entropy=config_id == 3,
+                           schedule="cascade", chunk=(max(mb // 4, 1), mb * 4), poll_every=4,
+                           config_id=config_id)
     if config_id == 1:
         return make_custom(name, 16, 4, 2, prompt_len=(16, 64), response=("uniform", 32, 256),
                            vocab=151936, micro_batch=8, seed=seed,

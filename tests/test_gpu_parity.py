@@ -221,6 +221,27 @@ def test_put_many_get_many_full_size(G, cid):
     _many_vs_serial(G, wl.make_config(cid))
 
 
+def test_one_request_for_the_whole_batch(G):
+    """A consumer that asks for everything at once: thousands of rows in one request (the large
+    finalize block, scalar elements spread over many chunks), alone and inside a plan."""
+    w = wl.make_config(2, schedule="none")
+    o = H.make_oracle(w)
+    g = G.GpuDock(w)
+    idx = np.arange(w.n, dtype=np.int32)
+    for c in range(len(w.columns)):
+        cu, data = w.pack(c, idx)
+        o.put(c, idx, cu, data); g.put(c, idx, cu, data)
+    upd = len(w.consumers) - 1
+    kw = G.stream_args(w, upd)
+    G.assert_batch_equal(g.get(upd, w.n, **kw), o.get(upd, w.n, **kw), "whole batch, td_get")
+    bufs = [g.buffers(c, w.n, key="plan") for c in range(upd)]
+    plan = g.dock.plan(bufs)
+    g.dock.get_many(plan)
+    for c in range(upd):
+        G.assert_batch_equal(g.read(bufs[c]), o.get(c, w.n), f"whole batch, plan, consumer {c}")
+    G.assert_state_equal(g, o, ctx="whole batch")
+
+
 # ------------------------------------------------------------------- fused token stream
 def test_fused_stream_every_alignment(G):
     """prompt row followed by response row at cu_seq, for every consumer, lengths 0..70 in every
