@@ -48,6 +48,9 @@ def parse_args():
     ap.add_argument("--fused", action="store_true",
                     help="the actor update's gets also ask for the fused prompt+response id stream and "
                          "its per-token advantage twin")
+    ap.add_argument("--graph", action="store_true",
+                    help="cascade only: capture the step's calls into one CUDA graph once and time its replay "
+                         "(nothing in the step needs the host, batch sizes are read on the device)")
     ap.add_argument("--scenario", default="dispatch", choices=["dispatch", "cascade"],
                     help="dispatch: put everything, then drain (the headline); cascade: generation puts in "
                          "chunks, inference states get a micro-batch and send their column back for it "
@@ -387,6 +390,8 @@ class CascadeStep:
                                    response_tokens_cap=int(lr[:m].sum(dtype=np.int64)))
                      for c in range(len(w.consumers))]
         pool = {c: dev(a) for c, a in w.pool.items()}
+        self.plans = {}
+        self.graph = None
         self.calls = []
         self.put_bytes = 0
         for op in w.ops:
@@ -397,6 +402,13 @@ class CascadeStep:
                 self.put_bytes += 2 * data.nbytes
             elif op.kind == "get":
                 self.calls.append(("get", self.bufs[op.consumer]))
+            elif op.kind == "get_many":
+                key = tuple(op.group)
+                if key not in self.plans:
+                    self.plans[key] = self.dock.plan([self.bufs[c] for c in op.group])
+                self.calls.append(("get_many", self.plans[key]))
+            elif op.kind == "put_back_many":
+                self.calls.append(("back_many", [(self.bufs[c], col, pool[col]) for c, col in op.group]))
             else:
                 self.calls.append(("back", self.bufs[op.consumer], [(c, pool[c]) for c in op.columns]))
         self.flush_buf = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=self.dev)
@@ -411,14 +423,33 @@ class CascadeStep:
                 d.put(call[1], call[2], call[3], call[4])
             elif call[0] == "get":
                 d.get(call[1])
+            elif call[0] == "get_many":
+                d.get_many(call[1])
+            elif call[0] == "back_many":
+                d.put_back_many(call[1])
             else:
                 d.put_back(call[1], call[2])
+
+    def capture(self):
+        """Records the step's calls into a CUDA graph; timed_step then replays it."""
+        torch = self.torch
+        self.run()
+        torch.cuda.synchronize()
+        self.graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(self.graph):
+            self.run()
+        torch.cuda.synchronize()
 
     def timed_step(self):
         torch = self.torch
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         self.flush_buf.zero_()
-        e0.record(); self.run(); e1.record()
+        e0.record()
+        if self.graph is not None:
+            self.graph.replay()
+        else:
+            self.run()
+        e1.record()
         torch.cuda.synchronize()
         return e0.elapsed_time(e1)
 
@@ -436,6 +467,11 @@ def run_cascade(args, w, local_rank, world, dist, config):
     """Times the cascade scenario and prints its JSON line (rank 0)."""
     import torch
     step = CascadeStep(w, local_rank)
+    launches_one_step = None
+    if args.graph:
+        n0 = step.dock.launch_count()
+        step.capture()
+        launches_one_step = (step.dock.launch_count() - n0) // 2      # run once eagerly, once under capture
     peak, peak_kind = load_peaks()
     sampler = make_sampler(torch, local_rank)
     sampler.start()
@@ -459,8 +495,11 @@ def run_cascade(args, w, local_rank, world, dist, config):
     torch.cuda.cudart().cudaProfilerStop()
     t_end = time.time()
     launches = step.dock.launch_count() - launches0
+    if launches_one_step is not None:
+        launches = launches_one_step * args.steps          # replayed from the graph
     clocks = sampler.stop(t_begin, t_end)
     ms_per_step, = max_over_ranks(dist, [sum(ms) / len(ms)], step.dev)
+    graph, step.graph = step.graph, None                    # the per-kernel pass below runs eagerly
     # algorithmic bytes: every stored row read and written once, every served row read and written once
     _put, _ragged, get_bytes = algorithmic_bytes(w)
     put_bytes = sum(2 * w.data[s.name].nbytes for s in w.columns)
@@ -481,13 +520,17 @@ def run_cascade(args, w, local_rank, world, dist, config):
     dom = "get_gather" if ms_ga >= ms_sc else "put_scatter"
     if int(os.environ.get("RANK", "0")) != 0:
         return
-    calls = {k: sum(1 for c in step.calls if c[0] == k) for k in ("put", "get", "back")}
+    calls = {k: sum(1 for c in step.calls if c[0] == k) for k in ("put", "get", "back", "get_many", "back_many")}
+    calls = {k: v for k, v in calls.items() if v}
     line = {
         "metric": METRIC, "value": whole_job_rate(world, n_dispatch, ms_per_step * 1e-3), "unit": "samples/s",
         "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "u8", "data": "synthetic",
         "config": dict(config, scenario="cascade", calls_per_step=calls,
-                       api="td_put per generation chunk, td_get + td_put_back per micro-batch, one stream, no host sync",
+                       launch="one CUDA graph replay per step" if graph is not None else "eager calls",
+                       api=("td_put per generation chunk, one td_get_many + one td_put_back_many per poll of all "
+                            "worker states, one stream, no host sync" if args.api == "many" else
+                            "td_put per generation chunk, td_get + td_put_back per micro-batch, one stream, no host sync"),
                        l2="flushed before each step (256 MiB write)"),
         "tokens_per_s": world * served_t / (ms_per_step * 1e-3),
         "step_GBps": (put_bytes + get_bytes) / (ms_per_step * 1e-3) / 1e9,
@@ -550,7 +593,7 @@ def main():
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
 
     from paper_2507_19017_b200 import workloads as wl
-    schedule = "bulk" if args.scenario == "dispatch" else "cascade"
+    schedule = "bulk" if args.scenario == "dispatch" else ("cascade_batched" if args.api == "many" else "cascade")
     w = wl.make_config(args.config, seed=wl.BASE_SEED + args.config + 1000 * rank, schedule=schedule)
     config = {"workload": f"configs[{args.config - 1}] {w.name}", "G": w.G, "N": w.N, "S": w.S,
               "samples": w.n, "tokens": w.tokens_total(), "micro_batch": w.micro_batch,

@@ -238,6 +238,19 @@ typedef struct {
 int td_put_back(td_dock *dock, const td_get_out *batch, uint32_t max_samples, const td_back_item *items,
                 uint32_t n_items, void *stream);
 
+/* The write-backs of several worker states in one call (three kernel launches for up to eight
+ * of them): request r sends column `column` back for the batch `batch` it names, exactly as
+ * td_put_back(dock, batch, max_samples, {column, d_data, data_elems}, 1, stream) would; the
+ * requests are stored in array order.  Together with td_get_many this serves one poll of every
+ * worker state with six launches, whatever their number. */
+typedef struct {
+    const td_get_out *batch;
+    uint32_t max_samples, column;
+    const void *d_data;
+    uint64_t data_elems;
+} td_back_req;
+int td_put_back_many(td_dock *dock, const td_back_req *reqs, uint32_t n_reqs, void *stream);
+
 /* Many gets served by one call.  Each worker state has its own controller and a step serves
  * several of them, each in several micro-batches; a plan fixes the list of requests (consumer,
  * max_samples, output buffers) once and td_get_many then serves all of them with three kernel

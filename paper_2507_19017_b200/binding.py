@@ -31,7 +31,7 @@ EXPORTS = ["td_query_workspace", "td_create", "td_destroy", "td_put", "td_get",
            "td_launch_count", "td_strerror", "td_kernel_timing", "td_kernel_timing_read",
            "td_put_host_stage_bytes", "td_put_host", "td_get_host", "td_put_many",
            "td_plan_bytes", "td_plan_create", "td_plan_destroy", "td_get_many", "td_get_static",
-           "td_model_bytes", "td_put_back"]
+           "td_model_bytes", "td_put_back", "td_put_back_many"]
 
 
 class TdModel(C.Structure):
@@ -80,6 +80,11 @@ class TdPutItem(C.Structure):
 class TdBackItem(C.Structure):
     _fields_ = [("column", C.c_uint32), ("reserved", C.c_uint32), ("d_data", C.c_void_p),
                 ("data_elems", C.c_uint64)]
+
+
+class TdBackReq(C.Structure):
+    _fields_ = [("batch", C.c_void_p), ("max_samples", C.c_uint32), ("column", C.c_uint32),
+                ("d_data", C.c_void_p), ("data_elems", C.c_uint64)]
 
 
 class TdGetReq(C.Structure):
@@ -155,6 +160,8 @@ def lib():
         L.td_put_many.argtypes = [vp, C.POINTER(TdPutItem), u32, vp]
         L.td_put_back.restype = C.c_int
         L.td_put_back.argtypes = [vp, C.POINTER(TdGetOut), u32, C.POINTER(TdBackItem), u32, vp]
+        L.td_put_back_many.restype = C.c_int
+        L.td_put_back_many.argtypes = [vp, C.POINTER(TdBackReq), u32, vp]
         L.td_plan_bytes.restype = C.c_size_t
         L.td_plan_bytes.argtypes = [vp, u32]
         L.td_plan_create.restype = C.c_int
@@ -409,6 +416,13 @@ class Dock:
             arr[j] = TdBackItem(column, 0, data.data_ptr(), data.numel())
         _check("td_put_back", lib().td_put_back(self.handle, C.byref(bufs.struct), bufs.max_samples,
                                                 arr, len(items), _stream_ptr(stream)))
+
+    def put_back_many(self, reqs: Sequence[Tuple], stream=None):
+        """reqs: (bufs, column, data): column sent back for the batch last served into bufs."""
+        arr = (TdBackReq * len(reqs))()
+        for j, (bufs, column, data) in enumerate(reqs):
+            arr[j] = TdBackReq(C.addressof(bufs.struct), bufs.max_samples, column, data.data_ptr(), data.numel())
+        _check("td_put_back_many", lib().td_put_back_many(self.handle, arr, len(reqs), _stream_ptr(stream)))
 
     def plan(self, bufs: Sequence[GetBuffers], stream=None) -> "Plan":
         return Plan(self, bufs, stream)

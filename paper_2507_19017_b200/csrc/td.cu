@@ -413,22 +413,42 @@ int td_put_many(td_dock *d, const td_put_item *items, uint32_t n_items, void *st
     return put_items(d, args.data(), n_items, (cudaStream_t)stream);
 }
 
+namespace {
+// One write-back as a put item: the samples and row boundaries are the batch's, the count is
+// read from its result block on the device.
+int back_args(const td_dock *d, const td_get_out *batch, uint32_t max_samples, uint32_t column,
+              const void *d_data, uint64_t data_elems, PutArgs *out) {
+    const DockView &v = d->dv;
+    if (!batch || !batch->indices || !batch->cu_prompt || !batch->cu_response || !batch->result) return TD_EINVAL;
+    if (column >= v.ncol || (!d_data && data_elems) || data_elems >= (1ull << 31)) return TD_EINVAL;
+    const uint32_t cls = v.col_cls[column];
+    const int32_t *cu = cls == TD_PROMPT ? batch->cu_prompt : cls == TD_RESPONSE ? batch->cu_response : nullptr;
+    *out = PutArgs{column, max_samples, batch->indices, cu, static_cast<const uint8_t *>(d_data), data_elems,
+                   &batch->result->n_samples};
+    return TD_OK;
+}
+}  // namespace
+
 int td_put_back(td_dock *d, const td_get_out *batch, uint32_t max_samples, const td_back_item *items,
                 uint32_t n_items, void *stream) {
     if (!d || !batch || (n_items && !items)) return TD_EINVAL;
-    if (!batch->indices || !batch->cu_prompt || !batch->cu_response || !batch->result) return TD_EINVAL;
-    if (max_samples == 0 || n_items == 0) return TD_OK;
-    const DockView &v = d->dv;
     std::vector<PutArgs> args(n_items);
     for (uint32_t i = 0; i < n_items; ++i) {
-        const td_back_item &it = items[i];
-        if (it.column >= v.ncol || (!it.d_data && it.data_elems) || it.data_elems >= (1ull << 31)) return TD_EINVAL;
-        const uint32_t cls = v.col_cls[it.column];
-        const int32_t *cu = cls == TD_PROMPT ? batch->cu_prompt : cls == TD_RESPONSE ? batch->cu_response : nullptr;
-        args[i] = PutArgs{it.column, max_samples, batch->indices, cu, static_cast<const uint8_t *>(it.d_data),
-                          it.data_elems, &batch->result->n_samples};
+        const int rc = back_args(d, batch, max_samples, items[i].column, items[i].d_data, items[i].data_elems, &args[i]);
+        if (rc != TD_OK) return rc;
     }
     return put_items(d, args.data(), n_items, (cudaStream_t)stream);
+}
+
+int td_put_back_many(td_dock *d, const td_back_req *reqs, uint32_t n_reqs, void *stream) {
+    if (!d || (n_reqs && !reqs)) return TD_EINVAL;
+    std::vector<PutArgs> args(n_reqs);
+    for (uint32_t i = 0; i < n_reqs; ++i) {
+        const int rc = back_args(d, reqs[i].batch, reqs[i].max_samples, reqs[i].column, reqs[i].d_data,
+                                 reqs[i].data_elems, &args[i]);
+        if (rc != TD_OK) return rc;
+    }
+    return put_items(d, args.data(), n_reqs, (cudaStream_t)stream);
 }
 
 int td_put(td_dock *d, uint32_t column, const int32_t *d_indices, uint32_t k, const int32_t *d_cu,
@@ -473,7 +493,8 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
                (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr) != cudaSuccess) return TD_ECUDA;
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
     if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, jpr), st, v, one,
-                     (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr, jpr, make_fastdiv(jpr)) != cudaSuccess) return TD_ECUDA;
+                     (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr, jpr, make_fastdiv(jpr),
+                     (const ConsumerSlot *)nullptr, 1u) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 
@@ -551,7 +572,8 @@ int td_get_static(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_
                (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr) != cudaSuccess) return TD_ECUDA;
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
     if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, jpr), st, v, one,
-                     (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr, jpr, make_fastdiv(jpr)) != cudaSuccess) return TD_ECUDA;
+                     (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr, jpr, make_fastdiv(jpr),
+                     (const ConsumerSlot *)nullptr, 1u) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 
@@ -662,7 +684,8 @@ int td_get_many(td_dock *d, td_plan *p, void *stream) {
     if (launch_timed(d, 1, get_gather_kernel, dim3(copy_grid(d, p->room_bytes)), dim3(kCopyThreads),
                      gather_smem_bytes(p->n_req, p->jobs_per_req), st, v, none,
                      (const GetReq *)p->d_reqs, p->n_req, p->d_counter, (const JobSize *)p->d_job_sizes,
-                     p->jobs_per_req, make_fastdiv(p->jobs_per_req)) != cudaSuccess) return TD_ECUDA;
+                     p->jobs_per_req, make_fastdiv(p->jobs_per_req), (const ConsumerSlot *)p->d_slots,
+                     p->n_slots) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
 

@@ -471,7 +471,8 @@ __device__ __noinline__ void warp_fill_seq_advantages(const td_get_out &out, uin
 __global__ void __launch_bounds__(kCopyThreads, kCopyBlocksPerSM)
 get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
                   const GetReq *reqs_dev, const uint32_t n_req, unsigned long long *work_counter,
-                  const JobSize *job_sizes, const uint32_t jpr, const FastDiv div_jpr) {
+                  const JobSize *job_sizes, const uint32_t jpr, const FastDiv div_jpr,
+                  const ConsumerSlot *slots_dev, const uint32_t n_slots) {
     const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
     extern __shared__ __align__(128) uint8_t gather_smem[];
     uint64_t *s_wsum = reinterpret_cast<uint64_t *>(gather_smem + (size_t)kCopyWarps * kPipeSmemPerWarp);
@@ -484,6 +485,18 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
     WarpPipe pipe;
     pipe.init(gather_smem + (size_t)warp * kPipeSmemPerWarp, lane, dv.spin_limit);
     griddep_wait();                                    // indices, cu_seqlens and result blocks are complete
+    // The scan and the finalize kernel are done with the scan scratch: leave its ticket and tile
+    // descriptors empty for the next call, so that a call which comes with the same launch
+    // sequence number again (a CUDA graph replayed) does not meet its own earlier descriptors.
+    if (blockIdx.x == 0) {
+        const ConsumerSlot *slots = slots_dev ? slots_dev : &one.cs;
+        const uint32_t tiles = sel_tiles(dv.G);
+        for (uint32_t i = threadIdx.x; i < n_slots * (tiles + 1u); i += kCopyThreads) {
+            const uint32_t sl = i / (tiles + 1u), t = i - sl * (tiles + 1u);
+            const SelScratch sc = sel_scratch(slots[sl].scratch, dv.G);
+            if (t == tiles) *sc.ticket = 0; else sc.desc[t] = 0;
+        }
+    }
     const uint32_t ncol = dv.ncol;                     // jpr = ncol, or ncol + kSeqJobs when a request wants the stream
     const uint32_t njobs = n_req * jpr;
 

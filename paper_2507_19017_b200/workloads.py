@@ -46,12 +46,14 @@ class ConsumerSpec:
 @dataclass
 class Op:
     """One call of a schedule: a put of `column` for `indices`, or a get."""
-    kind: str                         # "put" | "get" | "put_back"
+    kind: str                         # "put" | "get" | "put_back" | "get_many" | "put_back_many"
     column: int = -1                  # put: column number
     indices: Optional[np.ndarray] = None  # put: int32 sample indices, call order
     consumer: int = -1                # get: consumer number
     max_samples: int = 0              # get: micro-batch size
     columns: Optional[List[int]] = None   # put_back: columns `consumer` sends back for the batch it got last
+    group: Optional[List] = None          # get_many: consumers served by one call, in order (one micro-batch each);
+                                          # put_back_many: (consumer, column) pairs sent back by one call, in order
 
 
 @dataclass
@@ -268,10 +270,13 @@ CASCADE_PRODUCES = {"reference": ("ref_logprob",), "reward": ("reward",),
                     "actor_inference": ("old_logprob", "entropy")}
 
 
-def _cascade_ops(w: Workload, rng: np.random.Generator, lo: int, hi: int, poll_every: int) -> List[Op]:
+def _cascade_ops(w: Workload, rng: np.random.Generator, lo: int, hi: int, poll_every: int,
+                 batched: bool = False) -> List[Op]:
     """The whole sample flow on one dock: generation puts prompt and response ids in shuffled
     chunks; every `poll_every` puts each inference state takes a micro-batch and sends its
-    column back for exactly that batch, and the actor update takes what has become complete."""
+    column back for exactly that batch, and the actor update takes what has become complete.
+    batched: a poll is one get call for all worker states together and one write-back call for
+    all of them (the actor update then sees a poll's write-backs at the next poll)."""
     gen = [w.column_index("prompt_ids"), w.column_index("response_ids")]
     names = [c.name for c in w.columns]
     produces = {ci: [w.column_index(nm) for nm in CASCADE_PRODUCES.get(k.name, ()) if nm in names]
@@ -296,6 +301,11 @@ def _cascade_ops(w: Workload, rng: np.random.Generator, lo: int, hi: int, poll_e
     updaters = [ci for ci, cols in produces.items() if not cols]
 
     def poll(ops: List[Op], inference: bool = True):
+        if batched:
+            ops.append(Op("get_many", group=(workers if inference else []) + updaters, max_samples=w.micro_batch))
+            if inference:
+                ops.append(Op("put_back_many", group=[(ci, c) for ci in workers for c in produces[ci]]))
+            return
         if inference:
             for ci in workers:
                 ops.append(Op("get", consumer=ci, max_samples=w.micro_batch))
@@ -346,8 +356,8 @@ def make_custom(name: str, G: int, N: int, S: int, *, prompt_len: Tuple[int, int
         w.ops = _random_order_ops(w, rng, *chunk)
     elif schedule == "interleaved":
         w.ops = _interleaved_ops(w, rng, chunk[0], chunk[1], poll_every)
-    elif schedule == "cascade":
-        w.ops = _cascade_ops(w, rng, chunk[0], chunk[1], poll_every)
+    elif schedule in ("cascade", "cascade_batched"):
+        w.ops = _cascade_ops(w, rng, chunk[0], chunk[1], poll_every, batched=schedule == "cascade_batched")
     elif schedule == "none":
         w.ops = []
     else:
@@ -372,7 +382,7 @@ def make_config(config_id: int, seed: Optional[int] = None, sigma: float = SIGMA
     generation chunks of a quarter to four micro-batches, a poll every four puts)."""
     seed = BASE_SEED + config_id if seed is None else seed
     name = CONFIG_NAMES[config_id]
-    if schedule == "cascade":
+    if schedule in ("cascade", "cascade_batched"):
         base = make_config(config_id, seed, sigma, "none")
         spec = {1: ((16, 64), ("uniform", 32, 256), 151936), 2: ((128, 1024), ("lognormal", 1500.0, sigma, 4096), 152064),
                 3: ((256, 2048), ("lognormal", 3000.0, sigma, 16384), 152064),
@@ -381,7 +391,7 @@ def make_config(config_id: int, seed: Optional[int] = None, sigma: float = SIGMA
         mb = base.micro_batch
         return make_custom(name + "-cascade", base.G, base.N, base.S, prompt_len=spec[0], response=spec[1],
                            vocab=spec[2], micro_batch=mb, seed=seed, with_entropy=config_id == 3,
-                           schedule="cascade", chunk=(max(mb // 4, 1), mb * 4), poll_every=4,
+                           schedule=schedule, chunk=(max(mb // 4, 1), mb * 4), poll_every=4,
                            config_id=config_id)
     if config_id == 1:
         return make_custom(name, 16, 4, 2, prompt_len=(16, 64), response=("uniform", 32, 256),

@@ -217,6 +217,7 @@ def replay_both(w: wl.Workload, mode: int = td.PACKED, check_state_every: int = 
     n_get = 0
     batches = []
     last = {}
+    plans = {}
     pool_dev = {c: to_device(a, g.device) for c, a in w.pool.items()}
     for j, op in enumerate(w.ops):
         if op.kind == "put":
@@ -229,6 +230,26 @@ def replay_both(w: wl.Workload, mode: int = td.PACKED, check_state_every: int = 
             g.dock.put_back(bufs, [(c, pool_dev[c]) for c in op.columns])
             H.oracle_put_back(w, o, want, op.columns)
             assert_batch_equal(g.read(bufs), want, f"op {j} consumer {op.consumer} (after write-back)")
+        elif op.kind == "get_many":
+            bufs = [g.buffers(c, op.max_samples, mode, pad_p, pad_r) for c in op.group]
+            key = tuple(op.group)
+            if key not in plans:
+                plans[key] = g.dock.plan(bufs)
+            g.dock.get_many(plans[key])                      # read back only after the write-backs are enqueued
+            wants = [o.get(c, op.max_samples, mode, pad_p, pad_r) for c in op.group]
+            for c, want, b in zip(op.group, wants, bufs):
+                last[c] = (want, b)
+                batches.append((c, want))
+            nxt = w.ops[j + 1] if j + 1 < len(w.ops) else None
+            if nxt is None or nxt.kind != "put_back_many":
+                for c, want, b in zip(op.group, wants, bufs):
+                    assert_batch_equal(g.read(b), want, f"op {j} consumer {c}")
+        elif op.kind == "put_back_many":
+            g.dock.put_back_many([(last[c][1], col, pool_dev[col]) for c, col in op.group])
+            for c, col in op.group:
+                H.oracle_put_back(w, o, last[c][0], [col])
+            for c, (want, b) in last.items():
+                assert_batch_equal(g.read(b), want, f"op {j} consumer {c} (after write-backs)")
         elif any(k.kind == "put_back" and k.consumer == op.consumer for k in w.ops[j + 1:j + 2]):
             want = o.get(op.consumer, op.max_samples, mode, pad_p, pad_r)
             bufs = g.buffers(op.consumer, op.max_samples, mode, pad_p, pad_r)

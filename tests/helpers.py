@@ -50,6 +50,13 @@ def replay_oracle(w: wl.Workload, dock: ora.OracleDock, mode: int = ora.PACKED) 
             dock.put(op.column, op.indices, cu, data)
         elif op.kind == "put_back":
             oracle_put_back(w, dock, last[op.consumer], op.columns)
+        elif op.kind == "get_many":            # one call: the consumers are served in order
+            for c in op.group:
+                out.append((c, dock.get(c, op.max_samples, mode, w.pad_prompt_to, w.pad_response_to)))
+                last[c] = out[-1][1]
+        elif op.kind == "put_back_many":       # one call: the write-backs are stored in order
+            for c, col in op.group:
+                oracle_put_back(w, dock, last[c], [col])
         else:
             out.append((op.consumer, dock.get(op.consumer, op.max_samples, mode,
                                               w.pad_prompt_to, w.pad_response_to)))

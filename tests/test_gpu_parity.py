@@ -88,6 +88,73 @@ def test_cascade_write_back_small(G):
     assert sum(b.n_samples for c, b in batches if c == upd) == w.n
 
 
+def test_cascade_batched_polls(G):
+    """The same flow with one td_get_many and one td_put_back_many per poll."""
+    w = wl.make_custom("cascade-batched", 24, 4, 3, prompt_len=(5, 70), response=("uniform", 1, 300),
+                       vocab=50000, micro_batch=8, seed=33, schedule="cascade_batched", chunk=(1, 12),
+                       poll_every=3, with_entropy=True)
+    g, o, batches = G.replay_both(w, check_state_every=5)
+    upd = len(w.consumers) - 1
+    assert sum(b.n_samples for c, b in batches if c == upd) == w.n
+    w2 = wl.make_config(2, schedule="cascade_batched")
+    g, o, batches = G.replay_both(w2)
+    assert sum(b.n_samples for c, b in batches if c == upd) == w2.n
+
+
+def test_cascade_replayed_from_a_cuda_graph(G):
+    """Nothing in the flow needs the host (batch sizes are read on the device), so a whole
+    iteration - reset, generation puts, gets, write-backs - can be recorded once and replayed:
+    every get of the replay against the oracle, twice."""
+    import torch
+    w = wl.make_custom("cascade-graph", 16, 4, 2, prompt_len=(5, 70), response=("uniform", 1, 300),
+                       vocab=50000, micro_batch=8, seed=35, schedule="cascade_batched", chunk=(4, 12),
+                       poll_every=2)
+    o = H.make_oracle(w)
+    want = H.replay_oracle(w, o)
+    g = G.GpuDock(w)
+    pool_dev = {c: G.to_device(a, g.device) for c, a in w.pool.items()}
+    calls, bufs_of_get, last = [], [], {}
+    for j, op in enumerate(w.ops):
+        if op.kind == "put":
+            cu, data = w.pack(op.column, op.indices)
+            calls.append(("put", op.column, G.to_device(np.ascontiguousarray(op.indices, np.int32), g.device),
+                          G.to_device(cu, g.device), G.to_device(data, g.device)))
+        elif op.kind == "get_many":
+            bufs = [g.buffers(c, op.max_samples, key=("graph", j)) for c in op.group]      # one set per get
+            calls.append(("get_many", g.dock.plan(bufs)))
+            for c, b in zip(op.group, bufs):
+                last[c] = b
+                bufs_of_get.append((c, b))
+        else:
+            calls.append(("back_many", [(last[c], col, pool_dev[col]) for c, col in op.group]))
+
+    def run():
+        g.dock.reset()
+        for call in calls:
+            if call[0] == "put":
+                g.dock.put(call[1], call[2], call[3], call[4])
+            elif call[0] == "get_many":
+                g.dock.get_many(call[1])
+            else:
+                g.dock.put_back_many(call[1])
+
+    run()                                   # eager once (also the first use of every kernel)
+    torch.cuda.synchronize()
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        run()
+    for rep in range(2):
+        for _c, b in bufs_of_get:           # stale results must not pass for fresh ones
+            b.result.zero_()
+        graph.replay()
+        torch.cuda.synchronize()
+        assert len(bufs_of_get) == len(want)
+        for k, ((c, b), (wc, wb)) in enumerate(zip(bufs_of_get, want)):
+            assert c == wc
+            G.assert_batch_equal(g.read(b), wb, f"replay {rep} get {k} consumer {c}")
+        G.assert_state_equal(g, o, ctx=f"replay {rep}")
+
+
 @pytest.mark.parametrize("cid", [2, 3])
 def test_cascade_write_back_full_size(G, cid):
     base = wl.make_config(cid, schedule="none")
