@@ -328,24 +328,31 @@ class GpuStep:
     # end to end: host buffers in, host buffers out
     def prepare_e2e(self):
         td, torch = self.td, self.torch
-        need = max(self.dock.put_host_stage_bytes(c, i.numel(), d.numel()) for c, i, _cu, d in self.host_puts)
-        self.stage = [torch.empty(need, dtype=torch.uint8, device=self.dev) for _ in range(2)]
+        needs = [self.dock.put_host_stage_bytes(c, i.numel(), d.numel()) for c, i, _cu, d in self.host_puts]
+        if self.api == "many":
+            self.stage = [torch.empty(sum(needs), dtype=torch.uint8, device=self.dev)]
+        else:
+            self.stage = [torch.empty(max(needs), dtype=torch.uint8, device=self.dev) for _ in range(2)]
         self.host_gets = [td.HostGetBuffers(b) for b in self.gets]
+        self.host_put_arr = self.dock.put_items(self.host_puts)       # marshalled once, like a caller would
+        self.host_out_arr = self.dock.host_outs(self.host_gets)
 
     def e2e_step(self):
         torch = self.torch
         self.dock.reset()
+        if self.api == "many":          # one call in, one call out: two synchronisations per step
+            self.dock.put_many_host(self.host_put_arr, self.stage[0])
+            self.dock.get_many_host(self.plan, self.host_out_arr)
+            return None
         for j, (col, idx, cu, data) in enumerate(self.host_puts):
             if j >= 2:
                 self.stage_ev[j % 2].synchronize()      # staging buffer free again
             self.dock.put_host(col, idx, cu, data, self.stage[j % 2])
             self.stage_ev[j % 2].record()
-        d2h = 0
         for bufs, host in zip(self.gets, self.host_gets):
             self.dock.get_host(bufs, host)
-            d2h += host.bytes_valid(self.dock)
         torch.cuda.synchronize()
-        return d2h
+        return None
 
     def run_e2e(self, steps: int, warmup: int):
         torch = self.torch
@@ -355,11 +362,11 @@ class GpuStep:
             self.e2e_step()
         torch.cuda.synchronize()
         t0 = time.perf_counter()
-        d2h = 0
         for _ in range(steps):
-            d2h = self.e2e_step()
+            self.e2e_step()
         torch.cuda.synchronize()
-        return (time.perf_counter() - t0) / steps, d2h
+        el = (time.perf_counter() - t0) / steps
+        return el, sum(h.bytes_valid(self.dock) for h in self.host_gets)      # counted from what the last step copied
 
 
 class CascadeStep:

@@ -315,6 +315,19 @@ int td_put_host(td_dock *dock, uint32_t column, const int32_t *h_indices, uint32
                 void *d_stage, size_t stage_bytes, void *stream);
 int td_get_host(td_dock *dock, uint32_t consumer, uint32_t max_samples, const td_get_out *dev_out,
                 const td_get_out *host_out, void *stream);
+/* The batched calls with host buffers.
+ * td_put_many_host: td_put_many whose items' three pointers (named d_* in td_put_item) are HOST
+ * arrays here; they are copied, item after item, into d_stage (device, 256-byte aligned, at
+ * least the sum of td_put_host_stage_bytes() over the items, not reused until the put has
+ * executed) and put from there with one td_put_many.
+ * td_get_many_host: td_get_many on `plan`, then the valid part of every request's buffers is
+ * copied to the matching HOST pointers of host_outs[r] (one entry per request of the plan, in
+ * plan order; result and indices required, NULL elsewhere = skip).  All result blocks are
+ * fetched behind one synchronisation, all payload behind a second one: two per call however many
+ * requests the plan holds, where td_get_host takes two per request. */
+int td_put_many_host(td_dock *dock, const td_put_item *h_items, uint32_t n_items, void *d_stage,
+                     size_t stage_bytes, void *stream);
+int td_get_many_host(td_dock *dock, td_plan *plan, const td_get_out *host_outs, uint32_t n_req, void *stream);
 
 /* The communication-volume model of "Distributed Transfer Dock Strategy", in bytes, for sizing a
  * dock or a link (host arithmetic only; no device is touched):

@@ -31,7 +31,7 @@ EXPORTS = ["td_query_workspace", "td_create", "td_destroy", "td_put", "td_get",
            "td_launch_count", "td_strerror", "td_kernel_timing", "td_kernel_timing_read",
            "td_put_host_stage_bytes", "td_put_host", "td_get_host", "td_put_many",
            "td_plan_bytes", "td_plan_create", "td_plan_destroy", "td_get_many", "td_get_static",
-           "td_model_bytes", "td_put_back", "td_put_back_many"]
+           "td_model_bytes", "td_put_back", "td_put_back_many", "td_put_many_host", "td_get_many_host"]
 
 
 class TdModel(C.Structure):
@@ -162,6 +162,10 @@ def lib():
         L.td_put_back.argtypes = [vp, C.POINTER(TdGetOut), u32, C.POINTER(TdBackItem), u32, vp]
         L.td_put_back_many.restype = C.c_int
         L.td_put_back_many.argtypes = [vp, C.POINTER(TdBackReq), u32, vp]
+        L.td_put_many_host.restype = C.c_int
+        L.td_put_many_host.argtypes = [vp, C.POINTER(TdPutItem), u32, vp, C.c_size_t, vp]
+        L.td_get_many_host.restype = C.c_int
+        L.td_get_many_host.argtypes = [vp, vp, C.POINTER(TdGetOut), u32, vp]
         L.td_plan_bytes.restype = C.c_size_t
         L.td_plan_bytes.argtypes = [vp, u32]
         L.td_plan_create.restype = C.c_int
@@ -303,7 +307,9 @@ class HostGetBuffers:
         self.advantages = (torch.zeros(bufs.advantages.shape, dtype=torch.float32).pin_memory()
                            if bufs.advantages is not None else None)
         self.cols = {c: torch.zeros(t.shape, dtype=t.dtype).pin_memory() for c, t in bufs.cols.items()}
-        self.result = TdResult()
+        # the result block too lives in pinned memory: a copy into pageable memory stalls the caller
+        self._result_mem = torch.zeros(C.sizeof(TdResult), dtype=torch.uint8).pin_memory()
+        self.result = TdResult.from_address(self._result_mem.data_ptr())
         go = TdGetOut()
         go.mode, go.pad_prompt_to, go.pad_response_to = bufs.mode, bufs.pad_prompt_to, bufs.pad_response_to
         go.indices, go.cu_prompt = self.indices.data_ptr(), self.cu_prompt.data_ptr()
@@ -400,13 +406,11 @@ class Dock:
                                       cu.data_ptr() if cu is not None else None,
                                       data.data_ptr(), data.numel(), _stream_ptr(stream)))
 
-    def put_many(self, items: Sequence[Tuple], stream=None):
-        """items: (column, indices, cu or None, data) device tensors, stored in this order."""
-        arr = (TdPutItem * len(items))()
-        for j, (column, indices, cu, data) in enumerate(items):
-            arr[j] = TdPutItem(column, indices.numel(), indices.data_ptr(),
-                               cu.data_ptr() if cu is not None else None, data.data_ptr(), data.numel())
-        _check("td_put_many", lib().td_put_many(self.handle, arr, len(items), _stream_ptr(stream)))
+    def put_many(self, items, stream=None):
+        """items: (column, indices, cu or None, data) device tensors, stored in this order, or
+        put_items() of them."""
+        arr = items if isinstance(items, C.Array) else self.put_items(items)
+        _check("td_put_many", lib().td_put_many(self.handle, arr, len(arr), _stream_ptr(stream)))
 
     def put_back(self, bufs: GetBuffers, items: Sequence[Tuple], stream=None):
         """items: (column, data) device tensors holding the rows of the batch last served into
@@ -461,6 +465,33 @@ class Dock:
 
     def put_host_stage_bytes(self, column: int, k: int, data_elems: int) -> int:
         return lib().td_put_host_stage_bytes(self.handle, column, k, data_elems)
+
+    @staticmethod
+    def put_items(items: Sequence[Tuple]):
+        """The td_put_item array of (column, indices, cu or None, data) tensors, reusable across calls."""
+        arr = (TdPutItem * len(items))()
+        for j, (column, indices, cu, data) in enumerate(items):
+            arr[j] = TdPutItem(column, indices.numel(), indices.data_ptr(),
+                               cu.data_ptr() if cu is not None else None, data.data_ptr(), data.numel())
+        return arr
+
+    @staticmethod
+    def host_outs(hosts: Sequence["HostGetBuffers"]):
+        """The td_get_out array of a list of host mirrors, reusable across calls."""
+        return (TdGetOut * len(hosts))(*[h.struct for h in hosts])
+
+    def put_many_host(self, items, stage, stream=None):
+        """items: (column, indices, cu or None, data) HOST tensors, or put_items() of them; stage:
+        device uint8 tensor."""
+        arr = items if isinstance(items, C.Array) else self.put_items(items)
+        _check("td_put_many_host", lib().td_put_many_host(self.handle, arr, len(arr), stage.data_ptr(),
+                                                          stage.numel(), _stream_ptr(stream)))
+
+    def get_many_host(self, plan: "Plan", hosts, stream=None):
+        """hosts: HostGetBuffers per request of the plan, or host_outs() of them."""
+        arr = hosts if isinstance(hosts, C.Array) else self.host_outs(hosts)
+        _check("td_get_many_host", lib().td_get_many_host(self.handle, plan.handle, arr, len(arr),
+                                                          _stream_ptr(stream)))
 
     def get_host(self, bufs: GetBuffers, host: "HostGetBuffers", stream=None):
         _check("td_get_host", lib().td_get_host(self.handle, bufs.consumer, bufs.max_samples,

@@ -312,8 +312,23 @@ uint32_t copy_grid(const td_dock *d, uint64_t room_bytes) {
 
 // One launch group: alloc (if any ragged item), scatter, publish.  Items are taken in order;
 // a column appears at most once per group, so that duplicate detection sees earlier items.
-int put_group(td_dock *d, const PutBatch &b, cudaStream_t st) {
+int put_group(td_dock *d, PutBatch &b, cudaStream_t st) {
     const DockView &v = d->dv;
+    // Propose followers to the alloc kernel: an item may ride along with the latest item of its
+    // length class that takes passes of its own, when it has the same entry count and not more
+    // data behind it.
+    int leader[3] = {-1, -1, -1};
+    for (uint32_t i = 0; i < kMaxPutItems; ++i) b.follow[i] = 0;
+    for (uint32_t i = 0; i < b.n_items; ++i) {
+        const PutArgs &a = b.item[i];
+        const uint32_t cls = v.col_cls[a.column];
+        if (cls == TD_SCALAR) continue;
+        const int l = leader[cls];
+        if (l >= 0 && b.item[l].k == a.k && b.item[l].k_dev == a.k_dev && a.data_elems <= b.item[l].data_elems)
+            b.follow[i] = (uint8_t)(l + 1);
+        else
+            leader[cls] = (int)i;
+    }
     uint64_t ragged_bytes = 0, entries = 0;
     for (uint32_t i = 0; i < b.n_items; ++i) {
         entries += b.item[i].k;
@@ -785,16 +800,11 @@ int td_put_host(td_dock *d, uint32_t column, const int32_t *h_indices, uint32_t 
     return td_put(d, column, d_idx, k, ragged ? d_cu : nullptr, d_dat, data_elems, stream);
 }
 
-int td_get_host(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out *dev_out,
-                const td_get_out *host_out, void *stream) {
-    if (!d || !dev_out || !host_out || !host_out->result || !host_out->indices) return TD_EINVAL;
-    const int rc = td_get(d, consumer, max_samples, dev_out, stream);
-    if (rc != TD_OK) return rc;
-    cudaStream_t st = (cudaStream_t)stream;
-    const DockView &v = d->dv;
-    td_result *res = host_out->result;
-    if (cudaMemcpyAsync(res, dev_out->result, sizeof(td_result), cudaMemcpyDeviceToHost, st) != cudaSuccess) return TD_ECUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
+namespace {
+// Device -> host copies of the valid part of one served batch, sizes taken from its result block
+// (already on the host).  Enqueues only.
+int copy_batch_to_host(const DockView &v, uint32_t consumer, const td_get_out *dev_out, const td_get_out *host_out,
+                       const td_result *res, cudaStream_t st) {
     const size_t n = res->n_samples;
     auto d2h = [&](void *dst, const void *src, size_t bytes) {
         return !dst || !src || bytes == 0 || cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
@@ -824,8 +834,75 @@ int td_get_host(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_ge
         if (elems > host_out->seq_capacity_elems) return TD_EINVAL;
         ok = d2h(host_out->seq_advantages, dev_out->seq_advantages, elems * 4);
     }
-    if (!ok || cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
+    return ok ? TD_OK : TD_ECUDA;
+}
+}  // namespace
+
+int td_get_host(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out *dev_out,
+                const td_get_out *host_out, void *stream) {
+    if (!d || !dev_out || !host_out || !host_out->result || !host_out->indices) return TD_EINVAL;
+    const int rc = td_get(d, consumer, max_samples, dev_out, stream);
+    if (rc != TD_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    td_result *res = host_out->result;
+    if (cudaMemcpyAsync(res, dev_out->result, sizeof(td_result), cudaMemcpyDeviceToHost, st) != cudaSuccess) return TD_ECUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
+    const int rc2 = copy_batch_to_host(d->dv, consumer, dev_out, host_out, res, st);
+    if (rc2 != TD_OK) return rc2;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
+}
+
+int td_get_many_host(td_dock *d, td_plan *p, const td_get_out *host_outs, uint32_t n_req, void *stream) {
+    if (!d || !p || p->dock != d || !host_outs || n_req != p->n_req) return TD_EINVAL;
+    for (uint32_t q = 0; q < n_req; ++q)
+        if (!host_outs[q].result || !host_outs[q].indices) return TD_EINVAL;
+    const int rc = td_get_many(d, p, stream);
+    if (rc != TD_OK) return rc;
+    cudaStream_t st = (cudaStream_t)stream;
+    const GetReq *reqs = reinterpret_cast<const GetReq *>(p->host_image.data());     // the plan as uploaded
+    for (uint32_t q = 0; q < n_req; ++q)
+        if (cudaMemcpyAsync(host_outs[q].result, reqs[q].out.result, sizeof(td_result), cudaMemcpyDeviceToHost, st) !=
+            cudaSuccess) return TD_ECUDA;
+    if (cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
+    for (uint32_t q = 0; q < n_req; ++q) {
+        const int rc2 = copy_batch_to_host(d->dv, reqs[q].consumer, &reqs[q].out, &host_outs[q], host_outs[q].result, st);
+        if (rc2 != TD_OK) return rc2;
+    }
+    if (cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
+    return TD_OK;
+}
+
+int td_put_many_host(td_dock *d, const td_put_item *h_items, uint32_t n_items, void *d_stage, size_t stage_bytes,
+                     void *stream) {
+    if (!d || (n_items && !h_items)) return TD_EINVAL;
+    if (n_items == 0) return TD_OK;
+    if (!d_stage || (reinterpret_cast<uintptr_t>(d_stage) & 255u)) return TD_EWORKSPACE;
+    cudaStream_t st = (cudaStream_t)stream;
+    std::vector<td_put_item> dev(h_items, h_items + n_items);
+    uint8_t *p = static_cast<uint8_t *>(d_stage);
+    size_t used = 0;
+    for (uint32_t i = 0; i < n_items; ++i) {
+        const td_put_item &h = h_items[i];
+        if (h.column >= d->dv.ncol) return TD_EINVAL;
+        if (h.k == 0) continue;
+        const bool ragged = d->dv.col_cls[h.column] != TD_SCALAR;
+        if (!h.d_indices || (!h.d_data && h.data_elems) || (ragged && !h.d_cu)) return TD_EINVAL;
+        const size_t need = td_put_host_stage_bytes(d, h.column, h.k, h.data_elems);
+        if (used + need > stage_bytes) return TD_EWORKSPACE;
+        int32_t *d_idx = reinterpret_cast<int32_t *>(p + used);
+        int32_t *d_cu = reinterpret_cast<int32_t *>(p + used + align_up_sz((size_t)h.k * 4, 256));
+        uint8_t *d_dat = reinterpret_cast<uint8_t *>(d_cu) + align_up_sz(((size_t)h.k + 1) * 4, 256);
+        used += need;
+        const size_t esz = d->dv.col_esz[h.column];
+        if (cudaMemcpyAsync(d_idx, h.d_indices, (size_t)h.k * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TD_ECUDA;
+        if (ragged && cudaMemcpyAsync(d_cu, h.d_cu, ((size_t)h.k + 1) * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+            return TD_ECUDA;
+        if (h.data_elems && cudaMemcpyAsync(d_dat, h.d_data, (size_t)h.data_elems * esz, cudaMemcpyHostToDevice, st) !=
+            cudaSuccess) return TD_ECUDA;
+        dev[i].d_indices = d_idx; dev[i].d_cu = ragged ? d_cu : nullptr; dev[i].d_data = d_dat;
+    }
+    return td_put_many(d, dev.data(), n_items, stream);
 }
 
 }  // extern "C"

@@ -31,6 +31,10 @@ struct PutBatch {                              // the columns of one call, in ca
     uint32_t n_items;
     uint32_t pad;
     PutArgs item[kMaxPutItems];
+    // follow[i] = 1 + the index of an earlier item of the same length class that item i may
+    // ride along with in the alloc kernel (same entry count, not more data behind it), 0 = none.
+    // The host only proposes; the kernel checks that the index and cu arrays are equal.
+    uint8_t follow[kMaxPutItems];
 };
 
 static inline size_t put_alloc_smem_bytes(uint32_t S) {
@@ -87,6 +91,12 @@ __device__ __forceinline__ void warp_shard_prefix(bool alloc, uint32_t sh, uint3
 // A pass without a first arrival (a later column of a class whose rows exist) ends after 1.
 // A pass that would overflow a shard is replayed by one thread, entry by entry, so that only
 // the rows without room are refused.
+// A worker that sends a whole record puts several columns of one length class for the same
+// samples in the same order.  Such an item (a follower: its index and cu arrays equal those of
+// an earlier item of the call, its leader) never reserves a row, and everything it has to be
+// checked for follows from what the leader's thread already holds for the entry: the status
+// word, the row length and the length in force after the leader's CAS.  Followers are therefore
+// settled inside the leader's passes, without passes or atomics of their own.
 __global__ void __launch_bounds__(kAllocThreads)
 put_alloc_kernel(const DockView dv, const PutBatch batch) {
     extern __shared__ unsigned long long smem_u64[];
@@ -96,7 +106,8 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
     unsigned long long *s_start = s_run + S;                       // [S] where the pass's space begins
     __shared__ int32_t e_s[kAllocPass];
     __shared__ uint32_t e_room[kAllocPass];
-    __shared__ uint32_t s_overflow;
+    __shared__ uint8_t e_fok[kAllocPass];                          // bit f: follower f's entry was accepted
+    __shared__ uint32_t s_overflow, s_not_following;
 
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t L = blockIdx.x + 1;                             // TD_PROMPT or TD_RESPONSE
@@ -116,9 +127,39 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
         }
     }
 
+    // Which proposed followers really repeat their leader's index and cu arrays?
+    if (tid == 0) s_not_following = 0;
+    __syncthreads();
+    {
+        uint32_t differs = 0;
+        for (uint32_t it = 0; it < batch.n_items; ++it) {
+            if (!batch.follow[it] || dv.col_cls[batch.item[it].column] != L) continue;
+            const PutArgs &a = batch.item[it], &ld = batch.item[batch.follow[it] - 1u];
+            if (a.idx == ld.idx && a.cu == ld.cu) continue;
+            const uint32_t k = item_k(a);
+            bool d = false;
+            for (uint32_t i = tid; i <= k; i += kAllocThreads)
+                d |= (i < k && a.idx[i] != ld.idx[i]) || a.cu[i] != ld.cu[i];
+            if (d) differs |= 1u << it;
+        }
+        if (differs) atomicOr(&s_not_following, differs);
+    }
+    __syncthreads();
+    uint32_t not_following = s_not_following;
+    // an item that does not follow after all takes its own passes, in its place in the call; so
+    // do the later followers of its leader, which would otherwise overtake it
+    for (uint32_t it = 0; it < batch.n_items; ++it)
+        if ((not_following >> it) & 1u)
+            for (uint32_t f = it + 1; f < batch.n_items; ++f)
+                if (batch.follow[f] == batch.follow[it]) not_following |= 1u << f;
+
     for (uint32_t it = 0; it < batch.n_items; ++it) {
         const PutArgs &a = batch.item[it];
         if (dv.col_cls[a.column] != L) continue;
+        if (batch.follow[it] && !((not_following >> it) & 1u)) continue;      // settled with its leader
+        uint32_t followers = 0;
+        for (uint32_t f = it + 1; f < batch.n_items; ++f)
+            if (batch.follow[f] == it + 1u && !((not_following >> f) & 1u)) followers |= 1u << f;
         const uint32_t bit = 1u << a.column;
         const uint32_t k = item_k(a);
         for (uint32_t base = 0; base < k; base += kAllocPass) {
@@ -131,11 +172,12 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
             for (int j = 0; j < kAllocPer; ++j) {
                 const uint32_t i = base + j * kAllocThreads + tid;
                 alloc[j] = false; s[j] = -1; room[j] = 0; sh[j] = 0;
+                uint32_t fok = 0;
                 if (i < k) {
                     s[j] = a.idx[i];
                     const int64_t c0 = a.cu[i], c1 = a.cu[i + 1];
                     const int64_t l = c1 - c0;
-                    if (s[j] < 0 || (uint32_t)s[j] >= dv.n) { ++n_oob; }
+                    if (s[j] < 0 || (uint32_t)s[j] >= dv.n) { ++n_oob; n_oob += __popc(followers); }
                     else {
                         // The status word and the CAS travel side by side.  A column that is
                         // already stored has its class's length set, so the CAS of a repeated
@@ -152,8 +194,20 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
                             room[j] = (uint32_t)align_row((uint64_t)l);
                             sh[j] = shard_of(dv, (uint32_t)s[j]);
                         } else if (old != (int32_t)l) { ++n_mis; }
+                        // Followers: same sample, same row.  Their bound on the data is not
+                        // wider than the leader's, so where one of them is in order the leader
+                        // has done its CAS and the length in force is known.
+                        for (uint32_t fm = followers; fm; fm &= fm - 1u) {
+                            const uint32_t f = (uint32_t)__ffs(fm) - 1u;
+                            const PutArgs &b = batch.item[f];
+                            if (st & (1u << b.column)) ++n_dup;
+                            else if (l < 0 || c0 < 0 || (uint64_t)c1 > b.data_elems) ++n_bad;
+                            else if ((old == -1 ? (int32_t)l : old) != (int32_t)l) ++n_mis;
+                            else fok |= 1u << f;
+                        }
                     }
                 }
+                e_fok[j * kAllocThreads + tid] = (uint8_t)fok;
                 e_s[j * kAllocThreads + tid] = s[j];
                 e_room[j * kAllocThreads + tid] = alloc[j] ? room[j] : kNotAllocating;
                 any |= alloc[j];
@@ -221,7 +275,7 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
                         if (start + r > cap) {
                             atomicAdd(&dv.cursor[L][k2], 0ull - (unsigned long long)r);
                             atomicExch(&dv.len[L][ss], -1);
-                            ++n_full;
+                            n_full += 1u + __popc((uint32_t)e_fok[t]);      // its followers find no row either
                         } else {
                             dv.off[L][ss] = (long long)start;
                         }

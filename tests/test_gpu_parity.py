@@ -504,6 +504,69 @@ def test_output_capacity_truncation_matches(G):
     G.assert_stats_equal(g, o, "truncation")
 
 
+def _host_batch(G, g, bufs, host) -> "object":
+    """What td_get_host / td_get_many_host left in the pinned host mirrors, as a Batch."""
+    from oracle import td_oracle as ora
+    r = host.result
+    b = ora.Batch()
+    b.n_samples, b.n_groups, b.status = r.n_samples, r.n_groups, r.status
+    b.prompt_tokens, b.response_tokens = r.prompt_tokens, r.response_tokens
+    k = b.n_samples
+    b.indices = host.indices[:k].numpy().copy()
+    b.cu_prompt, b.cu_response = host.cu_prompt[:k + 1].numpy().copy(), host.cu_response[:k + 1].numpy().copy()
+    b.cu_seq = host.cu_seq[:k + 1].numpy().copy()
+    for c, t in host.cols.items():
+        cls = g.dock.columns[c][1]
+        tot = k if cls == td.SCALAR else (b.prompt_tokens if cls == td.PROMPT else b.response_tokens)
+        b.columns[c] = G.to_host(t[:tot])
+    if host.advantages is not None:
+        b.advantages = host.advantages[:k].numpy().copy()
+    return b
+
+
+def test_host_buffer_calls_single_and_batched(G):
+    """Host tensors in, host tensors out: td_put_host + td_get_host per call, and
+    td_put_many_host + td_get_many_host for a whole step, against the oracle."""
+    import torch
+    w = wl.make_custom("host", 24, 3, 4, prompt_len=(1, 70), response=("uniform", 0, 200), vocab=50000,
+                       micro_batch=9, seed=51, with_entropy=True, schedule="bulk")
+    gets = [op for op in w.ops if op.kind == "get"]
+
+    def pinned(a):
+        t = torch.from_numpy(np.ascontiguousarray(a).view(np.int16) if a.dtype == np.uint16 else np.ascontiguousarray(a))
+        return (t.view(torch.bfloat16) if a.dtype == np.uint16 else t).pin_memory()
+
+    for batched in (False, True):
+        o = H.make_oracle(w)
+        g = G.GpuDock(w)
+        items = []
+        for op in w.ops:
+            if op.kind == "put":
+                cu, data = w.pack(op.column, op.indices)
+                o.put(op.column, op.indices, cu, data)
+                items.append((op.column, pinned(np.ascontiguousarray(op.indices, np.int32)),
+                              pinned(cu) if cu is not None else None, pinned(data)))
+        need = [g.dock.put_host_stage_bytes(c, i.numel(), d.numel()) for c, i, _cu, d in items]
+        bufs = [g.buffers(op.consumer, op.max_samples, key=("host", j)) for j, op in enumerate(gets)]
+        hosts = [td.HostGetBuffers(b) for b in bufs]
+        if batched:
+            stage = torch.empty(sum(need), dtype=torch.uint8, device=g.device)
+            g.dock.put_many_host(items, stage)
+            plan = g.dock.plan(bufs)
+            g.dock.get_many_host(plan, hosts)
+        else:
+            stage = torch.empty(max(need), dtype=torch.uint8, device=g.device)
+            for c, i, cu, d in items:
+                g.dock.put_host(c, i, cu, d, stage)
+                torch.cuda.synchronize()          # one staging buffer: free again before the next put
+            for b, h in zip(bufs, hosts):
+                g.dock.get_host(b, h)
+        for j, op in enumerate(gets):
+            want = o.get(op.consumer, op.max_samples)
+            G.assert_batch_equal(_host_batch(G, g, bufs[j], hosts[j]), want, f"batched={batched} request {j}")
+        G.assert_state_equal(g, o, ctx=f"host batched={batched}")
+
+
 def test_host_argument_checks(G):
     w = wl.make_config(1)
     g = G.GpuDock(w)
