@@ -251,15 +251,27 @@ class GpuStep:
         self.puts = []        # (column, idx, cu, data) device tensors
         self.host_puts = []   # the same in pinned host memory
         self.h2d_bytes = 0
+        # A worker that sends a whole record has one index array for the batch and one cu array
+        # per length class: columns with equal arrays share them, on the host and on the device.
+        shared = {}
+
+        def share(a):
+            key = (a.dtype.str, a.shape, a.tobytes())
+            if key not in shared:
+                pinned = self._pin(a)
+                shared[key] = (pinned, pinned.to(self.dev))
+            return shared[key]
+
         for op in w.ops:
             if op.kind != "put":
                 continue
             cu, data = w.pack(op.column, op.indices)
             idx = np.ascontiguousarray(op.indices, dtype=np.int32)
-            h = (op.column, self._pin(idx), self._pin(cu) if cu is not None else None, self._pin(data))
-            self.host_puts.append(h)
-            self.puts.append((op.column, h[1].to(self.dev), h[2].to(self.dev) if h[2] is not None else None,
-                              h[3].to(self.dev)))
+            h_idx, d_idx = share(idx)
+            h_cu, d_cu = share(cu) if cu is not None else (None, None)
+            h_data = self._pin(data)
+            self.host_puts.append((op.column, h_idx, h_cu, h_data))
+            self.puts.append((op.column, d_idx, d_cu, h_data.to(self.dev)))
             self.h2d_bytes += idx.nbytes + (cu.nbytes if cu is not None else 0) + data.nbytes
         # one output buffer set per get call, sized by the longest rows it could meet
         lp = np.sort(w.len_prompt)[::-1]

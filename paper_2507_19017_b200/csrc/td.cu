@@ -338,7 +338,7 @@ int put_group(td_dock *d, PutBatch &b, cudaStream_t st) {
     if (entries == 0) return TD_OK;
     if (entries >= (1ull << 32)) return TD_EINVAL;
     if (ragged_bytes) {
-        if (launch(d, put_alloc_kernel, dim3(2), dim3(kAllocThreads), put_alloc_smem_bytes(v.S), st, v, b) != cudaSuccess)
+        if (launch_dep(d, put_alloc_kernel, dim3(2), dim3(kAllocThreads), put_alloc_smem_bytes(v.S), st, v, b) != cudaSuccess)
             return TD_ECUDA;
         if (launch_timed(d, 0, put_scatter_kernel, dim3(copy_grid(d, ragged_bytes)), dim3(kCopyThreads),
                          scatter_smem_bytes(), st, v, b) != cudaSuccess)
@@ -500,7 +500,7 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
     const uint32_t jpr = jobs_per_req(v, wants_stream(*out));
 
-    if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
+    if (launch_dep(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
@@ -579,7 +579,7 @@ int td_get_static(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
     const uint32_t jpr = jobs_per_req(v, wants_stream(*out));
 
-    if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
+    if (launch_dep(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
@@ -692,7 +692,7 @@ int td_get_many(td_dock *d, td_plan *p, void *stream) {
     GetInline none;
     std::memset(&none, 0, sizeof(none));
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
-    if (launch(d, get_select_kernel, dim3(sel_tiles(v.G), p->n_slots), dim3(kSelThreads), 0, st, v, none,
+    if (launch_dep(d, get_select_kernel, dim3(sel_tiles(v.G), p->n_slots), dim3(kSelThreads), 0, st, v, none,
                (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
     if (launch_finalize(d, p->n_req, p->max_req_samples, st, v, none, (const GetReq *)p->d_reqs,
                (const ConsumerSlot *)p->d_slots, seq, p->d_counter, p->d_job_sizes, p->jobs_per_req) != cudaSuccess) return TD_ECUDA;

@@ -127,6 +127,11 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
         }
     }
 
+    // From here on the call's arrays and the dock's tables are read: whatever ran before this
+    // kernel in the stream (a reset, the get whose batch is sent back, the caller's own producer)
+    // must have finished.  The prefetch above only asked for lines.
+    griddep_wait();
+
     // Which proposed followers really repeat their leader's index and cu arrays?
     if (tid == 0) s_not_following = 0;
     __syncthreads();

@@ -88,6 +88,7 @@ get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
     __shared__ uint32_t s_tile, s_excl, s_failed;
     __shared__ uint32_t s_warp[kSelWarps];
     griddep_launch_dependents();
+    griddep_wait();                                    // status and claim words as the work before this call left them
 
     if (tid == 0) {
         // ticket word = seq << 32 | tiles started; sequence numbers only grow
@@ -669,6 +670,7 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
 // Reset: every table, bitmap and counter back to the empty state; payload untouched.
 __global__ void __launch_bounds__(256)
 reset_kernel(const DockView dv) {
+    griddep_launch_dependents();                       // the first kernel of the next call may set itself up meanwhile
     const uint32_t t = blockIdx.x * blockDim.x + threadIdx.x;
     const uint32_t stride = gridDim.x * blockDim.x;
     for (uint32_t s = t; s < dv.n; s += stride) {
