@@ -20,8 +20,10 @@
  *     device memory and frees none.  "host" pointers are ordinary host memory.
  *   - td_put / td_get / td_get_many / td_reset only enqueue work on the given stream and return;
  *     they never synchronise.  Calls on one stream execute in call order.  Gets may run
- *     concurrently with each other and with puts on other streams; puts that touch the same
- *     (sample, length class) must be ordered by the caller.
+ *     concurrently with each other and with puts on other streams.  Puts that may reserve the
+ *     same row (the first columns of a length class to arrive for a sample) must be ordered by
+ *     the caller; puts of further columns for samples whose rows of that class are stored and
+ *     published (the write-backs of worker states) only read the tables and may overlap.
  *   - return value: TD_OK (0) or a negative td_error found on the host.  Conditions found on the
  *     device never trap: the offending sample is skipped, a TD_ERR_* bit is OR-ed into the
  *     dock's error word (td_status) and, for a get, into td_result.status.

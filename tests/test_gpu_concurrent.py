@@ -146,3 +146,93 @@ def test_config4_concurrent_full_size(G):
     w = wl.make_config(4)
     g, batches = run_concurrent(G, w, [0, 1, 2, 3])
     partial, st = check_outcome(G, w, g, [0, 1, 2, 3], batches)
+
+
+def test_concurrent_cascade_with_write_backs(G):
+    """The whole sample flow with every party on its own stream and thread: a producer puts the
+    id columns in shuffled chunks, three inference states poll, and send their column back for
+    each batch they are served (td_put_back, batch size read on the device), the actor update
+    polls for what has become complete.  Checked like the other concurrent runs: exactly once per
+    consumer, and every batch equal to what the oracle gathers for its indices once it holds
+    the same rows."""
+    w = wl.make_custom("conc-cascade", 96, 4, 8, prompt_len=(8, 200), response=("lognormal", 300.0, 0.4, 1200),
+                       vocab=32000, micro_batch=32, seed=45, schedule="cascade", chunk=(4, 40), poll_every=4,
+                       with_entropy=True)
+    g = G.GpuDock(w)
+    puts = [op for op in w.ops if op.kind == "put"]
+    produces = {}
+    for op in w.ops:
+        if op.kind == "put_back":
+            produces[op.consumer] = op.columns
+    workers = sorted(produces)
+    updater = [c for c in range(len(w.consumers)) if c not in produces][0]
+    pool_dev = {c: G.to_device(a, g.device) for c, a in w.pool.items()}
+    errors, lock = [], threading.Lock()
+    batches = {c: [] for c in range(len(w.consumers))}
+
+    def producer():
+        try:
+            s = torch.cuda.Stream()
+            with torch.cuda.stream(s):
+                for op in puts:
+                    g.put_op(op, stream=s)
+                s.synchronize()
+        except Exception as e:       # pragma: no cover
+            errors.append(e)
+
+    def party(c):
+        try:
+            s = torch.cuda.Stream()
+            with torch.cuda.stream(s):
+                pc, rc = g.token_caps(w.micro_batch)
+                bufs = td.GetBuffers(g.dock, c, w.micro_batch, prompt_tokens_cap=pc, response_tokens_cap=rc)
+                served, deadline = 0, time.time() + 120
+                while served < w.n:
+                    assert time.time() < deadline, f"consumer {c} did not finish in time"
+                    g.dock.get(bufs, stream=s)
+                    if c in produces:                      # enqueued before the host knows the batch size
+                        g.dock.put_back(bufs, [(col, pool_dev[col]) for col in produces[c]], stream=s)
+                    b = g.read(bufs, stream=s)
+                    assert b.status == 0
+                    if b.n_samples:
+                        batches[c].append(b)
+                        served += b.n_samples
+        except Exception as e:
+            errors.append(e)
+
+    threads = [threading.Thread(target=producer)] + [threading.Thread(target=party, args=(c,))
+                                                     for c in range(len(w.consumers))]
+    for t in threads:
+        t.start()
+    for t in threads:
+        t.join(timeout=150)
+    assert not any(t.is_alive() for t in threads), "a thread did not finish"
+    if errors:
+        raise errors[0]
+    torch.cuda.synchronize()
+
+    # the oracle is given the same rows: the ids, then every write-back as the workers made it
+    o = H.make_oracle(w)
+    idx = np.arange(w.n, dtype=np.int32)
+    for name in ("prompt_ids", "response_ids"):
+        c = w.column_index(name)
+        cu, data = w.pack(c, idx)
+        o.put(c, idx, cu, data)
+    for c in workers:
+        for b in batches[c]:
+            H.oracle_put_back(w, o, b, produces[c])
+    for c in range(len(w.consumers)):
+        got = []
+        for b in batches[c]:
+            assert b.n_samples % w.N == 0 and np.all(np.diff(b.indices) > 0)
+            want = o.gather(c, b.indices)
+            want.status = b.status
+            G.assert_batch_equal(b, want, f"consumer {c}")
+            got.extend(b.indices.tolist())
+        assert sorted(got) == list(range(w.n)), f"consumer {c}: not exactly once"
+    st = g.dock.status()
+    assert st.error_word == 0
+    for col in w.pool:
+        assert st.put_accepted[col] == w.n
+    full = (1 << len(w.columns)) - 1
+    assert np.all(g.table(0, 0, np.uint32) == full)           # every column of every sample stored
