@@ -29,7 +29,8 @@ METRIC = "td_put+td_get samples/s dispatched"
 L2_FLUSH_BYTES = 256 << 20
 # DRAM bytes (read + write) of one launch, from the ncu capture summarised under profiles/ for
 # the kernels as built; (config, kernel) pairs without a capture report null.
-NCU_TRAFFIC = {(2, "get_gather"): 80_401_152, (2, "put_scatter"): 45_302_784}
+NCU_TRAFFIC = {(2, "get_gather"): 80_714_752, (2, "put_scatter"): 45_192_448,
+               (3, "get_gather"): 1_146_963_200, (3, "put_scatter"): 733_966_080}
 
 
 def parse_args():
@@ -715,7 +716,7 @@ def main():
         k["GBps"] = k["bytes_per_launch"] / (k["avg_ms"] * 1e-3) / 1e9 if k["avg_ms"] > 0 else 0.0
     dom = "get_gather" if ms_ga >= ms_sc else "put_scatter"
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kern[dom]["GBps"], "peak": peak, "unit": "GB/s",
-                "frac": kern[dom]["GBps"] / peak, "traffic": NCU_TRAFFIC.get((args.config, dom)),
+                "frac": kern[dom]["GBps"] / peak, "traffic": None if args.fused else NCU_TRAFFIC.get((args.config, dom)),
                 "peak_kind": peak_kind,
                 "bytes_per_launch": kern[dom]["bytes_per_launch"], "avg_launch_ms": kern[dom]["avg_ms"]}
 
