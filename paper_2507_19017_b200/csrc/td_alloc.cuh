@@ -9,6 +9,7 @@ namespace td {
 
 constexpr int kAllocThreads = 1024;
 constexpr int kAllocWarps = kAllocThreads / 32;
+static_assert(kAllocWarps == 32, "the scan over the warps' sums gives one lane to each warp");
 constexpr int kAllocPer = 4;                                   // entries per thread and pass
 constexpr int kAllocPass = kAllocThreads * kAllocPer;          // entries per pass
 constexpr int kMaxPutItems = 8;                                // columns one put launch can carry
@@ -84,9 +85,9 @@ __device__ __forceinline__ void warp_shard_prefix(bool alloc, uint32_t sh, uint3
 // kAllocPass entries in call order.  Per pass:
 //   1. every thread validates kAllocPer entries and settles with a CAS on len[] which of them
 //      are first arrivals of their length class, i.e. reserve a row;
-//   2. round by round (kAllocThreads entries each) an ordered per-shard exclusive scan of the
-//      row sizes (warp shuffles, then the warps' sums through shared memory) gives every new
-//      row the place, relative to the pass, a sequential walk would have given it;
+//   2. an ordered per-shard exclusive scan of the row sizes (every warp over its own run of
+//      consecutive entries with shuffles, then the warps' sums through shared memory) gives
+//      every new row the place, relative to the pass, a sequential walk would have given it;
 //   3. one atomicAdd per shard reserves the pass's space; rows are placed behind it.
 // A pass without a first arrival (a later column of a class whose rows exist) ends after 1.
 // A pass that would overflow a shard is replayed by one thread, entry by entry, so that only
@@ -168,15 +169,19 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
         const uint32_t bit = 1u << a.column;
         const uint32_t k = item_k(a);
         for (uint32_t base = 0; base < k; base += kAllocPass) {
-            // 1. validate, CAS
+            // 1. validate, CAS.  A short pass is spread over all warps: each takes `per` rows of 32.
+            const uint32_t per = min((uint32_t)kAllocPer, (k - base + kAllocThreads - 1u) / kAllocThreads);
             int32_t s[kAllocPer];
             uint32_t room[kAllocPer], sh[kAllocPer];
             bool alloc[kAllocPer];
             bool any = false;
             #pragma unroll
             for (int j = 0; j < kAllocPer; ++j) {
-                const uint32_t i = base + j * kAllocThreads + tid;
+                // a warp owns 32 * per consecutive entries of the pass, in the order (j, lane)
+                const uint32_t eo = warp * (32u * per) + (uint32_t)j * 32u + lane;
+                const uint32_t i = base + eo;
                 alloc[j] = false; s[j] = -1; room[j] = 0; sh[j] = 0;
+                if ((uint32_t)j >= per) continue;
                 uint32_t fok = 0;
                 if (i < k) {
                     s[j] = a.idx[i];
@@ -212,45 +217,48 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
                         }
                     }
                 }
-                e_fok[j * kAllocThreads + tid] = (uint8_t)fok;
-                e_s[j * kAllocThreads + tid] = s[j];
-                e_room[j * kAllocThreads + tid] = alloc[j] ? room[j] : kNotAllocating;
+                e_fok[eo] = (uint8_t)fok;
+                e_s[eo] = s[j];
+                e_room[eo] = alloc[j] ? room[j] : kNotAllocating;
                 any |= alloc[j];
             }
-            for (uint32_t k2 = tid; k2 < S; k2 += kAllocThreads) s_run[k2] = 0;
             if (tid == 0) s_overflow = 0;
             if (!__syncthreads_or(any)) continue;                 // no first arrival in this pass
 
-            // 2. relative places, round by round
+            // 2. relative places: inside a warp its entries in order (four shuffle scans that
+            //    carry the warp's per-shard sums along), then the warps in order (one scan over
+            //    the warps' sums per shard)
+            for (uint32_t q = lane; q < S; q += 32) tot[warp * S + q] = 0;
+            __syncwarp();
             unsigned long long rel[kAllocPer];
             #pragma unroll
             for (int j = 0; j < kAllocPer; ++j) {
                 rel[j] = 0;
-                if (base + (uint32_t)j * kAllocThreads >= k) break;       // uniform
-                for (uint32_t q = tid; q < kAllocWarps * S; q += kAllocThreads) tot[q] = 0;
+                if ((uint32_t)j >= per) continue;                     // uniform
                 unsigned long long pre, wsum;
                 bool leader;
                 warp_shard_prefix(alloc[j], sh[j], room[j], lane, pre, wsum, leader);
-                __syncthreads();
-                if (leader) tot[warp * S + sh[j]] = wsum;
-                __syncthreads();
-                for (uint32_t k2 = warp; k2 < S; k2 += kAllocWarps) {
-                    const unsigned long long v = tot[lane * S + k2];
-                    unsigned long long inc = v;
-                    #pragma unroll
-                    for (int d = 1; d < 32; d <<= 1) {
-                        const unsigned long long t = shfl_up_u64(inc, d);
-                        if ((int)lane >= d) inc += t;
-                    }
-                    const unsigned long long run = s_run[k2];
-                    tot[lane * S + k2] = run + inc - v;
-                    __syncwarp();
-                    if (lane == 31) s_run[k2] = run + inc;
-                }
-                __syncthreads();
-                if (alloc[j]) rel[j] = tot[warp * S + sh[j]] + pre;
-                __syncthreads();
+                rel[j] = alloc[j] ? tot[warp * S + sh[j]] + pre : 0ull;
+                __syncwarp();
+                if (leader) tot[warp * S + sh[j]] += wsum;
+                __syncwarp();
             }
+            __syncthreads();
+            for (uint32_t k2 = warp; k2 < S; k2 += kAllocWarps) {
+                const unsigned long long v = tot[lane * S + k2];
+                unsigned long long inc = v;
+                #pragma unroll
+                for (int d = 1; d < 32; d <<= 1) {
+                    const unsigned long long t = shfl_up_u64(inc, d);
+                    if ((int)lane >= d) inc += t;
+                }
+                tot[lane * S + k2] = inc - v;                      // what the warps before this one ask for
+                if (lane == 31) s_run[k2] = inc;                   // what the pass asks for
+            }
+            __syncthreads();
+            #pragma unroll
+            for (int j = 0; j < kAllocPer; ++j)
+                if (alloc[j]) rel[j] += tot[warp * S + sh[j]];
 
             // 3. reserve the pass's space, place the rows
             for (uint32_t k2 = tid; k2 < S; k2 += kAllocThreads) {

@@ -33,6 +33,11 @@ static inline FastDiv make_fastdiv(uint32_t d) {
     const uint64_t m = (1ull << l) == d ? 0 : ((1ull << 32) * ((1ull << l) - d)) / d + 1;
     return FastDiv{(uint32_t)m, l};
 }
+__device__ __forceinline__ FastDiv make_fastdiv_dev(uint32_t d) {          // the same constants, computed on the device
+    const uint32_t l = d > 1u ? 32u - (uint32_t)__clz(d - 1u) : 0u;
+    const unsigned long long m = (1ull << l) == d ? 0ull : ((1ull << 32) * ((1ull << l) - d)) / d + 1ull;
+    return FastDiv{(uint32_t)m, l};
+}
 __device__ __forceinline__ uint32_t fast_div(uint32_t n, FastDiv f) {
     return (__umulhi(n, f.mul) + n) >> f.shr;
 }

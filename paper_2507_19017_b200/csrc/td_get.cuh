@@ -12,6 +12,7 @@ constexpr int kSelWarps = kSelThreads / 32;
 constexpr int kFinThreads = 256;            // finalize: threads per request; kFinThreadsBig when a request is large
 constexpr int kFinThreadsBig = 1024;
 constexpr uint32_t kFinBigSamples = 1024;   // a request that may serve more samples than this gets the large block
+constexpr uint32_t kFinGroupsKept = 1024;   // groups of a request whose numbers finalize keeps in shared memory
 constexpr int kMaxJobs = 4096;              // (request, column) pairs one gather launch serves
 // A request that wants the fused token stream has three more jobs behind its columns: the
 // stream's prompt half, its response half, and the advantage twin.
@@ -277,12 +278,18 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     const uint32_t tid = threadIdx.x;
     __shared__ uint64_t sh_a[kThreads / 32], sh_b[kThreads / 32];
     __shared__ uint32_t s_first_over;
+    // the groups served, for the first kFinGroupsKept of them: later steps take a sample's index
+    // from here instead of reading the index list back from global memory
+    __shared__ int32_t s_grp[kFinGroupsKept];
     griddep_launch_dependents();
     griddep_wait();                                    // the scan's candidate list is complete
     if (blockIdx.x == 0 && threadIdx.x == 0) *work_counter = 0;     // the gather hands out its chunks from zero
 
-    // how many groups were ready, from the last tile's inclusive prefix
+    // how many groups were ready, from the last tile's inclusive prefix; the first candidates are
+    // asked for in the same breath (which of them count is known once the prefix is here)
     const unsigned long long last = sc.desc[sel_tiles(dv.G) - 1];
+    int32_t g_first = -1;
+    if (tid < rq.max_groups && rq.rank_base + tid < dv.G) g_first = sc.cand[rq.rank_base + tid];
     uint32_t status = 0;
     uint32_t total = 0;
     if (desc_seq(last) != seq || desc_state(last) != kStatePrefix) status |= TD_ERR_LOOKBACK_TIMEOUT;
@@ -296,17 +303,24 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     for (uint32_t base = 0; base < ncand; base += kThreads) {
         const uint32_t r = base + tid;
         int32_t g = -1;
-        if (r < ncand) g = sc.cand[lo + r];
+        if (r < ncand) g = base == 0 ? g_first : sc.cand[lo + r];
         uint64_t dummy_b, ta, tb;
         const uint64_t inc = block_scan_incl_2<kThreads>(g >= 0 ? 1u : 0u, 0, dummy_b, sh_a, sh_b, ta, tb);
         if (g >= 0) {
             const uint32_t p = n_grp + (uint32_t)inc - 1u;
+            if (p < kFinGroupsKept) s_grp[p] = g;
             for (uint32_t j = 0; j < N; ++j) out.indices[(size_t)p * N + j] = g * (int32_t)N + (int32_t)j;
         }
         n_grp += (uint32_t)ta;
     }
     __syncthreads();
     uint32_t n_s = n_grp * N;
+    const FastDiv div_N = make_fastdiv_dev(N);
+    // sample at position i of the batch
+    auto sample_at = [&](uint32_t i) -> int32_t {
+        const uint32_t p = fast_div(i, div_N);
+        return p < kFinGroupsKept ? s_grp[p] * (int32_t)N + (int32_t)(i - p * N) : out.indices[i];
+    };
 
     // pass B: cu_seqlens and the fit test
     if (tid == 0) {
@@ -342,7 +356,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
         const uint32_t i = base + tid;
         uint64_t lp = 0, lr = 0;
         if (i < n_s) {
-            const int32_t s = out.indices[i];
+            const int32_t s = sample_at(i);
             const int32_t a = dv.len[TD_PROMPT][s], b = dv.len[TD_RESPONSE][s];
             lp = a > 0 ? (uint64_t)a : 0; lr = b > 0 ? (uint64_t)b : 0;
         }
@@ -363,6 +377,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
         carry_p += tp; carry_r += tr;
     }
     __syncthreads();
+    uint64_t tot_p = carry_p, tot_r = carry_r;         // the batch's token totals
     if (s_first_over != 0xffffffffu) {
         const uint32_t keep = s_first_over / N;
         for (uint32_t p = keep + tid; p < n_grp; p += kThreads) {
@@ -372,18 +387,20 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
         n_grp = keep; n_s = keep * N;
         status |= TD_ERR_OUT_TRUNCATED;
         if (tid == 0) flag_error(dv, TD_ERR_OUT_TRUNCATED, CNT_TRUNC);
+        tot_p = (uint64_t)(int64_t)out.cu_prompt[n_s];            // the cut batch ends here
+        tot_r = (uint64_t)(int64_t)out.cu_response[n_s];
     }
     // consumed bits
     uint32_t *consumed = dv.consumed + (size_t)c * dv.consumed_words;
     for (uint32_t i = tid; i < n_s; i += kThreads) {
-        const uint32_t s = (uint32_t)out.indices[i];
+        const uint32_t s = (uint32_t)sample_at(i);
         atomicOr(&consumed[s >> 5], 1u << (s & 31));
     }
     // group-normalised advantage, one thread per group, in double
     if ((dv.cflags[c] & TD_F_ADVANTAGE) && out.advantages) {
         const float *rew = reinterpret_cast<const float *>(dv.colbase[dv.reward_col]);
         for (uint32_t p = tid; p < n_grp; p += kThreads) {
-            const float *r = rew + out.indices[(size_t)p * N];       // a group's samples are consecutive
+            const float *r = rew + (p < kFinGroupsKept ? s_grp[p] * (int32_t)N : out.indices[(size_t)p * N]);   // a group's samples are consecutive
             double sum = 0.0;
             for (uint32_t j = 0; j < N; ++j) sum += (double)r[j];
             const double mean = sum / (double)N;
@@ -398,8 +415,8 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     if (tid == 0) {
         td_result r;
         r.n_samples = n_s; r.n_groups = n_grp;
-        r.prompt_tokens = (uint64_t)(int64_t)out.cu_prompt[n_s];
-        r.response_tokens = (uint64_t)(int64_t)out.cu_response[n_s];
+        r.prompt_tokens = tot_p;
+        r.response_tokens = tot_r;
         r.status = status; r.reserved = 0;
         *out.result = r;
         if (status & TD_ERR_LOOKBACK_TIMEOUT) atomicOr(dv.errword, TD_ERR_LOOKBACK_TIMEOUT);
@@ -409,8 +426,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     // the gather's job table: this request's output bytes per column and its row count
     if (job_sizes && tid < jobs_per_req) {
         JobSize js;
-        js.bytes = job_bytes_of(dv, rq, tid, n_s, (uint64_t)(int64_t)out.cu_prompt[n_s],
-                                (uint64_t)(int64_t)out.cu_response[n_s]);
+        js.bytes = job_bytes_of(dv, rq, tid, n_s, tot_p, tot_r);
         js.rows = n_s;
         js.cost_rows = job_cost_rows(dv, rq, tid, js.bytes, n_s);
         job_sizes[(size_t)blockIdx.x * jobs_per_req + tid] = js;
