@@ -349,13 +349,15 @@ class GpuStep:
         self.host_gets = [td.HostGetBuffers(b) for b in self.gets]
         self.host_put_arr = self.dock.put_items(self.host_puts)       # marshalled once, like a caller would
         self.host_out_arr = self.dock.host_outs(self.host_gets)
+        self.meta_stage = (torch.empty(self.dock.get_many_host_stage_bytes(self.plan), dtype=torch.uint8, device=self.dev)
+                           if self.api == "many" else None)
 
     def e2e_step(self):
         torch = self.torch
         self.dock.reset()
         if self.api == "many":          # one call in, one call out: two synchronisations per step
             self.dock.put_many_host(self.host_put_arr, self.stage[0])
-            self.dock.get_many_host(self.plan, self.host_out_arr)
+            self.dock.get_many_host(self.plan, self.host_out_arr, self.meta_stage)
             return None
         for j, (col, idx, cu, data) in enumerate(self.host_puts):
             if j >= 2:

@@ -326,10 +326,17 @@ int td_get_host(td_dock *dock, uint32_t consumer, uint32_t max_samples, const td
  * copied to the matching HOST pointers of host_outs[r] (one entry per request of the plan, in
  * plan order; result and indices required, NULL elsewhere = skip).  All result blocks are
  * fetched behind one synchronisation, all payload behind a second one: two per call however many
- * requests the plan holds, where td_get_host takes two per request. */
+ * requests the plan holds, where td_get_host takes two per request.  d_stage (device, 16-byte
+ * aligned, td_get_many_host_stage_bytes(plan) bytes, private to the call) is optional: with it
+ * the get writes every request's result block, indices, cu_seqlens and advantages a second time,
+ * side by side, and one transfer brings them all to the host (the first such call on a plan
+ * allocates a pinned host buffer of that size, freed by td_plan_destroy); NULL: one transfer per
+ * array and request. */
 int td_put_many_host(td_dock *dock, const td_put_item *h_items, uint32_t n_items, void *d_stage,
                      size_t stage_bytes, void *stream);
-int td_get_many_host(td_dock *dock, td_plan *plan, const td_get_out *host_outs, uint32_t n_req, void *stream);
+size_t td_get_many_host_stage_bytes(const td_plan *plan);
+int td_get_many_host(td_dock *dock, td_plan *plan, const td_get_out *host_outs, uint32_t n_req, void *d_stage,
+                     size_t stage_bytes, void *stream);
 
 /* The communication-volume model of "Distributed Transfer Dock Strategy", in bytes, for sizing a
  * dock or a link (host arithmetic only; no device is touched):

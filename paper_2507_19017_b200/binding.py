@@ -31,7 +31,7 @@ EXPORTS = ["td_query_workspace", "td_create", "td_destroy", "td_put", "td_get",
            "td_launch_count", "td_strerror", "td_kernel_timing", "td_kernel_timing_read",
            "td_put_host_stage_bytes", "td_put_host", "td_get_host", "td_put_many",
            "td_plan_bytes", "td_plan_create", "td_plan_destroy", "td_get_many", "td_get_static",
-           "td_model_bytes", "td_put_back", "td_put_back_many", "td_put_many_host", "td_get_many_host"]
+           "td_model_bytes", "td_put_back", "td_put_back_many", "td_put_many_host", "td_get_many_host", "td_get_many_host_stage_bytes"]
 
 
 class TdModel(C.Structure):
@@ -165,7 +165,9 @@ def lib():
         L.td_put_many_host.restype = C.c_int
         L.td_put_many_host.argtypes = [vp, C.POINTER(TdPutItem), u32, vp, C.c_size_t, vp]
         L.td_get_many_host.restype = C.c_int
-        L.td_get_many_host.argtypes = [vp, vp, C.POINTER(TdGetOut), u32, vp]
+        L.td_get_many_host.argtypes = [vp, vp, C.POINTER(TdGetOut), u32, vp, C.c_size_t, vp]
+        L.td_get_many_host_stage_bytes.restype = C.c_size_t
+        L.td_get_many_host_stage_bytes.argtypes = [vp]
         L.td_plan_bytes.restype = C.c_size_t
         L.td_plan_bytes.argtypes = [vp, u32]
         L.td_plan_create.restype = C.c_int
@@ -487,11 +489,17 @@ class Dock:
         _check("td_put_many_host", lib().td_put_many_host(self.handle, arr, len(arr), stage.data_ptr(),
                                                           stage.numel(), _stream_ptr(stream)))
 
-    def get_many_host(self, plan: "Plan", hosts, stream=None):
-        """hosts: HostGetBuffers per request of the plan, or host_outs() of them."""
+    def get_many_host(self, plan: "Plan", hosts, stage=None, stream=None):
+        """hosts: HostGetBuffers per request of the plan, or host_outs() of them; stage: device
+        uint8 tensor of get_many_host_stage_bytes(plan) bytes, or None."""
         arr = hosts if isinstance(hosts, C.Array) else self.host_outs(hosts)
         _check("td_get_many_host", lib().td_get_many_host(self.handle, plan.handle, arr, len(arr),
+                                                          stage.data_ptr() if stage is not None else None,
+                                                          stage.numel() if stage is not None else 0,
                                                           _stream_ptr(stream)))
+
+    def get_many_host_stage_bytes(self, plan: "Plan") -> int:
+        return lib().td_get_many_host_stage_bytes(plan.handle)
 
     def get_host(self, bufs: GetBuffers, host: "HostGetBuffers", stream=None):
         _check("td_get_host", lib().td_get_host(self.handle, bufs.consumer, bufs.max_samples,

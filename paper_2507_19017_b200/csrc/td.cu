@@ -505,7 +505,7 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
     if (launch_finalize(d, 1u, one.req.max_groups * v.N, st, v, one, (const GetReq *)nullptr,
-               (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr) != cudaSuccess) return TD_ECUDA;
+               (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr, (uint8_t *)nullptr) != cudaSuccess) return TD_ECUDA;
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
     if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, jpr), st, v, one,
                      (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr, jpr, make_fastdiv(jpr),
@@ -584,7 +584,7 @@ int td_get_static(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
     if (launch_finalize(d, 1u, one.req.max_groups * v.N, st, v, one, (const GetReq *)nullptr,
-               (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr) != cudaSuccess) return TD_ECUDA;
+               (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr, (uint8_t *)nullptr) != cudaSuccess) return TD_ECUDA;
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
     if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, jpr), st, v, one,
                      (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr, jpr, make_fastdiv(jpr),
@@ -601,6 +601,8 @@ struct td_plan {
     uint64_t room_bytes;
     uint32_t jobs_per_req;                // columns, plus the stream's jobs when a request wants it
     uint32_t max_req_samples;             // the largest request, in samples
+    size_t meta_total;                    // bytes of the staging buffer td_get_many_host may be given
+    uint8_t *h_meta;                      // its pinned host mirror, allocated by the first call that uses it
     unsigned long long *d_counter;        // the gather's chunk counter: word 1 of slot 0's scan scratch
     JobSize *d_job_sizes;                 // [n_req][n_columns] output bytes and rows, written by the finalize kernel
     std::vector<uint8_t> host_image;      // what was uploaded; kept until the plan dies
@@ -631,6 +633,7 @@ int td_plan_create(td_dock *d, const td_get_req *reqs, uint32_t n_req, void *d_p
     td_plan *p = new (std::nothrow) td_plan();
     if (!p) return TD_EINVAL;
     p->dock = d; p->n_req = n_req; p->jobs_per_req = jpr;
+    p->meta_total = 0; p->h_meta = nullptr; p->max_req_samples = 0;
     const size_t off_slots = align_up_sz((size_t)n_req * sizeof(GetReq), 256);
     const size_t off_scratch = off_slots + align_up_sz((size_t)v.ncons * sizeof(ConsumerSlot), 256);
     const size_t scratch_each = align_up_sz(sel_scratch_bytes(v.G), 256);
@@ -660,6 +663,9 @@ int td_plan_create(td_dock *d, const td_get_req *reqs, uint32_t n_req, void *d_p
         hr[q].rank_base = cs.max_groups;
         hr[q].max_groups = m;
         hr[q].cslot = (uint32_t)slot_of[c];
+        hr[q].meta_samples = std::min(m, v.G) * v.N;
+        hr[q].meta_off = p->meta_total;
+        p->meta_total += align_up_sz(meta_bytes(hr[q].meta_samples), 16);
         const uint64_t sum = (uint64_t)cs.max_groups + m;
         cs.max_groups = sum > v.G ? v.G : (uint32_t)sum;
         if (hr[q].rank_base > v.G) hr[q].rank_base = v.G;
@@ -681,11 +687,19 @@ int td_plan_create(td_dock *d, const td_get_req *reqs, uint32_t n_req, void *d_p
 }
 
 int td_plan_destroy(td_plan *p) {
+    if (p && p->h_meta) cudaFreeHost(p->h_meta);
     delete p;
     return TD_OK;
 }
 
-int td_get_many(td_dock *d, td_plan *p, void *stream) {
+namespace {
+int get_many(td_dock *d, td_plan *p, uint8_t *d_meta, void *stream);
+}
+int td_get_many(td_dock *d, td_plan *p, void *stream) { return get_many(d, p, nullptr, stream); }
+
+namespace {
+// d_meta: staging buffer for the second copy of the requests' small outputs, or nullptr.
+int get_many(td_dock *d, td_plan *p, uint8_t *d_meta, void *stream) {
     if (!d || !p || p->dock != d) return TD_EINVAL;
     const DockView &v = d->dv;
     cudaStream_t st = (cudaStream_t)stream;
@@ -695,7 +709,7 @@ int td_get_many(td_dock *d, td_plan *p, void *stream) {
     if (launch_dep(d, get_select_kernel, dim3(sel_tiles(v.G), p->n_slots), dim3(kSelThreads), 0, st, v, none,
                (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
     if (launch_finalize(d, p->n_req, p->max_req_samples, st, v, none, (const GetReq *)p->d_reqs,
-               (const ConsumerSlot *)p->d_slots, seq, p->d_counter, p->d_job_sizes, p->jobs_per_req) != cudaSuccess) return TD_ECUDA;
+               (const ConsumerSlot *)p->d_slots, seq, p->d_counter, p->d_job_sizes, p->jobs_per_req, d_meta) != cudaSuccess) return TD_ECUDA;
     if (launch_timed(d, 1, get_gather_kernel, dim3(copy_grid(d, p->room_bytes)), dim3(kCopyThreads),
                      gather_smem_bytes(p->n_req, p->jobs_per_req), st, v, none,
                      (const GetReq *)p->d_reqs, p->n_req, p->d_counter, (const JobSize *)p->d_job_sizes,
@@ -703,6 +717,7 @@ int td_get_many(td_dock *d, td_plan *p, void *stream) {
                      p->n_slots) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
+}  // namespace
 
 int td_status(td_dock *d, td_stats *host_out, void *stream) {
     if (!d || !host_out) return TD_EINVAL;
@@ -853,21 +868,51 @@ int td_get_host(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_ge
     return TD_OK;
 }
 
-int td_get_many_host(td_dock *d, td_plan *p, const td_get_out *host_outs, uint32_t n_req, void *stream) {
+size_t td_get_many_host_stage_bytes(const td_plan *p) { return p ? p->meta_total : 0; }
+
+int td_get_many_host(td_dock *d, td_plan *p, const td_get_out *host_outs, uint32_t n_req, void *d_stage,
+                     size_t stage_bytes, void *stream) {
     if (!d || !p || p->dock != d || !host_outs || n_req != p->n_req) return TD_EINVAL;
     for (uint32_t q = 0; q < n_req; ++q)
         if (!host_outs[q].result || !host_outs[q].indices) return TD_EINVAL;
-    const int rc = td_get_many(d, p, stream);
-    if (rc != TD_OK) return rc;
+    if (d_stage && ((reinterpret_cast<uintptr_t>(d_stage) & 15u) || stage_bytes < p->meta_total)) return TD_EWORKSPACE;
     cudaStream_t st = (cudaStream_t)stream;
     const GetReq *reqs = reinterpret_cast<const GetReq *>(p->host_image.data());     // the plan as uploaded
-    for (uint32_t q = 0; q < n_req; ++q)
-        if (cudaMemcpyAsync(host_outs[q].result, reqs[q].out.result, sizeof(td_result), cudaMemcpyDeviceToHost, st) !=
-            cudaSuccess) return TD_ECUDA;
-    if (cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
-    for (uint32_t q = 0; q < n_req; ++q) {
-        const int rc2 = copy_batch_to_host(d->dv, reqs[q].consumer, &reqs[q].out, &host_outs[q], host_outs[q].result, st);
-        if (rc2 != TD_OK) return rc2;
+    if (d_stage && !p->h_meta &&
+        cudaHostAlloc(reinterpret_cast<void **>(&p->h_meta), p->meta_total, cudaHostAllocDefault) != cudaSuccess)
+        return TD_ECUDA;
+    const int rc = get_many(d, p, static_cast<uint8_t *>(d_stage), stream);
+    if (rc != TD_OK) return rc;
+    if (d_stage) {
+        // one transfer brings every request's result block, indices, cu_seqlens and advantages
+        if (cudaMemcpyAsync(p->h_meta, d_stage, p->meta_total, cudaMemcpyDeviceToHost, st) != cudaSuccess) return TD_ECUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
+        for (uint32_t q = 0; q < n_req; ++q) {
+            const MetaView mv = meta_view(p->h_meta + reqs[q].meta_off, reqs[q].meta_samples);
+            const td_get_out &h = host_outs[q];
+            *h.result = *mv.result;
+            const size_t n = mv.result->n_samples;
+            std::memcpy(h.indices, mv.indices, n * 4);
+            if (h.cu_prompt) std::memcpy(h.cu_prompt, mv.cu_prompt, (n + 1) * 4);
+            if (h.cu_response) std::memcpy(h.cu_response, mv.cu_response, (n + 1) * 4);
+            if (h.cu_seq) std::memcpy(h.cu_seq, mv.cu_seq, (n + 1) * 4);
+            if (h.advantages && (d->dv.cflags[reqs[q].consumer] & TD_F_ADVANTAGE))
+                std::memcpy(h.advantages, mv.advantages, n * 4);
+            td_get_out payload_only = h;      // what is left to copy from the device: the columns
+            payload_only.indices = nullptr; payload_only.cu_prompt = nullptr; payload_only.cu_response = nullptr;
+            payload_only.cu_seq = nullptr; payload_only.advantages = nullptr;
+            const int rc2 = copy_batch_to_host(d->dv, reqs[q].consumer, &reqs[q].out, &payload_only, h.result, st);
+            if (rc2 != TD_OK) return rc2;
+        }
+    } else {
+        for (uint32_t q = 0; q < n_req; ++q)
+            if (cudaMemcpyAsync(host_outs[q].result, reqs[q].out.result, sizeof(td_result), cudaMemcpyDeviceToHost, st) !=
+                cudaSuccess) return TD_ECUDA;
+        if (cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
+        for (uint32_t q = 0; q < n_req; ++q) {
+            const int rc2 = copy_batch_to_host(d->dv, reqs[q].consumer, &reqs[q].out, &host_outs[q], host_outs[q].result, st);
+            if (rc2 != TD_OK) return rc2;
+        }
     }
     if (cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
     return TD_OK;

@@ -57,7 +57,33 @@ struct GetReq {
     uint32_t max_groups;      // floor(max_samples / N)
     uint32_t rank_base;       // first candidate rank this request may take
     uint32_t cslot;
+    // Plans only: where, in a staging buffer that a call may bring along, a second copy of the
+    // request's small outputs goes, so that a caller with host buffers fetches those of all
+    // requests with one transfer.  Layout of the block: td_result, indices[m], cu_prompt[m+1],
+    // cu_response[m+1], cu_seq[m+1], advantages[m], m = meta_samples.
+    uint64_t meta_off;
+    uint32_t meta_samples;
+    uint32_t pad;
 };
+// Views into such a block.
+struct MetaView {
+    td_result *result;
+    int32_t *indices, *cu_prompt, *cu_response, *cu_seq;
+    float *advantages;
+};
+__host__ __device__ __forceinline__ size_t meta_bytes(uint32_t m) {
+    return sizeof(td_result) + ((size_t)m * 2 + 3 * ((size_t)m + 1)) * 4;
+}
+__host__ __device__ __forceinline__ MetaView meta_view(uint8_t *p, uint32_t m) {
+    MetaView v;
+    v.result = reinterpret_cast<td_result *>(p);
+    v.indices = reinterpret_cast<int32_t *>(p + sizeof(td_result));
+    v.cu_prompt = v.indices + m;
+    v.cu_response = v.cu_prompt + (m + 1);
+    v.cu_seq = v.cu_response + (m + 1);
+    v.advantages = reinterpret_cast<float *>(v.cu_seq + (m + 1));
+    return v;
+}
 struct ConsumerSlot {
     uint32_t consumer;
     uint32_t max_groups;      // over all requests of the call that name this consumer
@@ -267,7 +293,8 @@ template <int kThreads>
 __global__ void __launch_bounds__(kThreads)
 get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
                     const GetReq *reqs_dev, const ConsumerSlot *slots_dev, const uint32_t seq,
-                    unsigned long long *work_counter, JobSize *job_sizes, const uint32_t jobs_per_req) {
+                    unsigned long long *work_counter, JobSize *job_sizes, const uint32_t jobs_per_req,
+                    uint8_t *meta_base) {
     const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
     const ConsumerSlot *slots = slots_dev ? slots_dev : &one.cs;
     const GetReq &rq = reqs[blockIdx.x];
@@ -276,6 +303,8 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     const SelScratch sc = sel_scratch(cs.scratch, dv.G);
     const uint32_t c = rq.consumer, N = dv.N;
     const uint32_t tid = threadIdx.x;
+    const bool mirror = meta_base != nullptr;                    // the call brought a staging buffer along
+    const MetaView mv = meta_view(meta_base + rq.meta_off, rq.meta_samples);
     __shared__ uint64_t sh_a[kThreads / 32], sh_b[kThreads / 32];
     __shared__ uint32_t s_first_over;
     // the groups served, for the first kFinGroupsKept of them: later steps take a sample's index
@@ -310,6 +339,8 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
             const uint32_t p = n_grp + (uint32_t)inc - 1u;
             if (p < kFinGroupsKept) s_grp[p] = g;
             for (uint32_t j = 0; j < N; ++j) out.indices[(size_t)p * N + j] = g * (int32_t)N + (int32_t)j;
+            if (mirror)
+                for (uint32_t j = 0; j < N; ++j) mv.indices[(size_t)p * N + j] = g * (int32_t)N + (int32_t)j;
         }
         n_grp += (uint32_t)ta;
     }
@@ -327,6 +358,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
         s_first_over = 0xffffffffu;
         out.cu_prompt[0] = 0; out.cu_response[0] = 0;
         if (out.cu_seq) out.cu_seq[0] = 0;
+        if (mirror) { mv.cu_prompt[0] = 0; mv.cu_response[0] = 0; mv.cu_seq[0] = 0; }
     }
     // tightest room per length class over the wanted columns
     uint64_t room_tok[3] = {~0ull, ~0ull, ~0ull};      // packed: tokens; scalar slot [0]: samples
@@ -367,6 +399,10 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
             out.cu_prompt[i + 1] = (int32_t)cp;
             out.cu_response[i + 1] = (int32_t)cr;
             if (out.cu_seq) out.cu_seq[i + 1] = (int32_t)(cp + cr);
+            if (mirror) {
+                mv.cu_prompt[i + 1] = (int32_t)cp; mv.cu_response[i + 1] = (int32_t)cr;
+                mv.cu_seq[i + 1] = (int32_t)(cp + cr);
+            }
             bool over = (uint64_t)(i + 1) > room_tok[0];
             if (!padded) over |= cp > room_tok[TD_PROMPT] || cr > room_tok[TD_RESPONSE];
             else over |= (uint64_t)(i + 1) > room_rows || (want_p && lp > out.pad_prompt_to) ||
@@ -407,8 +443,11 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
             double ss = 0.0;
             for (uint32_t j = 0; j < N; ++j) { const double d = (double)r[j] - mean; ss += d * d; }
             const double sd = sqrt(ss / (double)N);
-            for (uint32_t j = 0; j < N; ++j)
-                out.advantages[(size_t)p * N + j] = (float)(((double)r[j] - mean) / (sd + dv.eps));
+            for (uint32_t j = 0; j < N; ++j) {
+                const float adv = (float)(((double)r[j] - mean) / (sd + dv.eps));
+                out.advantages[(size_t)p * N + j] = adv;
+                if (mirror) mv.advantages[(size_t)p * N + j] = adv;
+            }
         }
     }
     __syncthreads();
@@ -419,6 +458,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
         r.response_tokens = tot_r;
         r.status = status; r.reserved = 0;
         *out.result = r;
+        if (mirror) *mv.result = r;
         if (status & TD_ERR_LOOKBACK_TIMEOUT) atomicOr(dv.errword, TD_ERR_LOOKBACK_TIMEOUT);
         atomicAdd(&dv.counters[CNT_GOT_SAMPLES + c], (unsigned long long)n_s);
         atomicAdd(&dv.counters[CNT_GOT_TOKENS + c], (unsigned long long)(r.prompt_tokens + r.response_tokens));

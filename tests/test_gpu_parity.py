@@ -536,7 +536,7 @@ def test_host_buffer_calls_single_and_batched(G):
         t = torch.from_numpy(np.ascontiguousarray(a).view(np.int16) if a.dtype == np.uint16 else np.ascontiguousarray(a))
         return (t.view(torch.bfloat16) if a.dtype == np.uint16 else t).pin_memory()
 
-    for batched in (False, True):
+    for batched in (False, True, "staged"):
         o = H.make_oracle(w)
         g = G.GpuDock(w)
         items = []
@@ -553,7 +553,10 @@ def test_host_buffer_calls_single_and_batched(G):
             stage = torch.empty(sum(need), dtype=torch.uint8, device=g.device)
             g.dock.put_many_host(items, stage)
             plan = g.dock.plan(bufs)
-            g.dock.get_many_host(plan, hosts)
+            meta = None
+            if batched == "staged":       # results, indices, cu_seqlens and advantages of all requests in one transfer
+                meta = torch.empty(g.dock.get_many_host_stage_bytes(plan), dtype=torch.uint8, device=g.device)
+            g.dock.get_many_host(plan, hosts, meta)
         else:
             stage = torch.empty(max(need), dtype=torch.uint8, device=g.device)
             for c, i, cu, d in items:
