@@ -289,6 +289,34 @@ int td_status(td_dock *dock, td_stats *host_out, void *stream);
  *          5 consumed bits (index = consumer) | 6 arena or scalar store (index = column) */
 int td_debug_table(const td_dock *dock, int which, uint32_t index, void **d_ptr, size_t *bytes);
 
+/* Self-check of the dock's bookkeeping, for tests and for tracking down a misbehaving caller:
+ * synchronises `stream`, copies the tables to the host and tests what must hold between any two
+ * calls: a stored column implies a reserved row; the rows of a warehouse (the split of the buffer
+ * along the batch, "Distributed Transfer Dock Strategy") start on row boundaries, do not overlap
+ * and end below the shard's cursor, which stays within the capacity; status words carry no
+ * unknown bits; a sample marked served belongs to a claimed group and had every column its
+ * consumer needs; the per-column and per-consumer counters equal what the tables say.
+ * (While a get is in flight on another stream the claim of a group may be ahead of its served
+ * marks; that is not reported.)  violations = 0 means all hold; first_sample names a sample,
+ * shard, column or consumer of the first violation found. */
+enum {
+    TD_BAD_STORED_WITHOUT_ROW = 1u << 0,
+    TD_BAD_ROW_PLACEMENT      = 1u << 1,
+    TD_BAD_ROW_OVERLAP        = 1u << 2,
+    TD_BAD_STATUS_BITS        = 1u << 3,
+    TD_BAD_SERVED_UNCLAIMED   = 1u << 4,
+    TD_BAD_SERVED_NOT_READY   = 1u << 5,
+    TD_BAD_COUNTERS           = 1u << 6
+};
+typedef struct {
+    uint32_t violations, reserved;
+    uint64_t first_sample;
+    uint64_t stored[32];             /* per column: samples whose status carries its bit */
+    uint64_t served[32];             /* per consumer: samples marked served */
+    uint64_t arena_elems_used[3];    /* by length class: elements taken by rows, padding included */
+} td_validate_report;
+int td_debug_validate(td_dock *dock, void *stream, td_validate_report *report);
+
 /* Kernels this dock has launched since td_create. */
 uint64_t td_launch_count(const td_dock *dock);
 

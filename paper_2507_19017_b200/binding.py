@@ -20,6 +20,8 @@ F_ADVANTAGE = 1
 OK, EINVAL, EWORKSPACE, ECUDA, ETOOLARGE = 0, -1, -2, -3, -4
 ERR_OOB_INDEX, ERR_DUP_PUT, ERR_LEN_MISMATCH, ERR_ARENA_FULL = 1, 2, 4, 8
 ERR_OUT_TRUNCATED, ERR_LOOKBACK_TIMEOUT, ERR_BAD_LENGTH, ERR_COPY_TIMEOUT = 16, 32, 64, 128
+(BAD_STORED_WITHOUT_ROW, BAD_ROW_PLACEMENT, BAD_ROW_OVERLAP, BAD_STATUS_BITS, BAD_SERVED_UNCLAIMED,
+ BAD_SERVED_NOT_READY, BAD_COUNTERS) = 1, 2, 4, 8, 16, 32, 64          # td_debug_validate
 
 DTYPE_TAG = {"i32": I32, "f32": F32, "bf16": BF16}
 CLASS_TAG = {"scalar": SCALAR, "prompt": PROMPT, "response": RESPONSE}
@@ -31,7 +33,7 @@ EXPORTS = ["td_query_workspace", "td_create", "td_destroy", "td_put", "td_get",
            "td_launch_count", "td_strerror", "td_kernel_timing", "td_kernel_timing_read",
            "td_put_host_stage_bytes", "td_put_host", "td_get_host", "td_put_many",
            "td_plan_bytes", "td_plan_create", "td_plan_destroy", "td_get_many", "td_get_static",
-           "td_model_bytes", "td_put_back", "td_put_back_many", "td_put_many_host", "td_get_many_host", "td_get_many_host_stage_bytes"]
+           "td_model_bytes", "td_put_back", "td_put_back_many", "td_put_many_host", "td_get_many_host", "td_get_many_host_stage_bytes", "td_debug_validate"]
 
 
 class TdModel(C.Structure):
@@ -85,6 +87,11 @@ class TdBackItem(C.Structure):
 class TdBackReq(C.Structure):
     _fields_ = [("batch", C.c_void_p), ("max_samples", C.c_uint32), ("column", C.c_uint32),
                 ("d_data", C.c_void_p), ("data_elems", C.c_uint64)]
+
+
+class TdValidateReport(C.Structure):
+    _fields_ = [("violations", C.c_uint32), ("reserved", C.c_uint32), ("first_sample", C.c_uint64),
+                ("stored", C.c_uint64 * 32), ("served", C.c_uint64 * 32), ("arena_elems_used", C.c_uint64 * 3)]
 
 
 class TdGetReq(C.Structure):
@@ -168,6 +175,8 @@ def lib():
         L.td_get_many_host.argtypes = [vp, vp, C.POINTER(TdGetOut), u32, vp, C.c_size_t, vp]
         L.td_get_many_host_stage_bytes.restype = C.c_size_t
         L.td_get_many_host_stage_bytes.argtypes = [vp]
+        L.td_debug_validate.restype = C.c_int
+        L.td_debug_validate.argtypes = [vp, vp, C.POINTER(TdValidateReport)]
         L.td_plan_bytes.restype = C.c_size_t
         L.td_plan_bytes.argtypes = [vp, u32]
         L.td_plan_create.restype = C.c_int
@@ -523,6 +532,12 @@ class Dock:
         _check("td_debug_table", lib().td_debug_table(self.handle, which, index, C.byref(ptr), C.byref(nbytes)))
         off = ptr.value - self.workspace.data_ptr()
         return self.workspace[off:off + nbytes.value]
+
+    def validate(self, stream=None) -> TdValidateReport:
+        """Self-check of the dock's tables (synchronises the stream); report.violations == 0 if sound."""
+        rep = TdValidateReport()
+        _check("td_debug_validate", lib().td_debug_validate(self.handle, _stream_ptr(stream), C.byref(rep)))
+        return rep
 
     def launch_count(self) -> int:
         return lib().td_launch_count(self.handle)

@@ -764,6 +764,91 @@ int td_debug_table(const td_dock *d, int which, uint32_t index, void **d_ptr, si
 
 uint64_t td_launch_count(const td_dock *d) { return d ? d->launches.load() : 0; }
 
+// Self-check of the dock's bookkeeping: copies the tables to the host and tests what must hold
+// between any two calls, whatever was put or served.  Synchronises the stream.
+int td_debug_validate(td_dock *d, void *stream, td_validate_report *rep) {
+    if (!d || !rep) return TD_EINVAL;
+    std::memset(rep, 0, sizeof(*rep));
+    const DockView &v = d->dv;
+    cudaStream_t st = (cudaStream_t)stream;
+    const size_t n = v.n;
+    std::vector<uint32_t> status(n), claim((size_t)v.ncons * v.claim_words), consumed((size_t)v.ncons * v.consumed_words);
+    std::vector<int32_t> len[3];
+    std::vector<long long> off[3];
+    std::vector<unsigned long long> cursor[3], counters(CNT_TOTAL);
+    auto d2h = [&](void *dst, const void *src, size_t bytes) {
+        return bytes == 0 || cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+    };
+    bool ok = d2h(status.data(), v.status, n * 4) && d2h(claim.data(), v.claim, claim.size() * 4) &&
+              d2h(consumed.data(), v.consumed, consumed.size() * 4) && d2h(counters.data(), v.counters, CNT_TOTAL * 8);
+    for (int L = 1; L <= 2 && ok; ++L) {
+        len[L].resize(n); off[L].resize(n); cursor[L].resize(v.S);
+        ok = d2h(len[L].data(), v.len[L], n * 4) && d2h(off[L].data(), v.off[L], n * 8) &&
+             d2h(cursor[L].data(), v.cursor[L], (size_t)v.S * 8);
+    }
+    if (!ok || cudaStreamSynchronize(st) != cudaSuccess) return TD_ECUDA;
+
+    auto fail = [&](uint32_t bit, uint64_t sample) {
+        if (!rep->violations) rep->first_sample = sample;
+        rep->violations |= bit;
+    };
+    uint32_t ragged_mask[3] = {0, 0, 0}, all_mask = 0;
+    for (uint32_t k = 0; k < v.ncol; ++k) { ragged_mask[v.col_cls[k]] |= 1u << k; all_mask |= 1u << k; }
+    const uint32_t per_shard = v.N * v.prompts_per_shard;
+    for (int L = 1; L <= 2; ++L) {
+        // rows of a shard, sorted by where they start, must not overlap and must end below the cursor
+        std::vector<std::vector<std::pair<long long, long long>>> rows(v.S);
+        for (size_t s = 0; s < n; ++s) {
+            const bool has_len = len[L][s] >= 0, has_off = off[L][s] >= 0;
+            if ((status[s] & ragged_mask[L]) && !(has_len && has_off)) fail(TD_BAD_STORED_WITHOUT_ROW, s);
+            if (has_off && !has_len) fail(TD_BAD_STORED_WITHOUT_ROW, s);
+            if (has_len && has_off) {
+                const long long room = ((long long)len[L][s] + (kRowAlign - 1)) / kRowAlign * kRowAlign;
+                rows[s / per_shard].emplace_back(off[L][s], off[L][s] + room);
+                if ((off[L][s] % kRowAlign) != 0) fail(TD_BAD_ROW_PLACEMENT, s);
+            }
+        }
+        for (uint32_t sh = 0; sh < v.S; ++sh) {
+            auto &r = rows[sh];
+            std::sort(r.begin(), r.end());
+            long long end = 0, used = 0;
+            for (auto &iv : r) {
+                if (iv.first < end && iv.second > iv.first) fail(TD_BAD_ROW_OVERLAP, sh);
+                end = std::max(end, iv.second);
+                used += iv.second - iv.first;
+            }
+            if ((unsigned long long)end > cursor[L][sh] || cursor[L][sh] > v.cap[L]) fail(TD_BAD_ROW_PLACEMENT, sh);
+            rep->arena_elems_used[L] += (uint64_t)used;
+        }
+    }
+    for (size_t s = 0; s < n; ++s)
+        if (status[s] & ~all_mask) fail(TD_BAD_STATUS_BITS, s);
+    for (uint32_t k = 0; k < v.ncol; ++k) {
+        uint64_t have = 0;
+        for (size_t s = 0; s < n; ++s) have += (status[s] >> k) & 1u;
+        if (have != counters[CNT_PUT_ACCEPTED + k]) fail(TD_BAD_COUNTERS, k);
+        rep->stored[k] = have;
+    }
+    for (uint32_t c = 0; c < v.ncons; ++c) {
+        const uint32_t *cl = &claim[(size_t)c * v.claim_words], *co = &consumed[(size_t)c * v.consumed_words];
+        uint64_t served = 0;
+        for (uint32_t g = 0; g < v.G; ++g) {
+            const bool claimed = (cl[g >> 5] >> (g & 31)) & 1u;
+            for (uint32_t j = 0; j < v.N; ++j) {
+                const size_t s = (size_t)g * v.N + j;
+                const bool done = (co[s >> 5] >> (s & 31)) & 1u;
+                served += done;
+                if (done && !claimed) fail(TD_BAD_SERVED_UNCLAIMED, s);
+                // a sample that was served had everything its consumer needs
+                if (done && (status[s] & v.need[c]) != v.need[c]) fail(TD_BAD_SERVED_NOT_READY, s);
+            }
+        }
+        if (served != counters[CNT_GOT_SAMPLES + c]) fail(TD_BAD_COUNTERS, c);
+        rep->served[c] = served;
+    }
+    return TD_OK;
+}
+
 int td_kernel_timing(td_dock *d, int enable) {
     if (!d) return TD_EINVAL;
     drop_timing(d);

@@ -159,6 +159,8 @@ def _same(got: np.ndarray, want: np.ndarray, what: str):
 
 def assert_state_equal(g: GpuDock, o: ora.OracleDock, arenas: bool = True, ctx=""):
     w = g.w
+    rep = g.dock.validate()
+    assert rep.violations == 0, f"{ctx} td_debug_validate: {rep.violations:#x} at {rep.first_sample}"
     _same(g.table(0, 0, np.uint32), o.status(), ctx + " status")
     for cls in (1, 2):
         _same(g.table(1, cls, np.int32), o.lengths(cls), ctx + f" len[{cls}]")

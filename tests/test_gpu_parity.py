@@ -570,6 +570,35 @@ def test_host_buffer_calls_single_and_batched(G):
         G.assert_state_equal(g, o, ctx=f"host batched={batched}")
 
 
+def test_validate_reports_planted_damage(G):
+    """td_debug_validate passes on a dock in use and names damage planted into its tables from
+    the host side (an unknown status bit, two rows at one place, a served mark without a claim)."""
+    import torch
+    w = wl.make_custom("validate", 8, 2, 2, prompt_len=(3, 30), response=("uniform", 1, 60), vocab=500,
+                       micro_batch=4, seed=61, schedule="bulk")
+    g, o, _ = G.replay_both(w)
+    rep = g.dock.validate()
+    assert rep.violations == 0
+    assert list(rep.stored[:len(w.columns)]) == [w.n] * len(w.columns)
+    assert list(rep.served[:len(w.consumers)]) == [w.n] * len(w.consumers)
+    used = int(((w.len_response.astype(np.int64) + 7) // 8 * 8).sum())
+    assert rep.arena_elems_used[2] == used
+    status = g.dock.table(0).view(torch.int32)
+    status[3] |= 1 << 20
+    assert g.dock.validate().violations & td.BAD_STATUS_BITS
+    status[3] &= ~(1 << 20)
+    off = g.dock.table(2, 2).view(torch.int64)
+    keep = off[1].item()
+    off[1] = off[0]
+    assert g.dock.validate().violations & td.BAD_ROW_OVERLAP
+    off[1] = keep
+    claim = g.dock.table(4, 1).view(torch.int32)
+    claim[0] &= ~1
+    assert g.dock.validate().violations & td.BAD_SERVED_UNCLAIMED
+    claim[0] |= 1
+    assert g.dock.validate().violations == 0
+
+
 def test_host_argument_checks(G):
     w = wl.make_config(1)
     g = G.GpuDock(w)
