@@ -49,6 +49,9 @@ def parse_args():
     ap.add_argument("--fused", action="store_true",
                     help="the actor update's gets also ask for the fused prompt+response id stream and "
                          "its per-token advantage twin")
+    ap.add_argument("--padded", action="store_true",
+                    help="gets write right-padded rows (row i at i * width, the column's pad bits behind it) "
+                         "instead of packed ones; widths are the workload's maximum lengths")
     ap.add_argument("--graph", action="store_true",
                     help="cascade only: capture the step's calls into one CUDA graph once and time its replay "
                          "(nothing in the step needs the host, batch sizes are read on the device)")
@@ -238,7 +241,7 @@ def algorithmic_bytes(w):
 class GpuStep:
     """Device-resident inputs and per-get output buffers of one step, and the step itself."""
 
-    def __init__(self, w, device_index: int, api: str = "many", fused: bool = False):
+    def __init__(self, w, device_index: int, api: str = "many", fused: bool = False, padded: bool = False):
         import torch
         self.api = api
         from paper_2507_19017_b200 import binding as td
@@ -283,7 +286,8 @@ class GpuStep:
                 continue
             m = op.max_samples
             stream = fused and w.consumers[op.consumer].advantage
-            bufs = td.GetBuffers(self.dock, op.consumer, m, td.PACKED,
+            bufs = td.GetBuffers(self.dock, op.consumer, m, td.PADDED if padded else td.PACKED,
+                                 w.pad_prompt_to if padded else 0, w.pad_response_to if padded else 0,
                                  prompt_tokens_cap=int(lp[:m].sum(dtype=np.int64)),
                                  response_tokens_cap=int(lr[:m].sum(dtype=np.int64)),
                                  seq=(w.column_index("prompt_ids"), w.column_index("response_ids")) if stream else None,
@@ -659,13 +663,24 @@ def main():
             dist.destroy_process_group()
         return
 
-    step = GpuStep(w, local_rank, args.api, args.fused)
+    step = GpuStep(w, local_rank, args.api, args.fused, args.padded)
+    if args.padded:
+        config["output"] = f"right-padded rows, widths {w.pad_prompt_to} / {w.pad_response_to}"
     if args.fused:
         config["fused_stream"] = "actor-update gets also write the prompt+response id stream and its advantage twin"
     config["api"] = ("td_put_many + td_get_many (one call each per step)" if args.api == "many"
                      else "td_put per column + td_get per micro-batch")
     peak, peak_kind = load_peaks()
     put_bytes, put_ragged_bytes, get_bytes = algorithmic_bytes(w)
+    if args.padded:      # the pad writes are part of what this mode must move
+        from paper_2507_19017_b200 import workloads as wl_
+        for k in w.consumers:
+            for name in k.out:
+                spec = w.columns[w.column_index(name)]
+                if spec.cls != wl_.SCALAR:
+                    width = w.pad_prompt_to if spec.cls == wl_.PROMPT else w.pad_response_to
+                    get_bytes += (w.n * width * w.data[name].itemsize) - w.data[name].nbytes
+
     if args.fused:       # the stream: both id columns read and written once more; the twin: one float written per token
         get_bytes += 2 * (w.data["prompt_ids"].nbytes + w.data["response_ids"].nbytes) + 4 * w.tokens_total()
 
@@ -718,12 +733,12 @@ def main():
         k["GBps"] = k["bytes_per_launch"] / (k["avg_ms"] * 1e-3) / 1e9 if k["avg_ms"] > 0 else 0.0
     dom = "get_gather" if ms_ga >= ms_sc else "put_scatter"
     roofline = {"bound": "hbm", "kernel": dom, "achieved": kern[dom]["GBps"], "peak": peak, "unit": "GB/s",
-                "frac": kern[dom]["GBps"] / peak, "traffic": None if args.fused else NCU_TRAFFIC.get((args.config, dom)),
+                "frac": kern[dom]["GBps"] / peak, "traffic": None if (args.fused or args.padded) else NCU_TRAFFIC.get((args.config, dom)),
                 "peak_kind": peak_kind,
                 "bytes_per_launch": kern[dom]["bytes_per_launch"], "avg_launch_ms": kern[dom]["avg_ms"]}
 
     e2e = None
-    if not args.no_e2e:
+    if not args.no_e2e and not args.padded:
         e2e_s, d2h = step.run_e2e(min(args.steps, 5), 1)
         e2e_s, = max_over_ranks(dist, [e2e_s], step.dev)
         e2e = {"value": whole_job_rate(world, n_dispatch, e2e_s), "unit": "samples/s", "ms_per_step": e2e_s * 1e3,
