@@ -245,7 +245,6 @@ int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **o
     v.ncol = cfg->n_columns; v.ncons = cfg->n_consumers;
     v.prompts_per_shard = v.G / v.S;
     v.div_shard = make_fastdiv(v.N * v.prompts_per_shard);
-    v.div_ncol = make_fastdiv(v.ncol);
     v.reward_col = cfg->reward_column;
     v.claim_words = L.claim_words; v.consumed_words = L.consumed_words;
     v.spin_limit = 1u << 20;

@@ -49,7 +49,6 @@ struct DockView {
     uint32_t prompts_per_shard;
     uint32_t reward_col;
     FastDiv  div_shard;                     // by samples per shard = N * prompts_per_shard
-    FastDiv  div_ncol;                      // by ncol
     uint32_t claim_words, consumed_words;   // words per consumer
     uint32_t spin_limit;                    // polls before a look-back wait gives up
     uint32_t pad0;

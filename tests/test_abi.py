@@ -96,6 +96,13 @@ def test_create_reports_workspace_and_argument_errors_before_any_cuda_call(td):
     assert td.lib().td_get(None, 0, 8, None, None) == td.EINVAL
     assert td.lib().td_launch_count(None) == 0
     assert td.lib().td_put_back(None, None, 8, None, 0, None) == td.EINVAL
+    assert td.lib().td_put_back_many(None, None, 0, None) == td.EINVAL
+    assert td.lib().td_get_many(None, None, None) == td.EINVAL
+    assert td.lib().td_get_many_host(None, None, None, 0, None, 0, None) == td.EINVAL
+    assert td.lib().td_put_many_host(None, None, 0, None, 0, None) == td.EINVAL
+    assert td.lib().td_get_many_host_stage_bytes(None) == 0
+    rep = td.TdValidateReport()
+    assert td.lib().td_debug_validate(None, None, C.byref(rep)) == td.EINVAL
 
 
 def test_create_fails_loudly_without_a_device(td):
