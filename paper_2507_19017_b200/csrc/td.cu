@@ -24,6 +24,8 @@ struct td_dock {
     size_t ws_bytes;
     size_t table_bytes[7];
     std::atomic<uint64_t> launches;
+    std::mutex slot_mu;
+    std::vector<cudaStream_t> slot_stream;     // which stream draws from which scatter chunk counter
     // optional per-kernel timing of the two copy kernels (0 = put scatter, 1 = get gather)
     std::atomic<bool> timing;
     std::mutex timing_mu;
@@ -46,7 +48,7 @@ size_t gather_smem_bytes(uint32_t n_req, uint32_t jobs_per_req) {
 }
 
 struct Layout {
-    size_t status, len[3], off[3], cursor[3], claim, consumed, errword, counters, col[kMaxColumns], total;
+    size_t status, len[3], off[3], cursor[3], claim, consumed, errword, counters, put_counters, col[kMaxColumns], total;
     uint32_t claim_words, consumed_words;
     uint64_t cap[3];
 };
@@ -88,6 +90,7 @@ Layout make_layout(const td_config *c) {
     auto take = [&](size_t bytes) { size_t at = p; p = align_up_sz(p + bytes, 256); return at; };
     L.errword = take(256);
     L.counters = take(CNT_TOTAL * 8);
+    L.put_counters = take((size_t)kPutCounterSlots * 8);
     L.status = take(n * 4);
     for (int k = 1; k <= 2; ++k) { L.len[k] = take(n * 4); L.off[k] = take(n * 8); L.cursor[k] = take(S * 8); }
     L.claim = take((size_t)c->n_consumers * L.claim_words * 4);
@@ -261,6 +264,7 @@ int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **o
     v.consumed = reinterpret_cast<uint32_t *>(w + L.consumed);
     v.errword = reinterpret_cast<uint32_t *>(w + L.errword);
     v.counters = reinterpret_cast<unsigned long long *>(w + L.counters);
+    v.put_counters = reinterpret_cast<unsigned long long *>(w + L.put_counters);
     for (uint32_t k = 0; k < v.ncol; ++k) {
         v.colbase[k] = w + L.col[k];
         v.col_esz[k] = (uint8_t)esize_of(cfg->columns[k].dtype);
@@ -309,6 +313,24 @@ uint32_t copy_grid(const td_dock *d, uint64_t room_bytes) {
     return (uint32_t)blocks;
 }
 
+// The chunk counter the scatter kernel of a call on stream `st` may draw from, or nullptr.  Calls
+// on one stream run one after the other, so a counter per stream is never shared by two launches
+// in flight.  A call that is being captured into a graph gets none: the graph may later run on
+// any stream, beside anything.
+unsigned long long *scatter_counter(td_dock *d, cudaStream_t st) {
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) {
+        cudaGetLastError();
+        return nullptr;
+    }
+    std::lock_guard<std::mutex> lk(d->slot_mu);
+    for (size_t i = 0; i < d->slot_stream.size(); ++i)
+        if (d->slot_stream[i] == st) return d->dv.put_counters + i;
+    if (d->slot_stream.size() >= (size_t)kPutCounterSlots) return nullptr;
+    d->slot_stream.push_back(st);
+    return d->dv.put_counters + (d->slot_stream.size() - 1);
+}
+
 // One launch group: alloc (if any ragged item), scatter, publish.  Items are taken in order;
 // a column appears at most once per group, so that duplicate detection sees earlier items.
 int put_group(td_dock *d, PutBatch &b, cudaStream_t st) {
@@ -336,6 +358,7 @@ int put_group(td_dock *d, PutBatch &b, cudaStream_t st) {
     }
     if (entries == 0) return TD_OK;
     if (entries >= (1ull << 32)) return TD_EINVAL;
+    b.work_counter = ragged_bytes ? scatter_counter(d, st) : nullptr;
     if (ragged_bytes) {
         if (launch_dep(d, put_alloc_kernel, dim3(2), dim3(kAllocThreads), put_alloc_smem_bytes(v.S), st, v, b) != cudaSuccess)
             return TD_ECUDA;

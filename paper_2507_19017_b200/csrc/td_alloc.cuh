@@ -36,6 +36,10 @@ struct PutBatch {                              // the columns of one call, in ca
     // ride along with in the alloc kernel (same entry count, not more data behind it), 0 = none.
     // The host only proposes; the kernel checks that the index and cu arrays are equal.
     uint8_t follow[kMaxPutItems];
+    // A counter in the dock's workspace from which the scatter kernel hands out its chunks, private
+    // to the stream the call was made on (calls on one stream run one after the other); nullptr:
+    // every warp takes a fixed share instead.  Zeroed by the alloc kernel.
+    unsigned long long *work_counter;
 };
 
 static inline size_t put_alloc_smem_bytes(uint32_t S) {
@@ -132,6 +136,7 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
     // kernel in the stream (a reset, the get whose batch is sent back, the caller's own producer)
     // must have finished.  The prefetch above only asked for lines.
     griddep_wait();
+    if (blockIdx.x == 0 && tid == 0 && batch.work_counter) *batch.work_counter = 0;
 
     // Which proposed followers really repeat their leader's index and cu arrays?
     if (tid == 0) s_not_following = 0;

@@ -9,6 +9,7 @@
 namespace td {
 
 constexpr int kMaxColumns = 32;
+constexpr int kPutCounterSlots = 64;         // streams that can put into a dock with chunks handed out by a counter
 constexpr uint32_t kRowAlign = 8;            // rows start on multiples of 8 elements (>= 16 bytes)
 constexpr uint32_t kFullMask = 0xffffffffu;
 
@@ -62,6 +63,7 @@ struct DockView {
     uint32_t *consumed;                     // [ncons][consumed_words]
     uint32_t *errword;
     unsigned long long *counters;           // [CNT_TOTAL]
+    unsigned long long *put_counters;       // [kPutCounterSlots] chunk counters of the scatter kernel, one per stream in use
     uint8_t  *colbase[kMaxColumns];         // arena (S * cap * esz) or scalar store (n * esz)
     uint32_t need[kMaxColumns];             // per consumer
     uint32_t outm[kMaxColumns];

@@ -67,10 +67,20 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
     }
     __syncthreads();
     const uint64_t n_warps = (uint64_t)gridDim.x * kCopyWarps;
-    const ChunkPlan plan = plan_chunks(item_end[batch.n_items - 1], n_warps);
-    const uint64_t warp0 = (uint64_t)blockIdx.x * kCopyWarps + (tid >> 5);
+    // With plenty to do (a full-size chunk and more per warp) and a counter to draw from, the
+    // chunks after a warp's first are handed out one by one: equal bytes are not equal time, and
+    // some SMs get through theirs sooner than others.  Otherwise every warp takes a fixed share.
+    const uint64_t total = item_end[batch.n_items - 1];
+    unsigned long long *work_counter = total >= n_warps * (uint64_t)kChunkTargetBytes ? batch.work_counter : nullptr;
+    const ChunkPlan plan = work_counter ? plan_chunks_dynamic(total, n_warps) : plan_chunks(total, n_warps);
+    unsigned long long ch = (uint64_t)blockIdx.x * kCopyWarps + (tid >> 5);
 
-    for (uint64_t ch = warp0; ch < plan.n_chunks; ch += n_warps) {
+    while (ch < plan.n_chunks) {
+        unsigned long long next = ch + n_warps;
+        if (work_counter) {
+            if (lane == 0) next = n_warps + atomicAdd(work_counter, 1ull);    // in flight while this chunk is copied
+            // (handed to the other lanes at the end of the loop body)
+        }
         uint64_t g0 = ch * plan.chunk_bytes;
         const uint64_t g1 = min(g0 + plan.chunk_bytes, item_end[batch.n_items - 1]);
         uint32_t it = 0;
@@ -104,6 +114,7 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
                                        return arena + ((uint64_t)shard_of(dv, (uint32_t)s) * cap + (uint64_t)off) * esz;
                                    });
         }
+        ch = work_counter ? shfl_u64(next, 0) : next;
     }
     if (pipe.finish(lane) && lane == 0) flag_error(dv, TD_ERR_COPY_TIMEOUT, CNT_TIMEOUT);
 }
