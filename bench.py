@@ -258,6 +258,7 @@ class GpuStep:
         # A worker that sends a whole record has one index array for the batch and one cu array
         # per length class: columns with equal arrays share them, on the host and on the device.
         shared = {}
+        counted = set()
 
         def share(a):
             key = (a.dtype.str, a.shape, a.tobytes())
@@ -276,7 +277,12 @@ class GpuStep:
             h_data = self._pin(data)
             self.host_puts.append((op.column, h_idx, h_cu, h_data))
             self.puts.append((op.column, d_idx, d_cu, h_data.to(self.dev)))
-            self.h2d_bytes += idx.nbytes + (cu.nbytes if cu is not None else 0) + data.nbytes
+            # the batched host call brings a shared array over once, the per-column call every time
+            for h, arr in ((h_idx, idx), (h_cu, cu)):
+                if arr is not None and not (api == "many" and h.data_ptr() in counted):
+                    self.h2d_bytes += arr.nbytes
+                    counted.add(h.data_ptr())
+            self.h2d_bytes += data.nbytes
         # one output buffer set per get call, sized by the longest rows it could meet
         lp = np.sort(w.len_prompt)[::-1]
         lr = np.sort(w.len_response)[::-1]

@@ -1047,8 +1047,17 @@ int td_put_many_host(td_dock *d, const td_put_item *h_items, uint32_t n_items, v
         uint8_t *d_dat = reinterpret_cast<uint8_t *>(d_cu) + align_up_sz(((size_t)h.k + 1) * 4, 256);
         used += need;
         const size_t esz = d->dv.col_esz[h.column];
-        if (cudaMemcpyAsync(d_idx, h.d_indices, (size_t)h.k * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TD_ECUDA;
-        if (ragged && cudaMemcpyAsync(d_cu, h.d_cu, ((size_t)h.k + 1) * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
+        // the columns of a record share their index array and, within a length class, their cu
+        // array: what an earlier item of the call already brought over is used again
+        for (uint32_t e = 0; e < i; ++e) {
+            if (h_items[e].k != h.k) continue;
+            if (h_items[e].d_indices == h.d_indices) d_idx = const_cast<int32_t *>(dev[e].d_indices);
+            if (ragged && h_items[e].d_cu == h.d_cu && dev[e].d_cu) d_cu = const_cast<int32_t *>(dev[e].d_cu);
+        }
+        if (d_idx == reinterpret_cast<int32_t *>(p + used - need) &&
+            cudaMemcpyAsync(d_idx, h.d_indices, (size_t)h.k * 4, cudaMemcpyHostToDevice, st) != cudaSuccess) return TD_ECUDA;
+        if (ragged && d_cu == reinterpret_cast<int32_t *>(p + used - need + align_up_sz((size_t)h.k * 4, 256)) &&
+            cudaMemcpyAsync(d_cu, h.d_cu, ((size_t)h.k + 1) * 4, cudaMemcpyHostToDevice, st) != cudaSuccess)
             return TD_ECUDA;
         if (h.data_elems && cudaMemcpyAsync(d_dat, h.d_data, (size_t)h.data_elems * esz, cudaMemcpyHostToDevice, st) !=
             cudaSuccess) return TD_ECUDA;
