@@ -349,7 +349,8 @@ int td_get_host(td_dock *dock, uint32_t consumer, uint32_t max_samples, const td
  * td_put_many_host: td_put_many whose items' three pointers (named d_* in td_put_item) are HOST
  * arrays here; they are copied, item after item, into d_stage (device, 256-byte aligned, at
  * least the sum of td_put_host_stage_bytes() over the items, not reused until the put has
- * executed) and put from there with one td_put_many.
+ * executed) and put from there with one td_put_many; an index or cu array that several items
+ * of the call name (same host pointer, same k) is brought over once.
  * td_get_many_host: td_get_many on `plan`, then the valid part of every request's buffers is
  * copied to the matching HOST pointers of host_outs[r] (one entry per request of the plan, in
  * plan order; result and indices required, NULL elsewhere = skip).  All result blocks are
