@@ -55,7 +55,7 @@ def parse_args():
     ap.add_argument("--graph", action="store_true",
                     help="cascade only: capture the step's calls into one CUDA graph once and time its replay "
                          "(nothing in the step needs the host, batch sizes are read on the device)")
-    ap.add_argument("--scenario", default="dispatch", choices=["dispatch", "cascade"],
+    ap.add_argument("--scenario", default="dispatch", choices=["dispatch", "cascade", "scan"],
                     help="dispatch: put everything, then drain (the headline); cascade: generation puts in "
                          "chunks, inference states get a micro-batch and send their column back for it "
                          "(td_put_back, no host round trip), the actor update takes what is complete")
@@ -495,6 +495,57 @@ class CascadeStep:
         return {self.w.columns[c].name: int(st.put_accepted[c]) for c in self.w.pool}
 
 
+def run_scan(args, local_rank):
+    """Readiness scan at sizes where bytes, not latency, bound it: docks of 2^20 .. 2^24 samples
+    that hold only the scalar reward, one consumer that needs just that.  Times a get of one
+    micro-batch (every group's status words are read, the lowest ready groups are served) with
+    every sample ready and with none ready, and prints one JSON line."""
+    import torch
+    from paper_2507_19017_b200 import binding as td
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    peak, peak_kind = load_peaks()
+    flush = torch.empty(L2_FLUSH_BYTES, dtype=torch.uint8, device=dev)
+    N = 16
+    rows = []
+    for log_n in (20, 22, 24):
+        n = 1 << log_n
+        G = n // N
+        dock = td.Dock(G, N, 16, [("i32", "prompt", 0), ("i32", "response", 0), ("f32", "scalar", 0)],
+                       [(4, 4, True)], 64, 64, 2, 1e-6, local_rank)
+        idx = torch.arange(n, dtype=torch.int32, device=dev)
+        rew = torch.randn(n, dtype=torch.float32, device=dev)
+        bufs = td.GetBuffers(dock, 0, 128, td.PACKED, prompt_tokens_cap=8, response_tokens_cap=8)
+
+        def timed_get():
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            flush.zero_()
+            e0.record(); dock.get(bufs); e1.record()
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1)
+
+        empty = min(timed_get() for _ in range(max(args.warmup, 3) + 5))
+        assert bufs.read_result().n_samples == 0
+        dock.put(2, idx, None, rew)
+        ready, served = [], 0
+        for _ in range(max(args.warmup, 3) + 5):
+            ready.append(timed_get())
+            r = bufs.read_result()
+            assert r.n_samples == 128 and r.status == 0
+            served += r.n_samples
+        scan_bytes = n * 4 + G // 8                     # status words + claim bits
+        rows.append({"samples": n, "groups": G, "tiles": -(-G // (256 * (4 if G > 65536 else 1))), "status_MB": scan_bytes / 1e6,
+                     "get_us_none_ready": empty * 1e3, "get_us_all_ready": min(ready) * 1e3,
+                     "scan_GBps_all_ready": scan_bytes / (min(ready) * 1e-3) / 1e9,
+                     "frac_of_peak": scan_bytes / (min(ready) * 1e-3) / 1e9 / peak})
+        assert dock.status().error_word == 0
+        dock.close()
+        del dock, idx, rew, bufs
+        torch.cuda.empty_cache()
+    print(json.dumps({"metric": "td_get readiness scan", "unit": "us per get of 128 samples (select + finalize + gather)",
+                      "peak_GBps": peak, "peak_kind": peak_kind, "l2": "flushed before each get", "sizes": rows}))
+
+
 def run_cascade(args, w, local_rank, world, dist, config):
     """Times the cascade scenario and prints its JSON line (rank 0)."""
     import torch
@@ -663,6 +714,12 @@ def main():
         torch.cuda.set_device(local_rank)
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
 
+    if args.scenario == "scan":
+        if rank == 0:
+            run_scan(args, local_rank)
+        if dist is not None:
+            dist.destroy_process_group()
+        return
     if args.scenario == "cascade":
         run_cascade(args, w, local_rank, world, dist, config)
         if dist is not None:

@@ -147,6 +147,18 @@ cudaError_t launch_timed(td_dock *d, int which, void (*kernel)(KArgs...), dim3 g
     return rc;
 }
 
+// Select of a launch over n_slots consumer slots: tiles of one or of several passes, by the
+// dock's size.
+template <typename... Args>
+cudaError_t launch_select(td_dock *d, uint32_t n_slots, cudaStream_t st, Args &&...args) {
+    const uint32_t G = d->dv.G;
+    if (sel_passes(G) > 1)
+        return launch_dep(d, get_select_kernel<(int)kSelWide>, dim3(sel_tiles(G), n_slots), dim3(kSelThreads), 0, st,
+                          std::forward<Args>(args)...);
+    return launch_dep(d, get_select_kernel<1>, dim3(sel_tiles(G), n_slots), dim3(kSelThreads), 0, st,
+                      std::forward<Args>(args)...);
+}
+
 // Finalize of a launch whose largest request may serve up to max_samples samples: one CTA per
 // request, a large block when a request is large (its scans then take a quarter of the rounds).
 template <typename... Args>
@@ -522,7 +534,7 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
     const uint32_t jpr = jobs_per_req(v, wants_stream(*out));
 
-    if (launch_dep(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
+    if (launch_select(d, 1u, st, v, one,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
@@ -601,7 +613,7 @@ int td_get_static(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
     const uint32_t jpr = jobs_per_req(v, wants_stream(*out));
 
-    if (launch_dep(d, get_select_kernel, dim3(sel_tiles(v.G), 1), dim3(kSelThreads), 0, st, v, one,
+    if (launch_select(d, 1u, st, v, one,
                (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
@@ -728,7 +740,7 @@ int get_many(td_dock *d, td_plan *p, uint8_t *d_meta, void *stream) {
     GetInline none;
     std::memset(&none, 0, sizeof(none));
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
-    if (launch_dep(d, get_select_kernel, dim3(sel_tiles(v.G), p->n_slots), dim3(kSelThreads), 0, st, v, none,
+    if (launch_select(d, p->n_slots, st, v, none,
                (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
     if (launch_finalize(d, p->n_req, p->max_req_samples, st, v, none, (const GetReq *)p->d_reqs,
                (const ConsumerSlot *)p->d_slots, seq, p->d_counter, p->d_job_sizes, p->jobs_per_req, d_meta) != cudaSuccess) return TD_ECUDA;

@@ -37,7 +37,15 @@ struct SelScratch {
     unsigned long long *desc;
     int32_t *cand;
 };
-__host__ __device__ __forceinline__ uint32_t sel_tiles(uint32_t G) { return (G + kSelThreads - 1) / kSelThreads; }
+// A tile is 256 groups per pass; a dock of more than kSelWideFrom groups gives every tile
+// kSelWide passes (the tiles' tickets and descriptors are a serial chain: about 10 ns per tile,
+// which outweighs the status words once there are thousands of tiles).
+constexpr uint32_t kSelWide = 4, kSelWideFrom = 65536;
+__host__ __device__ __forceinline__ uint32_t sel_passes(uint32_t G) { return G > kSelWideFrom ? kSelWide : 1u; }
+__host__ __device__ __forceinline__ uint32_t sel_tiles(uint32_t G) {
+    const uint32_t per = kSelThreads * sel_passes(G);
+    return (G + per - 1) / per;
+}
 __host__ __device__ __forceinline__ size_t sel_scratch_bytes(uint32_t G) {
     size_t b = (2 + (size_t)sel_tiles(G)) * 8 + (size_t)G * 4;
     return (b + 15) & ~size_t(15);
@@ -105,6 +113,7 @@ struct GetInline {            // a single get travels in the kernel parameters
 // warp.  Tiles take their number from a ticket, so a tile only ever waits for tiles that have
 // already started; the wait is bounded all the same.
 // ---------------------------------------------------------------------------------------------
+template <int kPasses>
 __global__ void __launch_bounds__(kSelThreads)
 get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
                   const ConsumerSlot *slots_dev, const uint32_t seq) {
@@ -116,7 +125,7 @@ get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
     uint32_t *claim = dv.claim + (size_t)c * dv.claim_words;
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     __shared__ uint32_t s_tile, s_excl, s_failed;
-    __shared__ uint32_t s_warp[kSelWarps];
+    __shared__ uint32_t s_warp[kPasses][kSelWarps];
     griddep_launch_dependents();
     griddep_wait();                                    // status and claim words as the work before this call left them
 
@@ -134,40 +143,55 @@ get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
         return;
     }
     const uint32_t tile = s_tile;
-    const uint32_t g = tile * kSelThreads + tid;
+    // pass u of the tile covers groups [tile * kPasses + u] * 256 ...: thread tid tests one of them
+    const uint32_t g0 = tile * (kSelThreads * kPasses) + tid;
 
     // The claim word and the group's N status words are read with relaxed loads, all in flight
     // together (four words per load when N allows), and one fence behind them makes the set an
     // acquire: a status bit seen here was published after its payload, and the gather that
     // follows in this stream reads that payload.
-    bool ready = false;
-    if (g < dv.G) {
-        const uint32_t cw = ld_relaxed_u32(&claim[g >> 5]);
-        const uint32_t *st = dv.status + (size_t)g * dv.N;
-        uint32_t all = need;
-        if ((dv.N & 3u) == 0) {
-            #pragma unroll 8
-            for (uint32_t j = 0; j < dv.N; j += 4) {
-                const uint4 w = ld_relaxed_u32x4(st + j);
-                all &= w.x & w.y & w.z & w.w;
+    bool ready[kPasses];
+    #pragma unroll
+    for (int u = 0; u < kPasses; ++u) {
+        const uint32_t g = g0 + (uint32_t)u * kSelThreads;
+        ready[u] = false;
+        if (g < dv.G) {
+            const uint32_t cw = ld_relaxed_u32(&claim[g >> 5]);
+            const uint32_t *st = dv.status + (size_t)g * dv.N;
+            uint32_t all = need;
+            if ((dv.N & 3u) == 0) {
+                #pragma unroll 8
+                for (uint32_t j = 0; j < dv.N; j += 4) {
+                    const uint4 w = ld_relaxed_u32x4(st + j);
+                    all &= w.x & w.y & w.z & w.w;
+                }
+            } else {
+                #pragma unroll 4
+                for (uint32_t j = 0; j < dv.N; ++j) all &= ld_relaxed_u32(st + j);
             }
-        } else {
-            #pragma unroll 4
-            for (uint32_t j = 0; j < dv.N; ++j) all &= ld_relaxed_u32(st + j);
+            ready[u] = !((cw >> (g & 31)) & 1u) && all == need;
         }
-        ready = !((cw >> (g & 31)) & 1u) && all == need;
     }
     __threadfence();
-    const uint32_t ballot = __ballot_sync(kFullMask, ready);
-    const uint32_t in_warp = __popc(ballot & ((1u << lane) - 1u));
-    if (lane == 0) s_warp[warp] = __popc(ballot);
-    __syncthreads();
-    uint32_t warp_off = 0, tile_count = 0;
+    uint32_t in_warp[kPasses];
     #pragma unroll
-    for (int w = 0; w < kSelWarps; ++w) {
-        const uint32_t v = s_warp[w];
-        if (w < (int)warp) warp_off += v;
-        tile_count += v;
+    for (int u = 0; u < kPasses; ++u) {
+        const uint32_t ballot = __ballot_sync(kFullMask, ready[u]);
+        in_warp[u] = __popc(ballot & ((1u << lane) - 1u));
+        if (lane == 0) s_warp[u][warp] = __popc(ballot);
+    }
+    __syncthreads();
+    // ready groups of the tile before this thread's group of pass u, and in the whole tile
+    uint32_t before[kPasses], tile_count = 0;
+    #pragma unroll
+    for (int u = 0; u < kPasses; ++u) {
+        before[u] = tile_count;
+        #pragma unroll
+        for (int w = 0; w < kSelWarps; ++w) {
+            const uint32_t v = s_warp[u][w];
+            if (w < (int)warp) before[u] += v;
+            tile_count += v;
+        }
     }
 
     if (warp == 0) {
@@ -214,15 +238,19 @@ get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
         if (tid == 0) flag_error(dv, TD_ERR_LOOKBACK_TIMEOUT, CNT_TIMEOUT);
         return;
     }
-    const uint32_t rank = s_excl + warp_off + in_warp;
-    const bool cand = ready && rank < cs.max_groups;
-    const uint32_t mask = __ballot_sync(kFullMask, cand);
-    uint32_t old = 0;
-    if (lane == 0 && mask) old = atomicOr(&claim[g >> 5], mask);   // the warp's 32 groups share a word
-    old = __shfl_sync(kFullMask, old, 0);
-    if (cand) sc.cand[rank] = ((old >> lane) & 1u) ? ~(int32_t)g : (int32_t)g;
-    const uint32_t lost = __popc(mask & old);
-    if (lane == 0 && lost) atomicAdd(&dv.counters[CNT_CONFLICT], (unsigned long long)lost);
+    #pragma unroll
+    for (int u = 0; u < kPasses; ++u) {
+        const uint32_t g = g0 + (uint32_t)u * kSelThreads;
+        const uint32_t rank = s_excl + before[u] + in_warp[u];
+        const bool cand = ready[u] && rank < cs.max_groups;
+        const uint32_t mask = __ballot_sync(kFullMask, cand);
+        uint32_t old = 0;
+        if (lane == 0 && mask) old = atomicOr(&claim[g >> 5], mask);   // the warp's 32 groups share a word
+        old = __shfl_sync(kFullMask, old, 0);
+        if (cand) sc.cand[rank] = ((old >> lane) & 1u) ? ~(int32_t)g : (int32_t)g;
+        const uint32_t lost = __popc(mask & old);
+        if (lane == 0 && lost) atomicAdd(&dv.counters[CNT_CONFLICT], (unsigned long long)lost);
+    }
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -242,6 +242,25 @@ def test_many_tiles_look_back(G):
     assert batches[0][1].n_samples == 2200
 
 
+def test_wide_tiles_of_a_large_dock(G):
+    """More than 65536 groups: scan tiles take four passes of 256 groups each.  Random partial
+    readiness, gets of thousands of groups and of a few, ranks across passes and tiles."""
+    w = wl.make_custom("wide", 70000, 1, 4, prompt_len=(0, 2), response=("uniform", 0, 3), vocab=100,
+                       micro_batch=9000, seed=23, schedule="interleaved", chunk=(1, 30000), poll_every=3)
+    g, o, batches = G.replay_both(w, arenas=False)
+    assert max(b.n_groups for _, b in batches) > 4096
+    w2 = wl.make_custom("wide2", 66048, 2, 8, prompt_len=(0, 2), response=("uniform", 0, 3), vocab=100,
+                        micro_batch=64, seed=24, schedule="none")
+    o2, g2 = H.make_oracle(w2), G.GpuDock(w2)
+    idx = np.arange(w2.n, dtype=np.int32)[::-1].copy()          # every sample, highest first
+    for c in range(len(w2.columns)):
+        cu, data = w2.pack(c, idx)
+        o2.put(c, idx, cu, data); g2.put(c, idx, cu, data)
+    for c in (0, 3, 0, 3):
+        G.assert_batch_equal(g2.get(c, 64), o2.get(c, 64), f"wide2 consumer {c}")
+    G.assert_state_equal(g2, o2, arenas=False, ctx="wide2")
+
+
 # ------------------------------------------------------------------- batched calls
 def _many_vs_serial(G, w, mode=td.PACKED, fused=False):
     """All columns in one td_put_many, all gets of the schedule in one td_get_many; the oracle
