@@ -163,12 +163,18 @@ class NvmlSampler:
         self.thread = threading.Thread(target=self._loop, daemon=True)
         self.thread.start()
 
-    def stop(self, t_begin: float, t_end: float):
+    def count_inside(self, t_begin: float, t_end: float) -> int:
+        return sum(1 for s in self.samples if t_begin <= s[0] <= t_end)
+
+    def stop(self, t_begin: float, t_end: float, t_soak_end: float = 0.0):
         self.stop_flag.set()
         if self.thread:
             self.thread.join(timeout=2)
         inside = [s for s in self.samples if t_begin <= s[0] <= t_end]
         window = "timed region"
+        if len(inside) < 3 and t_soak_end > t_end:
+            inside = [s for s in self.samples if t_begin <= s[0] <= t_soak_end]
+            window = "timed region and the same steps repeated right after it (the region is a few ms)"
         if len(inside) < 3:
             inside, window = self.samples, "warm-up and timed region"
         reasons = set()
@@ -771,7 +777,14 @@ def main():
     torch.cuda.cudart().cudaProfilerStop()
     t_end = time.time()
     launches = step.dock.launch_count() - launches0
-    clocks = sampler.stop(t_begin, t_end)
+    # A timed region of a few milliseconds holds too few clock samples: the same steps go on,
+    # untimed, until the sampler has seen the device under this load for a while.
+    t_soak_end = t_end
+    if isinstance(sampler, NvmlSampler) and sampler.count_inside(t_begin, t_end) < 3:
+        while time.time() - t_end < 0.25 and sampler.count_inside(t_begin, time.time()) < 8:
+            step.timed_step()
+        t_soak_end = time.time()
+    clocks = sampler.stop(t_begin, t_end, t_soak_end) if isinstance(sampler, NvmlSampler) else sampler.stop(t_begin, t_end)
 
     mean_put, mean_drain = sum(put_ms) / len(put_ms), sum(drain_ms) / len(drain_ms)
     ms_per_step = mean_put + mean_drain
