@@ -164,9 +164,21 @@ cudaError_t launch_select(td_dock *d, uint32_t n_slots, cudaStream_t st, Args &&
 template <typename... Args>
 cudaError_t launch_finalize(td_dock *d, uint32_t n_req, uint32_t max_samples, cudaStream_t st, Args &&...args) {
     if (max_samples > kFinBigSamples)
-        return launch_dep(d, get_finalize_kernel<kFinThreadsBig>, dim3(n_req), dim3(kFinThreadsBig), 0, st,
+        return launch_dep(d, get_finalize_kernel<kFinThreadsBig, false>, dim3(n_req), dim3(kFinThreadsBig), 0, st,
                           std::forward<Args>(args)...);
-    return launch_dep(d, get_finalize_kernel<kFinThreads>, dim3(n_req), dim3(kFinThreads), 0, st,
+    return launch_dep(d, get_finalize_kernel<kFinThreads, false>, dim3(n_req), dim3(kFinThreads), 0, st,
+                      std::forward<Args>(args)...);
+}
+
+// May the scan of a call run inside its finalize kernel?  The dock's groups fit one wide tile,
+// every consumer of the call has one request, and no request is large.
+bool scan_fits_finalize(const td_dock *d, uint32_t n_req, uint32_t n_slots, uint32_t max_samples) {
+    return d->dv.G <= kSelThreads * kSelWide && n_req == n_slots && max_samples <= kFinBigSamples;
+}
+template <typename... Args>
+cudaError_t launch_fused_finalize(td_dock *d, uint32_t n_req, cudaStream_t st, Args &&...args) {
+    static_assert(kFinThreads == kSelThreads, "the fused scan is one tile of the finalize kernel's threads");
+    return launch_dep(d, get_finalize_kernel<kFinThreads, true>, dim3(n_req), dim3(kFinThreads), 0, st,
                       std::forward<Args>(args)...);
 }
 
@@ -534,12 +546,17 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
     const uint32_t jpr = jobs_per_req(v, wants_stream(*out));
 
-    if (launch_select(d, 1u, st, v, one,
-               (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
-    if (launch_finalize(d, 1u, one.req.max_groups * v.N, st, v, one, (const GetReq *)nullptr,
-               (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr, (uint8_t *)nullptr) != cudaSuccess) return TD_ECUDA;
+    if (scan_fits_finalize(d, 1u, 1u, one.req.max_groups * v.N)) {
+        if (launch_fused_finalize(d, 1u, st, v, one, (const GetReq *)nullptr, (const ConsumerSlot *)nullptr, seq, counter,
+                                  (JobSize *)nullptr, jpr, (uint8_t *)nullptr) != cudaSuccess) return TD_ECUDA;
+    } else {
+        if (launch_select(d, 1u, st, v, one, (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
+        if (launch_finalize(d, 1u, one.req.max_groups * v.N, st, v, one, (const GetReq *)nullptr,
+                            (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr, (uint8_t *)nullptr) !=
+            cudaSuccess) return TD_ECUDA;
+    }
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
     if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, jpr), st, v, one,
                      (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr, jpr, make_fastdiv(jpr),
@@ -613,12 +630,17 @@ int td_get_static(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
     const uint32_t jpr = jobs_per_req(v, wants_stream(*out));
 
-    if (launch_select(d, 1u, st, v, one,
-               (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
-    if (launch_finalize(d, 1u, one.req.max_groups * v.N, st, v, one, (const GetReq *)nullptr,
-               (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr, (uint8_t *)nullptr) != cudaSuccess) return TD_ECUDA;
+    if (scan_fits_finalize(d, 1u, 1u, one.req.max_groups * v.N)) {
+        if (launch_fused_finalize(d, 1u, st, v, one, (const GetReq *)nullptr, (const ConsumerSlot *)nullptr, seq, counter,
+                                  (JobSize *)nullptr, jpr, (uint8_t *)nullptr) != cudaSuccess) return TD_ECUDA;
+    } else {
+        if (launch_select(d, 1u, st, v, one, (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
+        if (launch_finalize(d, 1u, one.req.max_groups * v.N, st, v, one, (const GetReq *)nullptr,
+                            (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr, (uint8_t *)nullptr) !=
+            cudaSuccess) return TD_ECUDA;
+    }
     const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
     if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, jpr), st, v, one,
                      (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr, jpr, make_fastdiv(jpr),
@@ -740,10 +762,15 @@ int get_many(td_dock *d, td_plan *p, uint8_t *d_meta, void *stream) {
     GetInline none;
     std::memset(&none, 0, sizeof(none));
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
-    if (launch_select(d, p->n_slots, st, v, none,
-               (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
-    if (launch_finalize(d, p->n_req, p->max_req_samples, st, v, none, (const GetReq *)p->d_reqs,
-               (const ConsumerSlot *)p->d_slots, seq, p->d_counter, p->d_job_sizes, p->jobs_per_req, d_meta) != cudaSuccess) return TD_ECUDA;
+    if (scan_fits_finalize(d, p->n_req, p->n_slots, p->max_req_samples)) {
+        if (launch_fused_finalize(d, p->n_req, st, v, none, (const GetReq *)p->d_reqs, (const ConsumerSlot *)p->d_slots, seq,
+                                  p->d_counter, p->d_job_sizes, p->jobs_per_req, d_meta) != cudaSuccess) return TD_ECUDA;
+    } else {
+        if (launch_select(d, p->n_slots, st, v, none, (const ConsumerSlot *)p->d_slots, seq) != cudaSuccess) return TD_ECUDA;
+        if (launch_finalize(d, p->n_req, p->max_req_samples, st, v, none, (const GetReq *)p->d_reqs,
+                            (const ConsumerSlot *)p->d_slots, seq, p->d_counter, p->d_job_sizes, p->jobs_per_req, d_meta) !=
+            cudaSuccess) return TD_ECUDA;
+    }
     if (launch_timed(d, 1, get_gather_kernel, dim3(copy_grid(d, p->room_bytes)), dim3(kCopyThreads),
                      gather_smem_bytes(p->n_req, p->jobs_per_req), st, v, none,
                      (const GetReq *)p->d_reqs, p->n_req, p->d_counter, (const JobSize *)p->d_job_sizes,

@@ -105,6 +105,89 @@ struct GetInline {            // a single get travels in the kernel parameters
     ConsumerSlot cs;
 };
 
+// The two halves of a tile's work, around whatever tells it how many ready groups come before
+// it.  select_eval: thread tid tests one group per pass (all N status words carry the
+// consumer's need bits, the group is not claimed) and the tile's ready groups are counted by
+// warp ballots.  select_claim: the ready groups whose rank is below max_groups are claimed with
+// one atomicOr per warp and pass and entered into the candidate list.
+template <int kPasses>
+struct TileState {
+    bool ready[kPasses];
+    uint32_t in_warp[kPasses];   // ready groups before this lane in its warp, per pass
+    uint32_t before[kPasses];    // ready groups of the tile before this thread's warp and pass
+    uint32_t g0;                 // group of pass 0
+};
+template <int kPasses>
+__device__ __forceinline__ uint32_t select_eval(const DockView &dv, const uint32_t *claim, uint32_t need, uint32_t tile,
+                                                uint32_t (*s_warp)[kSelWarps], TileState<kPasses> &ts) {
+    const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    // pass u of the tile covers groups [tile * kPasses + u] * 256 ...: thread tid tests one of them
+    ts.g0 = tile * (kSelThreads * kPasses) + tid;
+    // The claim word and the group's N status words are read with relaxed loads, all in flight
+    // together (four words per load when N allows), and one fence behind them makes the set an
+    // acquire: a status bit seen here was published after its payload, and the gather that
+    // follows in this stream reads that payload.
+    #pragma unroll
+    for (int u = 0; u < kPasses; ++u) {
+        const uint32_t g = ts.g0 + (uint32_t)u * kSelThreads;
+        ts.ready[u] = false;
+        if (g < dv.G) {
+            const uint32_t cw = ld_relaxed_u32(&claim[g >> 5]);
+            const uint32_t *st = dv.status + (size_t)g * dv.N;
+            uint32_t all = need;
+            if ((dv.N & 3u) == 0) {
+                #pragma unroll 8
+                for (uint32_t j = 0; j < dv.N; j += 4) {
+                    const uint4 w = ld_relaxed_u32x4(st + j);
+                    all &= w.x & w.y & w.z & w.w;
+                }
+            } else {
+                #pragma unroll 4
+                for (uint32_t j = 0; j < dv.N; ++j) all &= ld_relaxed_u32(st + j);
+            }
+            ts.ready[u] = !((cw >> (g & 31)) & 1u) && all == need;
+        }
+    }
+    __threadfence();
+    #pragma unroll
+    for (int u = 0; u < kPasses; ++u) {
+        const uint32_t ballot = __ballot_sync(kFullMask, ts.ready[u]);
+        ts.in_warp[u] = __popc(ballot & ((1u << lane) - 1u));
+        if (lane == 0) s_warp[u][warp] = __popc(ballot);
+    }
+    __syncthreads();
+    uint32_t tile_count = 0;
+    #pragma unroll
+    for (int u = 0; u < kPasses; ++u) {
+        ts.before[u] = tile_count;
+        #pragma unroll
+        for (int w = 0; w < kSelWarps; ++w) {
+            const uint32_t v = s_warp[u][w];
+            if (w < (int)warp) ts.before[u] += v;
+            tile_count += v;
+        }
+    }
+    return tile_count;
+}
+template <int kPasses>
+__device__ __forceinline__ void select_claim(const DockView &dv, uint32_t *claim, const SelScratch &sc, uint32_t excl,
+                                             uint32_t max_groups, const TileState<kPasses> &ts) {
+    const uint32_t lane = threadIdx.x & 31;
+    #pragma unroll
+    for (int u = 0; u < kPasses; ++u) {
+        const uint32_t g = ts.g0 + (uint32_t)u * kSelThreads;
+        const uint32_t rank = excl + ts.before[u] + ts.in_warp[u];
+        const bool cand = ts.ready[u] && rank < max_groups;
+        const uint32_t mask = __ballot_sync(kFullMask, cand);
+        uint32_t old = 0;
+        if (lane == 0 && mask) old = atomicOr(&claim[g >> 5], mask);   // the warp's 32 groups share a word
+        old = __shfl_sync(kFullMask, old, 0);
+        if (cand) sc.cand[rank] = ((old >> lane) & 1u) ? ~(int32_t)g : (int32_t)g;
+        const uint32_t lost = __popc(mask & old);
+        if (lane == 0 && lost) atomicAdd(&dv.counters[CNT_CONFLICT], (unsigned long long)lost);
+    }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Select.  grid = (tiles, consumer slots).  Thread g of a tile tests group g: all N status
 // words carry the consumer's need bits and the group is not claimed.  Warp ballots and popc
@@ -143,56 +226,8 @@ get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
         return;
     }
     const uint32_t tile = s_tile;
-    // pass u of the tile covers groups [tile * kPasses + u] * 256 ...: thread tid tests one of them
-    const uint32_t g0 = tile * (kSelThreads * kPasses) + tid;
-
-    // The claim word and the group's N status words are read with relaxed loads, all in flight
-    // together (four words per load when N allows), and one fence behind them makes the set an
-    // acquire: a status bit seen here was published after its payload, and the gather that
-    // follows in this stream reads that payload.
-    bool ready[kPasses];
-    #pragma unroll
-    for (int u = 0; u < kPasses; ++u) {
-        const uint32_t g = g0 + (uint32_t)u * kSelThreads;
-        ready[u] = false;
-        if (g < dv.G) {
-            const uint32_t cw = ld_relaxed_u32(&claim[g >> 5]);
-            const uint32_t *st = dv.status + (size_t)g * dv.N;
-            uint32_t all = need;
-            if ((dv.N & 3u) == 0) {
-                #pragma unroll 8
-                for (uint32_t j = 0; j < dv.N; j += 4) {
-                    const uint4 w = ld_relaxed_u32x4(st + j);
-                    all &= w.x & w.y & w.z & w.w;
-                }
-            } else {
-                #pragma unroll 4
-                for (uint32_t j = 0; j < dv.N; ++j) all &= ld_relaxed_u32(st + j);
-            }
-            ready[u] = !((cw >> (g & 31)) & 1u) && all == need;
-        }
-    }
-    __threadfence();
-    uint32_t in_warp[kPasses];
-    #pragma unroll
-    for (int u = 0; u < kPasses; ++u) {
-        const uint32_t ballot = __ballot_sync(kFullMask, ready[u]);
-        in_warp[u] = __popc(ballot & ((1u << lane) - 1u));
-        if (lane == 0) s_warp[u][warp] = __popc(ballot);
-    }
-    __syncthreads();
-    // ready groups of the tile before this thread's group of pass u, and in the whole tile
-    uint32_t before[kPasses], tile_count = 0;
-    #pragma unroll
-    for (int u = 0; u < kPasses; ++u) {
-        before[u] = tile_count;
-        #pragma unroll
-        for (int w = 0; w < kSelWarps; ++w) {
-            const uint32_t v = s_warp[u][w];
-            if (w < (int)warp) before[u] += v;
-            tile_count += v;
-        }
-    }
+    TileState<kPasses> ts;
+    const uint32_t tile_count = select_eval<kPasses>(dv, claim, need, tile, s_warp, ts);
 
     if (warp == 0) {
         uint32_t excl = 0;
@@ -238,19 +273,7 @@ get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
         if (tid == 0) flag_error(dv, TD_ERR_LOOKBACK_TIMEOUT, CNT_TIMEOUT);
         return;
     }
-    #pragma unroll
-    for (int u = 0; u < kPasses; ++u) {
-        const uint32_t g = g0 + (uint32_t)u * kSelThreads;
-        const uint32_t rank = s_excl + before[u] + in_warp[u];
-        const bool cand = ready[u] && rank < cs.max_groups;
-        const uint32_t mask = __ballot_sync(kFullMask, cand);
-        uint32_t old = 0;
-        if (lane == 0 && mask) old = atomicOr(&claim[g >> 5], mask);   // the warp's 32 groups share a word
-        old = __shfl_sync(kFullMask, old, 0);
-        if (cand) sc.cand[rank] = ((old >> lane) & 1u) ? ~(int32_t)g : (int32_t)g;
-        const uint32_t lost = __popc(mask & old);
-        if (lane == 0 && lost) atomicAdd(&dv.counters[CNT_CONFLICT], (unsigned long long)lost);
-    }
+    select_claim<kPasses>(dv, claim, sc, s_excl, cs.max_groups, ts);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -320,7 +343,9 @@ __device__ __forceinline__ uint32_t job_cost_rows(const DockView &dv, const GetR
     return (bytes != 0 && dv.col_cls[k] != TD_SCALAR && rq.out.mode == TD_PACKED) ? n_s : 0u;
 }
 
-template <int kThreads>
+// kFused: the dock has at most one (wide) tile of groups and every consumer of the call one
+// request, so the request's CTA does the scan and the claim itself first (one launch less).
+template <int kThreads, bool kFused>
 __global__ void __launch_bounds__(kThreads)
 get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
                     const GetReq *reqs_dev, const ConsumerSlot *slots_dev, const uint32_t seq,
@@ -345,15 +370,27 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     griddep_wait();                                    // the scan's candidate list is complete
     if (blockIdx.x == 0 && threadIdx.x == 0) *work_counter = 0;     // the gather hands out its chunks from zero
 
-    // how many groups were ready, from the last tile's inclusive prefix; the first candidates are
-    // asked for in the same breath (which of them count is known once the prefix is here)
-    const unsigned long long last = sc.desc[sel_tiles(dv.G) - 1];
-    int32_t g_first = -1;
-    if (tid < rq.max_groups && rq.rank_base + tid < dv.G) g_first = sc.cand[rq.rank_base + tid];
     uint32_t status = 0;
     uint32_t total = 0;
-    if (desc_seq(last) != seq || desc_state(last) != kStatePrefix) status |= TD_ERR_LOOKBACK_TIMEOUT;
-    else total = min(desc_count(last), cs.max_groups);
+    int32_t g_first = -1;
+    if constexpr (kFused) {
+        static_assert(!kFused || kThreads == kSelThreads, "the fused scan is one tile of kSelThreads threads");
+        __shared__ uint32_t s_warp[kSelWide][kSelWarps];
+        uint32_t *claim = dv.claim + (size_t)c * dv.claim_words;
+        TileState<(int)kSelWide> ts;
+        const uint32_t tile_count = select_eval<(int)kSelWide>(dv, claim, dv.need[c], 0u, s_warp, ts);
+        select_claim<(int)kSelWide>(dv, claim, sc, 0u, cs.max_groups, ts);
+        __syncthreads();                                   // the consumer's candidate list is complete
+        total = min(tile_count, cs.max_groups);
+        if (tid < rq.max_groups && rq.rank_base + tid < dv.G) g_first = sc.cand[rq.rank_base + tid];
+    } else {
+        // how many groups were ready, from the last tile's inclusive prefix; the first candidates
+        // are asked for in the same breath (which of them count is known once the prefix is here)
+        const unsigned long long last = sc.desc[sel_tiles(dv.G) - 1];
+        if (tid < rq.max_groups && rq.rank_base + tid < dv.G) g_first = sc.cand[rq.rank_base + tid];
+        if (desc_seq(last) != seq || desc_state(last) != kStatePrefix) status |= TD_ERR_LOOKBACK_TIMEOUT;
+        else total = min(desc_count(last), cs.max_groups);
+    }
     const uint32_t lo = rq.rank_base;
     const uint32_t hi = min(lo + rq.max_groups, total);
     const uint32_t ncand = hi > lo ? hi - lo : 0;
