@@ -390,7 +390,8 @@ int put_group(td_dock *d, PutBatch &b, cudaStream_t st) {
                          scatter_smem_bytes(), st, v, b) != cudaSuccess)
             return TD_ECUDA;
     }
-    if (launch_dep(d, put_publish_kernel, dim3((uint32_t)((entries + 255) / 256)), dim3(256), 0, st, v, b) != cudaSuccess)
+    if (launch_dep(d, put_publish_kernel, dim3((uint32_t)((entries + 255) / 256)), dim3(256), 0, st, v, b,
+                   ragged_bytes ? 1u : 0u) != cudaSuccess)
         return TD_ECUDA;
     return TD_OK;
 }

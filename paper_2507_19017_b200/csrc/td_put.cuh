@@ -42,8 +42,10 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
     const uint32_t tid = threadIdx.x, lane = tid & 31;
     WarpPipe pipe;                                                           // [warps][kPipeSmemPerWarp]
     pipe.init(scatter_smem + (size_t)(tid >> 5) * kPipeSmemPerWarp, lane, dv.spin_limit);
-    griddep_launch_dependents();
     griddep_wait();                                    // the alloc kernel's tables are complete
+    // Only now may the publish kernel be brought on: it reads the call's arrays and the tables
+    // ahead of its own wait, which is safe once everything before this kernel has finished.
+    griddep_launch_dependents();
 
     if (tid < batch.n_items) {                         // one thread per item: the totals load side by side
         const PutArgs &a = batch.item[tid];
@@ -123,8 +125,13 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
 // globally visible before a readiness bit is; the fence orders the bit behind them for readers
 // that acquire it.  A scalar item needs no scatter: its element is stored here, then published.
 __global__ void __launch_bounds__(256)
-put_publish_kernel(const DockView dv, const PutBatch batch) {
-    griddep_wait();                                    // every payload byte of the call is in place
+put_publish_kernel(const DockView dv, const PutBatch batch, const uint32_t behind_scatter) {
+    // behind_scatter: this launch follows the call's scatter kernel, which let it start only
+    // after the alloc kernel had finished: the entry and its table words can be fetched while the
+    // scatter is still copying, and only the readiness bit has to wait for it.  Otherwise (a
+    // call of scalar columns only) the kernel ahead may be the one that produces this call's
+    // index array, and everything waits.
+    if (!behind_scatter) griddep_wait();
     uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     uint32_t it = 0;
     for (; it < batch.n_items; ++it) {                 // grid slots are laid out by the items' largest counts
@@ -133,34 +140,39 @@ put_publish_kernel(const DockView dv, const PutBatch batch) {
     }
     if (it < batch.n_items && i >= item_k(batch.item[it])) it = batch.n_items;
     uint32_t ok = 0, n_oob = 0, n_dup = 0, n_bad = 0, column = 0;
+    int32_t s = -1;                                    // sample whose bit this thread sets, if any
+    uint32_t bit = 0, value = 0;
+    bool store_scalar = false;
     if (it < batch.n_items) {
         const PutArgs &a = batch.item[it];
         column = a.column;
         const uint32_t L = dv.col_cls[column];
-        const uint32_t bit = 1u << column;
+        bit = 1u << column;
         if (L != TD_SCALAR) {
-            int32_t s; int64_t l; long long off;
-            if (put_entry_live(dv, a, i, L, bit, s, l, off)) {
-                __threadfence();
-                const uint32_t old = atomicOr(&dv.status[s], bit);
-                ok = (old & bit) ? 0u : 1u;
-            }
+            int32_t ss; int64_t l; long long off;
+            if (put_entry_live(dv, a, i, L, bit, ss, l, off)) s = ss;
         } else {
-            const uint32_t esz = dv.col_esz[column];
-            const int32_t s = a.idx[i];
-            if (s < 0 || (uint32_t)s >= dv.n) ++n_oob;
+            const int32_t ss = a.idx[i];
+            if (ss < 0 || (uint32_t)ss >= dv.n) ++n_oob;
             else if ((uint64_t)i >= a.data_elems) ++n_bad;
-            else if (dv.status[s] & bit) ++n_dup;
+            else if (dv.status[ss] & bit) ++n_dup;
             else {
-                if (esz == 4)
-                    reinterpret_cast<uint32_t *>(dv.colbase[column])[s] = reinterpret_cast<const uint32_t *>(a.data)[i];
-                else
-                    reinterpret_cast<uint16_t *>(dv.colbase[column])[s] = reinterpret_cast<const uint16_t *>(a.data)[i];
-                __threadfence();
-                const uint32_t old = atomicOr(&dv.status[s], bit);
-                if (old & bit) ++n_dup; else ok = 1;
+                value = dv.col_esz[column] == 4 ? reinterpret_cast<const uint32_t *>(a.data)[i]
+                                                : (uint32_t)reinterpret_cast<const uint16_t *>(a.data)[i];
+                store_scalar = true;
+                s = ss;
             }
         }
+    }
+    if (behind_scatter) griddep_wait();                // every payload byte of the call is in place
+    if (s >= 0) {
+        if (store_scalar) {
+            if (dv.col_esz[column] == 4) reinterpret_cast<uint32_t *>(dv.colbase[column])[s] = value;
+            else reinterpret_cast<uint16_t *>(dv.colbase[column])[s] = (uint16_t)value;
+        }
+        __threadfence();
+        const uint32_t old = atomicOr(&dv.status[s], bit);
+        if (old & bit) { if (store_scalar) ++n_dup; } else ok = 1;
     }
     // a warp may straddle two items: count per column with a match on the column number
     const uint32_t peers = __match_any_sync(kFullMask, column);
