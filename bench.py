@@ -29,8 +29,8 @@ METRIC = "td_put+td_get samples/s dispatched"
 L2_FLUSH_BYTES = 256 << 20
 # DRAM bytes (read + write) of one launch, from the ncu capture summarised under profiles/ for
 # the kernels as built; (config, kernel) pairs without a capture report null.
-NCU_TRAFFIC = {(2, "get_gather"): 79_443_968, (2, "put_scatter"): 44_550_400,
-               (3, "get_gather"): 1_147_951_616, (3, "put_scatter"): 732_503_808}
+NCU_TRAFFIC = {(2, "get_gather"): 79_587_584, (2, "put_scatter"): 44_971_776,
+               (3, "get_gather"): 1_147_116_032, (3, "put_scatter"): 732_750_848}
 
 
 def parse_args():
