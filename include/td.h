@@ -244,7 +244,7 @@ int td_put_back(td_dock *dock, const td_get_out *batch, uint32_t max_samples, co
  * of them): request r sends column `column` back for the batch `batch` it names, exactly as
  * td_put_back(dock, batch, max_samples, {column, d_data, data_elems}, 1, stream) would; the
  * requests are stored in array order.  Together with td_get_many this serves one poll of every
- * worker state with six launches, whatever their number. */
+ * worker state with five or six launches, whatever their number. */
 typedef struct {
     const td_get_out *batch;
     uint32_t max_samples, column;
@@ -256,7 +256,7 @@ int td_put_back_many(td_dock *dock, const td_back_req *reqs, uint32_t n_reqs, vo
 /* Many gets served by one call.  Each worker state has its own controller and a step serves
  * several of them, each in several micro-batches; a plan fixes the list of requests (consumer,
  * max_samples, output buffers) once and td_get_many then serves all of them with three kernel
- * launches.  Requests that name the same consumer are served in array order: the result is the
+ * launches (two when the dock has at most 1024 prompts and every consumer one request).  Requests that name the same consumer are served in array order: the result is the
  * one td_get would give when called on each request in turn, except that a group cut off by
  * TD_ERR_OUT_TRUNCATED is not offered to the later requests of the same call.
  *   td_plan_bytes   device bytes a plan of n_req requests needs (request table + scan scratch).
