@@ -473,3 +473,19 @@ def test_fused_stream_takes_float_columns_and_respects_capacity():
     assert H.bits_equal(b.seq, want)
     b2 = d.get(0, 6, seq=(0, 1), seq_cap=64)          # the group that was cut is still there
     assert b2.n_groups == 1 and list(b2.indices) == [4, 5] and b2.status == 0
+
+
+def test_cascade_batched_polls_serve_everything_once():
+    """The batched form of the cascade (one get call for all worker states, one write-back call
+    for all of them per poll) drains like the per-call form: every consumer gets every sample
+    exactly once, every column ends up stored for every sample, nothing is flagged."""
+    w = small(schedule="cascade_batched", G=12, N=3, S=3, poll_every=4, with_entropy=True, micro_batch=6)
+    d = H.make_oracle(w)
+    out = H.replay_oracle(w, d)
+    for c in range(len(w.consumers)):
+        got = np.concatenate([b.indices for cc, b in out if cc == c])
+        assert sorted(got.tolist()) == list(range(w.n))
+    st = d.stats()
+    assert st.error_word == 0
+    assert all(st.put_accepted[c] == w.n for c in range(len(w.columns)))
+    assert np.all(d.status() == (1 << len(w.columns)) - 1)
