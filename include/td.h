@@ -17,7 +17,9 @@
  *
  * Conventions for every call:
  *   - "device" pointers are CUDA device memory owned by the caller; the library allocates no
- *     device memory and frees none.  "host" pointers are ordinary host memory.
+ *     device memory and frees none.  "host" pointers are ordinary host memory.  The one
+ *     allocation the library makes is pinned HOST memory: td_get_many_host with a staging
+ *     buffer allocates a host mirror of it once per plan (freed by td_plan_destroy).
  *   - td_put / td_get / td_get_many / td_reset only enqueue work on the given stream and return;
  *     they never synchronise.  Calls on one stream execute in call order.  Gets may run
  *     concurrently with each other and with puts on other streams.  Puts that may reserve the
@@ -61,7 +63,8 @@ enum {
     TD_ERR_LEN_MISMATCH     = 1u << 2,  /* put: length differs from the sample's length class   */
     TD_ERR_ARENA_FULL       = 1u << 3,  /* put: shard arena has no room for the row             */
     TD_ERR_OUT_TRUNCATED    = 1u << 4,  /* get: stopped before a group that would not fit       */
-    TD_ERR_LOOKBACK_TIMEOUT = 1u << 5,  /* get: a scan tile gave up waiting; nothing returned   */
+    TD_ERR_LOOKBACK_TIMEOUT = 1u << 5,  /* get: a scan tile gave up waiting; nothing is served,
+                                           nothing stays claimed, the groups remain available   */
     TD_ERR_BAD_LENGTH       = 1u << 6,  /* put: cu not monotone or beyond data_elems            */
     TD_ERR_COPY_TIMEOUT     = 1u << 7   /* a staged copy did not land in time; plain loads used  */
 };
@@ -198,9 +201,14 @@ size_t td_get_scratch_bytes(const td_dock *dock);
  *     outside any stream capture.
  *   - All calls share the one array, which still holds the previous call's contents; the words
  *     that must start at zero are cleared on `stream` before the scan.  Two td_get_static calls
- *     that overlap on the GPU (different streams, no ordering between them) race on it and may
- *     return nothing or report TD_ERR_LOOKBACK_TIMEOUT; order them, or use td_get with separate
- *     scratch for concurrent gets. */
+ *     that overlap on the GPU (different streams, no ordering between them) race on it: they
+ *     share the scan's ticket, its tile descriptors and its candidate list, so the outcome is
+ *     undefined within the dock's own tables: either call may return nothing, report
+ *     TD_ERR_LOOKBACK_TIMEOUT, be served groups that the other call selected (also groups of
+ *     the other call's consumer, whose served marks are then set for the wrong worker state),
+ *     or leave groups claimed and unserved until td_reset.  No memory outside the dock, the
+ *     array and the two calls' own output buffers is touched.  Order such calls (one stream,
+ *     or events), or use td_get with separate scratch for gets that may overlap. */
 int td_get_static(td_dock *dock, uint32_t consumer, uint32_t max_samples, const td_get_out *out,
                   void *stream);
 
@@ -316,6 +324,16 @@ typedef struct {
     uint64_t arena_elems_used[3];    /* by length class: elements taken by rows, padding included */
 } td_validate_report;
 int td_debug_validate(td_dock *dock, void *stream, td_validate_report *report);
+
+/* Test hook for the bounded wait of the readiness scan (workflow step 1): a scan tile waits at
+ * most poll_limit polls for the tiles ahead of it (0 restores the default, about 2^20), and the
+ * tile that draws number skip_tile withholds its descriptor (UINT32_MAX: none), so that the
+ * waits of the tiles behind it run out.  Such a get serves nothing, reports
+ * TD_ERR_LOOKBACK_TIMEOUT in its result and in the error word, counts n_lookback_timeouts, and
+ * hands every claim it made back.  Only this wait is affected; waits on staged copies keep
+ * their own limit.  Applies to gets enqueued after the call; not to be called while other host
+ * threads are using the dock. */
+int td_debug_lookback(td_dock *dock, uint32_t poll_limit, uint32_t skip_tile);
 
 /* Kernels this dock has launched since td_create. */
 uint64_t td_launch_count(const td_dock *dock);

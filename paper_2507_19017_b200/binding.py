@@ -33,7 +33,8 @@ EXPORTS = ["td_query_workspace", "td_create", "td_destroy", "td_put", "td_get",
            "td_launch_count", "td_strerror", "td_kernel_timing", "td_kernel_timing_read",
            "td_put_host_stage_bytes", "td_put_host", "td_get_host", "td_put_many",
            "td_plan_bytes", "td_plan_create", "td_plan_destroy", "td_get_many", "td_get_static",
-           "td_model_bytes", "td_put_back", "td_put_back_many", "td_put_many_host", "td_get_many_host", "td_get_many_host_stage_bytes", "td_debug_validate"]
+           "td_model_bytes", "td_put_back", "td_put_back_many", "td_put_many_host", "td_get_many_host", "td_get_many_host_stage_bytes", "td_debug_validate",
+           "td_debug_lookback"]
 
 
 class TdModel(C.Structure):
@@ -177,6 +178,8 @@ def lib():
         L.td_get_many_host_stage_bytes.argtypes = [vp]
         L.td_debug_validate.restype = C.c_int
         L.td_debug_validate.argtypes = [vp, vp, C.POINTER(TdValidateReport)]
+        L.td_debug_lookback.restype = C.c_int
+        L.td_debug_lookback.argtypes = [vp, u32, u32]
         L.td_plan_bytes.restype = C.c_size_t
         L.td_plan_bytes.argtypes = [vp, u32]
         L.td_plan_create.restype = C.c_int
@@ -538,6 +541,11 @@ class Dock:
         rep = TdValidateReport()
         _check("td_debug_validate", lib().td_debug_validate(self.handle, _stream_ptr(stream), C.byref(rep)))
         return rep
+
+    def debug_lookback(self, poll_limit: int = 0, skip_tile: int = 0xFFFFFFFF):
+        """Test hook: poll limit of the scan's look-back wait (0 = default) and a tile that withholds
+        its descriptor (0xFFFFFFFF = none)."""
+        _check("td_debug_lookback", lib().td_debug_lookback(self.handle, poll_limit, skip_tile))
 
     def launch_count(self) -> int:
         return lib().td_launch_count(self.handle)

@@ -35,6 +35,7 @@ struct td_dock {
 namespace {
 
 std::atomic<uint32_t> g_seq{1};     // launch sequence numbers for scan scratch, process wide
+constexpr uint32_t kDefaultPollLimit = 1u << 20;      // polls before a device-side wait gives up (tens of milliseconds)
 
 inline size_t align_up_sz(size_t x, size_t a) { return (x + a - 1) / a * a; }
 inline uint32_t esize_of(int32_t dtype) { return dtype == TD_BF16 ? 2u : 4u; }
@@ -274,7 +275,9 @@ int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **o
     v.div_shard = make_fastdiv(v.N * v.prompts_per_shard);
     v.reward_col = cfg->reward_column;
     v.claim_words = L.claim_words; v.consumed_words = L.consumed_words;
-    v.spin_limit = 1u << 20;
+    v.spin_limit = kDefaultPollLimit;
+    v.lookback_limit = kDefaultPollLimit;
+    v.debug_skip_tile = 0xffffffffu;
     v.eps = (double)cfg->adv_eps;
     v.cap[1] = L.cap[1]; v.cap[2] = L.cap[2];
     uint8_t *w = d->ws;
@@ -523,17 +526,13 @@ size_t td_get_scratch_bytes(const td_dock *d) {
     return d ? sel_scratch_bytes(d->dv.G) : 0;
 }
 
-int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out *out, void *stream) {
-    if (!d) return TD_EINVAL;
+namespace {
+// One get with its scan scratch at `scratch` (checked by the caller): select, finalize, gather,
+// or finalize and gather where the scan fits the finalize kernel.
+int get_one(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out *out, void *scratch,
+            cudaStream_t st) {
     const DockView &v = d->dv;
-    const int chk = check_get_out(v, consumer, max_samples, out);
-    if (chk != TD_OK) return chk;
-    if (!out->scratch || (reinterpret_cast<uintptr_t>(out->scratch) & 15u) ||
-        out->scratch_bytes < sel_scratch_bytes(v.G))
-        return TD_EWORKSPACE;
-    cudaStream_t st = (cudaStream_t)stream;
     const uint32_t m = max_samples / v.N;
-
     GetInline one;
     std::memset(&one, 0, sizeof(one));
     one.req.out = *out;
@@ -543,12 +542,12 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
     one.req.cslot = 0;
     one.cs.consumer = consumer;
     one.cs.max_groups = one.req.max_groups;
-    one.cs.scratch = out->scratch;
+    one.cs.scratch = scratch;
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
     const uint32_t jpr = jobs_per_req(v, wants_stream(*out));
 
     // word 1 of the scan scratch is the gather's chunk counter
-    unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
+    unsigned long long *counter = static_cast<unsigned long long *>(scratch) + 1;
     if (scan_fits_finalize(d, 1u, 1u, one.req.max_groups * v.N)) {
         if (launch_fused_finalize(d, 1u, st, v, one, (const GetReq *)nullptr, (const ConsumerSlot *)nullptr, seq, counter,
                                   (JobSize *)nullptr, jpr, (uint8_t *)nullptr) != cudaSuccess) return TD_ECUDA;
@@ -564,6 +563,18 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
                      (const ConsumerSlot *)nullptr, 1u) != cudaSuccess) return TD_ECUDA;
     return TD_OK;
 }
+}  // namespace
+
+int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out *out, void *stream) {
+    if (!d) return TD_EINVAL;
+    const DockView &v = d->dv;
+    const int chk = check_get_out(v, consumer, max_samples, out);
+    if (chk != TD_OK) return chk;
+    if (!out->scratch || (reinterpret_cast<uintptr_t>(out->scratch) & 15u) ||
+        out->scratch_bytes < sel_scratch_bytes(v.G))
+        return TD_EWORKSPACE;
+    return get_one(d, consumer, max_samples, out, out->scratch, (cudaStream_t)stream);
+}
 
 // ---- a get whose scan scratch is a fixed array inside the library ----
 // For callers that have nowhere to take scratch memory from: code running where device memory
@@ -573,8 +584,7 @@ int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out
 // variant keeps that scratch in the array below instead, which every device that loads the
 // library holds (kStaticScratchBytes, about 65 KB) until the process exits.
 constexpr uint32_t kStaticMaxGroups = 16384;          // docks with more prompts are refused
-constexpr size_t kStaticScratchBytes = (((2 + (kStaticMaxGroups + kSelThreads - 1) / kSelThreads) * 8 +
-                                         (size_t)kStaticMaxGroups * 4) + 15) & ~size_t(15);
+constexpr size_t kStaticScratchBytes = sel_scratch_bytes(kStaticMaxGroups);
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 namespace {
@@ -616,37 +626,7 @@ int td_get_static(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_
     // call's sequence number, but the ticket and the tile descriptors are cleared all the same,
     // so that nothing here depends on what ran before.
     if (cudaMemsetAsync(scratch, 0, (2 + (size_t)sel_tiles(v.G)) * 8, st) != cudaSuccess) return TD_ECUDA;
-    const uint32_t m = max_samples / v.N;
-
-    GetInline one;
-    std::memset(&one, 0, sizeof(one));
-    one.req.out = *out;
-    one.req.consumer = consumer;
-    one.req.max_groups = m < v.G ? m : v.G;
-    one.req.rank_base = 0;
-    one.req.cslot = 0;
-    one.cs.consumer = consumer;
-    one.cs.max_groups = one.req.max_groups;
-    one.cs.scratch = scratch;
-    const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
-    const uint32_t jpr = jobs_per_req(v, wants_stream(*out));
-
-    // word 1 of the scan scratch is the gather's chunk counter
-    unsigned long long *counter = static_cast<unsigned long long *>(one.cs.scratch) + 1;
-    if (scan_fits_finalize(d, 1u, 1u, one.req.max_groups * v.N)) {
-        if (launch_fused_finalize(d, 1u, st, v, one, (const GetReq *)nullptr, (const ConsumerSlot *)nullptr, seq, counter,
-                                  (JobSize *)nullptr, jpr, (uint8_t *)nullptr) != cudaSuccess) return TD_ECUDA;
-    } else {
-        if (launch_select(d, 1u, st, v, one, (const ConsumerSlot *)nullptr, seq) != cudaSuccess) return TD_ECUDA;
-        if (launch_finalize(d, 1u, one.req.max_groups * v.N, st, v, one, (const GetReq *)nullptr,
-                            (const ConsumerSlot *)nullptr, seq, counter, (JobSize *)nullptr, jpr, (uint8_t *)nullptr) !=
-            cudaSuccess) return TD_ECUDA;
-    }
-    const uint32_t blocks = copy_grid(d, room_bytes_of(v, consumer, max_samples, *out));
-    if (launch_timed(d, 1, get_gather_kernel, dim3(blocks), dim3(kCopyThreads), gather_smem_bytes(1, jpr), st, v, one,
-                     (const GetReq *)nullptr, 1u, counter, (const JobSize *)nullptr, jpr, make_fastdiv(jpr),
-                     (const ConsumerSlot *)nullptr, 1u) != cudaSuccess) return TD_ECUDA;
-    return TD_OK;
+    return get_one(d, consumer, max_samples, out, scratch, st);
 }
 
 // ---- plans: many gets served by one call ----
@@ -799,7 +779,16 @@ int td_status(td_dock *d, td_stats *host_out, void *stream) {
     host_out->n_len_mismatch = cnt[CNT_MISMATCH]; host_out->n_arena_full = cnt[CNT_FULL];
     host_out->n_truncated = cnt[CNT_TRUNC]; host_out->n_bad_length = cnt[CNT_BADLEN];
     host_out->n_claim_conflicts = cnt[CNT_CONFLICT]; host_out->n_lookback_timeouts = cnt[CNT_TIMEOUT];
-    host_out->error_word = err;
+    host_out->error_word = err & ~kErrIrregularCu;          // the internal bit is not a condition of the ABI
+    return TD_OK;
+}
+
+// Test hook: how long a scan tile waits for the tiles ahead of it, and one tile that never shows
+// up.  Only the look-back wait is touched; the waits on staged copies keep their limit.
+int td_debug_lookback(td_dock *d, uint32_t poll_limit, uint32_t skip_tile) {
+    if (!d) return TD_EINVAL;
+    d->dv.lookback_limit = poll_limit ? poll_limit : kDefaultPollLimit;
+    d->dv.debug_skip_tile = skip_tile;
     return TD_OK;
 }
 

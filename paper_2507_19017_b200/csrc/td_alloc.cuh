@@ -119,6 +119,7 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
     griddep_launch_dependents();                                   // the scatter may set itself up meanwhile
     const uint64_t cap = dv.cap[L];
     uint32_t n_oob = 0, n_dup = 0, n_bad = 0, n_mis = 0, n_full = 0;
+    bool irregular = false;                    // a cu entry out of order or out of range, whatever else is wrong with its row
 
     // The passes read the items' index and cu arrays one after the other, each read at the head
     // of a chain of dependent accesses: ask for all of them now, one request per 128-byte line.
@@ -192,13 +193,14 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
                     s[j] = a.idx[i];
                     const int64_t c0 = a.cu[i], c1 = a.cu[i + 1];
                     const int64_t l = c1 - c0;
+                    const bool bad = l < 0 || c0 < 0 || (uint64_t)c1 > a.data_elems;
+                    irregular |= bad;
                     if (s[j] < 0 || (uint32_t)s[j] >= dv.n) { ++n_oob; n_oob += __popc(followers); }
                     else {
                         // The status word and the CAS travel side by side.  A column that is
                         // already stored has its class's length set, so the CAS of a repeated
                         // put changes nothing; it is then counted as a repeat, whatever its
                         // length says.
-                        const bool bad = l < 0 || c0 < 0 || (uint64_t)c1 > a.data_elems;
                         const uint32_t st = dv.status[s[j]];
                         int32_t old = 0;
                         if (!bad) old = atomicCAS(&dv.len[L][s[j]], -1, (int32_t)l);
@@ -216,7 +218,7 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
                             const uint32_t f = (uint32_t)__ffs(fm) - 1u;
                             const PutArgs &b = batch.item[f];
                             if (st & (1u << b.column)) ++n_dup;
-                            else if (l < 0 || c0 < 0 || (uint64_t)c1 > b.data_elems) ++n_bad;
+                            else if (l < 0 || c0 < 0 || (uint64_t)c1 > b.data_elems) { ++n_bad; irregular = true; }
                             else if ((old == -1 ? (int32_t)l : old) != (int32_t)l) ++n_mis;
                             else fok |= 1u << f;
                         }
@@ -308,7 +310,10 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
     n_bad = __reduce_add_sync(kFullMask, n_bad);
     n_mis = __reduce_add_sync(kFullMask, n_mis);
     n_full = __reduce_add_sync(kFullMask, n_full);
+    irregular = __any_sync(kFullMask, irregular);
     if (lane == 0) {
+        // the scatter kernel of this call, and of later ones until a reset, then takes rows one by one
+        if (irregular) atomicOr(dv.errword, kErrIrregularCu);
         if (n_oob) flag_error(dv, TD_ERR_OOB_INDEX, CNT_OOB, n_oob);
         if (n_dup) flag_error(dv, TD_ERR_DUP_PUT, CNT_DUP, n_dup);
         if (n_bad) flag_error(dv, TD_ERR_BAD_LENGTH, CNT_BADLEN, n_bad);

@@ -12,6 +12,10 @@ constexpr int kMaxColumns = 32;
 constexpr int kPutCounterSlots = 64;         // streams that can put into a dock with chunks handed out by a counter
 constexpr uint32_t kRowAlign = 8;            // rows start on multiples of 8 elements (>= 16 bytes)
 constexpr uint32_t kFullMask = 0xffffffffu;
+// Internal bit of the dock's error word, never reported: a put since the last reset came with a
+// cu array that is not a non-decreasing sequence inside [0, data_elems].  Row positions in such
+// an array cannot be searched, so the scatter then takes its rows one by one.
+constexpr uint32_t kErrIrregularCu = 1u << 31;
 
 // counters[] slots (uint64 each)
 enum : int {
@@ -51,7 +55,9 @@ struct DockView {
     uint32_t reward_col;
     FastDiv  div_shard;                     // by samples per shard = N * prompts_per_shard
     uint32_t claim_words, consumed_words;   // words per consumer
-    uint32_t spin_limit;                    // polls before a look-back wait gives up
+    uint32_t spin_limit;                    // polls before a wait on a staged copy gives up
+    uint32_t lookback_limit;                // polls before a scan tile gives up waiting for a tile ahead of it
+    uint32_t debug_skip_tile;               // test hook: the scan tile of this number withholds its descriptor (none: ~0u)
     uint32_t pad0;
     double   eps;
     uint64_t cap[3];                        // elements per shard, by length class

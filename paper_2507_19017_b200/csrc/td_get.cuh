@@ -29,32 +29,34 @@ __device__ __forceinline__ uint32_t desc_seq(unsigned long long d) { return (uin
 __device__ __forceinline__ uint32_t desc_state(unsigned long long d) { return (uint32_t)(d >> 30) & 3u; }
 __device__ __forceinline__ uint32_t desc_count(unsigned long long d) { return (uint32_t)d & 0x3fffffffu; }
 
-// Scratch of one (call, consumer): [0] ticket, [1] reserved, [2 .. 2+T) tile descriptors, then
-// the candidate list int32[G]: the r-th ready group in index order, one's complement when the
-// claim was lost to a concurrent get.
+// Scratch of one (call, consumer): [0] ticket, [1] the gather's chunk counter, [2 .. 2+T) tile
+// descriptors, then uint32[T] (padded to a multiple of 8 bytes) the exclusive rank each tile
+// started from, then the candidate list int32[G]: the r-th ready group in index order, one's
+// complement when the claim was lost to a concurrent get.
 struct SelScratch {
     unsigned long long *ticket;
     unsigned long long *desc;
+    uint32_t *excl;
     int32_t *cand;
 };
 // A tile is 256 groups per pass; a dock of more than kSelWideFrom groups gives every tile
 // kSelWide passes (the tiles' tickets and descriptors are a serial chain: about 10 ns per tile,
 // which outweighs the status words once there are thousands of tiles).
 constexpr uint32_t kSelWide = 4, kSelWideFrom = 65536;
-__host__ __device__ __forceinline__ uint32_t sel_passes(uint32_t G) { return G > kSelWideFrom ? kSelWide : 1u; }
-__host__ __device__ __forceinline__ uint32_t sel_tiles(uint32_t G) {
-    const uint32_t per = kSelThreads * sel_passes(G);
-    return (G + per - 1) / per;
+__host__ __device__ constexpr uint32_t sel_passes(uint32_t G) { return G > kSelWideFrom ? kSelWide : 1u; }
+__host__ __device__ constexpr uint32_t sel_tiles(uint32_t G) {
+    return (G + kSelThreads * sel_passes(G) - 1) / (kSelThreads * sel_passes(G));
 }
-__host__ __device__ __forceinline__ size_t sel_scratch_bytes(uint32_t G) {
-    size_t b = (2 + (size_t)sel_tiles(G)) * 8 + (size_t)G * 4;
-    return (b + 15) & ~size_t(15);
+__host__ __device__ constexpr size_t sel_excl_bytes(uint32_t G) { return (((size_t)sel_tiles(G) * 4) + 7) & ~size_t(7); }
+__host__ __device__ constexpr size_t sel_scratch_bytes(uint32_t G) {
+    return ((2 + (size_t)sel_tiles(G)) * 8 + sel_excl_bytes(G) + (size_t)G * 4 + 15) & ~size_t(15);
 }
 __host__ __device__ __forceinline__ SelScratch sel_scratch(void *p, uint32_t G) {
     SelScratch s;
     s.ticket = reinterpret_cast<unsigned long long *>(p);
     s.desc = s.ticket + 2;
-    s.cand = reinterpret_cast<int32_t *>(s.desc + sel_tiles(G));
+    s.excl = reinterpret_cast<uint32_t *>(s.desc + sel_tiles(G));
+    s.cand = reinterpret_cast<int32_t *>(reinterpret_cast<uint8_t *>(s.excl) + sel_excl_bytes(G));
     return s;
 }
 
@@ -194,7 +196,11 @@ __device__ __forceinline__ void select_claim(const DockView &dv, uint32_t *claim
 // give the rank inside the tile, a decoupled look-back over the tile descriptors gives the
 // rank before it, and the first max_groups ready groups are claimed with one atomicOr per
 // warp.  Tiles take their number from a ticket, so a tile only ever waits for tiles that have
-// already started; the wait is bounded all the same.
+// already started; the wait is bounded all the same (dv.lookback_limit polls).  A tile that gives
+// up marks its descriptor failed and claims nothing; the tiles ahead of it may already have
+// claimed, which is why a tile records the rank it started from before it publishes its prefix:
+// the finalize kernel, which serves nothing from a scan that did not come through, hands exactly
+// those claims back.
 // ---------------------------------------------------------------------------------------------
 template <int kPasses>
 __global__ void __launch_bounds__(kSelThreads)
@@ -226,6 +232,7 @@ get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
         return;
     }
     const uint32_t tile = s_tile;
+    if (tile == dv.debug_skip_tile) return;            // test hook: this tile never shows up; its successors' waits run out
     TileState<kPasses> ts;
     const uint32_t tile_count = select_eval<kPasses>(dv, claim, need, tile, s_warp, ts);
 
@@ -233,7 +240,10 @@ get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
         uint32_t excl = 0;
         bool failed = s_failed;
         if (tile == 0) {
-            if (lane == 0) st_release_u64(&sc.desc[0], desc_pack(seq, kStatePrefix, tile_count));
+            if (lane == 0) {
+                sc.excl[0] = 0;
+                st_release_u64(&sc.desc[0], desc_pack(seq, kStatePrefix, tile_count));
+            }
         } else {
             if (lane == 0) st_release_u64(&sc.desc[tile], desc_pack(seq, kStateAggregate, tile_count));
             // look back over windows of 32 predecessors
@@ -249,7 +259,7 @@ get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
                         d = ld_acquire_u64(&sc.desc[t]);
                         if (desc_seq(d) == seq && desc_state(d) != 0) break;
                         __nanosleep(32);
-                    } while (++polls < dv.spin_limit);
+                    } while (++polls < dv.lookback_limit);
                     if (desc_seq(d) != seq || desc_state(d) == 0) state = kStateFailed;
                     else { state = desc_state(d); count = desc_count(d); }
                 }
@@ -262,9 +272,11 @@ get_select_kernel(const DockView dv, const __grid_constant__ GetInline one,
                 excl += __reduce_add_sync(kFullMask, lane <= upto ? count : 0u);
                 if (first < 32u) done = true; else look -= 32;
             }
-            if (lane == 0)
+            if (lane == 0) {
+                if (!failed) sc.excl[tile] = excl;     // ordered ahead of the descriptor by its release
                 st_release_u64(&sc.desc[tile], failed ? desc_pack(seq, kStateFailed, 0)
                                                       : desc_pack(seq, kStatePrefix, excl + tile_count));
+            }
         }
         if (lane == 0) { s_excl = excl; s_failed = failed; }
     }
@@ -386,10 +398,38 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     } else {
         // how many groups were ready, from the last tile's inclusive prefix; the first candidates
         // are asked for in the same breath (which of them count is known once the prefix is here)
-        const unsigned long long last = sc.desc[sel_tiles(dv.G) - 1];
+        const uint32_t tiles = sel_tiles(dv.G);
+        const unsigned long long last = sc.desc[tiles - 1];
         if (tid < rq.max_groups && rq.rank_base + tid < dv.G) g_first = sc.cand[rq.rank_base + tid];
-        if (desc_seq(last) != seq || desc_state(last) != kStatePrefix) status |= TD_ERR_LOOKBACK_TIMEOUT;
-        else total = min(desc_count(last), cs.max_groups);
+        // Every tile must have come through, not only the last one: a tile may give up on a slow
+        // predecessor that its own successors still catch, and its ranks of the candidate list
+        // are then never written.
+        bool bad = false;
+        for (uint32_t t = tid; t < tiles; t += kThreads) {
+            const unsigned long long d = t == tiles - 1 ? last : sc.desc[t];
+            bad |= desc_seq(d) != seq || desc_state(d) != kStatePrefix;
+        }
+        if (__syncthreads_or(bad)) {
+            // Nothing is served from this scan.  The tiles that did come through have claimed
+            // their groups (ranks [excl, inclusive prefix) below the consumer's limit, except the
+            // ones lost to another get): the consumer's first request of the call gives them back.
+            status |= TD_ERR_LOOKBACK_TIMEOUT;
+            if (rq.rank_base == 0) {
+                if (tid == 0) atomicAdd(&dv.counters[CNT_TIMEOUT], 1ull);      // once per consumer and call, whatever the tiles counted
+                uint32_t *claim = dv.claim + (size_t)c * dv.claim_words;
+                for (uint32_t t = tid; t < tiles; t += kThreads) {
+                    const unsigned long long d = sc.desc[t];
+                    if (desc_seq(d) != seq || desc_state(d) != kStatePrefix) continue;
+                    const uint32_t r1 = min(desc_count(d), cs.max_groups);
+                    for (uint32_t r = sc.excl[t]; r < r1; ++r) {
+                        const int32_t g = sc.cand[r];
+                        if (g >= 0) atomicAnd(&claim[(uint32_t)g >> 5], ~(1u << ((uint32_t)g & 31)));
+                    }
+                }
+            }
+        } else {
+            total = min(desc_count(last), cs.max_groups);
+        }
     }
     const uint32_t lo = rq.rank_base;
     const uint32_t hi = min(lo + rq.max_groups, total);

@@ -29,6 +29,21 @@ __device__ __forceinline__ bool put_entry_live(const DockView &dv, const PutArgs
     return true;
 }
 
+// Where row i of item `a` goes in its arena if the alloc kernel accepted it, else nullptr.
+__device__ __forceinline__ uint8_t *put_row_dst(const DockView &dv, const PutArgs &a, uint32_t L, uint32_t bit,
+                                                uint32_t esz, uint32_t i, int64_t c0, int64_t c1) {
+    const int32_t s = a.idx[i];
+    if (s < 0 || (uint32_t)s >= dv.n) return nullptr;
+    const uint32_t st = dv.status[s];          // three loads side by side
+    const int32_t ln = dv.len[L][s];
+    const long long off = dv.off[L][s];
+    if (st & bit) return nullptr;
+    if (c0 < 0 || c1 < c0 || (uint64_t)c1 > a.data_elems) return nullptr;
+    if ((int64_t)ln != c1 - c0) return nullptr;
+    if (off < 0) return nullptr;
+    return dv.colbase[a.column] + ((uint64_t)shard_of(dv, (uint32_t)s) * dv.cap[L] + (uint64_t)off) * esz;
+}
+
 // Scatter.  The packed sources of the call's ragged items, laid end to end with every row
 // charged kRowCost on top of its bytes, are cut into equal chunks, so that work is balanced
 // over tokens and rows rather than samples; warps stride over the chunks (see "Chunked ragged
@@ -69,6 +84,31 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
     }
     __syncthreads();
     const uint64_t n_warps = (uint64_t)gridDim.x * kCopyWarps;
+    // A cu array that is not a non-decreasing sequence inside its data (the alloc kernel of this
+    // call, or of an earlier one since the last reset, met one) gives rows no searchable position:
+    // the warps then take the rows of every item one by one, each row checked for itself, so that
+    // exactly the rows the alloc kernel accepted are copied, as the publish kernel assumes.
+    if (*dv.errword & kErrIrregularCu) {
+        for (uint32_t it = 0; it < batch.n_items; ++it) {
+            const PutArgs &a = batch.item[it];
+            const uint32_t L = dv.col_cls[a.column], esz = dv.col_esz[a.column];
+            if (L == TD_SCALAR) continue;
+            const uint8_t *lo = a.data, *hi = a.data + a.data_elems * esz;
+            for (uint64_t i = (uint64_t)blockIdx.x * kCopyWarps + (tid >> 5); i < item_rows[it]; i += n_warps) {
+                const int64_t c0 = a.cu[i], c1 = a.cu[i + 1];
+                uint8_t *dst = put_row_dst(dv, a, L, 1u << a.column, esz, (uint32_t)i, c0, c1);
+                if (!dst) continue;
+                const uint8_t *src = a.data + (uint64_t)c0 * esz;
+                for (uint64_t left = (uint64_t)(c1 - c0) * esz; left; ) {
+                    const uint32_t m = (uint32_t)min(left, (uint64_t)1 << 30);
+                    pipe.push<true>(dst, src, m, lane, lo, hi);
+                    dst += m; src += m; left -= m;
+                }
+            }
+        }
+        if (pipe.finish(lane) && lane == 0) flag_error(dv, TD_ERR_COPY_TIMEOUT, CNT_TIMEOUT);
+        return;
+    }
     // With plenty to do (a full-size chunk and more per warp) and a counter to draw from, the
     // chunks after a warp's first are handed out one by one: equal bytes are not equal time, and
     // some SMs get through theirs sooner than others.  Otherwise every warp takes a fixed share.
@@ -98,22 +138,10 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
             if (L == TD_SCALAR || item_rows[it] == 0) continue;
             const uint64_t b1 = min(g0 - start, item_bytes[it]);
             if (b1 <= b0) continue;
-            uint8_t *arena = dv.colbase[a.column];
-            const uint64_t cap = dv.cap[L];
             warp_copy_chunk<false>(a.cu, item_rows[it], b0, b1, const_cast<uint8_t *>(a.data), esz, lane,
                                    a.data, a.data + a.data_elems * esz, pipe, a.idx,
                                    [&](uint32_t i, int64_t c0, int64_t c1) -> uint8_t * {
-                                       // the row is live if the alloc kernel accepted it
-                                       const int32_t s = a.idx[i];
-                                       if (s < 0 || (uint32_t)s >= dv.n) return nullptr;
-                                       const uint32_t st = dv.status[s];          // three loads side by side
-                                       const int32_t ln = dv.len[L][s];
-                                       const long long off = dv.off[L][s];
-                                       if (st & bit) return nullptr;
-                                       if (c1 < c0 || (uint64_t)c1 > a.data_elems) return nullptr;
-                                       if ((int64_t)ln != c1 - c0) return nullptr;
-                                       if (off < 0) return nullptr;
-                                       return arena + ((uint64_t)shard_of(dv, (uint32_t)s) * cap + (uint64_t)off) * esz;
+                                       return put_row_dst(dv, a, L, bit, esz, i, c0, c1);   // live if the alloc kernel accepted it
                                    });
         }
         ch = work_counter ? shfl_u64(next, 0) : next;

@@ -43,23 +43,32 @@ def test_bulk_configs_full_size(G, cid):
     assert sum(b.n_samples for _, b in batches) == w.n * len(w.consumers)
 
 
-def test_config5_full_size_packed_and_padded(G):
+def test_config5_full_size_packed(G):
     w = wl.make_config(5)
     g, o, batches = G.replay_both(w)
     assert sum(b.n_samples for _, b in batches) == w.n * len(w.consumers)
-    # right-padded gets of the same dock: reset the claims by re-running puts on fresh docks is
-    # costly at this size, so gather parity is checked on sampled micro-batches instead
-    rng = np.random.default_rng(5)
-    g.dock.reset(); o.reset()
+
+
+def test_config5_full_size_padded_drain(G):
+    """The R1-shaped dock drained to exhaustion into right-padded rows for an id-only consumer and
+    for the actor update (one set of output buffers per consumer, reused get after get): every
+    batch and the final tables against the oracle."""
+    w = wl.make_config(5, schedule="none")
+    o, g = H.make_oracle(w), G.GpuDock(w)
+    idx = np.arange(w.n, dtype=np.int32)
     for c in range(len(w.columns)):
-        cu, data = w.pack(c, np.arange(w.n, dtype=np.int32))
-        o.put(c, np.arange(w.n), cu, data); g.put(c, np.arange(w.n), cu, data)
-    for _ in range(3):
+        cu, data = w.pack(c, idx)
+        o.put(c, idx, cu, data); g.put(c, idx, cu, data)
+    served = {0: 0, 3: 0}
+    for j in range(w.n // w.micro_batch + 1):                   # one get past the end: an empty batch
         for cons in (0, 3):
             want = o.get(cons, w.micro_batch, ora.PADDED, w.pad_prompt_to, w.pad_response_to)
             got = g.get(cons, w.micro_batch, td.PADDED, w.pad_prompt_to, w.pad_response_to)
-            G.assert_batch_equal(got, want, f"padded consumer {cons}")
-    del rng
+            G.assert_batch_equal(got, want, f"padded get {j} consumer {cons}")
+            served[cons] += got.n_samples
+    assert served == {0: w.n, 3: w.n}
+    G.assert_state_equal(g, o, arenas=False, ctx="padded drain")
+    G.assert_stats_equal(g, o, "padded drain")
 
 
 def test_config4_interleaved_serialized(G):
@@ -261,6 +270,87 @@ def test_wide_tiles_of_a_large_dock(G):
     G.assert_state_equal(g2, o2, arenas=False, ctx="wide2")
 
 
+def _twelve_tile_dock(G):
+    w = wl.make_custom("timeout", 12 * 256, 1, 4, prompt_len=(0, 3), response=("uniform", 0, 5), vocab=100,
+                       micro_batch=12 * 256, seed=31, schedule="none")
+    o, g = H.make_oracle(w), G.GpuDock(w)
+    idx = np.arange(w.n, dtype=np.int32)
+    for c in range(len(w.columns)):
+        cu, data = w.pack(c, idx)
+        o.put(c, idx, cu, data); g.put(c, idx, cu, data)
+    return w, o, g
+
+
+def _claimed(g, consumer):
+    return H.popcount_words(g.table(4, consumer, np.uint32))
+
+
+@pytest.mark.parametrize("skip_tile", [5, 0, 11])
+def test_lookback_wait_that_runs_out_serves_nothing_and_hands_claims_back(G, skip_tile):
+    """A scan tile that never publishes its descriptor: the tiles behind it wait their (short)
+    limit and give up, the get reports TD_ERR_LOOKBACK_TIMEOUT and serves nothing - and the
+    groups that the tiles ahead of it had already claimed are free again, so that the next get
+    serves the lowest groups as if nothing had happened."""
+    w, o, g = _twelve_tile_dock(G)
+    one = g.get(2, 256)                                          # an ordinary get first: groups 0..255 to consumer 2
+    G.assert_batch_equal(one, o.get(2, 256), "before")
+    before = {c: _claimed(g, c) for c in range(len(w.consumers))}
+    g.dock.debug_lookback(poll_limit=64, skip_tile=skip_tile)
+    for cons, m in ((3, w.n), (2, 1024)):
+        got = g.get(cons, m)
+        assert got.status == td.ERR_LOOKBACK_TIMEOUT and got.n_samples == 0 and got.n_groups == 0
+        assert got.prompt_tokens == 0 and got.response_tokens == 0
+    assert {c: _claimed(g, c) for c in range(len(w.consumers))} == before
+    rep = g.dock.validate()
+    assert rep.violations == 0 and rep.served[2] == 256 and rep.served[3] == 0
+    st = g.dock.status()
+    assert st.error_word == td.ERR_LOOKBACK_TIMEOUT and st.n_lookback_timeouts >= 2
+    assert st.got_samples[3] == 0 and st.got_samples[2] == 256
+    g.dock.debug_lookback()                                      # default limit, no tile withheld
+    for cons, m in ((3, 700), (2, 1024), (3, w.n), (2, w.n)):
+        G.assert_batch_equal(g.get(cons, m), o.get(cons, m), f"after, consumer {cons}")
+    G.assert_state_equal(g, o, arenas=False, ctx="after timeouts")
+    assert _claimed(g, 3) == w.G and _claimed(g, 2) == w.G
+
+
+def test_lookback_timeout_inside_a_plan(G):
+    """td_get_many over a scan that does not come through: every request of every consumer returns
+    nothing, no claim stays behind, and the same plan serves everything once the scan works."""
+    w, o, g = _twelve_tile_dock(G)
+    bufs = [g.buffers(c, 800, key=j) for j, c in enumerate((0, 3, 0, 3, 1))]
+    plan = g.dock.plan(bufs)
+    g.dock.debug_lookback(poll_limit=64, skip_tile=3)
+    g.dock.get_many(plan)
+    for b in bufs:
+        r = g.read(b)
+        assert r.status == td.ERR_LOOKBACK_TIMEOUT and r.n_samples == 0
+    assert all(_claimed(g, c) == 0 for c in range(len(w.consumers)))
+    assert g.dock.validate().violations == 0
+    g.dock.debug_lookback()
+    g.dock.get_many(plan)
+    for b, c in zip(bufs, (0, 3, 0, 3, 1)):
+        G.assert_batch_equal(g.read(b), o.get(c, 800), f"plan consumer {c}")
+    G.assert_state_equal(g, o, arenas=False, ctx="plan after timeout")
+
+
+def test_scan_scratch_in_use_by_a_later_launch_is_refused(G):
+    """A ticket word that carries a later launch's sequence number (what a tile finds when two
+    gets in flight were given the same scratch): the scan refuses, nothing is served or claimed,
+    and the scratch is usable again for the next get."""
+    w, o, g = _twelve_tile_dock(G)
+    bufs = g.buffers(0, 1024)
+    ticket = bufs.scratch[:8].view(torch.int64)
+    ticket.fill_(-(1 << 32))                                     # sequence number 0xffffffff, no tile started
+    g.dock.debug_lookback(poll_limit=64)
+    g.dock.get(bufs)
+    r = g.read(bufs)
+    assert r.status == td.ERR_LOOKBACK_TIMEOUT and r.n_samples == 0
+    assert _claimed(g, 0) == 0 and g.dock.validate().violations == 0
+    g.dock.debug_lookback()
+    g.dock.get(bufs)
+    G.assert_batch_equal(g.read(bufs), o.get(0, 1024), "after the refusal")
+
+
 # ------------------------------------------------------------------- batched calls
 def _many_vs_serial(G, w, mode=td.PACKED, fused=False):
     """All columns in one td_put_many, all gets of the schedule in one td_get_many; the oracle
@@ -456,6 +546,49 @@ def test_put_errors_are_counted_and_skipped(G):
     G.assert_stats_equal(g, o, "errors")
     st = g.dock.status()
     assert st.error_word == td.ERR_OOB_INDEX | td.ERR_DUP_PUT | td.ERR_LEN_MISMATCH | td.ERR_BAD_LENGTH
+
+
+def test_bad_cu_entry_in_the_middle_of_a_put_skips_only_that_row(G):
+    """cu arrays that go down in the middle of a many-row put, by a little and by more than any
+    row is long (row positions can then not be searched): only the offending rows are refused,
+    every other row of the call is stored with its payload, and later puts are not disturbed."""
+    w = wl.make_custom("badcu", 40, 4, 4, prompt_len=(3, 900), response=("uniform", 1, 3000), vocab=50000,
+                       micro_batch=160, seed=12, with_entropy=True, schedule="none")
+    room = 2 * w.shard_capacity(wl.RESPONSE)                    # the misread rows come out longer than the true ones
+    o, g = H.make_oracle(w, response_cap=room), G.GpuDock(w, response_cap=room)
+    rid, pid, ent = w.column_index("response_ids"), w.column_index("prompt_ids"), w.column_index("entropy")
+    idx = np.arange(w.n, dtype=np.int32)
+
+    def both(col, ind, cu, data):
+        o.put(col, ind, cu, data); g.put(col, ind, cu, data)
+
+    # response ids: one entry far below its predecessor (row 50 then ends before it starts, and row
+    # 51 reaches back over it), another one two elements below (row 100)
+    cu, data = w.pack(rid, idx)
+    bad = cu.copy()
+    bad[51] = cu[50] - 2000
+    bad[101] = cu[100] - 2
+    both(rid, idx, bad, data)
+    assert o.stats().n_bad_length == 2 and o.stats().put_accepted[rid] == w.n - 2
+    # prompt ids of the second half with a last entry of -1: the array's total is useless, every
+    # row but the last is in order
+    half = idx[w.n // 2:]
+    cu_p, data_p = w.pack(pid, half)
+    cu_p2 = cu_p.copy()
+    cu_p2[-1] = -1
+    both(pid, half, cu_p2, data_p)
+    assert o.stats().n_bad_length == 3 and o.stats().put_accepted[pid] == len(half) - 1
+    # clean puts afterwards (the dock has seen irregular arrays; results must not change); the
+    # entropy rows of the two samples whose response length was misread are refused
+    both(pid, idx[:w.n // 2], *w.pack(pid, idx[:w.n // 2]))
+    both(ent, idx, *w.pack(ent, idx))
+    assert o.stats().n_len_mismatch == 2
+    G.assert_state_equal(g, o, ctx="bad cu")
+    G.assert_stats_equal(g, o, "bad cu")
+    assert g.dock.status().error_word == td.ERR_BAD_LENGTH | td.ERR_LEN_MISMATCH
+    # what was stored can be served: the id-only consumers get every complete group
+    for cons in (0, 1):
+        G.assert_batch_equal(g.get(cons, w.n), o.get(cons, w.n), f"consumer {cons}")
 
 
 def test_arena_full_refuses_only_rows_without_room(G):

@@ -99,6 +99,17 @@ def test_every_sample_dispatched_exactly_once_per_consumer():
     # lowest index first: with everything ready, consumer batches come in index order
     for c in seen:
         assert seen[c] == list(range(w.n))
+    # the dispatch counters say what this test saw dispatched: samples per consumer, and their
+    # tokens counted from the generator's lengths
+    st = d.stats()
+    tokens = {c: 0 for c in seen}
+    for c, b in batches:
+        tokens[c] += int(w.len_prompt[b.indices].sum(dtype=np.int64) + w.len_response[b.indices].sum(dtype=np.int64))
+    for c in seen:
+        assert st.got_samples[c] == len(seen[c]) == w.n
+        assert st.got_tokens[c] == tokens[c] == w.tokens_total()
+    assert all(st.got_samples[c] == 0 and st.got_tokens[c] == 0 for c in range(len(w.consumers), 32))
+    assert st.n_truncated == 0 and st.error_word == 0
 
 
 def test_batches_match_generator_rows_and_cumsum():
@@ -322,6 +333,14 @@ def test_output_capacity_truncates_at_group_boundary():
     first_long = int(np.argmax(w.len_response == wide))
     b3 = d.get(1, w.n, ora.PADDED, int(w.len_prompt.max()), wide - 1)
     assert b3.n_samples == (first_long // w.N) * w.N and b3.status == ora.ERR_OUT_TRUNC
+    # counters: two of the three gets made here were cut; samples and tokens per consumer are
+    # those of the batches this test received
+    st = d.stats()
+    assert st.n_truncated == 2 and st.error_word == ora.ERR_OUT_TRUNC
+    tok = lambda idx: int(w.len_prompt[idx].sum() + w.len_response[idx].sum())
+    assert st.got_samples[0] == 8 and st.got_tokens[0] == tok(np.arange(8))
+    assert st.got_samples[1] == b3.n_samples and st.got_tokens[1] == tok(b3.indices)
+    assert st.got_samples[2] == 0 and st.got_tokens[2] == 0
 
 
 def test_reset_forgets_tables_keeps_payload():

@@ -37,11 +37,19 @@ def filled_dock(G, w):
 
 
 def test_static_scratch_get_matches_td_get_on_consecutive_calls(G):
-    # 600 prompts: three scan tiles, so the tile descriptors in the shared array are really used
-    w = wl.make_custom("noalloc", 600, 2, 4, prompt_len=(1, 40), response=("uniform", 0, 90), vocab=30000,
+    # 2000 prompts: more than one launch's finalize kernel can scan by itself, so every call runs
+    # the scan kernel (8 tiles: ticket, tile descriptors, start ranks and candidate list all live
+    # in the shared array) on top of whatever the call before it left there
+    from tests import helpers as H
+    w = wl.make_custom("noalloc", 2000, 2, 4, prompt_len=(1, 40), response=("uniform", 0, 90), vocab=30000,
                        micro_batch=500, seed=77, with_entropy=True, schedule="none")
     ref, sta = filled_dock(G, w), filled_dock(G, w)
-    calls = [(3, 500), (3, 500), (0, 64), (0, 2 * w.n), (1, 10), (1, 10)]      # two and more in a row
+    ora_dock = H.make_oracle(w)
+    idx = np.arange(w.n, dtype=np.int32)
+    for c in range(len(w.columns)):
+        ora_dock.put(c, idx, *w.pack(c, idx))
+    launches = sta.dock.launch_count()
+    calls = [(3, 500), (0, 500), (3, 500), (3, 64), (0, 2 * w.n), (1, 10), (1, 10), (3, 1500)]
     for j, (consumer, m) in enumerate(calls):
         want = ref.get(consumer, m, key=j)                    # td_get with caller-supplied scratch
         bufs = sta.buffers(consumer, m, key=j)
@@ -49,11 +57,13 @@ def test_static_scratch_get_matches_td_get_on_consecutive_calls(G):
         sta.dock.get_static(bufs)
         got = sta.read(bufs)
         G.assert_batch_equal(got, want, f"call {j}")
+        G.assert_batch_equal(got, ora_dock.get(consumer, m), f"call {j} against the oracle")
         assert got.status == 0
-    assert ref.get(3, 500, key="x").n_samples == 200          # the drains stayed in step to the end
-    b = sta.buffers(3, 500, key="x")
+    assert sta.dock.launch_count() - launches == 3 * len(calls)           # select, finalize, gather every time
+    assert ref.get(3, 4000, key="x").n_samples == w.n - 2564  # the drains stayed in step to the end
+    b = sta.buffers(3, 4000, key="x")
     sta.dock.get_static(b)
-    assert sta.read(b).n_samples == 200
+    assert sta.read(b).n_samples == w.n - 2564
     for c in range(len(w.consumers)):
         assert np.array_equal(sta.table(4, c, np.uint32), ref.table(4, c, np.uint32))
         assert np.array_equal(sta.table(5, c, np.uint32), ref.table(5, c, np.uint32))
