@@ -106,7 +106,12 @@ typedef struct {
 } td_result;
 
 /* Output buffers of one get.  The struct itself is host memory; every pointer in it is
- * caller-owned DEVICE memory that stays valid until the get has executed. */
+ * caller-owned DEVICE memory that stays valid until the get has executed.  The payload buffers
+ * (col[], seq, seq_advantages) may instead be page-locked host memory that the device can
+ * address (cudaHostAlloc / cudaHostRegister under unified addressing): the gather then writes
+ * the batch across the bus itself, in wide contiguous stores, and a worker whose tensors live on
+ * the host needs no copy afterwards.  indices, the cu arrays, advantages and result are read
+ * back by the kernels and belong in device memory. */
 typedef struct {
     int32_t  mode;                    /* TD_PACKED: column c holds its rows back to back, row i at
                                          cu_<class>[i]; TD_PADDED: row i at i * pad_<class>_to,
@@ -270,7 +275,8 @@ int td_put_back_many(td_dock *dock, const td_back_req *reqs, uint32_t n_reqs, vo
  *   td_plan_bytes   device bytes a plan of n_req requests needs (request table + scan scratch).
  *   td_plan_create  checks the requests (host array; out.scratch is not used), uploads them into
  *                   d_plan (device, 256-byte aligned, caller-owned, must outlive the plan) on
- *                   `stream`.  n_req * n_columns must not exceed 4096.
+ *                   `stream`.  n_req * n_columns must not exceed 4096, and the requests' output
+ *                   room together must stay below 256 GiB (TD_EINVAL).
  *   td_get_many     enqueues the gets.  A plan must not be in flight twice at the same time;
  *                   reusing it on one stream, call after call, is the intended use. */
 typedef struct {

@@ -245,11 +245,21 @@ class GetBuffers:
                  pad_prompt_to: int = 0, pad_response_to: int = 0,
                  capacities: Optional[Dict[int, int]] = None, want: Optional[Sequence[int]] = None,
                  prompt_tokens_cap: Optional[int] = None, response_tokens_cap: Optional[int] = None,
-                 seq: Optional[Tuple[int, int]] = None, seq_adv: bool = False, seq_cap: Optional[int] = None):
+                 seq: Optional[Tuple[int, int]] = None, seq_adv: bool = False, seq_cap: Optional[int] = None,
+                 host_payload: bool = False):
         """seq = (prompt column, response column) adds the fused token stream, seq_adv its
-        advantage twin; seq_cap is the room behind each (default: both token caps together)."""
+        advantage twin; seq_cap is the room behind each (default: both token caps together).
+        host_payload: the column buffers (and the stream) are pinned host memory that the device
+        writes directly; indices, cu_seqlens, advantages and the result block stay on the device."""
         import torch
         dev = dock.device
+        self.host_payload = host_payload
+
+        def payload(n, dtype):
+            if host_payload:
+                return torch.empty(n, dtype=dtype, pin_memory=True)
+            return torch.empty(n, dtype=dtype, device=dev)
+
         self.dock, self.consumer, self.max_samples, self.mode = dock, consumer, max_samples, mode
         self.pad_prompt_to, self.pad_response_to = pad_prompt_to, pad_response_to
         i32 = torch.int32
@@ -279,7 +289,7 @@ class GetBuffers:
                     raise ValueError("packed ragged columns need prompt_tokens_cap / response_tokens_cap "
                                      "or explicit capacities")
             self.caps[c] = cap
-            self.cols[c] = torch.empty(max(cap, 1), dtype=tdt[dt], device=dev)
+            self.cols[c] = payload(max(cap, 1), tdt[dt])
         go = TdGetOut()
         go.mode, go.pad_prompt_to, go.pad_response_to = mode, pad_prompt_to, pad_response_to
         go.indices, go.cu_prompt = self.indices.data_ptr(), self.cu_prompt.data_ptr()
@@ -296,10 +306,10 @@ class GetBuffers:
             go.seq_capacity_elems = cap
             if seq is not None:
                 go.seq_prompt_col, go.seq_response_col = seq
-                self.seq = torch.empty(max(cap, 1), dtype=tdt[dock.columns[seq[0]][0]], device=dev)
+                self.seq = payload(max(cap, 1), tdt[dock.columns[seq[0]][0]])
                 go.seq = self.seq.data_ptr()
             if seq_adv:
-                self.seq_advantages = torch.empty(max(cap, 1), dtype=torch.float32, device=dev)
+                self.seq_advantages = payload(max(cap, 1), torch.float32)
                 go.seq_advantages = self.seq_advantages.data_ptr()
         self.struct = go
 
@@ -320,7 +330,10 @@ class HostGetBuffers:
         self.cu_seq = torch.zeros(bufs.cu_seq.shape, dtype=torch.int32).pin_memory()
         self.advantages = (torch.zeros(bufs.advantages.shape, dtype=torch.float32).pin_memory()
                            if bufs.advantages is not None else None)
-        self.cols = {c: torch.zeros(t.shape, dtype=t.dtype).pin_memory() for c, t in bufs.cols.items()}
+        # payload that the device already writes into host memory needs no second buffer
+        self.payload_in_place = bool(getattr(bufs, "host_payload", False))
+        self.cols = ({c: t for c, t in bufs.cols.items()} if self.payload_in_place else
+                     {c: torch.zeros(t.shape, dtype=t.dtype).pin_memory() for c, t in bufs.cols.items()})
         # the result block too lives in pinned memory: a copy into pageable memory stalls the caller
         self._result_mem = torch.zeros(C.sizeof(TdResult), dtype=torch.uint8).pin_memory()
         self.result = TdResult.from_address(self._result_mem.data_ptr())
@@ -329,7 +342,7 @@ class HostGetBuffers:
         go.indices, go.cu_prompt = self.indices.data_ptr(), self.cu_prompt.data_ptr()
         go.cu_response, go.cu_seq = self.cu_response.data_ptr(), self.cu_seq.data_ptr()
         for c, t in self.cols.items():
-            go.col[c] = t.data_ptr()
+            go.col[c] = None if self.payload_in_place else t.data_ptr()      # NULL: nothing to copy
             go.col_capacity_elems[c] = t.numel()
         go.advantages = self.advantages.data_ptr() if self.advantages is not None else None
         go.result = C.addressof(self.result)

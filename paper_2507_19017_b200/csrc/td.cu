@@ -45,7 +45,7 @@ inline uint32_t esize_of(int32_t dtype) { return dtype == TD_BF16 ? 2u : 4u; }
 constexpr size_t kStageSmem = (size_t)kCopyWarps * kPipeSmemPerWarp;
 size_t scatter_smem_bytes() { return kStageSmem; }
 size_t gather_smem_bytes(uint32_t n_req, uint32_t jobs_per_req) {
-    return kStageSmem + (size_t)kCopyWarps * 8 + (size_t)n_req * jobs_per_req * 8 + (size_t)n_req * 4;
+    return kStageSmem + (size_t)kCopyWarps * 8 + (size_t)n_req * jobs_per_req * 4 + (size_t)n_req * 4;
 }
 
 struct Layout {
@@ -424,6 +424,13 @@ uint64_t room_bytes_of(const DockView &v, uint32_t consumer, uint32_t max_sample
 bool wants_stream(const td_get_out &out) { return out.seq || out.seq_advantages; }
 uint32_t jobs_per_req(const DockView &v, bool stream) { return v.ncol + (stream ? kSeqJobs : 0u); }
 
+// Upper bound of what a request adds to the space the gather cuts into chunks: its output room
+// plus the fixed charge of every row of every job.
+uint64_t extent_bound_of(const DockView &v, uint32_t consumer, uint32_t max_samples, const td_get_out &out, uint32_t jpr) {
+    const uint64_t rows = (uint64_t)std::min(max_samples / v.N, v.G) * v.N;
+    return room_bytes_of(v, consumer, max_samples, out) + rows * jpr * kRowCost + (uint64_t)jpr * kJobUnit;
+}
+
 int check_get_out(const DockView &v, uint32_t consumer, uint32_t max_samples, const td_get_out *out) {
     if (!out || consumer >= v.ncons) return TD_EINVAL;
     if (max_samples / v.N == 0) return TD_EINVAL;
@@ -545,6 +552,7 @@ int get_one(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_ou
     one.cs.scratch = scratch;
     const uint32_t seq = g_seq.fetch_add(1, std::memory_order_relaxed);
     const uint32_t jpr = jobs_per_req(v, wants_stream(*out));
+    if (extent_bound_of(v, consumer, max_samples, *out, jpr) >= kMaxLaunchExtent) return TD_EINVAL;
 
     // word 1 of the scan scratch is the gather's chunk counter
     unsigned long long *counter = static_cast<unsigned long long *>(scratch) + 1;
@@ -684,8 +692,10 @@ int td_plan_create(td_dock *d, const td_get_req *reqs, uint32_t n_req, void *d_p
     int slot_of[32];
     for (int &x : slot_of) x = -1;
     uint32_t n_slots = 0;
-    uint64_t room = 0;
+    uint64_t room = 0, extent = 0;
     for (uint32_t q = 0; q < n_req; ++q) {
+        extent += extent_bound_of(v, reqs[q].consumer, reqs[q].max_samples, reqs[q].out, jpr);
+        if (extent >= kMaxLaunchExtent) { delete p; return TD_EINVAL; }      // more than one launch can address
         const uint32_t c = reqs[q].consumer;
         if (slot_of[c] < 0) {
             slot_of[c] = (int)n_slots;
@@ -957,15 +967,25 @@ namespace {
 int copy_batch_to_host(const DockView &v, uint32_t consumer, const td_get_out *dev_out, const td_get_out *host_out,
                        const td_result *res, cudaStream_t st) {
     const size_t n = res->n_samples;
+    // the transfers wanted, in order; neighbours that continue each other on both sides go as one
+    struct Piece { uint8_t *dst; const uint8_t *src; size_t bytes; };
+    Piece todo[8 + 2 * kMaxColumns];
+    int n_todo = 0;
     auto d2h = [&](void *dst, const void *src, size_t bytes) {
-        return !dst || !src || bytes == 0 || cudaMemcpyAsync(dst, src, bytes, cudaMemcpyDeviceToHost, st) == cudaSuccess;
+        if (!dst || !src || bytes == 0) return;
+        Piece p{static_cast<uint8_t *>(dst), static_cast<const uint8_t *>(src), bytes};
+        if (n_todo && todo[n_todo - 1].dst + todo[n_todo - 1].bytes == p.dst &&
+            todo[n_todo - 1].src + todo[n_todo - 1].bytes == p.src)
+            todo[n_todo - 1].bytes += bytes;
+        else
+            todo[n_todo++] = p;
     };
-    bool ok = d2h(host_out->indices, dev_out->indices, n * 4);
-    ok = ok && d2h(host_out->cu_prompt, dev_out->cu_prompt, (n + 1) * 4);
-    ok = ok && d2h(host_out->cu_response, dev_out->cu_response, (n + 1) * 4);
-    ok = ok && d2h(host_out->cu_seq, dev_out->cu_seq, (n + 1) * 4);
-    ok = ok && d2h(host_out->advantages, dev_out->advantages, n * 4);
-    for (uint32_t k = 0; k < v.ncol && ok; ++k) {
+    d2h(host_out->indices, dev_out->indices, n * 4);
+    d2h(host_out->cu_prompt, dev_out->cu_prompt, (n + 1) * 4);
+    d2h(host_out->cu_response, dev_out->cu_response, (n + 1) * 4);
+    d2h(host_out->cu_seq, dev_out->cu_seq, (n + 1) * 4);
+    d2h(host_out->advantages, dev_out->advantages, n * 4);
+    for (uint32_t k = 0; k < v.ncol; ++k) {
         if (!((v.outm[consumer] >> k) & 1u) || !dev_out->col[k] || !host_out->col[k]) continue;
         const uint32_t cls = v.col_cls[k];
         size_t elems;
@@ -973,19 +993,22 @@ int copy_batch_to_host(const DockView &v, uint32_t consumer, const td_get_out *d
         else if (dev_out->mode == TD_PACKED) elems = cls == TD_PROMPT ? res->prompt_tokens : res->response_tokens;
         else elems = n * (size_t)(cls == TD_PROMPT ? dev_out->pad_prompt_to : dev_out->pad_response_to);
         if (elems > host_out->col_capacity_elems[k]) return TD_EINVAL;
-        ok = d2h(host_out->col[k], dev_out->col[k], elems * v.col_esz[k]);
+        d2h(host_out->col[k], dev_out->col[k], elems * v.col_esz[k]);
     }
-    if (ok && dev_out->seq && host_out->seq) {
+    if (dev_out->seq && host_out->seq) {
         const size_t elems = res->prompt_tokens + res->response_tokens;
         if (elems > host_out->seq_capacity_elems) return TD_EINVAL;
-        ok = d2h(host_out->seq, dev_out->seq, elems * v.col_esz[dev_out->seq_prompt_col]);
+        d2h(host_out->seq, dev_out->seq, elems * v.col_esz[dev_out->seq_prompt_col]);
     }
-    if (ok && dev_out->seq_advantages && host_out->seq_advantages) {
+    if (dev_out->seq_advantages && host_out->seq_advantages) {
         const size_t elems = res->prompt_tokens + res->response_tokens;
         if (elems > host_out->seq_capacity_elems) return TD_EINVAL;
-        ok = d2h(host_out->seq_advantages, dev_out->seq_advantages, elems * 4);
+        d2h(host_out->seq_advantages, dev_out->seq_advantages, elems * 4);
     }
-    return ok ? TD_OK : TD_ECUDA;
+    for (int i = 0; i < n_todo; ++i)
+        if (cudaMemcpyAsync(todo[i].dst, todo[i].src, todo[i].bytes, cudaMemcpyDeviceToHost, st) != cudaSuccess)
+            return TD_ECUDA;
+    return TD_OK;
 }
 }  // namespace
 

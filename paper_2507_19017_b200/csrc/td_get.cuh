@@ -347,6 +347,10 @@ struct JobSize {
 // chunk never holds more than a few hundred of them.
 constexpr uint32_t kScalarCost = 64;
 static_assert(kScalarCost % 16 == 0, "a job's extent stays a multiple of 16");
+// Jobs are laid end to end in the chunked space on multiples of kJobUnit bytes, and the gather
+// keeps their ends as 32-bit counts of units: 2^32 units are 256 GiB of extent per launch.
+constexpr uint32_t kJobUnit = 64;
+constexpr uint64_t kMaxLaunchExtent = (uint64_t)kJobUnit << 32;
 
 // Extent of a job in the space the gather cuts into chunks (see kRowCost).
 __device__ __forceinline__ uint32_t job_cost_rows(const DockView &dv, const GetReq &rq, uint32_t k,
@@ -641,11 +645,13 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
     const GetReq *reqs = reqs_dev ? reqs_dev : &one.req;
     extern __shared__ __align__(128) uint8_t gather_smem[];
     uint64_t *s_wsum = reinterpret_cast<uint64_t *>(gather_smem + (size_t)kCopyWarps * kPipeSmemPerWarp);
-    // [n_req * ncol] inclusive prefix of the jobs' extents, each job padded to 16; the low four
-    // bits hold the padding behind the job.  With this and the rows served per request in
-    // shared memory, a chunk's warp needs neither the result block nor the last cu entry.
-    uint64_t *job_end = s_wsum + kCopyWarps;
-    uint32_t *req_rows = reinterpret_cast<uint32_t *>(job_end + n_req * jpr);        // [n_req]
+    // [n_req * jpr] inclusive prefix of the jobs' extents in units of kJobUnit bytes, each job
+    // rounded up to a whole unit (four bytes per job: a plan of thousands of jobs still leaves
+    // room for two CTAs per SM).  With this and the rows served per request in shared memory, a
+    // chunk's warp needs neither the result block nor the last cu entry; that a job's last
+    // chunk reaches a few bytes past its true end does no harm, rows and elements bound it.
+    uint32_t *job_end = reinterpret_cast<uint32_t *>(s_wsum + kCopyWarps);
+    uint32_t *req_rows = job_end + n_req * jpr;                                       // [n_req]
     const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     WarpPipe pipe;
     pipe.init(gather_smem + (size_t)warp * kPipeSmemPerWarp, lane, dv.spin_limit);
@@ -684,19 +690,16 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
                 const uint32_t q = fast_div(j, div_jpr);
                 const uint32_t k = j - q * jpr;
                 const bool scalar = k < ncol && dv.col_cls[k] == TD_SCALAR;
-                job_end[j] = scalar ? (js.bytes ? (uint64_t)js.rows * kScalarCost : 0)
-                                    : js.bytes + (uint64_t)js.cost_rows * kRowCost;
+                const uint64_t extent = scalar ? (js.bytes ? (uint64_t)js.rows * kScalarCost : 0)
+                                               : js.bytes + (uint64_t)js.cost_rows * kRowCost;
+                job_end[j] = (uint32_t)((extent + (kJobUnit - 1)) / kJobUnit);
                 if (k == 0) req_rows[q] = js.rows;
             }
         }
         __syncthreads();
         const uint32_t j0 = min(tid * per, njobs), j1 = min(j0 + per, njobs);
         uint64_t local = 0;
-        for (uint32_t j = j0; j < j1; ++j) {
-            const uint64_t bytes = job_end[j], padded = (bytes + 15) & ~uint64_t(15);
-            local += padded;
-            job_end[j] = local | (padded - bytes);    // inclusive within the thread's run; padding in the low bits
-        }
+        for (uint32_t j = j0; j < j1; ++j) local += job_end[j];
         uint64_t inc = local;
         #pragma unroll
         for (int d = 1; d < 32; d <<= 1) {
@@ -705,12 +708,15 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
         }
         if (lane == 31) s_wsum[warp] = inc;
         __syncthreads();
-        uint64_t before = inc - local;
-        for (uint32_t w = 0; w < warp; ++w) before += s_wsum[w];
-        for (uint32_t j = j0; j < j1; ++j) job_end[j] += before;
+        uint64_t run = inc - local;
+        for (uint32_t w = 0; w < warp; ++w) run += s_wsum[w];
+        for (uint32_t j = j0; j < j1; ++j) {               // the host has checked that the total fits 32 bits of units
+            run += job_end[j];
+            job_end[j] = (uint32_t)run;
+        }
         __syncthreads();
     }
-    const uint64_t total_all = njobs ? job_end[njobs - 1] & ~uint64_t(15) : 0;
+    const uint64_t total_all = njobs ? (uint64_t)job_end[njobs - 1] * kJobUnit : 0;
     const uint64_t n_warps = (uint64_t)gridDim.x * kCopyWarps;
     // A warp starts on the chunk of its own number; the chunks after the first n_warps are
     // handed out by a counter in scratch memory (zeroed by the finalize kernel): equal bytes are
@@ -725,10 +731,10 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
         const uint64_t g1 = min(g0 + plan.chunk_bytes, total_all);
         // first job that reaches beyond g0
         uint32_t j = 0;
-        { uint32_t jhi = njobs - 1; while (j < jhi) { const uint32_t m = (j + jhi) >> 1; if ((job_end[m] & ~uint64_t(15)) > g0) jhi = m; else j = m + 1; } }
+        { uint32_t jhi = njobs - 1; while (j < jhi) { const uint32_t m = (j + jhi) >> 1; if ((uint64_t)job_end[m] * kJobUnit > g0) jhi = m; else j = m + 1; } }
         for (; g0 < g1; ++j) {
-            const uint64_t start = j ? job_end[j - 1] & ~uint64_t(15) : 0;
-            const uint64_t end = job_end[j] & ~uint64_t(15);
+            const uint64_t start = j ? (uint64_t)job_end[j - 1] * kJobUnit : 0;
+            const uint64_t end = (uint64_t)job_end[j] * kJobUnit;
             const uint64_t b0 = g0 - start;
             g0 = min(g1, end);
             if (end == start) continue;               // empty job
@@ -737,15 +743,14 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
             const GetReq &rq = reqs[q];
             const td_get_out &out = rq.out;
             const uint32_t n_s = req_rows[q];
-            const uint64_t job_exact = end - start - (job_end[j] & 15u);
-            const uint64_t b1_raw = g0 - start;          // end of this warp's part of the job, padded space
+            const uint64_t b1_raw = g0 - start;          // end of this warp's part of the job (it may lie in the job's padding)
             uint8_t *dst0;
             const int32_t *seq_cu = nullptr;             // set for the two halves of the fused stream
             bool seq_tail = false;
             if (k >= ncol) {
                 const uint32_t v = k - ncol;
                 if (v == 2) {
-                    warp_fill_seq_advantages(out, n_s, b0, min(b1_raw, job_exact), lane);
+                    warp_fill_seq_advantages(out, n_s, b0, b1_raw, lane);
                     continue;
                 }
                 k = v == 0 ? out.seq_prompt_col : out.seq_response_col;
@@ -791,8 +796,7 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
             };
             if (out.mode == TD_PACKED || seq_cu) {
                 const int32_t *cu = cls == TD_PROMPT ? out.cu_prompt : out.cu_response;
-                const uint64_t b1 = min(b1_raw, job_exact);
-                if (b1 <= b0) continue;
+                const uint64_t b1 = b1_raw;
                 warp_copy_chunk<true>(cu, n_s, b0, b1, dst0, esz, lane, src_lo, src_hi, pipe, indices,
                                       [&](uint32_t i, int64_t, int64_t) -> uint8_t * { return row_src(i); },
                                       seq_cu, seq_tail);

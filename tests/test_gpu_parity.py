@@ -688,7 +688,7 @@ def test_host_buffer_calls_single_and_batched(G):
         t = torch.from_numpy(np.ascontiguousarray(a).view(np.int16) if a.dtype == np.uint16 else np.ascontiguousarray(a))
         return (t.view(torch.bfloat16) if a.dtype == np.uint16 else t).pin_memory()
 
-    for batched in (False, True, "staged"):
+    for batched in (False, True, "staged", "in place"):
         o = H.make_oracle(w)
         g = G.GpuDock(w)
         items = []
@@ -700,13 +700,20 @@ def test_host_buffer_calls_single_and_batched(G):
                               pinned(cu) if cu is not None else None, pinned(data)))
         need = [g.dock.put_host_stage_bytes(c, i.numel(), d.numel()) for c, i, _cu, d in items]
         bufs = [g.buffers(op.consumer, op.max_samples, key=("host", j)) for j, op in enumerate(gets)]
+        if batched == "in place":         # payload buffers in pinned host memory, written by the gather itself
+            pc, rc = g.token_caps(w.micro_batch)
+            bufs = [td.GetBuffers(g.dock, op.consumer, op.max_samples, prompt_tokens_cap=pc, response_tokens_cap=rc,
+                                  host_payload=True) for op in gets]
+            for b in bufs:
+                for t in b.cols.values():
+                    t.view(torch.uint8).fill_(0xA5)
         hosts = [td.HostGetBuffers(b) for b in bufs]
         if batched:
             stage = torch.empty(sum(need), dtype=torch.uint8, device=g.device)
             g.dock.put_many_host(items, stage)
             plan = g.dock.plan(bufs)
             meta = None
-            if batched == "staged":       # results, indices, cu_seqlens and advantages of all requests in one transfer
+            if batched in ("staged", "in place"):   # results, indices, cu_seqlens and advantages of all requests in one transfer
                 meta = torch.empty(g.dock.get_many_host_stage_bytes(plan), dtype=torch.uint8, device=g.device)
             g.dock.get_many_host(plan, hosts, meta)
         else:
