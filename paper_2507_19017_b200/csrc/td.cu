@@ -35,6 +35,7 @@ struct td_dock {
 namespace {
 
 std::atomic<uint32_t> g_seq{1};     // launch sequence numbers for scan scratch, process wide
+std::atomic<unsigned long long> g_put_seq{1};         // numbers of the puts that tell their scatter kernel when to look
 constexpr uint32_t kDefaultPollLimit = 1u << 20;      // polls before a device-side wait gives up (tens of milliseconds)
 
 inline size_t align_up_sz(size_t x, size_t a) { return (x + a - 1) / a * a; }
@@ -49,7 +50,8 @@ size_t gather_smem_bytes(uint32_t n_req, uint32_t jobs_per_req) {
 }
 
 struct Layout {
-    size_t status, len[3], off[3], cursor[3], claim, consumed, errword, counters, put_counters, col[kMaxColumns], total;
+    size_t status, len[3], off[3], cursor[3], claim, consumed, errword, counters, put_counters, put_ready, progress,
+           col[kMaxColumns], total;
     uint32_t claim_words, consumed_words;
     uint64_t cap[3];
 };
@@ -92,6 +94,8 @@ Layout make_layout(const td_config *c) {
     L.errword = take(256);
     L.counters = take(CNT_TOTAL * 8);
     L.put_counters = take((size_t)kPutCounterSlots * 8);
+    L.put_ready = take((size_t)kPutCounterSlots * 8);
+    L.progress = take((size_t)c->n_columns * n * 4);
     L.status = take(n * 4);
     for (int k = 1; k <= 2; ++k) { L.len[k] = take(n * 4); L.off[k] = take(n * 8); L.cursor[k] = take(S * 8); }
     L.claim = take((size_t)c->n_consumers * L.claim_words * 4);
@@ -292,6 +296,8 @@ int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **o
     v.errword = reinterpret_cast<uint32_t *>(w + L.errword);
     v.counters = reinterpret_cast<unsigned long long *>(w + L.counters);
     v.put_counters = reinterpret_cast<unsigned long long *>(w + L.put_counters);
+    v.put_ready = reinterpret_cast<unsigned long long *>(w + L.put_ready);
+    v.progress = reinterpret_cast<uint32_t *>(w + L.progress);
     for (uint32_t k = 0; k < v.ncol; ++k) {
         v.colbase[k] = w + L.col[k];
         v.col_esz[k] = (uint8_t)esize_of(cfg->columns[k].dtype);
@@ -307,7 +313,8 @@ int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **o
     d->table_bytes[3] = (size_t)v.S * 8; d->table_bytes[4] = (size_t)v.claim_words * 4;
     d->table_bytes[5] = (size_t)v.consumed_words * 4; d->table_bytes[6] = 0;
 
-    int rc = td_reset(d, nullptr);
+    int rc = cudaMemsetAsync(w + L.put_ready, 0, (size_t)kPutCounterSlots * 8, nullptr) == cudaSuccess ? TD_OK : TD_ECUDA;
+    if (rc == TD_OK) rc = td_reset(d, nullptr);
     if (rc == TD_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) rc = TD_ECUDA;
     if (rc != TD_OK) { delete d; return rc; }
     *out = d;
@@ -340,26 +347,28 @@ uint32_t copy_grid(const td_dock *d, uint64_t room_bytes) {
     return (uint32_t)blocks;
 }
 
-// The chunk counter the scatter kernel of a call on stream `st` may draw from, or nullptr.  Calls
-// on one stream run one after the other, so a counter per stream is never shared by two launches
+// The slot of stream `st` in the dock's per-stream words (the scatter kernel's chunk counter, the
+// word in which the alloc kernel tells it that the call's inputs are complete), or -1.  Calls
+// on one stream run one after the other, so a slot per stream is never shared by two launches
 // in flight.  A call that is being captured into a graph gets none: the graph may later run on
 // any stream, beside anything.
-unsigned long long *scatter_counter(td_dock *d, cudaStream_t st) {
+int stream_slot(td_dock *d, cudaStream_t st) {
     cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
     if (cudaStreamIsCapturing(st, &cap) != cudaSuccess || cap != cudaStreamCaptureStatusNone) {
         cudaGetLastError();
-        return nullptr;
+        return -1;
     }
     std::lock_guard<std::mutex> lk(d->slot_mu);
     for (size_t i = 0; i < d->slot_stream.size(); ++i)
-        if (d->slot_stream[i] == st) return d->dv.put_counters + i;
-    if (d->slot_stream.size() >= (size_t)kPutCounterSlots) return nullptr;
+        if (d->slot_stream[i] == st) return (int)i;
+    if (d->slot_stream.size() >= (size_t)kPutCounterSlots) return -1;
     d->slot_stream.push_back(st);
-    return d->dv.put_counters + (d->slot_stream.size() - 1);
+    return (int)d->slot_stream.size() - 1;
 }
 
-// One launch group: alloc (if any ragged item), scatter, publish.  Items are taken in order;
-// a column appears at most once per group, so that duplicate detection sees earlier items.
+// One launch group: alloc and scatter (which also publishes), or, for scalar columns only, one
+// publish kernel.  Items are taken in order; a column appears at most once per group, so that
+// duplicate detection sees earlier items.
 int put_group(td_dock *d, PutBatch &b, cudaStream_t st) {
     const DockView &v = d->dv;
     // Propose followers to the alloc kernel: an item may ride along with the latest item of its
@@ -385,16 +394,23 @@ int put_group(td_dock *d, PutBatch &b, cudaStream_t st) {
     }
     if (entries == 0) return TD_OK;
     if (entries >= (1ull << 32)) return TD_EINVAL;
-    b.work_counter = ragged_bytes ? scatter_counter(d, st) : nullptr;
+    b.work_counter = nullptr; b.ready = nullptr; b.seq = 0;
     if (ragged_bytes) {
+        const int slot = stream_slot(d, st);
+        if (slot >= 0) {
+            b.work_counter = d->dv.put_counters + slot;
+            b.ready = d->dv.put_ready + slot;
+            b.seq = g_put_seq.fetch_add(1, std::memory_order_relaxed);
+        }
+        ragged_bytes += entries * kPutScalarCost;              // the scalar items of the call ride along
         if (launch_dep(d, put_alloc_kernel, dim3(2), dim3(kAllocThreads), put_alloc_smem_bytes(v.S), st, v, b) != cudaSuccess)
             return TD_ECUDA;
         if (launch_timed(d, 0, put_scatter_kernel, dim3(copy_grid(d, ragged_bytes)), dim3(kCopyThreads),
                          scatter_smem_bytes(), st, v, b) != cudaSuccess)
             return TD_ECUDA;
+        return TD_OK;
     }
-    if (launch_dep(d, put_publish_kernel, dim3((uint32_t)((entries + 255) / 256)), dim3(256), 0, st, v, b,
-                   ragged_bytes ? 1u : 0u) != cudaSuccess)
+    if (launch_dep(d, put_publish_kernel, dim3((uint32_t)((entries + 255) / 256)), dim3(256), 0, st, v, b) != cudaSuccess)
         return TD_ECUDA;
     return TD_OK;
 }

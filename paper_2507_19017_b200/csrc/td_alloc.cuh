@@ -40,6 +40,12 @@ struct PutBatch {                              // the columns of one call, in ca
     // to the stream the call was made on (calls on one stream run one after the other); nullptr:
     // every warp takes a fixed share instead.  Zeroed by the alloc kernel.
     unsigned long long *work_counter;
+    // A word in the dock's workspace, private to the stream like the counter, in which the alloc
+    // kernel stores `seq` (the call's number, growing from call to call) once everything ahead of
+    // the call has finished: the scatter kernel, launched early, may read the call's inputs from
+    // then on.  nullptr: the scatter kernel waits for the alloc kernel's end before it reads anything.
+    unsigned long long *ready;
+    unsigned long long seq;
 };
 
 static inline size_t put_alloc_smem_bytes(uint32_t S) {
@@ -137,7 +143,10 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
     // kernel in the stream (a reset, the get whose batch is sent back, the caller's own producer)
     // must have finished.  The prefetch above only asked for lines.
     griddep_wait();
-    if (blockIdx.x == 0 && tid == 0 && batch.work_counter) *batch.work_counter = 0;
+    if (blockIdx.x == 0 && tid == 0) {
+        if (batch.work_counter) *batch.work_counter = 0;
+        if (batch.ready) st_release_u64(batch.ready, batch.seq);       // the call's inputs are complete: the scatter may look
+    }
 
     // Which proposed followers really repeat their leader's index and cu arrays?
     if (tid == 0) s_not_following = 0;

@@ -70,6 +70,8 @@ struct DockView {
     uint32_t *errword;
     unsigned long long *counters;           // [CNT_TOTAL]
     unsigned long long *put_counters;       // [kPutCounterSlots] chunk counters of the scatter kernel, one per stream in use
+    unsigned long long *put_ready;          // [kPutCounterSlots] number of the latest put on that stream whose inputs are known to be complete
+    uint32_t *progress;                     // [ncol][n] elements of a row written so far by the put that stores it
     uint8_t  *colbase[kMaxColumns];         // arena (S * cap * esz) or scalar store (n * esz)
     uint32_t need[kMaxColumns];             // per consumer
     uint32_t outm[kMaxColumns];
@@ -439,6 +441,11 @@ struct WarpPipe {
         }
     }
 
+    // every copy issued so far written out to its destination
+    __device__ __forceinline__ void drain_all(uint32_t lane) {
+        while (tail != head) drain_one(lane);
+    }
+
     // before the warp returns: everything written out, nothing of its own still landing
     __device__ __forceinline__ uint32_t finish(uint32_t lane) {
         while (tail != head) drain_one(lane);
@@ -504,21 +511,89 @@ struct WarpPipe {
 constexpr uint32_t kRowCost = TD_ROW_COST;
 static_assert(kRowCost % 16 == 0, "a job's extent stays a multiple of 16");
 
+// Workflow step 3 for a put, row by row.  A row becomes visible to the controllers - its column
+// bit set in the sample's status word, behind a fence - once all of it is in its arena.  A row
+// that lies wholly inside one chunk is complete when that chunk's warp has written it out; a
+// row that chunk borders cut is complete when the parts written by all the warps that share it
+// add up to its length, which they count in progress[column][sample]; a row of no length
+// belongs to the chunk that holds its place in the space.  Waiting for the ring to run empty
+// and fencing after every chunk would cost more than the copying it interrupts, so a warp only
+// notes what it has written (sample, column, elements, row length: one row per lane) and
+// settles up to 32 notes at once: when the list is full, and when the warp is done.
+struct PublishQueue {
+    int32_t s;             // lane i: the i-th noted row's sample
+    uint32_t part, total;  //         elements written by this warp / in the row
+    uint32_t col;          //         its column
+    uint32_t n;            // rows noted (the same in every lane)
+};
+__device__ __forceinline__ void publish_queue_init(PublishQueue &q) { q.s = -1; q.part = q.total = q.col = 0; q.n = 0; }
+
+// Everything the warp has issued is written out and fenced; then the noted rows are settled.
+__device__ __forceinline__ void publish_queue_flush(const DockView &dv, PublishQueue &q, WarpPipe &pipe, uint32_t lane) {
+    if (q.n == 0) return;
+    pipe.drain_all(lane);
+    __threadfence();
+    __syncwarp();
+    bool ok = false;
+    if (lane < q.n) {
+        const uint32_t bit = 1u << q.col;
+        bool complete = q.part == q.total;             // the whole row, or a row of no length
+        if (!complete) {
+            // the first time the count reaches the row's length (the same sample twice in one
+            // call may push it beyond)
+            const uint32_t old = atomicAdd(&dv.progress[(size_t)q.col * dv.n + (uint32_t)q.s], q.part);
+            complete = old < q.total && old + q.part >= q.total;
+            if (complete) __threadfence();
+        }
+        if (complete) ok = !(atomicOr(&dv.status[q.s], bit) & bit);
+    }
+    // accepted rows are counted per column: one addition per column the list holds
+    const uint32_t live = __ballot_sync(kFullMask, lane < q.n);
+    if (lane < q.n) {
+        const uint32_t peers = __match_any_sync(live, q.col);
+        const uint32_t okc = __popc(__ballot_sync(live, ok) & peers);
+        if (okc && lane == (uint32_t)__ffs(peers) - 1u)
+            atomicAdd(&dv.counters[CNT_PUT_ACCEPTED + q.col], (unsigned long long)okc);
+    }
+    q.n = 0;
+}
+
+// Notes the rows of one round: lanes with s_row >= 0 each hold one.
+__device__ __forceinline__ void publish_queue_note(const DockView &dv, PublishQueue &q, WarpPipe &pipe, uint32_t lane,
+                                                   int32_t s_row, uint32_t part, uint32_t total, uint32_t col) {
+    const uint32_t m = __ballot_sync(kFullMask, s_row >= 0);
+    const uint32_t cnt = __popc(m);
+    if (cnt == 0) return;
+    if (q.n + cnt > 32u) publish_queue_flush(dv, q, pipe, lane);
+    // slot q.n + j takes the row of the j-th lane of m
+    const uint32_t j = lane - q.n;                                  // meaningful for q.n <= lane < q.n + cnt
+    const uint32_t src = (lane >= q.n && j < cnt) ? __fns(m, 0, (int)j + 1) : 0u;
+    const int32_t s_in = __shfl_sync(kFullMask, s_row, src);
+    const uint32_t part_in = __shfl_sync(kFullMask, part, src);
+    const uint32_t total_in = __shfl_sync(kFullMask, total, src);
+    if (lane >= q.n && j < cnt) { q.s = s_in; q.part = part_in; q.total = total_in; q.col = col; }
+    q.n += cnt;
+}
+
 // Steps 2 and 3 for one chunk [b0, b1) of that space (a chunk is shorter than 4 GB) of a packed
-// side described by cu[0..rows].  resolve(i) returns where row i starts on the other side, or
-// nullptr to skip the row; it is called by one lane per row; `along` is the index array it
-// reads (prefetched by the row search).  kToPacked: the packed side is the destination (get),
-// else the source (put, whose source window is tested against the caller's buffer).
+// side described by cu[0..rows].  resolve(i, c0, c1, s) returns where row i starts on the other
+// side, or nullptr to skip the row (and, for a put, the sample in s); it is called by one lane
+// per row; `along` is the index array it reads (prefetched by the row search).  kToPacked: the
+// packed side is the destination (get), else the source (put, whose source window is tested
+// against the caller's buffer).  kPublish (put): the rows, or parts of rows, that the chunk
+// holds are noted in `queue` for publication (see PublishQueue).
 // seq_cu, when given, moves the rows on the packed side: row i then sits at element seq_cu[i]
 // (seq_tail false) or ends at element seq_cu[i + 1] (seq_tail true) instead of starting at
 // cu[i] - the two halves of a stream in which each sample's prompt row is followed by its
 // response row; cu still says how long the rows are and where they lie in the chunked space.
-template <bool kToPacked, typename Resolve>
+template <bool kToPacked, bool kPublish, typename Resolve>
 __device__ __forceinline__ void warp_copy_chunk(const int32_t *cu, uint32_t rows, uint64_t b0, uint64_t b1,
                                                 uint8_t *packed, uint32_t esz, uint32_t lane,
                                                 const uint8_t *src_lo, const uint8_t *src_hi, WarpPipe &pipe,
                                                 const int32_t *along, Resolve resolve,
-                                                const int32_t *seq_cu = nullptr, bool seq_tail = false) {
+                                                const int32_t *seq_cu = nullptr, bool seq_tail = false,
+                                                const DockView *dvp = nullptr, PublishQueue *queue = nullptr,
+                                                uint32_t column = 0) {
     uint32_t r0 = warp_find_row(cu, rows, (int64_t)b0, esz, kRowCost, lane, along);
     for (;;) {
         // lane l: the part of row r0 + l that falls inside the chunk, as (address on the packed
@@ -527,6 +602,8 @@ __device__ __forceinline__ void warp_copy_chunk(const int32_t *cu, uint32_t rows
         bool in = false;
         uint32_t len = 0;
         uint8_t *mine = nullptr, *other = nullptr;
+        int32_t s_row = -1;                // put: the sample of a row this lane has a part of, or owns
+        uint32_t total = 0;                // put: the row's length in elements
         if (i < rows) {
             const int64_t c0 = __ldg(cu + i);
             const uint64_t row0 = (uint64_t)c0 * esz + (uint64_t)i * kRowCost;
@@ -536,15 +613,21 @@ __device__ __forceinline__ void warp_copy_chunk(const int32_t *cu, uint32_t rows
                 const uint64_t dlo = row0 + kRowCost;                       // the row's bytes, in the chunked space
                 const uint64_t dhi = c1 > c0 ? dlo + (uint64_t)(c1 - c0) * esz : dlo;
                 const uint64_t lo = max(dlo, b0), hi = min(dhi, b1);
-                if (hi > lo) {
-                    uint8_t *row = resolve(i, c0, c1);
+                const bool empty_here = kPublish && c1 == c0 && row0 >= b0;   // a row of no length whose place is in this chunk
+                if (hi > lo || empty_here) {
+                    int32_t s = -1;
+                    uint8_t *row = resolve(i, c0, c1, s);
                     if (row) {
-                        other = row + (lo - dlo);
-                        uint64_t at = (uint64_t)c0;
-                        if (seq_cu) at = seq_tail ? (uint64_t)((int64_t)__ldg(seq_cu + i + 1) - (c1 - c0))
-                                                  : (uint64_t)__ldg(seq_cu + i);
-                        mine = packed + at * esz + (lo - dlo);
-                        len = (uint32_t)(hi - lo);
+                        s_row = s;
+                        total = (uint32_t)(c1 - c0);
+                        if (hi > lo) {
+                            other = row + (lo - dlo);
+                            uint64_t at = (uint64_t)c0;
+                            if (seq_cu) at = seq_tail ? (uint64_t)((int64_t)__ldg(seq_cu + i + 1) - (c1 - c0))
+                                                      : (uint64_t)__ldg(seq_cu + i);
+                            mine = packed + at * esz + (lo - dlo);
+                            len = (uint32_t)(hi - lo);
+                        }
                     }
                 }
             }
@@ -561,6 +644,7 @@ __device__ __forceinline__ void warp_copy_chunk(const int32_t *cu, uint32_t rows
             if (kToPacked) pipe.template push<false>(p, o, len_r, lane, src_lo, src_hi);
             else pipe.template push<true>(o, p, len_r, lane, src_lo, src_hi);
         }
+        if (kPublish) publish_queue_note(*dvp, *queue, pipe, lane, s_row, len / esz, total, column);
         if (n_rows < 32u) break;
         r0 += 32u;
     }

@@ -797,9 +797,9 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
             if (out.mode == TD_PACKED || seq_cu) {
                 const int32_t *cu = cls == TD_PROMPT ? out.cu_prompt : out.cu_response;
                 const uint64_t b1 = b1_raw;
-                warp_copy_chunk<true>(cu, n_s, b0, b1, dst0, esz, lane, src_lo, src_hi, pipe, indices,
-                                      [&](uint32_t i, int64_t, int64_t) -> uint8_t * { return row_src(i); },
-                                      seq_cu, seq_tail);
+                warp_copy_chunk<true, false>(cu, n_s, b0, b1, dst0, esz, lane, src_lo, src_hi, pipe, indices,
+                                             [&](uint32_t i, int64_t, int64_t, int32_t &) -> uint8_t * { return row_src(i); },
+                                             seq_cu, seq_tail);
             } else {
                 // fixed-width rows: payload part, then the pad pattern up to the row's end
                 const uint32_t W = cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to;
@@ -849,6 +849,7 @@ reset_kernel(const DockView dv) {
     for (uint32_t i = t; i < dv.S; i += stride) { dv.cursor[1][i] = 0; dv.cursor[2][i] = 0; }
     for (uint32_t i = t; i < dv.ncons * dv.claim_words; i += stride) dv.claim[i] = 0;
     for (uint32_t i = t; i < dv.ncons * dv.consumed_words; i += stride) dv.consumed[i] = 0;
+    for (uint64_t i = t; i < (uint64_t)dv.ncol * dv.n; i += stride) dv.progress[i] = 0;
     for (uint32_t i = t; i < CNT_TOTAL; i += stride) dv.counters[i] = 0;
     if (t == 0) *dv.errword = 0;
 }
