@@ -255,7 +255,9 @@ int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **o
     int sms = 0;
     if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, cfg->device) != cudaSuccess) return TD_ECUDA;
     const size_t alloc_smem = put_alloc_smem_bytes(cfg->n_shards);
-    if (cudaFuncSetAttribute(put_alloc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)alloc_smem) != cudaSuccess)
+    if (cudaFuncSetAttribute(put_alloc_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)alloc_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(put_alloc_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)alloc_smem) != cudaSuccess ||
+        cudaFuncSetAttribute(put_alloc_kernel<4>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)alloc_smem) != cudaSuccess)
         return TD_ECUDA;
 
     if (cudaFuncSetAttribute(put_scatter_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -403,7 +405,13 @@ int put_group(td_dock *d, PutBatch &b, cudaStream_t st) {
             b.seq = g_put_seq.fetch_add(1, std::memory_order_relaxed);
         }
         ragged_bytes += entries * kPutScalarCost;              // the scalar items of the call ride along
-        if (launch_dep(d, put_alloc_kernel, dim3(2), dim3(kAllocThreads), put_alloc_smem_bytes(v.S), st, v, b) != cudaSuccess)
+        // entries per thread and pass of the alloc kernel: enough for the largest item in one pass, up to four
+        uint32_t k_max = 0;
+        for (uint32_t i = 0; i < b.n_items; ++i)
+            if (v.col_cls[b.item[i].column] != TD_SCALAR) k_max = std::max(k_max, b.item[i].k);
+        auto alloc_kernel = k_max <= (uint32_t)kAllocThreads ? put_alloc_kernel<1>
+                            : k_max <= 2u * kAllocThreads ? put_alloc_kernel<2> : put_alloc_kernel<4>;
+        if (launch_dep(d, alloc_kernel, dim3(2), dim3(kAllocThreads), put_alloc_smem_bytes(v.S), st, v, b) != cudaSuccess)
             return TD_ECUDA;
         if (launch_timed(d, 0, put_scatter_kernel, dim3(copy_grid(d, ragged_bytes)), dim3(kCopyThreads),
                          scatter_smem_bytes(), st, v, b) != cudaSuccess)

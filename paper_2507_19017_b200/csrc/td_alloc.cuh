@@ -10,8 +10,7 @@ namespace td {
 constexpr int kAllocThreads = 1024;
 constexpr int kAllocWarps = kAllocThreads / 32;
 static_assert(kAllocWarps == 32, "the scan over the warps' sums gives one lane to each warp");
-constexpr int kAllocPer = 4;                                   // entries per thread and pass
-constexpr int kAllocPass = kAllocThreads * kAllocPer;          // entries per pass
+constexpr int kAllocPerMax = 4;                                // entries per thread and pass: 1, 2 or 4, by the size of the call
 constexpr int kMaxPutItems = 8;                                // columns one put launch can carry
 constexpr uint32_t kNotAllocating = 0xffffffffu;
 
@@ -54,7 +53,7 @@ static inline size_t put_alloc_smem_bytes(uint32_t S) {
 
 // Ordered exclusive prefix of `room` over the lanes that allocate in the same shard, and that
 // shard's sum over the warp.  leader: the first allocating lane of its shard.
-__device__ __forceinline__ void warp_shard_prefix(bool alloc, uint32_t sh, uint32_t room, uint32_t lane,
+__device__ __noinline__ void warp_shard_prefix(bool alloc, uint32_t sh, uint32_t room, uint32_t lane,
                                                   unsigned long long &pre, unsigned long long &wsum, bool &leader) {
     pre = 0; wsum = 0; leader = false;
     const uint32_t mask = __ballot_sync(kFullMask, alloc);
@@ -67,7 +66,7 @@ __device__ __forceinline__ void warp_shard_prefix(bool alloc, uint32_t sh, uint3
     __match_all_sync(kFullMask, key, &same);
     if (same) {
         unsigned long long inc = alloc ? room : 0u;
-        #pragma unroll
+        #pragma unroll 1
         for (int d = 1; d < 32; d <<= 1) {
             const unsigned long long t = shfl_up_u64(inc, d);
             if ((int)lane >= d) inc += t;
@@ -79,7 +78,7 @@ __device__ __forceinline__ void warp_shard_prefix(bool alloc, uint32_t sh, uint3
     }
     const uint32_t k2 = alloc ? sh : kNotAllocating;
     leader = alloc;
-    #pragma unroll 8
+    #pragma unroll 1
     for (uint32_t j = 0; j < 32; ++j) {
         const uint32_t kj = __shfl_sync(kFullMask, k2, j);
         const uint32_t rj = __shfl_sync(kFullMask, room, j);
@@ -108,8 +107,12 @@ __device__ __forceinline__ void warp_shard_prefix(bool alloc, uint32_t sh, uint3
 // checked for follows from what the leader's thread already holds for the entry: the status
 // word, the row length and the length in force after the leader's CAS.  Followers are therefore
 // settled inside the leader's passes, without passes or atomics of their own.
+// kAllocPer entries per thread and pass (a call of up to 1024 entries per length class runs the
+// instance with one: a quarter of the code, which on a cold instruction cache is what counts).
+template <int kAllocPer>
 __global__ void __launch_bounds__(kAllocThreads)
 put_alloc_kernel(const DockView dv, const PutBatch batch) {
+    constexpr int kAllocPass = kAllocThreads * kAllocPer;          // entries per pass
     extern __shared__ unsigned long long smem_u64[];
     const uint32_t S = dv.S;
     unsigned long long *tot = smem_u64;                            // [kAllocWarps][S]
@@ -148,11 +151,22 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
         if (batch.ready) st_release_u64(batch.ready, batch.seq);       // the call's inputs are complete: the scatter may look
     }
 
-    // Which proposed followers really repeat their leader's index and cu arrays?
+    // Which proposed followers really repeat their leader's index and cu arrays?  (Nothing to
+    // find out, and no barrier to pass, when every one of them names its leader's own arrays.)
+    bool to_compare = false;
+    #pragma unroll 1
+    for (uint32_t it = 0; it < batch.n_items; ++it)
+        if (batch.follow[it] && dv.col_cls[batch.item[it].column] == L) {
+            const PutArgs &a = batch.item[it], &ld = batch.item[batch.follow[it] - 1u];
+            to_compare |= a.idx != ld.idx || a.cu != ld.cu;
+        }
+    uint32_t not_following = 0;
+    if (to_compare) {
     if (tid == 0) s_not_following = 0;
     __syncthreads();
     {
         uint32_t differs = 0;
+        #pragma unroll 1
         for (uint32_t it = 0; it < batch.n_items; ++it) {
             if (!batch.follow[it] || dv.col_cls[batch.item[it].column] != L) continue;
             const PutArgs &a = batch.item[it], &ld = batch.item[batch.follow[it] - 1u];
@@ -166,14 +180,17 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
         if (differs) atomicOr(&s_not_following, differs);
     }
     __syncthreads();
-    uint32_t not_following = s_not_following;
+    not_following = s_not_following;
     // an item that does not follow after all takes its own passes, in its place in the call; so
     // do the later followers of its leader, which would otherwise overtake it
+    #pragma unroll 1
     for (uint32_t it = 0; it < batch.n_items; ++it)
         if ((not_following >> it) & 1u)
             for (uint32_t f = it + 1; f < batch.n_items; ++f)
                 if (batch.follow[f] == batch.follow[it]) not_following |= 1u << f;
+    }
 
+    #pragma unroll 1
     for (uint32_t it = 0; it < batch.n_items; ++it) {
         const PutArgs &a = batch.item[it];
         if (dv.col_cls[a.column] != L) continue;
@@ -183,6 +200,7 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
             if (batch.follow[f] == it + 1u && !((not_following >> f) & 1u)) followers |= 1u << f;
         const uint32_t bit = 1u << a.column;
         const uint32_t k = item_k(a);
+        #pragma unroll 1
         for (uint32_t base = 0; base < k; base += kAllocPass) {
             // 1. validate, CAS.  A short pass is spread over all warps: each takes `per` rows of 32.
             const uint32_t per = min((uint32_t)kAllocPer, (k - base + kAllocThreads - 1u) / kAllocThreads);
@@ -223,6 +241,7 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
                         // Followers: same sample, same row.  Their bound on the data is not
                         // wider than the leader's, so where one of them is in order the leader
                         // has done its CAS and the length in force is known.
+                        #pragma unroll 1
                         for (uint32_t fm = followers; fm; fm &= fm - 1u) {
                             const uint32_t f = (uint32_t)__ffs(fm) - 1u;
                             const PutArgs &b = batch.item[f];
@@ -263,7 +282,7 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
             for (uint32_t k2 = warp; k2 < S; k2 += kAllocWarps) {
                 const unsigned long long v = tot[lane * S + k2];
                 unsigned long long inc = v;
-                #pragma unroll
+                #pragma unroll 1
                 for (int d = 1; d < 32; d <<= 1) {
                     const unsigned long long t = shfl_up_u64(inc, d);
                     if ((int)lane >= d) inc += t;

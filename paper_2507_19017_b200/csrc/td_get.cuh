@@ -476,6 +476,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     uint64_t room_tok[3] = {~0ull, ~0ull, ~0ull};      // packed: tokens; scalar slot [0]: samples
     uint64_t room_rows = ~0ull;                         // padded: rows
     const uint32_t outm = dv.outm[c];
+    #pragma unroll 1
     for (uint32_t k = 0; k < dv.ncol; ++k) {
         if (!((outm >> k) & 1u) || out.col[k] == nullptr) continue;
         const uint32_t cls = dv.col_cls[k];
@@ -490,6 +491,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     const uint64_t room_seq = (out.seq || out.seq_advantages) ? out.seq_capacity_elems : ~0ull;
     const bool padded = out.mode == TD_PADDED;
     bool want_p = false, want_r = false;
+    #pragma unroll 1
     for (uint32_t k = 0; k < dv.ncol; ++k)
         if (((outm >> k) & 1u) && out.col[k] != nullptr) {
             want_p |= dv.col_cls[k] == TD_PROMPT;
@@ -528,6 +530,7 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     uint64_t tot_p = carry_p, tot_r = carry_r;         // the batch's token totals
     if (s_first_over != 0xffffffffu) {
         const uint32_t keep = s_first_over / N;
+        #pragma unroll 1
         for (uint32_t p = keep + tid; p < n_grp; p += kThreads) {
             const uint32_t g = (uint32_t)out.indices[(size_t)p * N] / N;
             atomicAnd(&dv.claim[(size_t)c * dv.claim_words + (g >> 5)], ~(1u << (g & 31)));
