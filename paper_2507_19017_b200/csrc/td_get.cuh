@@ -458,6 +458,12 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
     }
     __syncthreads();
     uint32_t n_s = n_grp * N;
+    // the groups' rewards are wanted last, behind the cu scans: ask for their lines now
+    if ((dv.cflags[c] & TD_F_ADVANTAGE) && tid < n_grp && tid < kFinGroupsKept) {
+        const float *r = reinterpret_cast<const float *>(dv.colbase[dv.reward_col]) + (size_t)s_grp[tid] * N;
+        asm volatile("prefetch.global.L1 [%0];" ::"l"(r));
+        if (N > 32u) asm volatile("prefetch.global.L1 [%0];" ::"l"(r + N - 1));
+    }
     const FastDiv div_N = make_fastdiv_dev(N);
     // sample at position i of the batch
     auto sample_at = [&](uint32_t i) -> int32_t {
