@@ -51,6 +51,7 @@ def parse_args():
                     help="workload shape 1..5; default: shapes 5 (headline), 2, 3 and 4 in one run")
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-cpu-all-cores", action="store_true", help="skip the oracle-on-several-cores leg")
     ap.add_argument("--no-e2e", action="store_true")
     ap.add_argument("--no-variants", action="store_true", help="skip the warm-L2 and heavy-tail records")
     ap.add_argument("--e2e-path", default="auto", choices=["auto", "in-place", "copy"],
@@ -59,7 +60,7 @@ def parse_args():
     ap.add_argument("--api", default="many", choices=["many", "single"],
                     help="many: one td_put_many and one td_get_many per step; single: one td_put per "
                          "column and one td_get per micro-batch")
-    ap.add_argument("--cpu-seconds", type=float, default=6.0, help="CPU-oracle time budget per shape")
+    ap.add_argument("--cpu-seconds", type=float, default=4.0, help="CPU-oracle time budget per shape and leg")
     ap.add_argument("--sigma", type=float, default=None,
                     help="spread of the lognormal response lengths (default 0.25; 0.75 is the heavy tail)")
     ap.add_argument("--warm-l2", action="store_true", help="do not flush the L2 before the phases")
@@ -792,6 +793,27 @@ def time_oracle(w, budget_s: float, steps: int = 0, warmup: int = 0):
     return samples / el, done, el
 
 
+def _oracle_worker(args):
+    """One host process of the all-cores leg: its own copy of the workload and of the oracle."""
+    cid, sigma, budget = args
+    from oracle import td_oracle
+    td_oracle.build()
+    w = make_workload(cid, 0, sigma, "bulk")
+    return time_oracle(w, budget)
+
+
+def time_oracle_all_cores(cid: int, sigma, budget_s: float, max_workers: int = 8):
+    """The same oracle, unchanged, on several host cores at once: one process per core, each with
+    its own dock over the same workload (the oracle is one thread by design; this is what the
+    host can dispatch when every core runs one).  Processes are spawned, not forked.  Returns
+    (samples/s summed over the processes, processes, seconds of the slowest)."""
+    import multiprocessing as mp
+    workers = max(1, min(os.cpu_count() or 1, max_workers))
+    with mp.get_context("spawn").Pool(workers) as pool:
+        res = pool.map(_oracle_worker, [(cid, sigma, budget_s)] * workers)
+    return sum(r[0] for r in res), workers, max(r[2] for r in res)
+
+
 # --------------------------------------------------------------------------- one shape, measured
 def make_workload(cid: int, rank: int, sigma, schedule: str):
     from paper_2507_19017_b200 import workloads as wl
@@ -948,6 +970,11 @@ def measure_dispatch(args, cid: int, rank: int, local_rank: int, world: int, dis
         rate, steps_o, el = time_oracle(w, args.cpu_seconds)
         cpu = {"value": rate, "unit": "samples/s", "cores": 1, "kind": "oracle",
                "sample": f"{steps_o} whole step(s) of the same workload in {el:.1f} s"}
+        if not args.no_cpu_all_cores:
+            rate_all, procs, el_all = time_oracle_all_cores(cid, sigma, args.cpu_seconds)
+            cpu["all_cores"] = {"value": rate_all, "unit": "samples/s", "cores": procs, "kind": "oracle",
+                                "sample": f"{procs} processes, one dock each over the same workload, whole steps "
+                                          f"for {el_all:.1f} s; host has {os.cpu_count()} logical cores"}
     rec["cpu_baseline"] = cpu
     return rec
 

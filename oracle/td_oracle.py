@@ -27,15 +27,24 @@ ERR_OOB_INDEX, ERR_DUP_PUT, ERR_LEN_MISMATCH, ERR_ARENA_FULL, ERR_OUT_TRUNC = 1,
 ERR_BAD_LENGTH = 64
 
 
-def build(force: bool = False) -> str:
-    """Compile the oracle with gcc (no optimisation flags beyond -O2)."""
+_LIB_SAN = os.path.join(_HERE, "libtd_oracle_san.so")
+SANITIZED_ENV = "TD_ORACLE_SANITIZED"      # set: lib() loads the build below instead of the plain one
+
+
+def build(force: bool = False, sanitize: bool = False) -> str:
+    """Compile the oracle with gcc (no optimisation flags beyond -O2).  sanitize: a second build
+    with AddressSanitizer and UndefinedBehaviorSanitizer (errors abort), for the test that runs
+    the oracle's own pins under them; the process that loads it must have libasan preloaded."""
     hdr = os.path.join(_HERE, "td_oracle.h")
-    stale = (not os.path.exists(_LIB)
-             or os.path.getmtime(_LIB) < max(os.path.getmtime(_SRC), os.path.getmtime(hdr)))
+    out = _LIB_SAN if sanitize else _LIB
+    stale = (not os.path.exists(out)
+             or os.path.getmtime(out) < max(os.path.getmtime(_SRC), os.path.getmtime(hdr)))
     if force or stale:
-        subprocess.check_call(["gcc", "-O2", "-std=c11", "-Wall", "-Wextra", "-shared", "-fPIC",
-                               "-o", _LIB, _SRC, "-lm"])
-    return _LIB
+        extra = (["-g", "-O1", "-fno-omit-frame-pointer", "-fsanitize=address,undefined",
+                  "-fno-sanitize-recover=all"] if sanitize else ["-O2"])
+        subprocess.check_call(["gcc", *extra, "-std=c11", "-Wall", "-Wextra", "-shared", "-fPIC",
+                               "-o", out, _SRC, "-lm"])
+    return out
 
 
 class _Column(C.Structure):
@@ -84,7 +93,7 @@ _lib = None
 def lib():
     global _lib
     if _lib is None:
-        L = C.CDLL(build())
+        L = C.CDLL(build(sanitize=bool(os.environ.get(SANITIZED_ENV))))
         L.ora_create.restype = C.c_void_p
         L.ora_create.argtypes = [C.POINTER(_Config)]
         L.ora_destroy.argtypes = [C.c_void_p]

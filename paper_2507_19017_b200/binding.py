@@ -119,7 +119,9 @@ _lib = None
 
 
 def lib_path() -> str:
-    return _build.LIB_PATH
+    """The library to load: libtd.so beside this file, or the build named by TD_LIB_PATH (a build
+    of the same sources with other compiler flags: sanitizers, NVTX ranges)."""
+    return os.environ.get("TD_LIB_PATH") or _build.LIB_PATH
 
 
 def lib():

@@ -15,6 +15,21 @@
 
 using namespace td;
 
+// Named ranges around the public calls for timeline tools (NVTX; compiled in with -DTD_NVTX, the
+// header-only nvtx3 that ships with the toolkit; otherwise the macro is empty).
+#ifdef TD_NVTX
+#include <nvtx3/nvToolsExt.h>
+namespace {
+struct TdRange {
+    explicit TdRange(const char *name) { nvtxRangePushA(name); }
+    ~TdRange() { nvtxRangePop(); }
+};
+}  // namespace
+#define TD_RANGE(name) TdRange td_range_guard(name)
+#else
+#define TD_RANGE(name) do { } while (0)
+#endif
+
 struct td_dock {
     DockView dv;
     td_config cfg;                 // columns / consumers pointers are not kept
@@ -330,6 +345,7 @@ int td_destroy(td_dock *dock) {
 }
 
 int td_reset(td_dock *d, void *stream) {
+    TD_RANGE("td_reset");
     if (!d) return TD_EINVAL;
     const uint32_t blocks = (uint32_t)std::min<size_t>((d->dv.n + 255) / 256, (size_t)d->sm_count * 4);
     if (launch(d, reset_kernel, dim3(blocks ? blocks : 1), dim3(256), 0, (cudaStream_t)stream, d->dv) != cudaSuccess)
@@ -497,6 +513,7 @@ int put_items(td_dock *d, const PutArgs *items, uint32_t n_items, cudaStream_t s
 }  // namespace
 
 int td_put_many(td_dock *d, const td_put_item *items, uint32_t n_items, void *stream) {
+    TD_RANGE("td_put_many");
     if (!d || (n_items && !items)) return TD_EINVAL;
     for (uint32_t i = 0; i < n_items; ++i)
         if (!valid_put_item(d, items[i])) return TD_EINVAL;
@@ -527,6 +544,7 @@ int back_args(const td_dock *d, const td_get_out *batch, uint32_t max_samples, u
 
 int td_put_back(td_dock *d, const td_get_out *batch, uint32_t max_samples, const td_back_item *items,
                 uint32_t n_items, void *stream) {
+    TD_RANGE("td_put_back");
     if (!d || !batch || (n_items && !items)) return TD_EINVAL;
     std::vector<PutArgs> args(n_items);
     for (uint32_t i = 0; i < n_items; ++i) {
@@ -537,6 +555,7 @@ int td_put_back(td_dock *d, const td_get_out *batch, uint32_t max_samples, const
 }
 
 int td_put_back_many(td_dock *d, const td_back_req *reqs, uint32_t n_reqs, void *stream) {
+    TD_RANGE("td_put_back_many");
     if (!d || (n_reqs && !reqs)) return TD_EINVAL;
     std::vector<PutArgs> args(n_reqs);
     for (uint32_t i = 0; i < n_reqs; ++i) {
@@ -598,6 +617,7 @@ int get_one(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_ou
 }  // namespace
 
 int td_get(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out *out, void *stream) {
+    TD_RANGE("td_get");
     if (!d) return TD_EINVAL;
     const DockView &v = d->dv;
     const int chk = check_get_out(v, consumer, max_samples, out);
@@ -645,6 +665,7 @@ int static_scratch_address(int device, void **out) {
 }  // namespace
 
 int td_get_static(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out *out, void *stream) {
+    TD_RANGE("td_get_static");
     if (!d) return TD_EINVAL;
     const DockView &v = d->dv;
     const int chk = check_get_out(v, consumer, max_samples, out);
@@ -766,7 +787,8 @@ int td_plan_destroy(td_plan *p) {
 namespace {
 int get_many(td_dock *d, td_plan *p, uint8_t *d_meta, void *stream);
 }
-int td_get_many(td_dock *d, td_plan *p, void *stream) { return get_many(d, p, nullptr, stream); }
+int td_get_many(td_dock *d, td_plan *p, void *stream) {
+    TD_RANGE("td_get_many"); return get_many(d, p, nullptr, stream); }
 
 namespace {
 // d_meta: staging buffer for the second copy of the requests' small outputs, or nullptr.
@@ -965,6 +987,7 @@ size_t td_put_host_stage_bytes(const td_dock *d, uint32_t column, uint32_t k, ui
 
 int td_put_host(td_dock *d, uint32_t column, const int32_t *h_indices, uint32_t k, const int32_t *h_cu,
                 const void *h_data, uint64_t data_elems, void *d_stage, size_t stage_bytes, void *stream) {
+    TD_RANGE("td_put_host");
     if (!d || column >= d->dv.ncol) return TD_EINVAL;
     if (k == 0) return TD_OK;
     if (!h_indices || (!h_data && data_elems) || !d_stage) return TD_EINVAL;
@@ -993,7 +1016,7 @@ int copy_batch_to_host(const DockView &v, uint32_t consumer, const td_get_out *d
     const size_t n = res->n_samples;
     // the transfers wanted, in order; neighbours that continue each other on both sides go as one
     struct Piece { uint8_t *dst; const uint8_t *src; size_t bytes; };
-    Piece todo[8 + 2 * kMaxColumns];
+    Piece todo[8 + 2 * kMaxColumns] = {};
     int n_todo = 0;
     auto d2h = [&](void *dst, const void *src, size_t bytes) {
         if (!dst || !src || bytes == 0) return;
@@ -1038,6 +1061,7 @@ int copy_batch_to_host(const DockView &v, uint32_t consumer, const td_get_out *d
 
 int td_get_host(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_out *dev_out,
                 const td_get_out *host_out, void *stream) {
+    TD_RANGE("td_get_host");
     if (!d || !dev_out || !host_out || !host_out->result || !host_out->indices) return TD_EINVAL;
     const int rc = td_get(d, consumer, max_samples, dev_out, stream);
     if (rc != TD_OK) return rc;
@@ -1055,6 +1079,7 @@ size_t td_get_many_host_stage_bytes(const td_plan *p) { return p ? p->meta_total
 
 int td_get_many_host(td_dock *d, td_plan *p, const td_get_out *host_outs, uint32_t n_req, void *d_stage,
                      size_t stage_bytes, void *stream) {
+    TD_RANGE("td_get_many_host");
     if (!d || !p || p->dock != d || !host_outs || n_req != p->n_req) return TD_EINVAL;
     for (uint32_t q = 0; q < n_req; ++q)
         if (!host_outs[q].result || !host_outs[q].indices) return TD_EINVAL;
@@ -1103,6 +1128,7 @@ int td_get_many_host(td_dock *d, td_plan *p, const td_get_out *host_outs, uint32
 
 int td_put_many_host(td_dock *d, const td_put_item *h_items, uint32_t n_items, void *d_stage, size_t stage_bytes,
                      void *stream) {
+    TD_RANGE("td_put_many_host");
     if (!d || (n_items && !h_items)) return TD_EINVAL;
     if (n_items == 0) return TD_OK;
     if (!d_stage || (reinterpret_cast<uintptr_t>(d_stage) & 255u)) return TD_EWORKSPACE;

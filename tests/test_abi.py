@@ -117,6 +117,23 @@ def test_create_fails_loudly_without_a_device(td):
 
 def test_missing_library_raises(td, monkeypatch):
     monkeypatch.setattr(td, "_lib", None)
+    monkeypatch.delenv("TD_LIB_PATH", raising=False)
     monkeypatch.setattr(td._build, "LIB_PATH", "/nonexistent/libtd.so")
     with pytest.raises(RuntimeError):
         td.lib()
+
+
+def test_build_with_nvtx_ranges_exports_the_same_symbols(td, tmp_path):
+    """-DTD_NVTX wraps the public calls in named ranges for timeline tools; the build must succeed
+    against the toolkit's header-only nvtx3 and change nothing about the ABI."""
+    from paper_2507_19017_b200 import build as b
+    out = str(tmp_path / "libtd_nvtx.so")
+    cmd = [b._nvcc()] + b.NVCC_FLAGS + ["-DTD_NVTX", "-o", out] + [os.path.join(b.CSRC, s) for s in b.SOURCES] + ["-ldl"]
+    env = {k: v for k, v in os.environ.items() if k != "LD_PRELOAD"}      # the compiler runs without any preloaded runtime
+    res = subprocess.run(cmd, capture_output=True, text=True, timeout=900, env=env)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lib = C.CDLL(out)
+    for name in declared_functions():
+        assert hasattr(lib, name), name
+    lib.td_strerror.restype = C.c_char_p
+    assert lib.td_strerror(0) == b"ok"
