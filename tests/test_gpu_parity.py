@@ -591,6 +591,30 @@ def test_bad_cu_entry_in_the_middle_of_a_put_skips_only_that_row(G):
         G.assert_batch_equal(g.get(cons, w.n), o.get(cons, w.n), f"consumer {cons}")
 
 
+def test_same_sample_twice_in_one_call_is_safe(G):
+    """The same index more than once inside one put is outside what the dock specifies (which copy
+    stays is open), but it must be safe: the row ends up stored once, the tables stay sound, the
+    counters agree with the tables, and - both copies being equal here - the row reads back."""
+    w = wl.make_custom("twice", 6, 4, 2, prompt_len=(3, 40), response=("uniform", 5000, 9000), vocab=1000,
+                       micro_batch=24, seed=17, schedule="none")
+    g = G.GpuDock(w)
+    rid, pid, rew = w.column_index("response_ids"), w.column_index("prompt_ids"), w.column_index("reward")
+    order = np.array([0, 1, 1, 2, 3, 3, 3] + list(range(4, w.n)) + [w.n - 1], np.int32)     # long rows: several chunks each
+    for c in (rid, pid, rew, w.column_index("old_logprob"), w.column_index("ref_logprob")):
+        cu, data = w.pack(c, order)
+        g.put(c, order, cu, data)
+    rep = g.dock.validate()
+    assert rep.violations == 0
+    assert list(rep.stored[:len(w.columns)]) == [w.n] * len(w.columns)
+    st = g.dock.status()
+    assert all(st.put_accepted[c] == w.n for c in range(len(w.columns)))
+    assert st.error_word & ~td.ERR_DUP_PUT == 0
+    got = g.get(3, w.n)
+    assert got.n_samples == w.n and got.status == 0
+    for c, spec in enumerate(w.columns):
+        assert H.bits_equal(got.columns[c], w.data[spec.name]), spec.name
+
+
 def test_arena_full_refuses_only_rows_without_room(G):
     w = wl.make_custom("full", 4, 4, 2, prompt_len=(10, 10), response=("uniform", 5, 60), vocab=1000,
                        micro_batch=16, seed=9, schedule="none")
