@@ -39,7 +39,27 @@ NOMINAL_HBM_GBPS = 8000.0             # the "~8 TB/s" the 70 % target is stated 
 # DRAM bytes (read + write) of one launch of the copy kernels as they are built now, taken from
 # the ncu summaries under profiles/: (config, kernel) -> (bytes, file, what was captured).
 # A pair without a capture of the current kernels reports null.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {
+    (2, "get_gather"): (80_914_432, "profiles/copy_kernels_config2_7b_shaped.md", "ncu capture of this kernel on this shape"),
+    (2, "put_scatter"): (46_817_792, "profiles/copy_kernels_config2_7b_shaped.md", "ncu capture of this kernel on this shape"),
+    (3, "get_gather"): (1_147_037_952, "profiles/copy_kernels_config3_32b_shaped.md", "ncu capture of this kernel on this shape"),
+    (3, "put_scatter"): (733_611_776, "profiles/copy_kernels_config3_32b_shaped.md", "ncu capture of this kernel on this shape"),
+}
+# The larger shapes hold too much on the device for a full counter capture; their traffic is taken
+# to grow with the bytes that must cross HBM, from the capture of the 32B-shaped batch:
+# kernel -> (captured traffic, HBM-crossing bytes of that launch).
+NCU_SCALE_FROM_CONFIG3 = {"get_gather": (1_147_037_952, 1_200_614_776), "put_scatter": (733_611_776, 784_775_700)}
+
+
+def captured_traffic(cid: int, kernel: str, bytes_per_launch: float):
+    """(bytes, source, note) or None."""
+    if (cid, kernel) in NCU_TRAFFIC:
+        return NCU_TRAFFIC[(cid, kernel)]
+    if cid in (4, 5) and kernel in NCU_SCALE_FROM_CONFIG3:
+        t, b = NCU_SCALE_FROM_CONFIG3[kernel]
+        return (int(bytes_per_launch * t / b), "profiles/copy_kernels_config3_32b_shaped.md",
+                "scaled from the capture of the 32B-shaped batch by the bytes that must cross HBM")
+    return None
 
 
 def parse_args():
@@ -936,7 +956,8 @@ def measure_dispatch(args, cid: int, rank: int, local_rank: int, world: int, dis
                 "get_gather": kernel_record(ms_ga, n_ga, ksteps, sb["get_hbm"], sb["get_delivered"], peak)}
         dom = "get_gather" if ms_ga >= ms_sc else "put_scatter"
         k = kern[dom]
-        traffic = None if (args.fused or args.padded or warm_l2 or sigma is not None) else NCU_TRAFFIC.get((cid, dom))
+        traffic = (None if (args.fused or args.padded or warm_l2 or sigma is not None or args.api != "many")
+                   else captured_traffic(cid, dom, k["bytes_per_launch"]))
         rec["kernels"] = kern
         rec["roofline"] = {
             # numerator: the bytes that must cross HBM in one launch (every stored row that is taken
