@@ -20,9 +20,9 @@ rows that rank owns).  What this module adds is the part between the ranks:
          The owners' packed rows then travel to the home rank, which lays them out in global
          group order and rebuilds cu_seqlens from the lengths.
 
-No data-path collective exists inside a rank's dock, and nothing here uses a load with cluster
-multicast or hands a peer's memory to a library kernel: the exchange is torch.distributed
-(NCCL on GPUs, gloo in the CPU tests) into local buffers.  With one rank every exchange
+No data-path collective exists inside a rank's dock, and no kernel, this library's or anyone's,
+is handed another GPU's memory: the exchange is torch.distributed (NCCL on GPUs, gloo in the CPU
+tests) into local buffers.  With one rank every exchange
 degenerates to a local copy and the results are those of the plain dock.
 
 The local dock is reached through a small adapter (`CudaLocal` below; the tests plug a CPU
