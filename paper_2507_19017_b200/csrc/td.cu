@@ -109,7 +109,7 @@ Layout make_layout(const td_config *c) {
     L.errword = take(256);
     L.counters = take(CNT_TOTAL * 8);
     L.put_counters = take((size_t)kPutCounterSlots * 8);
-    L.put_ready = take((size_t)kPutCounterSlots * 8);
+    L.put_ready = take((size_t)kPutCounterSlots * 4 * 8);
     L.progress = take((size_t)c->n_columns * n * 4);
     L.status = take(n * 4);
     for (int k = 1; k <= 2; ++k) { L.len[k] = take(n * 4); L.off[k] = take(n * 8); L.cursor[k] = take(S * 8); }
@@ -330,7 +330,7 @@ int td_create(const td_config *cfg, void *d_workspace, size_t bytes, td_dock **o
     d->table_bytes[3] = (size_t)v.S * 8; d->table_bytes[4] = (size_t)v.claim_words * 4;
     d->table_bytes[5] = (size_t)v.consumed_words * 4; d->table_bytes[6] = 0;
 
-    int rc = cudaMemsetAsync(w + L.put_ready, 0, (size_t)kPutCounterSlots * 8, nullptr) == cudaSuccess ? TD_OK : TD_ECUDA;
+    int rc = cudaMemsetAsync(w + L.put_ready, 0, (size_t)kPutCounterSlots * 4 * 8, nullptr) == cudaSuccess ? TD_OK : TD_ECUDA;
     if (rc == TD_OK) rc = td_reset(d, nullptr);
     if (rc == TD_OK && cudaStreamSynchronize(nullptr) != cudaSuccess) rc = TD_ECUDA;
     if (rc != TD_OK) { delete d; return rc; }
@@ -412,13 +412,22 @@ int put_group(td_dock *d, PutBatch &b, cudaStream_t st) {
     }
     if (entries == 0) return TD_OK;
     if (entries >= (1ull << 32)) return TD_EINVAL;
-    b.work_counter = nullptr; b.ready = nullptr; b.seq = 0;
+    b.work_counter = nullptr; b.ready = nullptr; b.progress = nullptr; b.seq = 0;
     if (ragged_bytes) {
         const int slot = stream_slot(d, st);
         if (slot >= 0) {
             b.work_counter = d->dv.put_counters + slot;
-            b.ready = d->dv.put_ready + slot;
+            b.ready = d->dv.put_ready + 4 * (size_t)slot;
             b.seq = g_put_seq.fetch_add(1, std::memory_order_relaxed);
+            // the per-class counts of allocated entries go by the order of the leader items, which is
+            // only known here when no follower has to be compared with its leader on the device
+            bool settled = true;
+            for (uint32_t i = 0; i < b.n_items; ++i)
+                if (b.follow[i]) {
+                    const PutArgs &a = b.item[i], &ld = b.item[b.follow[i] - 1u];
+                    settled = settled && a.idx == ld.idx && a.cu == ld.cu;
+                }
+            if (settled) b.progress = b.ready + 1;
         }
         ragged_bytes += entries * kPutScalarCost;              // the scalar items of the call ride along
         // entries per thread and pass of the alloc kernel: enough for the largest item in one pass, up to four

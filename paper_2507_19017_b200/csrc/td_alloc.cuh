@@ -45,7 +45,16 @@ struct PutBatch {                              // the columns of one call, in ca
     // then on.  nullptr: the scatter kernel waits for the alloc kernel's end before it reads anything.
     unsigned long long *ready;
     unsigned long long seq;
+    // Two more words behind `ready`, one per length class, when the call's followers are settled
+    // on the host (progress != nullptr): the alloc kernel stores there, pass after pass, how
+    // many entries of its class it has dealt with - counted over the class's leader items in call
+    // order, tagged with the call's number - and the scatter kernel copies a row as soon as the
+    // count has passed it, instead of waiting for the whole allocation.
+    unsigned long long *progress;
 };
+__host__ __device__ __forceinline__ unsigned long long progress_pack(unsigned long long seq, uint32_t done) {
+    return (seq << 32) | done;
+}
 
 static inline size_t put_alloc_smem_bytes(uint32_t S) {
     return (size_t)(kAllocWarps + 2) * S * sizeof(unsigned long long);
@@ -146,10 +155,30 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
     // kernel in the stream (a reset, the get whose batch is sent back, the caller's own producer)
     // must have finished.  The prefetch above only asked for lines.
     griddep_wait();
-    if (blockIdx.x == 0 && tid == 0) {
-        if (batch.work_counter) *batch.work_counter = 0;
-        if (batch.ready) st_release_u64(batch.ready, batch.seq);       // the call's inputs are complete: the scatter may look
+    if (blockIdx.x == 0 && tid == 0 && batch.work_counter) *batch.work_counter = 0;
+    // Ahead of everything else: is every cu array of this class a non-decreasing sequence inside
+    // its data?  The scatter kernel searches those arrays and must know before it starts; one
+    // sweep over entries whose lines were asked for above.  Then the class reports its inputs
+    // complete (the second class to do so makes the word read seq * 4 + 2).
+    if (batch.ready) {
+        #pragma unroll 1
+        for (uint32_t it = 0; it < batch.n_items; ++it) {
+            const PutArgs &a = batch.item[it];
+            if (dv.col_cls[a.column] != L) continue;
+            const uint32_t k = item_k(a);
+            for (uint32_t i = tid; i < k; i += kAllocThreads) {
+                const int64_t c0 = a.cu[i], c1 = a.cu[i + 1];
+                irregular |= c1 < c0 || c0 < 0 || (uint64_t)c1 > a.data_elems;
+            }
+        }
+        if (__syncthreads_or(irregular) && tid == 0) atomicOr(dv.errword, kErrIrregularCu);
+        if (tid == 0) {
+            __threadfence();
+            atomicMax(batch.ready, batch.seq << 2);
+            atomicAdd(batch.ready, 1ull);
+        }
     }
+    uint32_t done_before = 0;                  // entries of this class's earlier leader items
 
     // Which proposed followers really repeat their leader's index and cu arrays?  (Nothing to
     // find out, and no barrier to pass, when every one of them names its leader's own arrays.)
@@ -258,7 +287,7 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
                 any |= alloc[j];
             }
             if (tid == 0) s_overflow = 0;
-            if (!__syncthreads_or(any)) continue;                 // no first arrival in this pass
+            if (__syncthreads_or(any)) {                          // else: no first arrival in this pass
 
             // 2. relative places: inside a warp its entries in order (four shuffle scans that
             //    carry the warp's per-shard sums along), then the warps in order (one scan over
@@ -331,7 +360,15 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
                 }
             }
             __syncthreads();
+            }
+            // the rows of this pass have their places: whoever copies them may go ahead
+            if (batch.progress && tid == 0) {
+                __threadfence();
+                st_release_u64(&batch.progress[L - 1],
+                               progress_pack(batch.seq, done_before + min(base + (uint32_t)kAllocPass, k)));
+            }
         }
+        done_before += k;
     }
     n_oob = __reduce_add_sync(kFullMask, n_oob);
     n_dup = __reduce_add_sync(kFullMask, n_dup);

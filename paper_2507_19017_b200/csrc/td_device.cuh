@@ -70,7 +70,7 @@ struct DockView {
     uint32_t *errword;
     unsigned long long *counters;           // [CNT_TOTAL]
     unsigned long long *put_counters;       // [kPutCounterSlots] chunk counters of the scatter kernel, one per stream in use
-    unsigned long long *put_ready;          // [kPutCounterSlots] number of the latest put on that stream whose inputs are known to be complete
+    unsigned long long *put_ready;          // [kPutCounterSlots][4] per stream that puts: "inputs complete" word, entries allocated so far per length class (see PutBatch)
     uint32_t *progress;                     // [ncol][n] elements of a row written so far by the put that stores it
     uint8_t  *colbase[kMaxColumns];         // arena (S * cap * esz) or scalar store (n * esz)
     uint32_t need[kMaxColumns];             // per consumer
@@ -586,54 +586,61 @@ __device__ __forceinline__ void publish_queue_note(const DockView &dv, PublishQu
 // (seq_tail false) or ends at element seq_cu[i + 1] (seq_tail true) instead of starting at
 // cu[i] - the two halves of a stream in which each sample's prompt row is followed by its
 // response row; cu still says how long the rows are and where they lie in the chunked space.
-template <bool kToPacked, bool kPublish, typename Resolve>
+struct NoAwait {
+    __device__ __forceinline__ void operator()(uint32_t) const {}
+};
+template <bool kToPacked, bool kPublish, typename Resolve, typename Await = NoAwait>
 __device__ __forceinline__ void warp_copy_chunk(const int32_t *cu, uint32_t rows, uint64_t b0, uint64_t b1,
                                                 uint8_t *packed, uint32_t esz, uint32_t lane,
                                                 const uint8_t *src_lo, const uint8_t *src_hi, WarpPipe &pipe,
                                                 const int32_t *along, Resolve resolve,
                                                 const int32_t *seq_cu = nullptr, bool seq_tail = false,
                                                 const DockView *dvp = nullptr, PublishQueue *queue = nullptr,
-                                                uint32_t column = 0) {
+                                                uint32_t column = 0, Await await = Await()) {
     uint32_t r0 = warp_find_row(cu, rows, (int64_t)b0, esz, kRowCost, lane, along);
     for (;;) {
         // lane l: the part of row r0 + l that falls inside the chunk, as (address on the packed
         // side, address on the other side, bytes); bytes = 0 when there is nothing to copy
         const uint32_t i = r0 + lane;
-        bool in = false;
+        bool in = false, wanted = false;
         uint32_t len = 0;
         uint8_t *mine = nullptr, *other = nullptr;
         int32_t s_row = -1;                // put: the sample of a row this lane has a part of, or owns
         uint32_t total = 0;                // put: the row's length in elements
+        int64_t c0 = 0, c1 = 0;
+        uint64_t dlo = 0, lo = 0, hi = 0;
         if (i < rows) {
-            const int64_t c0 = __ldg(cu + i);
+            c0 = __ldg(cu + i);
             const uint64_t row0 = (uint64_t)c0 * esz + (uint64_t)i * kRowCost;
             in = c0 >= 0 && row0 < b1;
             if (in) {
-                const int64_t c1 = __ldg(cu + i + 1);
-                const uint64_t dlo = row0 + kRowCost;                       // the row's bytes, in the chunked space
+                c1 = __ldg(cu + i + 1);
+                dlo = row0 + kRowCost;                                       // the row's bytes, in the chunked space
                 const uint64_t dhi = c1 > c0 ? dlo + (uint64_t)(c1 - c0) * esz : dlo;
-                const uint64_t lo = max(dlo, b0), hi = min(dhi, b1);
+                lo = max(dlo, b0); hi = min(dhi, b1);
                 const bool empty_here = kPublish && c1 == c0 && row0 >= b0;   // a row of no length whose place is in this chunk
-                if (hi > lo || empty_here) {
-                    int32_t s = -1;
-                    uint8_t *row = resolve(i, c0, c1, s);
-                    if (row) {
-                        s_row = s;
-                        total = (uint32_t)(c1 - c0);
-                        if (hi > lo) {
-                            other = row + (lo - dlo);
-                            uint64_t at = (uint64_t)c0;
-                            if (seq_cu) at = seq_tail ? (uint64_t)((int64_t)__ldg(seq_cu + i + 1) - (c1 - c0))
-                                                      : (uint64_t)__ldg(seq_cu + i);
-                            mine = packed + at * esz + (lo - dlo);
-                            len = (uint32_t)(hi - lo);
-                        }
-                    }
-                }
+                wanted = hi > lo || empty_here;
             }
         }
         // rows inside the chunk form a prefix of the lanes
         const uint32_t n_rows = (uint32_t)__ffs(~__ballot_sync(kFullMask, in)) - 1u;   // 32 when all lanes are in
+        await(r0 + n_rows);                // put: until the rows before that number have their places
+        if (wanted) {
+            int32_t s = -1;
+            uint8_t *row = resolve(i, c0, c1, s);
+            if (row) {
+                s_row = s;
+                total = (uint32_t)(c1 - c0);
+                if (hi > lo) {
+                    other = row + (lo - dlo);
+                    uint64_t at = (uint64_t)c0;
+                    if (seq_cu) at = seq_tail ? (uint64_t)((int64_t)__ldg(seq_cu + i + 1) - (c1 - c0))
+                                              : (uint64_t)__ldg(seq_cu + i);
+                    mine = packed + at * esz + (lo - dlo);
+                    len = (uint32_t)(hi - lo);
+                }
+            }
+        }
         uint32_t todo = __ballot_sync(kFullMask, len != 0);
         while (todo) {
             const uint32_t r = (uint32_t)__ffs(todo) - 1u;

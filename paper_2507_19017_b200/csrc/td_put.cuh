@@ -106,11 +106,13 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
     // Inputs complete?  The alloc kernel says so ahead of its own work; if the word does not show
     // up within the limit, the wait for that kernel's end says the same, only later.
     __shared__ uint32_t s_gave_up;
+    __shared__ uint32_t item_base[kMaxPutItems];      // entries of the same class's leader items ahead of the item's leader
+    __shared__ uint32_t class_total[3];               // entries of a class's leader items
     bool waited = true;
     if (batch.ready) {
         if (tid == 0) {
             uint32_t polls = 0;
-            while (ld_acquire_u64(batch.ready) != batch.seq && ++polls < 4096u) __nanosleep(64);
+            while (ld_acquire_u64(batch.ready) != (batch.seq << 2) + 2u && ++polls < 4096u) __nanosleep(64);
             s_gave_up = polls >= 4096u;
         }
         __syncthreads();
@@ -137,10 +139,17 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
     __syncthreads();
     if (tid == 0) {
         uint64_t acc = 0;
+        uint32_t seen[3] = {0, 0, 0};
         for (uint32_t it = 0; it < batch.n_items; ++it) {
             acc += (item_bytes[it] + 15) & ~uint64_t(15);
             item_end[it] = acc;
+            // where the alloc kernel's count of entries stands when it reaches this item's rows:
+            // a follower's rows are settled with its leader's
+            const uint32_t L = dv.col_cls[batch.item[it].column];
+            if (batch.follow[it]) item_base[it] = item_base[batch.follow[it] - 1u];
+            else { item_base[it] = seen[L]; seen[L] += item_rows[it]; }
         }
+        class_total[0] = 0; class_total[1] = seen[1]; class_total[2] = seen[2];
     }
     __syncthreads();
     const uint64_t n_warps = (uint64_t)gridDim.x * kCopyWarps;
@@ -185,10 +194,38 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
                 }
             }
         }
-        griddep_wait();                                // the alloc kernel's tables are complete
+        // with a count of the entries allocated so far, rows are waited for one chunk at a time
+        if (!batch.progress || (*dv.errword & kErrIrregularCu)) { griddep_wait(); waited = true; }
     }
     // Nothing behind this kernel needs it to have finished before it starts setting itself up.
     griddep_launch_dependents();
+    // Rows [0, need) of the item being copied have their places once the alloc kernel's count for
+    // the item's class has reached item_base + need.  One lane polls; when the count does not get
+    // there within the limit, the wait for that kernel's end settles it, as it does once for all
+    // when the call has no such count.
+    bool done_prompt = waited, done_response = waited;       // the class's count has reached its total
+    uint32_t cur_item = 0, cur_class = 0;
+    auto await = [&](uint32_t need_rows) {
+        if (cur_class == TD_PROMPT ? done_prompt : done_response) return;
+        const uint32_t need = item_base[cur_item] + need_rows;
+        unsigned long long v = 0;
+        if (lane == 0) {
+            uint32_t polls = 0;
+            for (;;) {
+                v = ld_acquire_u64(&batch.progress[cur_class - 1u]);
+                if (((uint32_t)(v >> 32) == (uint32_t)batch.seq && (uint32_t)v >= need) || ++polls >= 16384u) break;
+                __nanosleep(100);
+            }
+        }
+        v = shfl_u64(v, 0);
+        if ((uint32_t)(v >> 32) != (uint32_t)batch.seq || (uint32_t)v < need) {
+            griddep_wait();
+            done_prompt = done_response = true;
+        } else if ((uint32_t)v >= class_total[cur_class]) {
+            if (cur_class == TD_PROMPT) done_prompt = true; else done_response = true;
+        }
+        __syncwarp();
+    };
 
     ScalarCounts cnt{0, 0, 0};
     PublishQueue queue;
@@ -257,13 +294,14 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
                     const uint32_t n_ok = warp_put_scalars(dv, a, e0, e1, lane, cnt);
                     if (lane == 0 && n_ok) atomicAdd(&dv.counters[CNT_PUT_ACCEPTED + a.column], (unsigned long long)n_ok);
                 } else {
+                    cur_item = it; cur_class = L;
                     warp_copy_chunk<false, true>(
                         a.cu, item_rows[it], b0, b1, const_cast<uint8_t *>(a.data), esz, lane,
                         a.data, a.data + a.data_elems * esz, pipe, a.idx,
                         [&](uint32_t i, int64_t c0, int64_t c1, int32_t &s) -> uint8_t * {
                             return put_row_dst(dv, a, L, bit, esz, i, c0, c1, s);     // live if the alloc kernel accepted it
                         },
-                        nullptr, false, &dv, &queue, a.column);
+                        nullptr, false, &dv, &queue, a.column, await);
                 }
             }
             ch = work_counter ? shfl_u64(next, 0) : next;
@@ -271,6 +309,9 @@ put_scatter_kernel(const DockView dv, const PutBatch batch) {
     }
     publish_queue_flush(dv, queue, pipe, lane);
     if (pipe.finish(lane) && lane == 0) flag_error(dv, TD_ERR_COPY_TIMEOUT, CNT_TIMEOUT);
+    // This kernel's end must imply the alloc kernel's (whatever follows in the stream waits for
+    // this one only); by now that kernel is long done.
+    if (!waited) griddep_wait();
     cnt.oob = __reduce_add_sync(kFullMask, cnt.oob);
     cnt.dup = __reduce_add_sync(kFullMask, cnt.dup);
     cnt.bad = __reduce_add_sync(kFullMask, cnt.bad);
