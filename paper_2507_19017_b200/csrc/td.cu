@@ -41,6 +41,7 @@ struct td_dock {
     std::atomic<uint64_t> launches;
     std::mutex slot_mu;
     std::vector<cudaStream_t> slot_stream;     // which stream draws from which scatter chunk counter
+    std::mutex put_mu;                         // a put takes its number and enqueues its kernels as one step
     // optional per-kernel timing of the two copy kernels (0 = put scatter, 1 = get gather)
     std::atomic<bool> timing;
     std::mutex timing_mu;
@@ -414,6 +415,10 @@ int put_group(td_dock *d, PutBatch &b, cudaStream_t st) {
     if (entries >= (1ull << 32)) return TD_EINVAL;
     b.work_counter = nullptr; b.ready = nullptr; b.progress = nullptr; b.seq = 0;
     if (ragged_bytes) {
+        // The words the two kernels talk through carry the call's number, and numbers must grow in
+        // the order the calls reach their stream: two host threads putting on one stream take
+        // their number and enqueue under one lock.
+        std::lock_guard<std::mutex> order(d->put_mu);
         const int slot = stream_slot(d, st);
         if (slot >= 0) {
             b.work_counter = d->dv.put_counters + slot;
