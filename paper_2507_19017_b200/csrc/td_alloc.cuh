@@ -166,6 +166,11 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
             const PutArgs &a = batch.item[it];
             if (dv.col_cls[a.column] != L) continue;
             const uint32_t k = item_k(a);
+            if (batch.follow[it] && a.cu == batch.item[batch.follow[it] - 1u].cu) {
+                // the leader's very array, swept with the leader: only this item's own bound is left
+                if (tid == 0 && k) irregular |= (uint64_t)a.cu[k] > a.data_elems;
+                continue;
+            }
             for (uint32_t i = tid; i < k; i += kAllocThreads) {
                 const int64_t c0 = a.cu[i], c1 = a.cu[i + 1];
                 irregular |= c1 < c0 || c0 < 0 || (uint64_t)c1 > a.data_elems;
