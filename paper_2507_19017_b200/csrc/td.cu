@@ -478,6 +478,25 @@ uint64_t room_bytes_of(const DockView &v, uint32_t consumer, uint32_t max_sample
 bool wants_stream(const td_get_out &out) { return out.seq || out.seq_advantages; }
 uint32_t jobs_per_req(const DockView &v, bool stream) { return v.ncol + (stream ? kSeqJobs : 0u); }
 
+// The room a request's output buffers leave (see GetReq): by class, over the wanted columns.
+void fill_room(const DockView &v, uint32_t consumer, const td_get_out &out, GetReq &rq) {
+    rq.room_tok[0] = rq.room_tok[1] = rq.room_tok[2] = ~0ull;
+    rq.room_rows = ~0ull;
+    rq.want_classes = 0;
+    for (uint32_t k = 0; k < v.ncol; ++k) {
+        if (!((v.outm[consumer] >> k) & 1u) || out.col[k] == nullptr) continue;
+        const uint32_t cls = v.col_cls[k];
+        const uint64_t capk = out.col_capacity_elems[k];
+        rq.want_classes |= 1u << cls;
+        if (cls == TD_SCALAR) rq.room_tok[0] = std::min<uint64_t>(rq.room_tok[0], capk);
+        else if (out.mode == TD_PACKED) rq.room_tok[cls] = std::min<uint64_t>(rq.room_tok[cls], capk);
+        else {
+            const uint32_t W = cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to;
+            rq.room_rows = std::min<uint64_t>(rq.room_rows, W ? capk / W : 0);
+        }
+    }
+}
+
 // Upper bound of what a request adds to the space the gather cuts into chunks: its output room
 // plus the fixed charge of every row of every job.
 uint64_t extent_bound_of(const DockView &v, uint32_t consumer, uint32_t max_samples, const td_get_out &out, uint32_t jpr) {
@@ -604,6 +623,7 @@ int get_one(td_dock *d, uint32_t consumer, uint32_t max_samples, const td_get_ou
     one.req.max_groups = m < v.G ? m : v.G;
     one.req.rank_base = 0;
     one.req.cslot = 0;
+    fill_room(v, consumer, *out, one.req);
     one.cs.consumer = consumer;
     one.cs.max_groups = one.req.max_groups;
     one.cs.scratch = scratch;
@@ -770,6 +790,7 @@ int td_plan_create(td_dock *d, const td_get_req *reqs, uint32_t n_req, void *d_p
         hr[q].max_groups = m;
         hr[q].cslot = (uint32_t)slot_of[c];
         hr[q].meta_samples = std::min(m, v.G) * v.N;
+        fill_room(v, c, reqs[q].out, hr[q]);
         hr[q].meta_off = p->meta_total;
         p->meta_total += align_up_sz(meta_bytes(hr[q].meta_samples), 16);
         const uint64_t sum = (uint64_t)cs.max_groups + m;

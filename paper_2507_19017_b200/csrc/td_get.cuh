@@ -76,8 +76,16 @@ struct alignas(128) GetReq {
     // cu_response[m+1], cu_seq[m+1], advantages[m], m = meta_samples.
     uint64_t meta_off;
     uint32_t meta_samples;
-    uint32_t pad;
+    // What the output buffers leave room for, worked out on the host when the request is set up
+    // (the finalize kernel would otherwise walk the column pointers and capacities one dependent
+    // load after the other): samples by the tightest scalar column, prompt / response tokens by the
+    // tightest packed column of the class, rows by the tightest padded column; which classes
+    // have a wanted ragged column at all.
+    uint32_t want_classes;     // bit 1: a prompt-length column is wanted, bit 2: a response-length one
+    uint64_t room_tok[3];
+    uint64_t room_rows;
 };
+static_assert(sizeof(GetReq) == 768, "requests of a plan are read in whole 128-byte lines");
 // Views into such a block.
 struct MetaView {
     td_result *result;
@@ -478,31 +486,12 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
         if (out.cu_seq) out.cu_seq[0] = 0;
         if (mirror) { mv.cu_prompt[0] = 0; mv.cu_response[0] = 0; mv.cu_seq[0] = 0; }
     }
-    // tightest room per length class over the wanted columns
-    uint64_t room_tok[3] = {~0ull, ~0ull, ~0ull};      // packed: tokens; scalar slot [0]: samples
-    uint64_t room_rows = ~0ull;                         // padded: rows
-    const uint32_t outm = dv.outm[c];
-    #pragma unroll 1
-    for (uint32_t k = 0; k < dv.ncol; ++k) {
-        if (!((outm >> k) & 1u) || out.col[k] == nullptr) continue;
-        const uint32_t cls = dv.col_cls[k];
-        const uint64_t capk = out.col_capacity_elems[k];
-        if (cls == TD_SCALAR) room_tok[0] = min(room_tok[0], capk);
-        else if (out.mode == TD_PACKED) room_tok[cls] = min(room_tok[cls], capk);
-        else {
-            const uint32_t W = cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to;
-            room_rows = min(room_rows, W ? (uint64_t)(capk / W) : (uint64_t)0);
-        }
-    }
+    // tightest room per length class over the wanted columns (set up on the host)
+    const uint64_t room_tok[3] = {rq.room_tok[0], rq.room_tok[1], rq.room_tok[2]};
+    const uint64_t room_rows = rq.room_rows;
     const uint64_t room_seq = (out.seq || out.seq_advantages) ? out.seq_capacity_elems : ~0ull;
     const bool padded = out.mode == TD_PADDED;
-    bool want_p = false, want_r = false;
-    #pragma unroll 1
-    for (uint32_t k = 0; k < dv.ncol; ++k)
-        if (((outm >> k) & 1u) && out.col[k] != nullptr) {
-            want_p |= dv.col_cls[k] == TD_PROMPT;
-            want_r |= dv.col_cls[k] == TD_RESPONSE;
-        }
+    const bool want_p = (rq.want_classes >> TD_PROMPT) & 1u, want_r = (rq.want_classes >> TD_RESPONSE) & 1u;
     uint64_t carry_p = 0, carry_r = 0;
     for (uint32_t base = 0; base < n_s; base += kThreads) {
         const uint32_t i = base + tid;
