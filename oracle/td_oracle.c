@@ -249,9 +249,13 @@ static void emit(const ora_dock *d, const ora_consumer *K, const int32_t *idx, u
                 memcpy(dst + at * es, src, l * es);
                 at += l;
             } else {
+                /* a row of W elements: the l stored ones and W - l copies of the pad pattern,
+                 * behind them, or in front of them for a prompt that is asked for left-padded */
                 uint8_t *row = dst + (size_t)i * W * es;
-                memcpy(row, src, l * es);
-                for (size_t j = l; j < W; ++j) memcpy(row + j * es, &C->pad_bits, es);
+                const size_t lead = (L == ORA_PROMPT && (out->flags & ORA_OUT_LEFT_PAD_PROMPT)) ? W - l : 0;
+                for (size_t j = 0; j < lead; ++j) memcpy(row + j * es, &C->pad_bits, es);
+                memcpy(row + lead * es, src, l * es);
+                for (size_t j = lead + l; j < W; ++j) memcpy(row + j * es, &C->pad_bits, es);
             }
         }
     }
@@ -309,6 +313,7 @@ static void emit(const ora_dock *d, const ora_consumer *K, const int32_t *idx, u
  */
 int ora_get(ora_dock *d, uint32_t consumer, uint32_t max_samples, const ora_get_out *out) {
     if (!d || !out || consumer >= d->ncons || !out->indices || !out->result) return -1;
+    if (out->flags & ~(uint32_t)ORA_OUT_LEFT_PAD_PROMPT) return -1;
     const uint32_t m = max_samples / d->N;
     if (m == 0) return -1;
     ora_consumer *K = &d->cons[consumer];
@@ -359,6 +364,7 @@ int ora_get(ora_dock *d, uint32_t consumer, uint32_t max_samples, const ora_get_
 int ora_gather(const ora_dock *d, uint32_t consumer, const int32_t *indices, uint32_t count,
                const ora_get_out *out) {
     if (!d || !out || consumer >= d->ncons || (count && !indices)) return -1;
+    if (out->flags & ~(uint32_t)ORA_OUT_LEFT_PAD_PROMPT) return -1;
     const ora_consumer *K = &d->cons[consumer];
     if (!seq_args_ok(d, K, out)) return -1;
     uint64_t tokP = 0, tokR = 0; uint32_t maxP = 0, maxR = 0;

@@ -41,6 +41,7 @@ extern "C" {
 enum { ORA_I32 = 0, ORA_F32 = 1, ORA_BF16 = 2 };
 enum { ORA_SCALAR = 0, ORA_PROMPT = 1, ORA_RESPONSE = 2 };
 enum { ORA_PACKED = 0, ORA_PADDED = 1 };
+enum { ORA_OUT_LEFT_PAD_PROMPT = 1u };             /* ora_get_out.flags */
 enum { ORA_F_ADVANTAGE = 1u };
 
 /* condition bits, OR-ed into ora_result.status and the dock's error word */
@@ -74,6 +75,8 @@ typedef struct {
 typedef struct {
     int32_t  mode;                       /* ORA_PACKED | ORA_PADDED */
     uint32_t pad_prompt_to, pad_response_to;
+    uint32_t flags;                      /* ORA_OUT_LEFT_PAD_PROMPT (ORA_PADDED only): rows of prompt
+                                            columns end at their width, the pad comes first */
     int32_t *indices;                    /* [max_samples] */
     int32_t *cu_prompt, *cu_response, *cu_seq;   /* [max_samples + 1] */
     void    *col[32];                    /* NULL = not wanted */

@@ -21,6 +21,7 @@ DTYPES = {"i32": 0, "f32": 1, "bf16": 2}
 CLASSES = {"scalar": 0, "prompt": 1, "response": 2}
 NP_DTYPE = {0: np.int32, 1: np.float32, 2: np.uint16}
 PACKED, PADDED = 0, 1
+OUT_LEFT_PAD_PROMPT = 1            # flag of a get's output: prompt rows end at their width (PADDED only)
 F_ADVANTAGE = 1
 
 ERR_OOB_INDEX, ERR_DUP_PUT, ERR_LEN_MISMATCH, ERR_ARENA_FULL, ERR_OUT_TRUNC = 1, 2, 4, 8, 16
@@ -71,7 +72,7 @@ class _Result(C.Structure):
 
 class _GetOut(C.Structure):
     _fields_ = [("mode", C.c_int32), ("pad_prompt_to", C.c_uint32), ("pad_response_to", C.c_uint32),
-                ("indices", C.c_void_p), ("cu_prompt", C.c_void_p), ("cu_response", C.c_void_p),
+                ("flags", C.c_uint32), ("indices", C.c_void_p), ("cu_prompt", C.c_void_p), ("cu_response", C.c_void_p),
                 ("cu_seq", C.c_void_p), ("col", C.c_void_p * 32),
                 ("col_capacity_elems", C.c_uint64 * 32), ("advantages", C.c_void_p),
                 ("result", C.POINTER(_Result)),
@@ -198,11 +199,12 @@ class OracleDock:
     # -- get / gather -----------------------------------------------------
     def _alloc(self, consumer: int, max_samples: int, mode: int, pad_p: int, pad_r: int,
                capacities: Optional[Dict[int, int]], want: Optional[Sequence[int]],
-               lens_bound: Sequence[int], seq=None, seq_adv: bool = False, seq_cap: Optional[int] = None):
+               lens_bound: Sequence[int], seq=None, seq_adv: bool = False, seq_cap: Optional[int] = None,
+               out_flags: int = 0):
         need, outm, flags = self.consumers[consumer]
         res = _Result()
         go = _GetOut()
-        go.mode, go.pad_prompt_to, go.pad_response_to = mode, pad_p, pad_r
+        go.mode, go.pad_prompt_to, go.pad_response_to, go.flags = mode, pad_p, pad_r, out_flags
         bufs = {"indices": np.zeros(max_samples, np.int32)}
         for nm in ("cu_prompt", "cu_response", "cu_seq"):
             bufs[nm] = np.zeros(max_samples + 1, np.int32)
@@ -284,16 +286,18 @@ class OracleDock:
     def get(self, consumer: int, max_samples: int, mode: int = PACKED, pad_prompt_to: int = 0,
             pad_response_to: int = 0, capacities: Optional[Dict[int, int]] = None,
             want: Optional[Sequence[int]] = None, seq=None, seq_adv: bool = False,
-            seq_cap: Optional[int] = None) -> Batch:
+            seq_cap: Optional[int] = None, out_flags: int = 0) -> Batch:
         """seq = (prompt column, response column) asks for the fused token stream, seq_adv for
-        its advantage twin; seq_cap bounds both (default: room for the longest rows)."""
+        its advantage twin; seq_cap bounds both (default: room for the longest rows).
+        out_flags = OUT_LEFT_PAD_PROMPT: padded prompt rows carry their pad in front."""
         ragged = [c for c, (_d, cls, _p) in enumerate(self.columns)
                   if cls != 0 and (self.consumers[consumer][1] >> c) & 1 and (want is None or c in want)]
         need_bound = mode == PACKED and any(capacities is None or c not in capacities for c in ragged)
         need_bound = need_bound or ((seq is not None or seq_adv) and seq_cap is None)
         bound = self._bounds(max_samples) if need_bound else [0, 0, 0]
         go, res, bufs, cols, adv = self._alloc(consumer, max_samples, mode, pad_prompt_to,
-                                               pad_response_to, capacities, want, bound, seq, seq_adv, seq_cap)
+                                               pad_response_to, capacities, want, bound, seq, seq_adv, seq_cap,
+                                               out_flags)
         rc = lib().ora_get(self._h, consumer, max_samples, C.byref(go))
         if rc != 0:
             raise ValueError("ora_get: bad argument")
@@ -319,14 +323,14 @@ class OracleDock:
 
     def gather(self, consumer: int, indices: np.ndarray, mode: int = PACKED, pad_prompt_to: int = 0,
                pad_response_to: int = 0, want: Optional[Sequence[int]] = None, seq=None,
-               seq_adv: bool = False) -> Batch:
+               seq_adv: bool = False, out_flags: int = 0) -> Batch:
         idx = np.ascontiguousarray(indices, dtype=np.int32)
         k = len(idx)
         bound = [0, 0, 0]
         for cls in (1, 2):
             bound[cls] = int(np.maximum(self.lengths(cls)[idx], 0).sum(dtype=np.int64)) if k else 0
         go, res, bufs, cols, adv = self._alloc(consumer, max(k, 1), mode, pad_prompt_to,
-                                               pad_response_to, None, want, bound, seq, seq_adv)
+                                               pad_response_to, None, want, bound, seq, seq_adv, None, out_flags)
         rc = lib().ora_gather(self._h, consumer, idx.ctypes.data, k, C.byref(go))
         if rc != 0:
             raise ValueError("ora_gather: bad argument")

@@ -75,7 +75,9 @@ def expected_packed(w: wl.Workload, column: int, indices: np.ndarray) -> np.ndar
     return np.concatenate(parts) if parts else np.zeros(0, src.dtype)
 
 
-def expected_padded(w: wl.Workload, column: int, indices: np.ndarray, width: int) -> np.ndarray:
+def expected_padded(w: wl.Workload, column: int, indices: np.ndarray, width: int, left: bool = False) -> np.ndarray:
+    """The dense [len(indices), width] matrix of a ragged column from the generator's arrays: each
+    row's elements at the row's start, or (left) flush with its end, the pad pattern elsewhere."""
     spec = w.columns[column]
     src = w.data[spec.name]
     st = w.row_starts(spec.cls)
@@ -87,7 +89,10 @@ def expected_padded(w: wl.Workload, column: int, indices: np.ndarray, width: int
         out.view(np.uint16)[:] = np.uint16(spec.pad_bits & 0xFFFF)
     for i, s in enumerate(indices):
         row = src[st[s]:st[s + 1]]
-        out[i, :len(row)] = row
+        if left:
+            out[i, width - len(row):] = row
+        else:
+            out[i, :len(row)] = row
     del pad
     return out
 

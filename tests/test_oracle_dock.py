@@ -54,6 +54,46 @@ def test_identity_round_trip_padded():
             assert H.bits_equal(b.columns[c], H.expected_padded(w, c, idx, width)), spec.name
 
 
+def test_identity_round_trip_left_padded_prompts():
+    """Prompt rows flush right in their width (the pad in front), response rows as before:
+    expected values from the generator's arrays; the flag changes nothing else of the batch."""
+    w = small(with_entropy=True)
+    d = H.make_oracle(w)
+    for c in range(len(w.columns)):
+        cu, data = w.pack(c, np.arange(w.n, dtype=np.int32))
+        d.put(c, np.arange(w.n), cu, data)
+    upd = len(w.consumers) - 1
+    b = d.get(upd, w.n, ora.PADDED, 40, 96, out_flags=ora.OUT_LEFT_PAD_PROMPT)
+    idx = np.arange(w.n)
+    assert b.n_samples == w.n and b.status == 0
+    assert np.array_equal(b.cu_prompt, np.concatenate(([0], np.cumsum(w.len_prompt))))
+    for c, spec in enumerate(w.columns):
+        if spec.cls == wl.SCALAR:
+            assert H.bits_equal(b.columns[c], w.data[spec.name])
+        else:
+            width = 40 if spec.cls == wl.PROMPT else 96
+            assert H.bits_equal(b.columns[c], H.expected_padded(w, c, idx, width, left=spec.cls == wl.PROMPT)), spec.name
+    # a packed get ignores the flag; an unknown flag is refused
+    g = d.gather(upd, idx[:8], out_flags=ora.OUT_LEFT_PAD_PROMPT)
+    assert H.bits_equal(g.columns[0], w.pack(0, idx[:8].astype(np.int32))[1])
+    with pytest.raises(ValueError):
+        d.gather(upd, idx[:8], out_flags=2)
+
+
+def test_left_padded_prompts_by_hand():
+    cols = [("i32", "prompt", 0xDEADBEEF), ("bf16", "prompt", 0xABCD), ("f32", "response", 0x7FC00001)]
+    d = ora.OracleDock(1, 3, 1, cols, [(0x7, 0x7, False)], 64, 64, 0)
+    d.put(0, [0, 1, 2], np.array([0, 2, 2, 5], np.int32), np.array([5, 6, 7, 8, 9], np.int32))
+    d.put(1, [0, 1, 2], np.array([0, 2, 2, 5], np.int32), np.array([1, 2, 3, 4, 5], np.uint16))
+    d.put(2, [0, 1, 2], np.array([0, 1, 3, 3], np.int32), np.array([1, 2, 3], np.float32))
+    b = d.get(0, 3, ora.PADDED, 3, 2, out_flags=ora.OUT_LEFT_PAD_PROMPT)
+    P = 0xDEADBEEF
+    assert b.columns[0].view(np.uint32).tolist() == [[P, 5, 6], [P, P, P], [7, 8, 9]]      # widths 2, 0 and 3 of 3
+    assert b.columns[1].tolist() == [[0xABCD, 1, 2], [0xABCD] * 3, [3, 4, 5]]
+    assert b.columns[2].view(np.uint32).tolist() == [[0x3F800000, 0x7FC00001], [0x40000000, 0x40400000],
+                                                     [0x7FC00001, 0x7FC00001]]               # responses: pad behind
+
+
 def test_padded_uses_the_columns_pad_bits():
     cols = [("i32", "prompt", 0xDEADBEEF), ("f32", "response", 0x7FC00001), ("bf16", "response", 0xABCD),
             ("f32", "scalar", 0)]
