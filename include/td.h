@@ -46,6 +46,7 @@ typedef struct td_dock td_dock;          /* opaque host object */
 enum { TD_I32 = 0, TD_F32 = 1, TD_BF16 = 2 };             /* td_column.dtype */
 enum { TD_SCALAR = 0, TD_PROMPT = 1, TD_RESPONSE = 2 };   /* td_column.cls   */
 enum { TD_PACKED = 0, TD_PADDED = 1 };                    /* td_get_out.mode */
+enum { TD_OUT_LEFT_PAD_PROMPT = 1u };                     /* td_get_out.flags */
 enum { TD_F_ADVANTAGE = 1u };                             /* td_consumer.flags */
 
 typedef enum {
@@ -117,7 +118,13 @@ typedef struct {
                                          cu_<class>[i]; TD_PADDED: row i at i * pad_<class>_to,
                                          filled up with the column's pad_bits */
     uint32_t pad_prompt_to, pad_response_to;   /* row widths in elements (TD_PADDED only) */
-    uint32_t reserved;
+    uint32_t flags;                   /* 0, or TD_OUT_LEFT_PAD_PROMPT: in TD_PADDED mode a row of a
+                                         TD_PROMPT column ends at its width, (pad_prompt_to - length)
+                                         copies of pad_bits in front of it, so that in a dense
+                                         [prompt | response] batch every response starts at the same
+                                         position, as batched generation lays its sequences out;
+                                         TD_RESPONSE rows are padded behind as always, TD_PACKED
+                                         ignores the flag.  Any other bit: TD_EINVAL */
     int32_t *indices;                 /* [max_samples] sample indices, ascending          required */
     int32_t *cu_prompt, *cu_response; /* [max_samples + 1] prefix sums of the true lengths required */
     int32_t *cu_seq;                  /* [max_samples + 1] cu_prompt + cu_response, or NULL */

@@ -16,6 +16,7 @@ from . import build as _build
 I32, F32, BF16 = 0, 1, 2
 SCALAR, PROMPT, RESPONSE = 0, 1, 2
 PACKED, PADDED = 0, 1
+OUT_LEFT_PAD_PROMPT = 1            # td_get_out.flags
 F_ADVANTAGE = 1
 OK, EINVAL, EWORKSPACE, ECUDA, ETOOLARGE = 0, -1, -2, -3, -4
 ERR_OOB_INDEX, ERR_DUP_PUT, ERR_LEN_MISMATCH, ERR_ARENA_FULL = 1, 2, 4, 8
@@ -66,7 +67,7 @@ class TdResult(C.Structure):
 
 class TdGetOut(C.Structure):
     _fields_ = [("mode", C.c_int32), ("pad_prompt_to", C.c_uint32), ("pad_response_to", C.c_uint32),
-                ("reserved", C.c_uint32),
+                ("flags", C.c_uint32),
                 ("indices", C.c_void_p), ("cu_prompt", C.c_void_p), ("cu_response", C.c_void_p),
                 ("cu_seq", C.c_void_p), ("col", C.c_void_p * 32),
                 ("col_capacity_elems", C.c_uint64 * 32), ("advantages", C.c_void_p),
@@ -248,9 +249,10 @@ class GetBuffers:
                  capacities: Optional[Dict[int, int]] = None, want: Optional[Sequence[int]] = None,
                  prompt_tokens_cap: Optional[int] = None, response_tokens_cap: Optional[int] = None,
                  seq: Optional[Tuple[int, int]] = None, seq_adv: bool = False, seq_cap: Optional[int] = None,
-                 host_payload: bool = False):
+                 host_payload: bool = False, left_pad_prompts: bool = False):
         """seq = (prompt column, response column) adds the fused token stream, seq_adv its
         advantage twin; seq_cap is the room behind each (default: both token caps together).
+        left_pad_prompts (PADDED mode): prompt rows end at their width, the pad in front.
         host_payload: the column buffers (and the stream) are pinned host memory that the device
         writes directly; indices, cu_seqlens, advantages and the result block stay on the device."""
         import torch
@@ -264,6 +266,7 @@ class GetBuffers:
 
         self.dock, self.consumer, self.max_samples, self.mode = dock, consumer, max_samples, mode
         self.pad_prompt_to, self.pad_response_to = pad_prompt_to, pad_response_to
+        self.flags = OUT_LEFT_PAD_PROMPT if left_pad_prompts else 0
         i32 = torch.int32
         self.indices = torch.zeros(max_samples, dtype=i32, device=dev)
         self.cu_prompt = torch.zeros(max_samples + 1, dtype=i32, device=dev)
@@ -294,6 +297,7 @@ class GetBuffers:
             self.cols[c] = payload(max(cap, 1), tdt[dt])
         go = TdGetOut()
         go.mode, go.pad_prompt_to, go.pad_response_to = mode, pad_prompt_to, pad_response_to
+        go.flags = self.flags
         go.indices, go.cu_prompt = self.indices.data_ptr(), self.cu_prompt.data_ptr()
         go.cu_response, go.cu_seq = self.cu_response.data_ptr(), self.cu_seq.data_ptr()
         for c, t in self.cols.items():
@@ -341,6 +345,7 @@ class HostGetBuffers:
         self.result = TdResult.from_address(self._result_mem.data_ptr())
         go = TdGetOut()
         go.mode, go.pad_prompt_to, go.pad_response_to = bufs.mode, bufs.pad_prompt_to, bufs.pad_response_to
+        go.flags = getattr(bufs, "flags", 0)
         go.indices, go.cu_prompt = self.indices.data_ptr(), self.cu_prompt.data_ptr()
         go.cu_response, go.cu_seq = self.cu_response.data_ptr(), self.cu_seq.data_ptr()
         for c, t in self.cols.items():

@@ -509,6 +509,7 @@ int check_get_out(const DockView &v, uint32_t consumer, uint32_t max_samples, co
     if (max_samples / v.N == 0) return TD_EINVAL;
     if (!out->indices || !out->cu_prompt || !out->cu_response || !out->result) return TD_EINVAL;
     if (out->mode != TD_PACKED && out->mode != TD_PADDED) return TD_EINVAL;
+    if (out->flags & ~(uint32_t)TD_OUT_LEFT_PAD_PROMPT) return TD_EINVAL;
     if ((v.cflags[consumer] & TD_F_ADVANTAGE) && !out->advantages) return TD_EINVAL;
     if (wants_stream(*out) && !out->cu_seq) return TD_EINVAL;
     if (out->seq) {

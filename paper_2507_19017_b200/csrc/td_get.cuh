@@ -799,10 +799,12 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
                                              [&](uint32_t i, int64_t, int64_t, int32_t &) -> uint8_t * { return row_src(i); },
                                              seq_cu, seq_tail);
             } else {
-                // fixed-width rows: payload part, then the pad pattern up to the row's end
+                // fixed-width rows: payload part, then the pad pattern up to the row's end; a
+                // prompt row asked for left-padded has the pad pattern first and ends at its width
                 const uint32_t W = cls == TD_PROMPT ? out.pad_prompt_to : out.pad_response_to;
                 const uint64_t row_bytes = (uint64_t)W * esz;
                 const uint64_t b1 = min(b1_raw, (uint64_t)n_s * row_bytes);
+                const bool left = cls == TD_PROMPT && (out.flags & TD_OUT_LEFT_PAD_PROMPT);
                 const int32_t *lent = dv.len[cls];
                 for (uint64_t r0 = b0 / row_bytes; r0 < n_s && r0 * row_bytes < b1; r0 += 32) {
                     const uint64_t i = r0 + lane;
@@ -816,14 +818,21 @@ get_gather_kernel(const DockView dv, const __grid_constant__ GetInline one,
                     for (uint32_t r = 0; r < 32; ++r) {
                         const uint64_t rlo = (r0 + r) * row_bytes;
                         if (r0 + r >= n_s || rlo >= b1) break;
-                        const uint64_t valid_hi = rlo + shfl_u64(valid, r);
+                        // the row's payload lies at [v0, v1) of the job, this warp's part of the row is [lo, hi)
+                        const uint64_t v_bytes = shfl_u64(valid, r);
+                        const uint64_t v0 = left ? rlo + row_bytes - v_bytes : rlo, v1 = v0 + v_bytes;
                         uint8_t *o = reinterpret_cast<uint8_t *>(shfl_u64(reinterpret_cast<uint64_t>(src), r));
                         const uint64_t lo = max(rlo, b0), hi = min(rlo + row_bytes, b1);
-                        const uint64_t phi = min(hi, valid_hi);
-                        if (phi > lo && o)
-                            pipe.push<false>(dst0 + lo, o + (lo - rlo), (uint32_t)(phi - lo), lane, src_lo, src_hi);
-                        const uint64_t plo = max(lo, valid_hi);
-                        if (hi > plo) warp_fill(dst0 + plo, hi - plo, dv.col_pad[k], esz, lane);
+                        const uint64_t p0 = max(lo, v0), p1 = min(hi, v1);
+                        if (p1 > p0 && o)
+                            pipe.push<false>(dst0 + p0, o + (p0 - v0), (uint32_t)(p1 - p0), lane, src_lo, src_hi);
+                        if (left) {
+                            const uint64_t fhi = min(hi, v0);
+                            if (fhi > lo) warp_fill(dst0 + lo, fhi - lo, dv.col_pad[k], esz, lane);
+                        } else {
+                            const uint64_t flo = max(lo, v1);
+                            if (hi > flo) warp_fill(dst0 + flo, hi - flo, dv.col_pad[k], esz, lane);
+                        }
                     }
                 }
             }

@@ -63,20 +63,22 @@ class GpuDock:
 
     def buffers(self, consumer: int, max_samples: int, mode: int = td.PACKED, pad_p: int = 0,
                 pad_r: int = 0, capacities=None, want=None, key=None, seq=None, seq_adv=False,
-                seq_cap=None) -> td.GetBuffers:
+                seq_cap=None, left_pad=False) -> td.GetBuffers:
         k = (consumer, max_samples, mode, pad_p, pad_r, key,
              tuple(sorted(capacities.items())) if capacities else None, tuple(want) if want else None,
-             seq, seq_adv, seq_cap)
+             seq, seq_adv, seq_cap, left_pad)
         if k not in self._bufs:
             pc, rc = self.token_caps(max_samples)
             self._bufs[k] = td.GetBuffers(self.dock, consumer, max_samples, mode, pad_p, pad_r,
-                                          capacities, want, pc, rc, seq, seq_adv, seq_cap)
+                                          capacities, want, pc, rc, seq, seq_adv, seq_cap,
+                                          left_pad_prompts=left_pad)
         return self._bufs[k]
 
     def get(self, consumer: int, max_samples: int, mode: int = td.PACKED, pad_p: int = 0, pad_r: int = 0,
             capacities=None, want=None, stream=None, key=None, seq=None, seq_adv=False,
-            seq_cap=None) -> ora.Batch:
-        bufs = self.buffers(consumer, max_samples, mode, pad_p, pad_r, capacities, want, key, seq, seq_adv, seq_cap)
+            seq_cap=None, left_pad=False) -> ora.Batch:
+        bufs = self.buffers(consumer, max_samples, mode, pad_p, pad_r, capacities, want, key, seq, seq_adv, seq_cap,
+                            left_pad)
         self.dock.get(bufs, stream)
         return self.read(bufs, stream)
 

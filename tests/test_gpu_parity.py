@@ -1,6 +1,8 @@
 """Parity of the CUDA library with the CPU oracle on the same seeded inputs, through the C ABI.
 Indices, offsets, bitmaps, cu_seqlens and payload are compared bit for bit; the fp32 advantages
 within 1e-6 relative / 1e-7 absolute (both sides accumulate in double)."""
+import dataclasses
+
 import numpy as np
 import pytest
 
@@ -441,6 +443,72 @@ def test_fused_stream_in_a_plan(G):
 @pytest.mark.parametrize("cid", [2, 3])
 def test_fused_stream_full_size(G, cid):
     _many_vs_serial(G, wl.make_config(cid), fused=True)
+
+
+# ------------------------------------------------------------------- left-padded prompts
+def _put_everything(w, o, g):
+    idx = np.arange(w.n, dtype=np.int32)
+    for c in range(len(w.columns)):
+        cu, data = w.pack(c, idx)
+        o.put(c, idx, cu, data); g.put(c, idx, cu, data)
+
+
+def test_left_padded_prompts_every_alignment(G):
+    """TD_OUT_LEFT_PAD_PROMPT: prompt rows flush with the end of their width.  Lengths 0..37 (rows
+    of no length and rows that fill the width included) at widths whose rows start on every
+    4-byte phase, drained in small gets, in one get of everything and through a plan; the fused
+    stream beside it is unchanged by the flag."""
+    w = wl.make_custom("lpad", 64, 2, 4, prompt_len=(0, 37), response=("uniform", 0, 70), vocab=1 << 20,
+                       micro_batch=6, seed=13, with_entropy=True, schedule="none")
+    # a 2-byte prompt column beside the ids, and pad patterns that are not zero
+    pads = {"prompt_ids": 0xDEADBEEF, "response_ids": 0x7FC00001, "entropy": 0xABCD}
+    w.columns = [dataclasses.replace(c, pad_bits=pads.get(c.name, 0)) for c in w.columns]
+    w.columns.append(wl.ColumnSpec("prompt_weight", "bf16", wl.PROMPT, 0x3F80))
+    w.data["prompt_weight"] = np.random.Generator(np.random.PCG64(5)).integers(
+        0, 1 << 16, size=int(w.len_prompt.sum()), dtype=np.uint16)
+    w.consumers = wl.standard_consumers(w.columns)
+    upd = len(w.consumers) - 1
+    for widths in ((37, 70), (38, 71), (39, 73), (40, 72)):
+        o, g = H.make_oracle(w), G.GpuDock(w)
+        _put_everything(w, o, g)
+        kw = G.stream_args(w, upd)
+        for j in range(w.n // 6 + 1):
+            for cons, extra in ((0, {}), (upd, kw)):
+                want = o.get(cons, 6, ora.PADDED, *widths, out_flags=ora.OUT_LEFT_PAD_PROMPT, **extra)
+                got = g.get(cons, 6, td.PADDED, *widths, left_pad=True, **extra)
+                G.assert_batch_equal(got, want, f"widths {widths} get {j} consumer {cons}")
+        # everything at once for another consumer, and two more consumers through one plan
+        G.assert_batch_equal(g.get(1, w.n, td.PADDED, *widths, left_pad=True),
+                             o.get(1, w.n, ora.PADDED, *widths, out_flags=ora.OUT_LEFT_PAD_PROMPT), "whole batch")
+        bufs = [g.buffers(2, 20, td.PADDED, *widths, key=f"plan{q}", left_pad=True) for q in range(3)]
+        g.dock.get_many(g.dock.plan(bufs))
+        for q in range(3):
+            G.assert_batch_equal(g.read(bufs[q]), o.get(2, 20, ora.PADDED, *widths, out_flags=ora.OUT_LEFT_PAD_PROMPT),
+                                 f"plan request {q}")
+        G.assert_state_equal(g, o, ctx=f"left-padded, widths {widths}")
+    # rows right-padded when the flag is absent, on the same buffers' shapes; unknown flags refused
+    G.assert_batch_equal(g.get(2, 20, td.PADDED, 40, 72), o.get(2, 20, ora.PADDED, 40, 72), "flag absent")
+    bad = g.buffers(2, 20, td.PADDED, 40, 72, key="bad flags")
+    bad.struct.flags = 2
+    with pytest.raises(td.TdError):
+        g.dock.get(bad)
+
+
+def test_left_padded_prompts_long_rows(G):
+    """Rows of many pipeline stages, widths far beyond the longest row, chunk borders inside pad
+    and payload alike: the 7B-shaped dock's prompts and responses, 64-sample gets."""
+    w = wl.make_config(2, schedule="none")
+    o, g = H.make_oracle(w), G.GpuDock(w)
+    _put_everything(w, o, g)
+    upd = len(w.consumers) - 1
+    for j in range(3):
+        for cons in (0, upd):
+            want = o.get(cons, 64, ora.PADDED, w.pad_prompt_to + 3, w.pad_response_to, out_flags=ora.OUT_LEFT_PAD_PROMPT)
+            got = g.get(cons, 64, td.PADDED, w.pad_prompt_to + 3, w.pad_response_to, left_pad=True)
+            G.assert_batch_equal(got, want, f"get {j} consumer {cons}")
+            # independent of the oracle: a prompt row ends with its tokens, the pad fills the front
+            c0 = w.column_index("prompt_ids")
+            assert H.bits_equal(got.columns[c0], H.expected_padded(w, c0, got.indices, w.pad_prompt_to + 3, left=True))
 
 
 def test_fused_stream_of_a_float_pair_and_truncation(G):
