@@ -390,8 +390,13 @@ class GpuStep:
         return t.pin_memory()
 
     def flush_l2(self):
+        """Ahead of a timed phase: the 256 MiB write that empties L2, or (warm variant) a spin of
+        about 100 us that touches no memory.  Either keeps the device busy while the host
+        enqueues the phase's launches, so that the events time the device, not the host."""
         if not self.warm_l2:
             self.flush_buf.zero_()
+        else:
+            self.torch.cuda._sleep(200_000)
 
     def close(self):
         """Gives the device memory back (the next shape of the run needs it)."""
