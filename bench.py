@@ -12,7 +12,7 @@ for the 7B-, 32B- and MoE-shaped batches (the MoE shape twice: bulk, and as the 
 configuration describes, a producer stream against four polling consumer streams).
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--sigma S] [--warm-l2]
-                  [--scenario dispatch|concurrent|cascade|scan] [--impl reference]
+                  [--scenario dispatch|concurrent|cascade|scan|fixed-cost] [--impl reference]
 """
 from __future__ import annotations
 
@@ -95,7 +95,7 @@ def parse_args():
     ap.add_argument("--graph", action="store_true",
                     help="cascade only: capture the step's calls into one CUDA graph once and time its replay "
                          "(nothing in the step needs the host, batch sizes are read on the device)")
-    ap.add_argument("--scenario", default="dispatch", choices=["dispatch", "concurrent", "cascade", "scan"],
+    ap.add_argument("--scenario", default="dispatch", choices=["dispatch", "concurrent", "cascade", "scan", "fixed-cost"],
                     help="dispatch: put everything, then drain (the headline); concurrent: one producer stream "
                          "putting shuffled chunks of 1-64 samples while four consumer threads poll td_get on "
                          "their own streams (the out-of-order stress); cascade: generation puts in "
@@ -626,6 +626,53 @@ class CascadeStep:
     def written_back(self):
         st = self.dock.status()
         return {self.w.columns[c].name: int(st.put_accepted[c]) for c in self.w.pool}
+
+
+def run_fixed_cost(args, local_rank):
+    """What a put phase and a drain cost before any byte moves: the 7B-shaped dock (2048 samples,
+    128 requests of 64) with every row length divided by 64, 16, 4, 2 and 1, and the same rows
+    in docks of 64 to 8192 samples.  Prints one JSON line with the times and, for the first
+    series, the straight line time = fixed + bytes / rate fitted through them."""
+    import torch
+    from paper_2507_19017_b200 import workloads as wl
+    peak, peak_kind = load_peaks()
+    reps = max(2 * args.steps, 20)
+
+    def timed(w):
+        step = GpuStep(w, local_rank)
+        for _ in range(5):
+            step.timed_step()
+        t = [step.timed_step() for _ in range(reps)]
+        sb = step_bytes(w)
+        put_b, drain_b = sb["put"], sb["get_hbm"]
+        step.close()
+        return statistics.mean(x[0] for x in t) * 1e3, statistics.mean(x[1] for x in t) * 1e3, put_b, drain_b
+
+    by_length = []
+    for scale in (64, 16, 4, 2, 1):
+        w = wl.make_custom(f"7b-shaped-rows-1/{scale}", 256, 8, 4, prompt_len=(max(128 // scale, 1), max(1024 // scale, 2)),
+                           response=("lognormal", 1500.0 / scale, wl.SIGMA_HEADLINE, max(4096 // scale, 4)),
+                           vocab=152064, micro_batch=64, seed=wl.BASE_SEED, schedule="bulk", config_id=2)
+        put_us, drain_us, put_b, drain_b = timed(w)
+        by_length.append({"row_length_scale": f"1/{scale}", "put_us": put_us, "drain_us": drain_us,
+                          "put_hbm_bytes": put_b, "drain_hbm_bytes": drain_b})
+    fit = {}
+    for ph in ("put", "drain"):
+        x = np.array([r[f"{ph}_hbm_bytes"] for r in by_length], dtype=np.float64)
+        y = np.array([r[f"{ph}_us"] for r in by_length], dtype=np.float64)
+        slope, fixed = np.polyfit(x, y, 1)
+        fit[ph] = {"fixed_us": float(fixed), "GBps_of_the_rest": float(1e-3 / slope) if slope > 0 else None,
+                   "frac_of_measured_copy": float(1e-3 / slope / peak) if slope > 0 else None}
+    by_samples = []
+    for G, mb in ((8, 64), (32, 64), (128, 64), (256, 64), (1024, 64)):
+        w = wl.make_custom(f"short-rows-{G * 8}", G, 8, 4, prompt_len=(2, 16), response=("lognormal", 24.0, wl.SIGMA_HEADLINE, 64),
+                           vocab=152064, micro_batch=mb, seed=wl.BASE_SEED, schedule="bulk", config_id=2)
+        put_us, drain_us, _pb, _db = timed(w)
+        by_samples.append({"samples": w.n, "requests": 4 * (w.n // mb), "put_us": put_us, "drain_us": drain_us})
+    print(json.dumps({"scenario": "fixed-cost", "api": "td_put_many + td_get_many (3 + 3 launches per step)",
+                      "l2": "flushed before each phase (256 MiB write)", "timed_steps_per_point": reps,
+                      "by_row_length": by_length, "fit_time_us_equals_fixed_plus_bytes_over_rate": fit,
+                      "by_samples_with_rows_of_a_few_tokens": by_samples, "peak_GBps": peak, "peak_kind": peak_kind}))
 
 
 def run_scan(args, local_rank):
@@ -1190,6 +1237,10 @@ def main():
     if args.scenario == "scan":
         if rank == 0:
             run_scan(args, local_rank)
+        return finish()
+    if args.scenario == "fixed-cost":
+        if rank == 0:
+            run_fixed_cost(args, local_rank)
         return finish()
     if args.scenario == "cascade":
         from paper_2507_19017_b200 import workloads as wl
