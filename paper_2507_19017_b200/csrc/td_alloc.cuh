@@ -70,19 +70,28 @@ __device__ __noinline__ void warp_shard_prefix(bool alloc, uint32_t sh, uint32_t
     const uint32_t first = (uint32_t)__ffs(mask) - 1u;
     // usual case: every allocating lane of the warp is in one shard -> one shuffle scan
     const uint32_t first_sh = __shfl_sync(kFullMask, sh, first);      // every lane takes part
-    const uint32_t key = alloc ? sh : first_sh;
-    int same;
-    __match_all_sync(kFullMask, key, &same);
-    if (same) {
-        unsigned long long inc = alloc ? room : 0u;
+    if (__ballot_sync(kFullMask, alloc && sh != first_sh) == 0) {
+        const uint32_t mine = alloc ? room : 0u;
+        leader = alloc && lane == first;
+        if (__ballot_sync(kFullMask, mine >> 26) == 0) {              // rows of the usual sizes: the warp's sum fits 32 bits
+            uint32_t inc = mine;
+            #pragma unroll
+            for (int d = 1; d < 32; d <<= 1) {
+                const uint32_t t = __shfl_up_sync(kFullMask, inc, d);
+                if ((int)lane >= d) inc += t;
+            }
+            wsum = __shfl_sync(kFullMask, inc, 31);
+            pre = inc - mine;
+            return;
+        }
+        unsigned long long inc = mine;
         #pragma unroll 1
         for (int d = 1; d < 32; d <<= 1) {
             const unsigned long long t = shfl_up_u64(inc, d);
             if ((int)lane >= d) inc += t;
         }
         wsum = shfl_u64(inc, 31);
-        pre = inc - (alloc ? room : 0u);
-        leader = alloc && lane == first;
+        pre = inc - mine;
         return;
     }
     const uint32_t k2 = alloc ? sh : kNotAllocating;
@@ -237,41 +246,54 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
         #pragma unroll 1
         for (uint32_t base = 0; base < k; base += kAllocPass) {
             // 1. validate, CAS.  A short pass is spread over all warps: each takes `per` rows of 32.
+            //    A thread's entries go through the step side by side - their own words first,
+            //    then every status word and CAS, then the verdicts - so that the dependent
+            //    accesses of one entry do not wait for those of the one before.
             const uint32_t per = min((uint32_t)kAllocPer, (k - base + kAllocThreads - 1u) / kAllocThreads);
             int32_t s[kAllocPer];
-            uint32_t room[kAllocPer], sh[kAllocPer];
-            bool alloc[kAllocPer];
+            int64_t c0[kAllocPer], c1[kAllocPer];
+            uint32_t room[kAllocPer], sh[kAllocPer], st[kAllocPer];
+            int32_t old[kAllocPer];
+            bool alloc[kAllocPer], have[kAllocPer], bad[kAllocPer];
             bool any = false;
             #pragma unroll
             for (int j = 0; j < kAllocPer; ++j) {
                 // a warp owns 32 * per consecutive entries of the pass, in the order (j, lane)
+                const uint32_t i = base + warp * (32u * per) + (uint32_t)j * 32u + lane;
+                have[j] = (uint32_t)j < per && i < k;
+                s[j] = -1; c0[j] = 0; c1[j] = 0;
+                if (have[j]) { s[j] = a.idx[i]; c0[j] = a.cu[i]; c1[j] = a.cu[i + 1]; }
+            }
+            #pragma unroll
+            for (int j = 0; j < kAllocPer; ++j) {
+                st[j] = 0; old[j] = 0; bad[j] = false;
+                if (!have[j]) continue;
+                bad[j] = c1[j] < c0[j] || c0[j] < 0 || (uint64_t)c1[j] > a.data_elems;
+                irregular |= bad[j];
+                if (s[j] < 0 || (uint32_t)s[j] >= dv.n) continue;
+                // The status word and the CAS travel side by side.  A column that is already
+                // stored has its class's length set, so the CAS of a repeated put changes
+                // nothing; it is then counted as a repeat, whatever its length says.
+                st[j] = dv.status[s[j]];
+                if (!bad[j]) old[j] = atomicCAS(&dv.len[L][s[j]], -1, (int32_t)(c1[j] - c0[j]));
+            }
+            #pragma unroll
+            for (int j = 0; j < kAllocPer; ++j) {
                 const uint32_t eo = warp * (32u * per) + (uint32_t)j * 32u + lane;
-                const uint32_t i = base + eo;
-                alloc[j] = false; s[j] = -1; room[j] = 0; sh[j] = 0;
+                alloc[j] = false; room[j] = 0; sh[j] = 0;
                 if ((uint32_t)j >= per) continue;
                 uint32_t fok = 0;
-                if (i < k) {
-                    s[j] = a.idx[i];
-                    const int64_t c0 = a.cu[i], c1 = a.cu[i + 1];
-                    const int64_t l = c1 - c0;
-                    const bool bad = l < 0 || c0 < 0 || (uint64_t)c1 > a.data_elems;
-                    irregular |= bad;
+                if (have[j]) {
+                    const int64_t l = c1[j] - c0[j];
                     if (s[j] < 0 || (uint32_t)s[j] >= dv.n) { ++n_oob; n_oob += __popc(followers); }
                     else {
-                        // The status word and the CAS travel side by side.  A column that is
-                        // already stored has its class's length set, so the CAS of a repeated
-                        // put changes nothing; it is then counted as a repeat, whatever its
-                        // length says.
-                        const uint32_t st = dv.status[s[j]];
-                        int32_t old = 0;
-                        if (!bad) old = atomicCAS(&dv.len[L][s[j]], -1, (int32_t)l);
-                        if (st & bit) { ++n_dup; }
-                        else if (bad) { ++n_bad; }
-                        else if (old == -1) {
+                        if (st[j] & bit) { ++n_dup; }
+                        else if (bad[j]) { ++n_bad; }
+                        else if (old[j] == -1) {
                             alloc[j] = true;
                             room[j] = (uint32_t)align_row((uint64_t)l);
                             sh[j] = shard_of(dv, (uint32_t)s[j]);
-                        } else if (old != (int32_t)l) { ++n_mis; }
+                        } else if (old[j] != (int32_t)l) { ++n_mis; }
                         // Followers: same sample, same row.  Their bound on the data is not
                         // wider than the leader's, so where one of them is in order the leader
                         // has done its CAS and the length in force is known.
@@ -279,9 +301,9 @@ put_alloc_kernel(const DockView dv, const PutBatch batch) {
                         for (uint32_t fm = followers; fm; fm &= fm - 1u) {
                             const uint32_t f = (uint32_t)__ffs(fm) - 1u;
                             const PutArgs &b = batch.item[f];
-                            if (st & (1u << b.column)) ++n_dup;
-                            else if (l < 0 || c0 < 0 || (uint64_t)c1 > b.data_elems) { ++n_bad; irregular = true; }
-                            else if ((old == -1 ? (int32_t)l : old) != (int32_t)l) ++n_mis;
+                            if (st[j] & (1u << b.column)) ++n_dup;
+                            else if (l < 0 || c0[j] < 0 || (uint64_t)c1[j] > b.data_elems) { ++n_bad; irregular = true; }
+                            else if ((old[j] == -1 ? (int32_t)l : old[j]) != (int32_t)l) ++n_mis;
                             else fok |= 1u << f;
                         }
                     }
