@@ -472,6 +472,24 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
         asm volatile("prefetch.global.L1 [%0];" ::"l"(r));
         if (N > 32u) asm volatile("prefetch.global.L1 [%0];" ::"l"(r + N - 1));
     }
+    // A request of at most 32 groups has its groups' statistics worked out now, by the lanes of the
+    // block's last warp, one group each, while the first warps are at the cu scans: the reward
+    // loads and the double-precision sums then wait side by side with the length loads instead
+    // of behind them.  (Groups that the fit test below cuts off were looked at in vain.)
+    const bool adv_wanted = (dv.cflags[c] & TD_F_ADVANTAGE) && out.advantages;
+    const bool adv_early = adv_wanted && n_grp <= 32u;
+    __shared__ double s_mean[32], s_den[32];
+    if (adv_early && tid >= (uint32_t)kThreads - 32u && tid - ((uint32_t)kThreads - 32u) < n_grp) {
+        const uint32_t p = tid - ((uint32_t)kThreads - 32u);
+        const float *r = reinterpret_cast<const float *>(dv.colbase[dv.reward_col]) + (size_t)s_grp[p] * N;
+        double sum = 0.0;
+        for (uint32_t j = 0; j < N; ++j) sum += (double)r[j];
+        const double mean = sum / (double)N;
+        double ss = 0.0;
+        for (uint32_t j = 0; j < N; ++j) { const double d = (double)r[j] - mean; ss += d * d; }
+        s_mean[p] = mean;
+        s_den[p] = sqrt(ss / (double)N) + dv.eps;
+    }
     const FastDiv div_N = make_fastdiv_dev(N);
     // sample at position i of the batch
     auto sample_at = [&](uint32_t i) -> int32_t {
@@ -542,8 +560,17 @@ get_finalize_kernel(const DockView dv, const __grid_constant__ GetInline one,
         const uint32_t s = (uint32_t)sample_at(i);
         atomicOr(&consumed[s >> 5], 1u << (s & 31));
     }
-    // group-normalised advantage, one thread per group, in double
-    if ((dv.cflags[c] & TD_F_ADVANTAGE) && out.advantages) {
+    // group-normalised advantage in double: one thread per sample from the statistics taken
+    // above, or (a large request) one thread per group
+    if (adv_early) {
+        const float *rew = reinterpret_cast<const float *>(dv.colbase[dv.reward_col]);
+        for (uint32_t i = tid; i < n_s; i += kThreads) {
+            const uint32_t p = fast_div(i, div_N);
+            const float adv = (float)(((double)rew[sample_at(i)] - s_mean[p]) / s_den[p]);
+            out.advantages[i] = adv;
+            if (mirror) mv.advantages[i] = adv;
+        }
+    } else if (adv_wanted) {
         const float *rew = reinterpret_cast<const float *>(dv.colbase[dv.reward_col]);
         for (uint32_t p = tid; p < n_grp; p += kThreads) {
             const float *r = rew + (p < kFinGroupsKept ? s_grp[p] * (int32_t)N : out.indices[(size_t)p * N]);   // a group's samples are consecutive
