@@ -40,15 +40,15 @@ NOMINAL_HBM_GBPS = 8000.0             # the "~8 TB/s" the 70 % target is stated 
 # the ncu summaries under profiles/: (config, kernel) -> (bytes, file, what was captured).
 # A pair without a capture of the current kernels reports null.
 NCU_TRAFFIC = {
-    (2, "get_gather"): (79_659_264, "profiles/copy_kernels_config2_7b_shaped.md", "ncu capture of this kernel on this shape"),
-    (2, "put_scatter"): (44_827_136, "profiles/copy_kernels_config2_7b_shaped.md", "ncu capture of this kernel on this shape"),
-    (3, "get_gather"): (1_147_407_360, "profiles/copy_kernels_config3_32b_shaped.md", "ncu capture of this kernel on this shape"),
-    (3, "put_scatter"): (732_837_632, "profiles/copy_kernels_config3_32b_shaped.md", "ncu capture of this kernel on this shape"),
+    (2, "get_gather"): (80_016_128, "profiles/copy_kernels_config2_7b_shaped.md", "ncu capture of this kernel on this shape"),
+    (2, "put_scatter"): (45_304_064, "profiles/copy_kernels_config2_7b_shaped.md", "ncu capture of this kernel on this shape"),
+    (3, "get_gather"): (1_147_490_816, "profiles/copy_kernels_config3_32b_shaped.md", "ncu capture of this kernel on this shape"),
+    (3, "put_scatter"): (733_361_920, "profiles/copy_kernels_config3_32b_shaped.md", "ncu capture of this kernel on this shape"),
 }
 # The larger shapes hold too much on the device for a full counter capture; their traffic is taken
 # to grow with the bytes that must cross HBM, from the capture of the 32B-shaped batch:
 # kernel -> (captured traffic, HBM-crossing bytes of that launch).
-NCU_SCALE_FROM_CONFIG3 = {"get_gather": (1_147_407_360, 1_200_614_776), "put_scatter": (732_837_632, 784_775_700)}
+NCU_SCALE_FROM_CONFIG3 = {"get_gather": (1_147_490_816, 1_200_614_776), "put_scatter": (733_361_920, 784_775_700)}
 
 
 def captured_traffic(cid: int, kernel: str, bytes_per_launch: float):
