@@ -77,6 +77,10 @@ def parse_args():
     ap.add_argument("--e2e-path", default="auto", choices=["auto", "in-place", "copy"],
                     help="end-to-end step: where the gets leave their payload (in-place: pinned host buffers written "
                          "by the gather kernel; copy: device buffers, one transfer per column and request; auto: by size)")
+    ap.add_argument("--e2e-schedule", default="pipelined", choices=["pipelined", "serial"],
+                    help="end-to-end step with the batched calls: serial = one put of every column, then one "
+                         "drain; pipelined = the columns every worker state needs first, the gets of the states "
+                         "that need nothing else on a second stream while the other columns are still coming in")
     ap.add_argument("--api", default="many", choices=["many", "single"],
                     help="many: one td_put_many and one td_get_many per step; single: one td_put per "
                          "column and one td_get per micro-batch")
@@ -323,6 +327,8 @@ class GpuStep:
         self.api = api
         self.warm_l2 = warm_l2
         self.e2e_path = "auto"
+        self.e2e_schedule = "pipelined"
+        self.e2e_waves = None
         from paper_2507_19017_b200 import binding as td
         from paper_2507_19017_b200 import workloads as wl
         self.torch, self.td, self.w = torch, td, w
@@ -468,6 +474,33 @@ class GpuStep:
             self.e2e_plan = self.dock.plan(self.e2e_gets) if self.e2e_in_place else self.plan
             self.host_gets = [td.HostGetBuffers(b) for b in self.e2e_gets]
             self.meta_stage = torch.empty(self.dock.get_many_host_stage_bytes(self.e2e_plan), dtype=torch.uint8, device=self.dev)
+            # Pipelined schedule: the columns that every worker state needs go first; the states
+            # that need nothing else are served on a second stream as soon as those are stored,
+            # while the remaining columns are still crossing the bus in the other direction.
+            need = [set(w.column_index(nm) for nm in k.need) for k in w.consumers]
+            first_cols = set.intersection(*need)
+            early = {c for c, nd in enumerate(need) if nd <= first_cols}
+            self.e2e_waves = None
+            if self.e2e_schedule == "pipelined" and early and len(early) < len(need) and first_cols:
+                waves = []
+                for cols, cons in ((first_cols, early), (None, set(range(len(need))) - early)):
+                    puts = [p for p in self.host_puts if (p[0] in first_cols) == (cols is not None)]
+                    gets = [b for b in self.e2e_gets if b.consumer in cons]
+                    hosts = [h for b, h in zip(self.e2e_gets, self.host_gets) if b.consumer in cons]
+                    plan = self.dock.plan(gets)
+                    waves.append({
+                        "put_arr": self.dock.put_items(puts),
+                        "stage": torch.empty(sum(self.dock.put_host_stage_bytes(c, i.numel(), d.numel()) for c, i, _cu, d in puts),
+                                             dtype=torch.uint8, device=self.dev),
+                        "plan": plan, "out_arr": self.dock.host_outs(hosts),
+                        "meta": torch.empty(self.dock.get_many_host_stage_bytes(plan), dtype=torch.uint8, device=self.dev),
+                        "h2d": sum(d.numel() * d.element_size() for _c, _i, _cu, d in puts)
+                               + sum(t.numel() * 4 for t in {id(x): x for _c, i, cu, _d in puts for x in (i, cu) if x is not None}.values()),
+                        "h2d_copies": len(puts) + len({x.data_ptr() for _c, i, cu, _d in puts for x in (i, cu) if x is not None}),
+                        "d2h_copies": sum(len(b.cols) for b in gets)})
+                self.e2e_waves = waves
+                self.e2e_stream = torch.cuda.Stream(device=self.dev)
+                self.e2e_event = torch.cuda.Event()
         else:
             self.stage = [torch.empty(max(needs), dtype=torch.uint8, device=self.dev) for _ in range(2)]
             self.host_gets = [td.HostGetBuffers(b) for b in self.gets]
@@ -477,6 +510,15 @@ class GpuStep:
     def e2e_step(self):
         torch = self.torch
         self.dock.reset()
+        if self.api == "many" and self.e2e_waves:
+            a, b = self.e2e_waves
+            self.dock.put_many_host(a["put_arr"], a["stage"])
+            self.e2e_event.record()
+            self.dock.put_many_host(b["put_arr"], b["stage"])                  # on its way while the first states are served
+            self.e2e_stream.wait_event(self.e2e_event)
+            self.dock.get_many_host(a["plan"], a["out_arr"], a["meta"], stream=self.e2e_stream)
+            self.dock.get_many_host(b["plan"], b["out_arr"], b["meta"])
+            return None
         if self.api == "many":          # one call in, one call out: two synchronisations per step
             self.dock.put_many_host(self.host_put_arr, self.stage[0])
             self.dock.get_many_host(self.e2e_plan, self.host_out_arr, self.meta_stage)
@@ -506,7 +548,21 @@ class GpuStep:
         served = sum(h.result.n_samples for h in self.host_gets)
         assert served == self.w.n * len(self.w.consumers), f"end-to-end drain served {served} samples"
         d2h = sum(h.bytes_valid(self.dock) for h in self.host_gets)      # counted from what the last step brought over
-        if self.api == "many":
+        if self.api == "many" and self.e2e_waves:
+            self.e2e_h2d_bytes = sum(wv["h2d"] for wv in self.e2e_waves)
+            copies = {"h2d_copies_per_step": sum(wv["h2d_copies"] for wv in self.e2e_waves),
+                      "d2h_copies_per_step": 2 if self.e2e_in_place else 2 + sum(wv["d2h_copies"] for wv in self.e2e_waves),
+                      "d2h_path": ("payload written into pinned host buffers by the gather kernel" if self.e2e_in_place else
+                                   "one transfer per served column and request from device buffers") +
+                                  "; one more transfer per wave for all its result blocks, indices, cu_seqlens and advantages",
+                      "schedule": "two waves: td_put_many_host of the columns every worker state needs, then of the "
+                                  "rest, on one stream; td_get_many_host for the states that need only the first "
+                                  "columns on a second stream behind the first put (its transfers to the host run "
+                                  "while the second put's come in), then td_get_many_host for the other states"}
+            for wv in self.e2e_waves:
+                wv["plan"].close()
+            self.e2e_waves = None
+        elif self.api == "many":
             shared = len({h.data_ptr() for _c, h, _cu, _d in self.host_puts}) + \
                 len({cu.data_ptr() for _c, _h, cu, _d in self.host_puts if cu is not None})
             if self.e2e_in_place:
@@ -966,6 +1022,7 @@ def measure_dispatch(args, cid: int, rank: int, local_rank: int, world: int, dis
     n_dispatch = w.n * len(w.consumers)
     step = GpuStep(w, local_rank, args.api, args.fused, args.padded, warm_l2)
     step.e2e_path = args.e2e_path
+    step.e2e_schedule = args.e2e_schedule
     if args.padded:
         config["output"] = f"right-padded rows, widths {w.pad_prompt_to} / {w.pad_response_to}"
     if args.fused:
@@ -1031,7 +1088,7 @@ def measure_dispatch(args, cid: int, rank: int, local_rank: int, world: int, dis
         e2e_s, d2h, copies = step.run_e2e(min(args.steps, 5), 1)
         e2e_s, = max_over_ranks(dist, [e2e_s], step.dev)
         e2e = {"value": whole_job_rate(world, n_dispatch, e2e_s), "unit": "samples/s", "ms_per_step": e2e_s * 1e3,
-               "h2d_bytes_per_step": step.h2d_bytes, "d2h_bytes_per_step": d2h}
+               "h2d_bytes_per_step": getattr(step, "e2e_h2d_bytes", None) or step.h2d_bytes, "d2h_bytes_per_step": d2h}
         e2e.update(copies)
     rec["e2e"] = e2e
     step.close()

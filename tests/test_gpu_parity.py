@@ -821,6 +821,66 @@ def test_host_buffer_calls_single_and_batched(G):
         G.assert_state_equal(g, o, ctx=f"host batched={batched}")
 
 
+@pytest.mark.parametrize("in_place", [False, True])
+def test_two_waves_with_host_buffers_on_two_streams(G, in_place):
+    """The columns every worker state needs are put first; the states that need nothing else are
+    served on a second stream behind that put while the other columns are still being put on the
+    first; the actor update follows the second put.  Every batch is the oracle's: which samples
+    an id-only state is served, and what it is handed, does not depend on the columns still in
+    flight."""
+    import torch
+    w = wl.make_custom("waves", 48, 4, 4, prompt_len=(1, 300), response=("uniform", 0, 3000), vocab=50000,
+                       micro_batch=32, seed=53, with_entropy=True, schedule="bulk")
+    gets = [op for op in w.ops if op.kind == "get"]
+
+    def pinned(a):
+        t = torch.from_numpy(np.ascontiguousarray(a).view(np.int16) if a.dtype == np.uint16 else np.ascontiguousarray(a))
+        return (t.view(torch.bfloat16) if a.dtype == np.uint16 else t).pin_memory()
+
+    o, g = H.make_oracle(w), G.GpuDock(w)
+    first = {w.column_index("prompt_ids"), w.column_index("response_ids")}
+    upd = len(w.consumers) - 1
+    items = {True: [], False: []}
+    for op in w.ops:
+        if op.kind == "put":
+            cu, data = w.pack(op.column, op.indices)
+            o.put(op.column, op.indices, cu, data)
+            items[op.column in first].append((op.column, pinned(np.ascontiguousarray(op.indices, np.int32)),
+                                              pinned(cu) if cu is not None else None, pinned(data)))
+    pc, rc = g.token_caps(w.micro_batch)
+    bufs = [td.GetBuffers(g.dock, op.consumer, op.max_samples, prompt_tokens_cap=pc, response_tokens_cap=rc,
+                          host_payload=in_place) for op in gets]
+    hosts = [td.HostGetBuffers(b) for b in bufs]
+    waves = []
+    for early in (True, False):
+        sel = [j for j, op in enumerate(gets) if (op.consumer != upd) == early]
+        plan = g.dock.plan([bufs[j] for j in sel])
+        stage = torch.empty(sum(g.dock.put_host_stage_bytes(c, i.numel(), d.numel()) for c, i, _cu, d in items[early]),
+                            dtype=torch.uint8, device=g.device)
+        meta = torch.empty(g.dock.get_many_host_stage_bytes(plan), dtype=torch.uint8, device=g.device)
+        waves.append((items[early], stage, plan, [hosts[j] for j in sel], meta))
+    side = torch.cuda.Stream()
+    ev = torch.cuda.Event()
+    for rep in range(3):                       # the buffers, plans and staging areas are reused step after step
+        if rep:
+            g.dock.reset(); o.reset()
+            for op in w.ops:
+                if op.kind == "put":
+                    o.put(op.column, op.indices, *w.pack(op.column, op.indices))
+        (it_a, st_a, plan_a, hosts_a, meta_a), (it_b, st_b, plan_b, hosts_b, meta_b) = waves
+        g.dock.put_many_host(it_a, st_a)
+        ev.record()
+        g.dock.put_many_host(it_b, st_b)
+        side.wait_event(ev)
+        g.dock.get_many_host(plan_a, hosts_a, meta_a, stream=side)
+        g.dock.get_many_host(plan_b, hosts_b, meta_b)
+        for j, op in enumerate(gets):
+            want = o.get(op.consumer, op.max_samples)
+            G.assert_batch_equal(_host_batch(G, g, bufs[j], hosts[j]), want, f"step {rep} request {j}")
+        G.assert_state_equal(g, o, ctx=f"two waves, step {rep}")
+        G.assert_stats_equal(g, o, f"two waves, step {rep}")
+
+
 def test_validate_reports_planted_damage(G):
     """td_debug_validate passes on a dock in use and names damage planted into its tables from
     the host side (an unknown status bit, two rows at one place, a served mark without a claim)."""
