@@ -13,6 +13,11 @@ configuration describes, a producer stream against four polling consumer streams
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--config C] [--sigma S] [--warm-l2]
                   [--scenario dispatch|concurrent|cascade|scan|fixed-cost] [--impl reference]
+                  [--e2e-schedule pipelined|serial] [--e2e-path auto|in-place|copy]
+
+`e2e` is the same step through the calls that take HOST buffers, bus transfers inside the timed
+region; by default it is issued in two waves (the columns every worker state needs first, the
+states that need nothing else served on a second stream while the other columns come in).
 """
 from __future__ import annotations
 
